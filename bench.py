@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the Fathom decode-step hot path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic Qwen3-8B-shaped layer:
+    fathom_build_planes -> fathom_alloc_depth -> fathom_scan -> fathom_topk -> fathom_sparse_attend
+at n = 1,048,576 tokens, 8 KV heads / 32 query heads, d = 128, budget B = 48, k = 4096, planes in HBM
+(the million-token configuration the metric is quoted on).  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+--impl reference times the CPU oracle (oracle/, numpy fp64, as it stands) on a bounded sample of the
+same workload on the host cores; it is a deliberately slow baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2609_17652_b200 import dist as fdist
+
+METRIC = "keys_scanned_per_s"
+UNIT = "keys/s"
+WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3, planes in HBM)",
+                n=1 << 20, Hkv=8, Hq=32, d=128, B=48, k=4096, heads_per_plan=4)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (captured at n = 131072 and scaled by the tokens a full launch processes); None = not captured yet.
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": None, "scan_kernel": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=WORKLOAD["n"], help="tokens per session (default: the 1M configuration)")
+    ap.add_argument("--budget", type=int, default=WORKLOAD["B"])
+    ap.add_argument("--k", type=int, default=WORKLOAD["k"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-host-resident", action="store_true", help="skip the pinned-host-planes scan leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
+    ap.add_argument("--ref-sample-tokens", type=int, default=65536)
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def bits_per_token(depth_row) -> float:
+    t = np.asarray(depth_row).astype(np.int64)
+    return float(t.sum()) + float((t > 0).sum()) * 16.0 / 64.0
+
+
+# ------------------------------------------------------------------------------------------------ ours
+def run_ours(args):
+    from paper_2609_17652_b200 import binding as fb
+    from workloads.synth import make_layer
+
+    rank, world, local_rank = fdist.init_from_env(args.gpus, backend="nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    n, Hkv, Hq, d = args.n, WORKLOAD["Hkv"], WORKLOAD["Hq"], WORKLOAD["d"]
+    B, k, hpp = args.budget, args.k, WORKLOAD["heads_per_plan"]
+    G = Hq // Hkv
+
+    # weak scaling: every rank owns one independent session (its own seed); no data-path collective
+    session = fdist.sessions_of_rank(rank, world, n_sessions=world)[0]
+    L = make_layer(n, Hkv, Hq, d, seed=2, session=session, device=str(dev))
+    lay = fb.make_layout(Hkv, Hq, n, d)
+    ctx = fb.Context(local_rank, fb.fathom_scratch_bytes(lay, k))
+    planes = torch.zeros((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
+    scales = torch.zeros((Hkv, d, lay.scale_stride), dtype=torch.int16, device=dev)
+    depth = torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev)
+    scores = torch.zeros((Hq, lay.score_stride), dtype=torch.float32, device=dev)
+    idx = torch.zeros((Hq, k), dtype=torch.int32, device=dev)
+    out = torch.zeros((Hq, d), dtype=torch.float32, device=dev)
+    sm_scale = 1.0 / math.sqrt(d)
+    stream = torch.cuda.current_stream()
+
+    stage_names = ["build_planes", "alloc_depth", "scan", "topk", "sparse_attend"]
+    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 4, "sparse_attend": 2}
+
+    def stage(i, K=L.K, Kr=L.Krows, Vr=L.Vrows, q=L.q, var=L.var, pl=planes, sc=scales):
+        if i == 0:
+            ctx.fathom_build_planes(lay, K, pl, sc, stream)
+        elif i == 1:
+            ctx.fathom_alloc_depth(lay, q, var, fb.DEPTH_WATERFILL, B, hpp, depth, stream)
+        elif i == 2:
+            ctx.fathom_scan(lay, pl, sc, q, depth, hpp, scores, stream)
+        elif i == 3:
+            ctx.fathom_topk(lay, scores, k, 0, 0, idx, stream)
+        else:
+            ctx.fathom_sparse_attend(lay, q, Kr, Vr, idx, k, sm_scale, out, stream)
+
+    def step(events=None):
+        for i in range(5):
+            if events is not None:
+                events[i].record(stream)
+            stage(i)
+        if events is not None:
+            events[5].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: exactly `steps` steps, CUDA events on the launching stream, clocks sampled meanwhile
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    fdist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    t_wall = time.perf_counter()
+    for s in range(args.steps):
+        step(ev[s])
+    torch.cuda.synchronize()
+    t_wall = time.perf_counter() - t_wall
+    fdist.barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = ev[0][0].elapsed_time(ev[-1][5])
+    total_ms = fdist.max_over_ranks(total_ms)
+    ms_per_step = total_ms / args.steps
+    stage_us = {nm: 1e3 * statistics.mean(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps))
+                for i, nm in enumerate(stage_names)}
+    status = ctx.fathom_device_status()
+
+    depth_h = depth.cpu().numpy()
+    bits = float(np.mean([bits_per_token(r) for r in depth_h]))
+    plane_bytes_read = sum(bits_per_token(r) for r in depth_h) / 8.0 * n * (hpp / G)    # per launch, all KV heads
+    alg_bytes = {
+        "build_planes": n * Hkv * (d * 4 + 68.0),
+        "scan": plane_bytes_read + 4.0 * Hq * n,
+        "topk": 2 * 4.0 * Hq * n,
+        "sparse_attend": Hq * k * d * 2 * 2.0,
+    }
+    peak, peak_src = measured_peaks()
+
+    def roof(stage_key, t_us, kernel, unit_count):
+        ach = alg_bytes[stage_key] / (t_us * 1e-6) / 1e9
+        tr = NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD.get(kernel)
+        return {"kernel": kernel, "bound": "hbm", "achieved": round(ach, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(ach / peak, 4), "traffic": (tr * unit_count if tr else None),
+                "algorithmic_bytes": alg_bytes[stage_key], "launch_us": round(t_us, 2), "peak_source": peak_src}
+
+    # ---- isolated stage timings with an L2 flush before every launch (cold-cache view of each stage)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    iso_us = {}
+    for i, nm in enumerate(stage_names):
+        ts = []
+        for _ in range(10):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); stage(i); b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        iso_us[nm] = statistics.median(ts)
+
+    result = {
+        "metric": METRIC, "value": None, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64 bit planes + f32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD["name"], "n": n, "kv_heads": Hkv, "q_heads": Hq, "d": d, "budget_bits": B,
+                   "k": k, "heads_per_plan": hpp, "sessions_per_gpu": 1, "parallelism": f"{world} independent session(s), one per GPU",
+                   "l2": "step inputs (4 GiB of fp32 keys, 4 GiB of bf16 rows) exceed the 126 MB L2; no explicit flush in the timed region"},
+    }
+    keys_per_step = n * Hkv * world
+    result["value"] = keys_per_step / (ms_per_step * 1e-3)
+    result["gpu_launches"] = args.steps * sum(launches_per_step.values())
+    result["clocks"] = clocks
+    result["stage_us"] = {k_: round(v, 2) for k_, v in stage_us.items()}
+    result["stage_us_isolated_l2_flushed"] = {k_: round(v, 2) for k_, v in iso_us.items()}
+    result["decode_step_us_per_layer"] = round(sum(v for k_, v in stage_us.items() if k_ != "build_planes"), 2)
+    result["bits_per_token"] = round(bits, 2)
+    result["scan"] = {
+        "keys_per_s": n * Hkv / (stage_us["scan"] * 1e-6),
+        "plane_and_scale_bytes_read": plane_bytes_read,
+        "gbs_index_bytes_only": round(plane_bytes_read / (stage_us["scan"] * 1e-6) / 1e9, 1),
+        "gbs_with_score_writes": round(alg_bytes["scan"] / (stage_us["scan"] * 1e-6) / 1e9, 1),
+    }
+    result["roofline"] = roof("build_planes", stage_us["build_planes"], "build_planes_kernel", n * Hkv)
+    result["roofline_other_kernels"] = {
+        "scan": roof("scan", stage_us["scan"], "scan_kernel", n * Hkv),
+        "topk (4 kernels, 2 passes over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
+        "sparse_attend (2 kernels)": roof("sparse_attend", stage_us["sparse_attend"], "attend_*", n * Hkv),
+    }
+    result["device_status"] = status
+    result["wall_ms_per_step"] = round(1e3 * t_wall / args.steps, 4)
+
+    # ---- planes in pinned host memory, read zero-copy by the scan kernel over the host link
+    if rank == 0 and not args.no_host_resident:
+        result["host_resident_scan"] = host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, plane_bytes_read)
+
+    # ---- end to end through the C ABI from HOST buffers: H2D of the step's inputs and D2H of its result are timed
+    if not args.no_e2e:
+        result["e2e"] = e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step)
+    else:
+        result["e2e"] = None
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(args.cpu_sample_tokens, B, min(k, 2048), hpp)
+    fdist.barrier()
+    if rank == 0:
+        print(json.dumps(result))
+    ctx.close()
+    fdist.shutdown()
+
+
+def host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, plane_bytes_read):
+    hp = torch.empty(planes.shape, dtype=planes.dtype, pin_memory=True); hp.copy_(planes)
+    hs = torch.empty(scales.shape, dtype=scales.dtype, pin_memory=True); hs.copy_(scales)
+    # host-link probe: one pinned -> device copy of 1 GiB, best of 10
+    src = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(1 << 30, dtype=torch.uint8, device=planes.device)
+    best = 1e9
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); dst.copy_(src, non_blocking=True); b.record(stream)
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b))
+    link_gbs = (1 << 30) / (best * 1e-3) / 1e9
+    ts = []
+    for it in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        ctx.fathom_scan(lay, hp, hs, L.q, depth, hpp, scores, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            ts.append(a.elapsed_time(b))
+    t = statistics.median(ts)
+    gbs = plane_bytes_read / (t * 1e-3) / 1e9
+    del src, dst
+    return {"scan_ms": round(t, 4), "bytes_over_link": plane_bytes_read, "gbs": round(gbs, 2),
+            "link_peak_gbs": round(link_gbs, 2), "frac_of_measured_link": round(gbs / link_gbs, 4),
+            "link_probe": "1 GiB pinned->device copy, best of 10"}
+
+
+def e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step):
+    hK = torch.empty(L.K.shape, dtype=L.K.dtype, pin_memory=True); hK.copy_(L.K)
+    hKr = torch.empty(L.Krows.shape, dtype=L.Krows.dtype, pin_memory=True); hKr.copy_(L.Krows)
+    hVr = torch.empty(L.Vrows.shape, dtype=L.Vrows.dtype, pin_memory=True); hVr.copy_(L.Vrows)
+    hq = torch.empty(L.q.shape, dtype=L.q.dtype, pin_memory=True); hq.copy_(L.q)
+    hvar = torch.empty(L.var.shape, dtype=L.var.dtype, pin_memory=True); hvar.copy_(L.var)
+    hout = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+    dK, dKr, dVr, dq, dvar = (torch.empty_like(L.K), torch.empty_like(L.Krows), torch.empty_like(L.Vrows),
+                              torch.empty_like(L.q), torch.empty_like(L.var))
+    h2d = sum(t.numel() * t.element_size() for t in (hK, hKr, hVr, hq, hvar))
+    d2h = hout.numel() * hout.element_size()
+
+    def e2e_step():
+        dK.copy_(hK, non_blocking=True); dKr.copy_(hKr, non_blocking=True); dVr.copy_(hVr, non_blocking=True)
+        dq.copy_(hq, non_blocking=True); dvar.copy_(hvar, non_blocking=True)
+        for i in range(5):
+            stage(i, K=dK, Kr=dKr, Vr=dVr, q=dq, var=dvar)
+        hout.copy_(out, non_blocking=True)
+
+    steps = max(3, min(args.steps, 5))
+    e2e_step(); torch.cuda.synchronize()
+    fdist.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        e2e_step()
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = fdist.max_over_ranks(a.elapsed_time(b)) / steps
+    return {"value": keys_per_step / (ms * 1e-3), "unit": UNIT, "ms_per_step": round(ms, 3), "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "what": "pinned host K (fp32), K/V rows (bf16), q, var copied to the device, five C-ABI calls, result copied back"}
+
+
+# ------------------------------------------------------------------------------------------------ oracle legs
+def oracle_step(n_s, B, k, hpp, seed):
+    from oracle import fathom_oracle as O
+    from workloads.synth import make_layer
+    L = make_layer(n_s, WORKLOAD["Hkv"], WORKLOAD["Hq"], WORKLOAD["d"], seed=seed, device="cpu")
+    K, q, var = L.K.numpy(), L.q.numpy(), L.var.numpy()
+    Kr, Vr = L.Krows.float().numpy(), L.Vrows.float().numpy()
+    t0 = time.perf_counter()
+    planes, scales = O.build_planes(K)
+    depth = O.alloc_depth(q, var, "waterfill", B, hpp)
+    s = O.scan(planes, scales, q, depth, n_s, hpp)
+    idx = O.topk(s, k)
+    O.sparse_attend(q, Kr, Vr, idx, 1.0 / math.sqrt(WORKLOAD["d"]))
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(n_s, B, k, hpp):
+    from threadpoolctl import threadpool_limits
+    torch.set_num_threads(1)
+    with threadpool_limits(limits=1):
+        dt = oracle_step(n_s, B, k, hpp, seed=2)
+    return {"value": n_s * WORKLOAD["Hkv"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
+            "host_cores_available": os.cpu_count(),
+            "sample": f"one step of the same layer shape at n = {n_s} tokens (8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from threadpoolctl import threadpool_limits
+    torch.set_num_threads(1)
+    n_s, B, hpp = args.ref_sample_tokens, args.budget, WORKLOAD["heads_per_plan"]
+    k = min(args.k, 2048)
+    with threadpool_limits(limits=1):
+        for w in range(args.warmup):
+            oracle_step(n_s, B, k, hpp, seed=100 + w)
+        ts = [oracle_step(n_s, B, k, hpp, seed=200 + s) for s in range(args.steps)]
+    dt = sum(ts) / len(ts)
+    val = n_s * WORKLOAD["Hkv"] / dt
+    sample = f"each step = one layer of the same shape at n = {n_s} tokens (8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD["name"], "n": args.n, "kv_heads": 8, "q_heads": 32, "d": 128,
+                   "budget_bits": B, "k": args.k, "heads_per_plan": hpp},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

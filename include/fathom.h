@@ -1,0 +1,152 @@
+/*
+ * fathom.h — C ABI of the B200 (sm_100a) implementation of Fathom's decode-step hot path:
+ * bit-plane key store, per-query depth allocation, variable-depth bit-plane scan, top-k
+ * selection and exact attention over the selected rows.
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Shapes: Hkv KV heads, Hq query heads, G = Hq / Hkv query heads per KV head (query head h
+ *    reads KV head h / G), d = 128 channels, n tokens, nb = ceil(n / 64) blocks of 64 tokens.
+ *  - Every data pointer is a DEVICE pointer unless the argument says otherwise.  `planes` and
+ *    `scales` may instead point to pinned host memory that the device can address (the paper's
+ *    host-resident store, Sec. 3.5): the scan then reads it directly over the host link.
+ *  - All buffers are allocated and owned by the caller.  The library allocates only the scratch
+ *    arena and one status word when a context is created, and frees them when it is destroyed.
+ *  - The five data-path calls only ENQUEUE work on `stream` (a cudaStream_t passed as void*;
+ *    NULL = the legacy default stream).  None of them synchronises; results (`depth`, `scores`,
+ *    `idx`) stay on the device and feed the next call, so a decode step needs no host round trip
+ *    (Sec. 3.5, Appendix A6: fixed-size plan, no host synchronisation).
+ *  - Return value: FATHOM_OK (0) or a negative fathom_status.  Arguments that can be checked on
+ *    the host (null pointers, d != 128, strides too small or misaligned, k out of range, scratch
+ *    too small) are rejected before anything is launched and leave all outputs untouched.
+ *    Conditions only the device can see are recorded in a status word read back with
+ *    fathom_device_status(); kernels never trap, assert or wait without a bound.
+ *  - Determinism: the same inputs give the same bytes in `planes`, `scales`, `depth`, `idx`,
+ *    `scores` and `out` on every run (no floating-point atomics anywhere).
+ *  - Inputs must be finite; |k| must stay below 8 * 65504 so that a block scale fits fp16.
+ *  - One context may be used by one host thread at a time; calls on different streams that use
+ *    the same context share its scratch arena and must not overlap on the device.
+ */
+#ifndef FATHOM_H_
+#define FATHOM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FATHOM_OK = 0,
+  FATHOM_ERR_INVALID_ARG = -1,      /* null pointer, non-positive size, k or budget out of range */
+  FATHOM_ERR_UNSUPPORTED = -2,      /* d != 128, heads_per_plan not in {1,2,4,8}, unknown mode/dtype */
+  FATHOM_ERR_ALIGNMENT = -3,        /* pointer or stride not aligned as the layout requires */
+  FATHOM_ERR_SCRATCH_TOO_SMALL = -4,/* context scratch smaller than fathom_scratch_bytes() for this call */
+  FATHOM_ERR_CUDA = -5              /* a CUDA runtime call failed (see fathom_last_cuda_error) */
+} fathom_status;
+
+typedef enum { FATHOM_F32 = 0, FATHOM_BF16 = 1 } fathom_dtype;
+
+typedef enum {
+  FATHOM_DEPTH_WATERFILL = 0,       /* reverse water-filling of `budget` bits (Sec. 3.3, Eq. 3-4) */
+  FATHOM_DEPTH_FIXED_TOP_R = 1,     /* `budget` = r channels with the largest sum_h |q_j| at depth 4 (Sec. 2, SparQ's grouped rule) */
+  FATHOM_DEPTH_UNIFORM = 2          /* every channel at depth `budget` in 0..4 (Sec. 2, thumbnail scans) */
+} fathom_depth_mode;
+
+/* Bits of the device status word (fathom_device_status). */
+#define FATHOM_DEV_TOPK_SHORT     0x1u  /* top-k found fewer than k eligible tokens (non-finite scores) */
+#define FATHOM_DEV_WAIT_EXPIRED   0x2u  /* a bounded device-side wait gave up */
+
+/* One session's store for one layer.  Strides are in elements of the respective array. */
+typedef struct {
+  int32_t n_kv_heads;          /* Hkv >= 1 */
+  int32_t n_q_heads;           /* Hq, a multiple of Hkv */
+  int32_t d;                   /* channels per head; must be 128 */
+  int32_t reserved;            /* set to 0 */
+  int64_t n;                   /* tokens, n >= 1 */
+  int64_t plane_stride_words;  /* uint64 words per (KV head, channel, plane) row; >= nb, multiple of 2 (16 B) */
+  int64_t scale_stride;        /* fp16 elements per (KV head, channel) row; >= nb, multiple of 8 (16 B) */
+  int64_t score_stride;        /* floats per query-head score row; >= n, multiple of 4 (16 B) */
+} fathom_layout;
+
+typedef struct fathom_ctx fathom_ctx;   /* opaque: device id, scratch arena, status word */
+
+/* ---- context ------------------------------------------------------------------------------
+ * fathom_create allocates `scratch_bytes` of device memory on `device` (plus a status word) and
+ * returns a context in *ctx (host pointer).  fathom_destroy frees both; passing NULL is a no-op.
+ * fathom_scratch_bytes returns the scratch a context needs so that every call with this layout
+ * and this k succeeds (top-k: histograms, candidate and winner lists; attention: split partials).
+ * The paper has no counterpart of these three; they exist so that the data path never allocates. */
+int fathom_create(fathom_ctx** ctx, int device, size_t scratch_bytes);
+int fathom_destroy(fathom_ctx* ctx);
+size_t fathom_scratch_bytes(const fathom_layout* layout, int k);
+
+/* Human-readable text for a fathom_status (static string, never NULL). */
+const char* fathom_strerror(int status);
+/* Text of the last CUDA error seen by this context (static or context-owned string). */
+const char* fathom_last_cuda_error(const fathom_ctx* ctx);
+/* Copies the device status word to *status (host pointer) and clears it.  Synchronises `stream`. */
+int fathom_device_status(fathom_ctx* ctx, void* stream, uint32_t* status);
+/* Library version, major * 100 + minor. */
+int fathom_version(void);
+
+/* ---- (1) plane builder — Sec. 3.2, Eq. 2 and the paragraph that follows it ----------------
+ * For every KV head, 64-token block beta and channel j:  a = max_{i in beta, i < n} |k_ij|, the stored
+ * scale is s = fp16_round_nearest(a / 8) and the code is c = clip(floor(k / s), -8, 7) + 8 taken with
+ * the stored scale (s == 0 gives c = 8).  Bit p (0 = most significant = sign) of the 64 codes is packed
+ * into one 64-bit word, token i at bit (i mod 64), absent tail tokens as 0.
+ *   K       in   [Hkv][n][d], token-major, k_dtype FATHOM_F32 or FATHOM_BF16, 16-byte aligned
+ *   planes  out  [Hkv][d][4][plane_stride_words] uint64; words beta >= nb of a row are not written
+ *   scales  out  [Hkv][d][scale_stride] fp16 bit patterns; elements beta >= nb are not written
+ * A prefix of t planes of a channel is its t-bit mid-rise quantiser with the same block scale. */
+int fathom_build_planes(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype,
+                        uint64_t* planes, uint16_t* scales, void* stream);
+
+/* ---- (2) depth allocator — Sec. 3.3, Eq. 3 and Eq. 4; Appendix A -------------------------
+ * One plan per `heads_per_plan` consecutive query heads (G = the paper's group-shared plan; 1 = one
+ * plan per query head).  WATERFILL: g_j = (sum_h q_hj^2) * var_j in fp64; the 4d candidate planes
+ * (j, m = 1..4) are ranked by g_j 4^-m (ties: lower channel, then lower plane) and the first
+ * min(budget, 4d) are granted; depth_j = planes granted to channel j.  This is Eq. 4 at the smallest
+ * water line whose depths fit the budget, evaluated exactly, so sum_j depth_j == min(budget, 4d).
+ *   q      in   [Hq][d] fp32          var  in  [Hkv][d] fp32 (unused by the other two modes)
+ *   depth  out  [Hq / heads_per_plan][d] uint8, values 0..4 */
+int fathom_alloc_depth(fathom_ctx* ctx, const fathom_layout* layout, const float* q, const float* var,
+                       int mode, int budget, int heads_per_plan, uint8_t* depth, void* stream);
+
+/* ---- (3) scan — Sec. 3.2 (prefix dequantiser), Sec. 3.3 (inactive channels are skipped) ---
+ * For every plan, every query head h of it and every token i < n:
+ *   scores[h][i] = sum_{j : depth_j > 0} q_hj * (c_ij >> (4 - t_j) + 1/2 - 2^(t_j - 1)) * (8 s_{beta(i), j}) / 2^(t_j - 1)
+ * reading only planes p < t_j and the scales of the active channels; fp32 accumulation; no 1/sqrt(d)
+ * factor.  `planes` / `scales` may be device memory or device-addressable pinned host memory.
+ *   scores  out  [Hq][score_stride] fp32; elements i >= n of a row are not written
+ * heads_per_plan must be 1, 2, 4 or 8 and divide G. */
+int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes,
+                const uint16_t* scales, const float* q, const uint8_t* depth, int heads_per_plan,
+                float* scores, void* stream);
+
+/* ---- (4) top-k — Sec. 2 "Top-k decoding" ---------------------------------------------------
+ * Per query head: the first n_sink and the last n_local tokens are always selected; the remaining
+ * k - |forced| are the tokens with the highest scores among the others, ties to the lower token
+ * index, -0 equal to +0.  Requires 1 <= k <= n, forced count <= k, k <= FATHOM_MAX_K.
+ *   scores  in   [Hq][score_stride] fp32 (finite)
+ *   idx     out  [Hq][k] int32, ascending token indices
+ * Uses the context scratch (fathom_scratch_bytes). */
+#define FATHOM_MAX_K 16384
+int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* scores, int k,
+                int n_sink, int n_local, int32_t* idx, void* stream);
+
+/* ---- (5) gather + exact attention — Sec. 2 "Top-k decoding" --------------------------------
+ * Per query head h with KV head h / G:  out[h] = softmax_i(softmax_scale * q_h . K[idx[h][i]]) . V[idx[h][i]]
+ * over its own k selected rows (fp32 arithmetic on rows of `row_dtype`).
+ *   Krows, Vrows  in  [Hkv][n][d] FATHOM_BF16 or FATHOM_F32, 16-byte aligned
+ *   idx           in  [Hq][k] int32, each in [0, n)        out  [Hq][d] fp32
+ * Uses the context scratch (fathom_scratch_bytes). */
+int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* layout, const float* q,
+                         const void* Krows, const void* Vrows, int row_dtype, const int32_t* idx,
+                         int k, float softmax_scale, float* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FATHOM_H_ */

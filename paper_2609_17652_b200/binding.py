@@ -1,0 +1,160 @@
+"""ctypes binding of libfathom.so: argument marshalling only, every step runs in the CUDA kernels.
+
+The function names are those of the C ABI (include/fathom.h).  Tensors are torch tensors used as
+plain device (or pinned host) buffers; their data pointers are passed through unchanged.  There is
+no CPU fallback: if the library cannot be loaded, importing raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfathom.so")
+
+F32, BF16 = 0, 1
+DEPTH_WATERFILL, DEPTH_FIXED_TOP_R, DEPTH_UNIFORM = 0, 1, 2
+MAX_K = 16384
+DEV_TOPK_SHORT, DEV_WAIT_EXPIRED = 0x1, 0x2
+
+EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error",
+           "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
+           "fathom_topk", "fathom_sparse_attend"]
+
+
+class Layout(C.Structure):
+    _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("d", C.c_int32), ("reserved", C.c_int32),
+                ("n", C.c_int64), ("plane_stride_words", C.c_int64), ("scale_stride", C.c_int64),
+                ("score_stride", C.c_int64)]
+
+
+def make_layout(Hkv: int, Hq: int, n: int, d: int = 128) -> Layout:
+    """Tight strides rounded up to the 16-byte multiples the layout requires."""
+    nb = (n + 63) // 64
+    return Layout(Hkv, Hq, d, 0, n, (nb + 1) // 2 * 2, (nb + 7) // 8 * 8, (n + 3) // 4 * 4)
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2609_17652_b200.build` (needs nvcc); "
+                          "there is no fallback path")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int, C.c_int64
+    LP = C.POINTER(Layout)
+    lib.fathom_create.argtypes = [C.POINTER(vp), i32, C.c_size_t]
+    lib.fathom_destroy.argtypes = [vp]
+    lib.fathom_scratch_bytes.argtypes = [LP, i32]
+    lib.fathom_scratch_bytes.restype = C.c_size_t
+    lib.fathom_strerror.argtypes = [i32]
+    lib.fathom_strerror.restype = C.c_char_p
+    lib.fathom_last_cuda_error.argtypes = [vp]
+    lib.fathom_last_cuda_error.restype = C.c_char_p
+    lib.fathom_device_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    lib.fathom_version.argtypes = []
+    lib.fathom_build_planes.argtypes = [vp, LP, vp, i32, vp, vp, vp]
+    lib.fathom_alloc_depth.argtypes = [vp, LP, vp, vp, i32, i32, i32, vp, vp]
+    lib.fathom_scan.argtypes = [vp, LP, vp, vp, vp, vp, i32, vp, vp]
+    lib.fathom_topk.argtypes = [vp, LP, vp, i32, i32, i32, vp, vp]
+    lib.fathom_sparse_attend.argtypes = [vp, LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
+    for name in EXPORTS:
+        if name not in ("fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error"):
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+class FathomError(RuntimeError):
+    def __init__(self, status: int, ctx=None):
+        msg = lib.fathom_strerror(status).decode()
+        if status == -5 and ctx is not None:
+            msg += ": " + lib.fathom_last_cuda_error(ctx).decode()
+        super().__init__(f"fathom status {status}: {msg}")
+        self.status = status
+
+
+def _ptr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+class Context:
+    """Owns one fathom_ctx (scratch arena + status word) on one device."""
+
+    def __init__(self, device: int = 0, scratch_bytes: int = 0):
+        self._h = C.c_void_p()
+        rc = lib.fathom_create(C.byref(self._h), device, scratch_bytes)
+        if rc != 0:
+            raise FathomError(rc)
+        self.device, self.scratch_bytes = device, scratch_bytes
+
+    def close(self):
+        if self._h:
+            lib.fathom_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != 0:
+            raise FathomError(rc, self._h)
+
+    # ---- the five calls (raw status returned by the *_rc variants is used by the error-path tests)
+    def fathom_build_planes(self, layout, K, planes, scales, stream=None, k_dtype=None):
+        self._check(lib.fathom_build_planes(self._h, C.byref(layout), _ptr(K), _dtype_code(K) if k_dtype is None else k_dtype,
+                                            _ptr(planes), _ptr(scales), _stream(stream)))
+
+    def fathom_alloc_depth(self, layout, q, var, mode, budget, heads_per_plan, depth, stream=None):
+        self._check(lib.fathom_alloc_depth(self._h, C.byref(layout), _ptr(q), _ptr(var), mode, budget, heads_per_plan,
+                                           _ptr(depth), _stream(stream)))
+
+    def fathom_scan(self, layout, planes, scales, q, depth, heads_per_plan, scores, stream=None):
+        self._check(lib.fathom_scan(self._h, C.byref(layout), _ptr(planes), _ptr(scales), _ptr(q), _ptr(depth),
+                                    heads_per_plan, _ptr(scores), _stream(stream)))
+
+    def fathom_topk(self, layout, scores, k, n_sink, n_local, idx, stream=None):
+        self._check(lib.fathom_topk(self._h, C.byref(layout), _ptr(scores), k, n_sink, n_local, _ptr(idx), _stream(stream)))
+
+    def fathom_sparse_attend(self, layout, q, Krows, Vrows, idx, k, softmax_scale, out, stream=None, row_dtype=None):
+        self._check(lib.fathom_sparse_attend(self._h, C.byref(layout), _ptr(q), _ptr(Krows), _ptr(Vrows),
+                                             _dtype_code(Krows) if row_dtype is None else row_dtype, _ptr(idx), k,
+                                             C.c_float(softmax_scale), _ptr(out), _stream(stream)))
+
+    def fathom_device_status(self, stream=None) -> int:
+        st = C.c_uint32(0)
+        self._check(lib.fathom_device_status(self._h, _stream(stream), C.byref(st)))
+        return st.value
+
+
+def fathom_scratch_bytes(layout: Layout, k: int) -> int:
+    return int(lib.fathom_scratch_bytes(C.byref(layout), k))
+
+
+def fathom_version() -> int:
+    return int(lib.fathom_version())

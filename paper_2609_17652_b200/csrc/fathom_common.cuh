@@ -1,0 +1,58 @@
+// Internal definitions shared by the translation units of libfathom (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "fathom.h"
+
+#define FATHOM_D 128            // channels per head (Sec. 1: Qwen3-8B head size)
+#define FATHOM_BLOCK 64         // tokens per scale block (Sec. 3.2)
+#define FATHOM_NPLANES 4        // bits per code (Sec. 3.2)
+
+struct fathom_ctx {
+  int device;
+  void* scratch;               // device arena, 256-byte aligned
+  size_t scratch_bytes;
+  uint32_t* dev_status;        // device status word
+  cudaError_t last_cuda;
+};
+
+static inline int fathom_cuda_fail(fathom_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda = e;
+  return FATHOM_ERR_CUDA;
+}
+
+#define FATHOM_CUDA_TRY(ctx, expr)                              \
+  do {                                                          \
+    cudaError_t e__ = (expr);                                   \
+    if (e__ != cudaSuccess) return fathom_cuda_fail((ctx), e__);\
+  } while (0)
+
+// Checks every host-visible property of a layout.  Returns FATHOM_OK or the error.
+int fathom_check_layout(const fathom_layout* L);
+
+static inline int64_t fathom_nblocks(int64_t n) { return (n + FATHOM_BLOCK - 1) / FATHOM_BLOCK; }
+static inline bool fathom_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t fathom_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- scratch arena carving (one place, used by fathom_scratch_bytes and by the calls) --------
+#define FATHOM_TOPK_BINS 4096            // 12 leading bits of the ordered score key
+#define FATHOM_ATTN_CHUNK 128            // selected rows handled by one CTA of the partial kernel
+
+struct fathom_topk_scratch {
+  uint32_t* hist;        // [Hq][FATHOM_TOPK_BINS]
+  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 3 winners written, 4 candidates written
+  int32_t* cand;         // [Hq][n] token indices of the threshold bin
+  int32_t* winners;      // [Hq][k] unordered winners
+  size_t bytes;
+};
+struct fathom_attn_scratch {
+  float* partial;        // [Hq][splits][d + 2]: running max, denominator, weighted V sum
+  int splits;
+  size_t bytes;
+};
+fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k);
+fathom_attn_scratch fathom_carve_attn(void* base, int Hq, int k);

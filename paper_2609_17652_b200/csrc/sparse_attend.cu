@@ -1,0 +1,157 @@
+// fathom_sparse_attend: gather of the selected K/V rows + exact softmax attention (Sec. 2 "Top-k decoding").
+//
+// Split-k: CTA (split, head) handles FATHOM_ATTN_CHUNK selected rows.  Logits: one thread per row reads
+// its whole K row with 16-byte loads (a row is 256 B in bf16) against q held in shared memory.  After the
+// chunk maximum and exp, each warp walks 32 rows of V with a lane owning 4 channels (one coalesced
+// 256/512-byte row per load instruction) and the four warps are summed in a fixed order.  A second kernel
+// merges the per-chunk (max, denominator, weighted sum) triples in split order, so the output is
+// bit-reproducible.
+#include "fathom_common.cuh"
+
+namespace {
+
+constexpr int AT_THREADS = FATHOM_ATTN_CHUNK;   // 128 threads: one per row, then one per channel
+constexpr int AT_WARPS = AT_THREADS / 32;
+
+__device__ __forceinline__ float dot_row(const __nv_bfloat16* row, const float* sq) {
+  const uint4* r = reinterpret_cast<const uint4*>(row);
+  float acc = 0.0f;
+#pragma unroll
+  for (int v = 0; v < FATHOM_D / 8; ++v) {
+    const uint4 x = __ldg(r + v);
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      acc = fmaf(__uint_as_float(w[c] << 16), sq[v * 8 + 2 * c], acc);
+      acc = fmaf(__uint_as_float(w[c] & 0xffff0000u), sq[v * 8 + 2 * c + 1], acc);
+    }
+  }
+  return acc;
+}
+__device__ __forceinline__ float dot_row(const float* row, const float* sq) {
+  const float4* r = reinterpret_cast<const float4*>(row);
+  float acc = 0.0f;
+#pragma unroll
+  for (int v = 0; v < FATHOM_D / 4; ++v) {
+    const float4 x = __ldg(r + v);
+    acc = fmaf(x.x, sq[v * 4 + 0], acc);
+    acc = fmaf(x.y, sq[v * 4 + 1], acc);
+    acc = fmaf(x.z, sq[v * 4 + 2], acc);
+    acc = fmaf(x.w, sq[v * 4 + 3], acc);
+  }
+  return acc;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float v[4]) {
+  const uint2 x = __ldg(reinterpret_cast<const uint2*>(p));
+  v[0] = __uint_as_float(x.x << 16); v[1] = __uint_as_float(x.x & 0xffff0000u);
+  v[2] = __uint_as_float(x.y << 16); v[3] = __uint_as_float(x.y & 0xffff0000u);
+}
+__device__ __forceinline__ void load4(const float* p, float v[4]) {
+  const float4 x = __ldg(reinterpret_cast<const float4*>(p));
+  v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(AT_THREADS)
+attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, const T* __restrict__ Vrows,
+                      const int32_t* __restrict__ idx, int k, long long n, int G, float softmax_scale,
+                      float* __restrict__ partial, int splits) {
+  __shared__ float s_q[FATHOM_D];
+  __shared__ float s_p[AT_THREADS];
+  __shared__ int32_t s_idx[AT_THREADS];
+  __shared__ float s_red[AT_WARPS];
+  __shared__ float s_acc[AT_WARPS][FATHOM_D];
+  const int split = blockIdx.x, head = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kv = head / G;
+  const T* Kh = Krows + (size_t)kv * (size_t)n * FATHOM_D;
+  const T* Vh = Vrows + (size_t)kv * (size_t)n * FATHOM_D;
+  s_q[tid] = q[(size_t)head * FATHOM_D + tid];
+  const int pos = split * AT_THREADS + tid;
+  const bool valid = pos < k;
+  int32_t row = 0;
+  if (valid) {
+    row = idx[(size_t)head * k + pos];
+    row = (row < 0) ? 0 : ((long long)row >= n ? (int32_t)(n - 1) : row);   // out-of-range indices are clamped, never dereferenced
+  }
+  s_idx[tid] = row;
+  __syncthreads();
+
+  float e = -INFINITY;
+  if (valid) e = dot_row(Kh + (size_t)row * FATHOM_D, s_q) * softmax_scale;
+  float m = e;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) s_red[warp] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  const float p = valid ? expf(e - m) : 0.0f;
+  s_p[tid] = p;
+  float l = p;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  __syncthreads();                                           // s_red reads done, s_p visible
+  if (lane == 0) s_red[warp] = l;
+
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const int rows_here = min(AT_THREADS, k - split * AT_THREADS);
+  const int r_end = min(rows_here, (warp + 1) * 32);
+#pragma unroll 8
+  for (int r = warp * 32; r < r_end; ++r) {
+    float v[4];
+    load4(Vh + (size_t)s_idx[r] * FATHOM_D + 4 * lane, v);
+    const float pr = s_p[r];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[c] = fmaf(pr, v[c], acc[c]);
+  }
+#pragma unroll
+  for (int c = 0; c < 4; ++c) s_acc[warp][4 * lane + c] = acc[c];
+  __syncthreads();
+  float* out = partial + ((size_t)head * splits + split) * (FATHOM_D + 2);
+  out[2 + tid] = ((s_acc[0][tid] + s_acc[1][tid]) + s_acc[2][tid]) + s_acc[3][tid];
+  if (tid == 0) { out[0] = m; out[1] = ((s_red[0] + s_red[1]) + s_red[2]) + s_red[3]; }
+}
+
+__global__ void __launch_bounds__(FATHOM_D)
+attend_combine_kernel(const float* __restrict__ partial, int splits, float* __restrict__ out) {
+  const int head = blockIdx.x, tid = threadIdx.x;
+  const float* P = partial + (size_t)head * splits * (FATHOM_D + 2);
+  float M = -INFINITY;
+  for (int s = 0; s < splits; ++s) M = fmaxf(M, P[(size_t)s * (FATHOM_D + 2)]);
+  float num = 0.0f, den = 0.0f;
+  for (int s = 0; s < splits; ++s) {
+    const float* ps = P + (size_t)s * (FATHOM_D + 2);
+    const float w = expf(ps[0] - M);
+    den = fmaf(w, ps[1], den);
+    num = fmaf(w, ps[2 + tid], num);
+  }
+  out[(size_t)head * FATHOM_D + tid] = num / den;
+}
+
+}  // namespace
+
+extern "C" int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* L, const float* q, const void* Krows,
+                                    const void* Vrows, int row_dtype, const int32_t* idx, int k, float softmax_scale,
+                                    float* out, void* stream) {
+  if (!ctx || !q || !Krows || !Vrows || !idx || !out) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k < 1 || k > L->n) return FATHOM_ERR_INVALID_ARG;
+  if (row_dtype != FATHOM_BF16 && row_dtype != FATHOM_F32) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(Krows) || !fathom_aligned16(Vrows)) return FATHOM_ERR_ALIGNMENT;
+  const int Hq = L->n_q_heads, G = Hq / L->n_kv_heads;
+  fathom_attn_scratch S = fathom_carve_attn(ctx->scratch, Hq, k);
+  if (S.bytes > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid((unsigned)S.splits, (unsigned)Hq);
+  if (row_dtype == FATHOM_BF16)
+    attend_partial_kernel<__nv_bfloat16><<<grid, AT_THREADS, 0, st>>>(
+        q, static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k, L->n, G,
+        softmax_scale, S.partial, S.splits);
+  else
+    attend_partial_kernel<float><<<grid, AT_THREADS, 0, st>>>(q, static_cast<const float*>(Krows),
+                                                              static_cast<const float*>(Vrows), idx, k, L->n, G,
+                                                              softmax_scale, S.partial, S.splits);
+  attend_combine_kernel<<<Hq, FATHOM_D, 0, st>>>(S.partial, S.splits, out);
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}

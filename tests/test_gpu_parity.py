@@ -1,0 +1,192 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fathom_oracle as O
+from workloads.synth import make_layer
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from tests._pipeline import run_gpu, score_tolerance
+
+
+def host(L):
+    return {"K": L.K.cpu().numpy(), "q": L.q.cpu().numpy(), "var": L.var.cpu().numpy(),
+            "Krows": L.Krows.float().cpu().numpy(), "Vrows": L.Vrows.float().cpu().numpy()}
+
+
+def check_all(L, B, k, hpp, mode=0, n_sink=0, n_local=0, **kw):
+    H = host(L)
+    g = run_gpu(L, B, k, hpp, mode=mode, n_sink=n_sink, n_local=n_local, **kw)
+    # (1) planes / scales bit-exact; padding untouched
+    planes, scales = O.build_planes(H["K"])
+    assert np.array_equal(g["scales"].view(np.uint16), scales.view(np.uint16))
+    assert np.array_equal(g["planes"], planes)
+    assert np.all(g["planes_pad"] == -1)
+    # (2) depths bit-exact
+    mode_name = {0: "waterfill", 1: "fixed_top_r", 2: "uniform"}[mode]
+    depth = O.alloc_depth(H["q"], H["var"], mode_name, B, hpp)
+    assert np.array_equal(g["depth"], depth)
+    # (3) scores within 1e-5 (relative to max(|s|, rms))
+    ref = O.scan(planes, scales, H["q"], depth, L.n, hpp)
+    err = np.abs(g["scores"].astype(np.float64) - ref)
+    assert np.all(err <= score_tolerance(ref)), float((err / score_tolerance(ref)).max())
+    assert np.all(np.isnan(g["scores_pad"]))
+    # (4) top-k, stage-isolated: oracle top-k of the GPU's own scores, bit-exact index lists
+    idx = O.topk(g["scores"].astype(np.float64), k, n_sink, n_local)
+    assert np.array_equal(g["idx"], idx)
+    # end to end: sets may differ only inside the tolerance band around the k-th oracle score
+    idx_ref = O.topk(ref, k, n_sink, n_local)
+    for h in range(L.Hq):
+        diff = np.setxor1d(idx_ref[h], g["idx"][h])
+        if len(diff):
+            kth = np.sort(ref[h])[::-1][k - 1]
+            assert np.all(np.abs(ref[h, diff] - kth) <= 4 * score_tolerance(ref)[h].max())
+    # (5) attention over the same index lists
+    Kr = H["K"] if kw.get("rows_dtype") == torch.float32 else H["Krows"]       # rows at the precision the GPU was given
+    o_ref = O.sparse_attend(H["q"], Kr, H["Vrows"], g["idx"], 1.0 / math.sqrt(L.d))
+    rel = np.linalg.norm(g["out"] - o_ref, axis=1) / np.linalg.norm(o_ref, axis=1)
+    assert rel.max() <= 2e-3, rel.max()
+    assert g["status"] == 0
+    return g, ref
+
+
+def test_config1_tiny_single_head():
+    L = make_layer(4096, Hkv=1, Hq=1, seed=0, device="cuda")
+    g, _ = check_all(L, B=48, k=64, hpp=1)
+    assert set(L.needles[0].tolist()) <= set(g["idx"][0].tolist())
+
+
+@pytest.mark.parametrize("n", [1, 63, 64, 65, 127, 200, 2047, 2049, 4100, 9001])
+def test_ragged_lengths(n):
+    L = make_layer(n, Hkv=2, Hq=8, seed=n, device="cuda")
+    k = max(1, min(n, 37 if n > 40 else n))
+    check_all(L, B=48, k=k, hpp=4)
+
+
+@pytest.mark.parametrize("hpp", [1, 2, 4])
+def test_plan_granularity(hpp):
+    L = make_layer(5000, Hkv=2, Hq=8, seed=3, device="cuda")
+    check_all(L, B=48, k=100, hpp=hpp)
+
+
+def test_eight_heads_per_plan():
+    L = make_layer(3000, Hkv=1, Hq=8, seed=4, device="cuda")
+    check_all(L, B=64, k=50, hpp=8)
+
+
+@pytest.mark.parametrize("mode,budget", [(1, 16), (1, 32), (2, 2), (2, 0), (0, 0), (0, 1), (0, 136), (0, 511), (0, 512), (0, 600)])
+def test_depth_modes_and_budgets(mode, budget):
+    L = make_layer(4500, Hkv=2, Hq=8, seed=5, device="cuda")
+    check_all(L, B=budget, k=77, hpp=4, mode=mode)
+
+
+def test_sink_and_local_tokens():
+    L = make_layer(6000, Hkv=2, Hq=8, seed=6, device="cuda")
+    g, _ = check_all(L, B=48, k=128, hpp=4, n_sink=4, n_local=32)
+    for h in range(8):
+        s = set(g["idx"][h].tolist())
+        assert set(range(4)) <= s and set(range(6000 - 32, 6000)) <= s
+    check_all(L, B=48, k=36, hpp=4, n_sink=4, n_local=32)       # nothing left to select
+
+
+def test_all_planes_equals_dense_4bit_dot_product():
+    L = make_layer(8192, Hkv=2, Hq=8, seed=7, device="cuda")
+    g, _ = check_all(L, B=512, k=256, hpp=4)
+    codes, scales = O.quantise_block_codes(L.K.cpu().numpy())
+    S = np.repeat(scales.astype(np.float64), 64, axis=2)[:, :, :L.n].transpose(0, 2, 1)
+    deq = (codes.astype(np.float64) - 7.5) * S
+    qh = L.q.cpu().numpy().astype(np.float64)
+    for h in range(8):
+        ref = deq[h // 4] @ qh[h]
+        assert np.all(np.abs(g["scores"][h] - ref) <= score_tolerance(ref[None])[0])
+
+
+def test_topk_heavy_ties_and_signed_zero():
+    from paper_2609_17652_b200 import binding as fb
+    n, Hq = 20000, 4
+    lay = fb.make_layout(1, Hq, n)
+    r = np.random.default_rng(0)
+    s = np.zeros((Hq, lay.score_stride), dtype=np.float32)
+    s[0, :n] = np.round(r.standard_normal(n), 1)                # many exact ties
+    s[1, :n] = 1.0                                              # all equal: the k lowest indices win
+    s[2, :n] = np.where(r.random(n) < 0.5, 0.0, -0.0)           # +0 / -0 are equal
+    s[3, :n] = -np.abs(np.round(r.standard_normal(n), 2))       # all non-positive
+    sc = torch.from_numpy(s).cuda()
+    for k in (1, 5, 1000, 4096):
+        ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+        idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+        ctx.fathom_topk(lay, sc, k, 0, 0, idx)
+        want = O.topk(s[:, :n].astype(np.float64), k)
+        assert np.array_equal(idx.cpu().numpy(), want)
+        assert ctx.fathom_device_status() == 0
+        ctx.close()
+
+
+def test_attention_fp32_rows_and_k_equals_n():
+    L = make_layer(300, Hkv=2, Hq=8, seed=8, device="cuda")
+    check_all(L, B=48, k=300, hpp=4, rows_dtype=torch.float32)
+
+
+def test_planes_in_pinned_host_memory_give_identical_scores():
+    L = make_layer(70000, Hkv=2, Hq=8, seed=9, device="cuda")
+    a = run_gpu(L, 48, 64, 4, stages=("scan",))
+    b = run_gpu(L, 48, 64, 4, stages=("scan",), host_planes=True)
+    assert np.array_equal(a["scores"], b["scores"])
+
+
+def test_bf16_keys_build():
+    L = make_layer(1000, Hkv=2, Hq=8, seed=10, device="cuda")
+    from paper_2609_17652_b200 import binding as fb
+    lay = fb.make_layout(2, 8, 1000)
+    ctx = fb.Context(0, 0)
+    planes = torch.zeros((2, 128, 4, lay.plane_stride_words), dtype=torch.int64, device="cuda")
+    scales = torch.zeros((2, 128, lay.scale_stride), dtype=torch.int16, device="cuda")
+    ctx.fathom_build_planes(lay, L.Krows, planes, scales)
+    torch.cuda.synchronize()
+    p_ref, s_ref = O.build_planes(L.Krows.float().cpu().numpy())
+    nb = 16
+    assert np.array_equal(planes[..., :nb].cpu().numpy().view(np.uint64), p_ref)
+    assert np.array_equal(scales[..., :nb].cpu().numpy().view(np.uint16), s_ref.view(np.uint16))
+    ctx.close()
+
+
+def test_argument_validation_returns_codes():
+    from paper_2609_17652_b200 import binding as fb
+    import ctypes as C
+    lay = fb.make_layout(2, 8, 1000)
+    ctx = fb.Context(0, 1024)
+    x = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_topk(lay, x, 100, 0, 0, x)
+    assert e.value.status == -4                                   # scratch too small
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_topk(lay, x, 2000, 0, 0, x)
+    assert e.value.status == -1                                   # k > n
+    bad = fb.make_layout(2, 8, 1000); bad.d = 64
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_scan(bad, x, x, x, x, 4, x)
+    assert e.value.status == -2
+    bad = fb.make_layout(2, 8, 1000); bad.plane_stride_words = 17
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_scan(bad, x, x, x, x, 4, x)
+    assert e.value.status == -3
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_scan(lay, x, x, x, x, 3, x)
+    assert e.value.status == -1
+    with pytest.raises(fb.FathomError) as e:
+        ctx.fathom_scan(lay, 0, x, x, x, 4, x)
+    assert e.value.status == -1
+    ctx.close()
+
+
+def test_determinism_two_runs_same_bytes():
+    L = make_layer(10000, Hkv=2, Hq=8, seed=11, device="cuda")
+    a = run_gpu(L, 48, 256, 4)
+    b = run_gpu(L, 48, 256, 4)
+    for key in ("planes", "depth", "scores", "idx", "out"):
+        assert np.array_equal(a[key], b[key]), key
