@@ -44,9 +44,10 @@ static inline size_t fathom_round_up(size_t x, size_t a) { return (x + a - 1) / 
 
 struct fathom_topk_scratch {
   uint32_t* hist;        // [Hq][FATHOM_TOPK_BINS]
-  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 3 winners written, 4 candidates written
+  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 4 candidates written
+  uint32_t* bitmap;      // [Hq][bitmap_words] selection bitmap, token i at bit (i % 32) of word i / 32
   int32_t* cand;         // [Hq][n] token indices of the threshold bin
-  int32_t* winners;      // [Hq][k] unordered winners
+  long long bitmap_words;
   size_t bytes;
 };
 struct fathom_attn_scratch {

@@ -3,21 +3,25 @@
 // Bucket select on the order-preserving integer image of the fp32 score (-0 folded onto +0):
 //   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores);
 //   2. per head, the threshold bin b* whose suffix count first reaches the number wanted;
-//   3. filter (second read): tokens in bins above b* are winners, tokens in b* are candidates;
-//      both are appended with warp-aggregated atomics (ballot + popc), order irrelevant;
-//   4. per head, an 8-bit radix select over the candidates on the 64-bit composite
-//      (key << 32 | ~index), which makes every element distinct and encodes "ties go to the lower
-//      token index"; the chosen candidates join the winners, the forced sink/local tokens are
-//      added and the k indices are sorted ascending in shared memory (bitonic network).
-// The set is unique, so the arbitrary append order never shows in the output.
+//   3. filter (second read): a lane owns one token, so the warp ballot of "bin above b*" IS the 32-token
+//      word of a selection bitmap, written without atomics; tokens in bin b* itself are candidates,
+//      appended with warp-aggregated atomics (ballot + popc), order irrelevant;
+//   4. per head, a radix select over the candidates on the 64-bit composite (key << 32 | ~index), which
+//      makes every element distinct and encodes "ties go to the lower token index"; the chosen
+//      candidates and the forced sink/local tokens are OR-ed into the bitmap, and the k indices are
+//      emitted in ascending order by a popcount prefix sum over the bitmap words.
+// The selected set is unique, so neither the append order nor atomics can show in the output.
 #include "fathom_common.cuh"
 
 namespace {
 
-constexpr int TK_THREADS = 256;
-constexpr int TK_PER_THREAD = 16;                            // 4 x float4
-constexpr int TK_TILE = TK_THREADS * TK_PER_THREAD;          // 4096 scores per CTA
+constexpr int HIST_THREADS = 256;
+constexpr int HIST_TILE = 32768;                             // scores per CTA of the histogram pass
+constexpr int FILT_THREADS = 256;
+constexpr int FILT_WARP_TOKENS = 1024;                       // 32 ballots -> 32 bitmap words per warp
+constexpr int FILT_TILE = (FILT_THREADS / 32) * FILT_WARP_TOKENS;   // 8192 tokens per CTA
 constexpr int FIN_THREADS = 1024;
+constexpr int FIN_CACHE = 4096;                              // candidate composites kept in shared memory
 
 __device__ __forceinline__ uint32_t ordered_key(float f) {
   uint32_t u = __float_as_uint(f);
@@ -27,37 +31,37 @@ __device__ __forceinline__ uint32_t ordered_key(float f) {
 
 struct Forced { long long sink_end, local_begin; };          // eligible tokens: sink_end <= i < local_begin
 
-__global__ void __launch_bounds__(TK_THREADS)
+__global__ void __launch_bounds__(HIST_THREADS)
 topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                  uint32_t* __restrict__ hist) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   const int head = blockIdx.y;
-  for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += TK_THREADS) sh[b] = 0u;
+  for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  const long long base = (long long)blockIdx.x * TK_TILE;
+  const long long base = (long long)blockIdx.x * HIST_TILE;
+  const long long end = min(base + HIST_TILE, n);
+#pragma unroll 4
+  for (long long i = base + (long long)threadIdx.x * 4; i < end; i += HIST_THREADS * 4) {
+    // score_stride is a multiple of 4, so the float4 stays inside the row even when it straddles n
+    const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
+    const float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-  for (int v = 0; v < TK_PER_THREAD / 4; ++v) {
-    const long long i = base + ((long long)v * TK_THREADS + threadIdx.x) * 4;
-    if (i < n) {                                             // score_stride is a multiple of 4: the float4 stays in the row
-      const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
-      const float e[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const long long t = i + c;
-        if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
-      }
+    for (int c = 0; c < 4; ++c) {
+      const long long t = i + c;
+      if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
     }
   }
   __syncthreads();
   uint32_t* g = hist + (size_t)head * FATHOM_TOPK_BINS;
-  for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += TK_THREADS) {
+  for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) {
     const uint32_t c = sh[b];
     if (c) atomicAdd(&g[b], c);
   }
 }
 
-// state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it
+// state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it,
+// [4] = candidates appended by the filter
 __global__ void __launch_bounds__(FIN_THREADS)
 topk_find_bin_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ state, uint32_t want,
                      uint32_t* __restrict__ dev_status) {
@@ -87,7 +91,7 @@ topk_find_bin_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ s
   }
   __syncthreads();
   const uint32_t above = warp_sum[warp] + incl - local;       // tokens in bins above this thread's four
-  if (want == 0) {
+  if (want == 0) {                                            // nothing to select: no bin is above or equal
     if (tid == 0) { state[head * 8 + 0] = FATHOM_TOPK_BINS; state[head * 8 + 1] = 0; state[head * 8 + 2] = 0; }
     return;
   }
@@ -103,52 +107,43 @@ topk_find_bin_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ s
       run += c[x];
     }
   }
-  if (tid == FIN_THREADS - 1 && above + local < want) {       // fewer eligible tokens than wanted
+  if (tid == FIN_THREADS - 1 && above + local < want) {       // fewer eligible tokens than wanted: take them all
     atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
     state[head * 8 + 0] = 0; state[head * 8 + 1] = above + local - c[3]; state[head * 8 + 2] = c[3];
   }
 }
 
-__global__ void __launch_bounds__(TK_THREADS)
+__global__ void __launch_bounds__(FILT_THREADS)
 topk_filter_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
-                   uint32_t* __restrict__ state, int32_t* __restrict__ cand, int32_t* __restrict__ winners, int k) {
-  const int head = blockIdx.y, lane = threadIdx.x & 31;
+                   uint32_t* __restrict__ state, int32_t* __restrict__ cand, uint32_t* __restrict__ bitmap,
+                   long long bitmap_words) {
+  const int head = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t bstar = state[head * 8 + 0];
   const float* row = scores + (size_t)head * (size_t)score_stride;
   int32_t* cand_h = cand + (size_t)head * (size_t)n;
-  int32_t* win_h = winners + (size_t)head * (size_t)k;
-  const long long base = (long long)blockIdx.x * TK_TILE;
-#pragma unroll
-  for (int v = 0; v < TK_PER_THREAD / 4; ++v) {
-    const long long i = base + ((long long)v * TK_THREADS + threadIdx.x) * 4;
-    float e[4] = {0.f, 0.f, 0.f, 0.f};
-    if (i < n) {
-      const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
-      e[0] = x.x; e[1] = x.y; e[2] = x.z; e[3] = x.w;
-    }
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const long long t = i + c;
-      const bool elig = t < n && t >= F.sink_end && t < F.local_begin;
-      const uint32_t bin = ordered_key(e[c]) >> 20;
-      const bool is_win = elig && bin > bstar;
-      const bool is_cand = elig && bin == bstar;
-      const unsigned mw = __ballot_sync(0xffffffffu, is_win);
-      const unsigned mc = __ballot_sync(0xffffffffu, is_cand);
-      if (mw) {
-        uint32_t pos = 0;
-        if (lane == __ffs(mw) - 1) pos = atomicAdd(&state[head * 8 + 3], (uint32_t)__popc(mw));
-        pos = __shfl_sync(0xffffffffu, pos, __ffs(mw) - 1);
-        if (is_win) win_h[pos + __popc(mw & ((1u << lane) - 1u))] = (int32_t)t;
-      }
-      if (mc) {
-        uint32_t pos = 0;
-        if (lane == __ffs(mc) - 1) pos = atomicAdd(&state[head * 8 + 4], (uint32_t)__popc(mc));
-        pos = __shfl_sync(0xffffffffu, pos, __ffs(mc) - 1);
-        if (is_cand) cand_h[pos + __popc(mc & ((1u << lane) - 1u))] = (int32_t)t;
-      }
+  uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
+  const long long wbase = (long long)blockIdx.x * FILT_TILE + (long long)warp * FILT_WARP_TOKENS;
+  if (wbase >= n) return;
+  uint32_t my_word = 0u;                                      // lane i keeps the ballot of iteration i
+#pragma unroll 8
+  for (int it = 0; it < 32; ++it) {
+    const long long t = wbase + it * 32 + lane;
+    const bool elig = t < n && t >= F.sink_end && t < F.local_begin;
+    const float s = (t < n) ? __ldg(row + t) : 0.0f;
+    const uint32_t bin = ordered_key(s) >> 20;
+    const bool is_cand = elig && bin == bstar;
+    const unsigned mw = __ballot_sync(0xffffffffu, elig && bin > bstar);
+    const unsigned mc = __ballot_sync(0xffffffffu, is_cand);
+    if (lane == it) my_word = mw;
+    if (mc) {
+      uint32_t pos = 0;
+      const int leader = __ffs(mc) - 1;
+      if (lane == leader) pos = atomicAdd(&state[head * 8 + 4], (uint32_t)__popc(mc));
+      pos = __shfl_sync(0xffffffffu, pos, leader);
+      if (is_cand) cand_h[pos + __popc(mc & ((1u << lane) - 1u))] = (int32_t)t;
     }
   }
+  bm[wbase / 32 + lane] = my_word;                            // 32 consecutive words, one coalesced store
 }
 
 // low 52 bits of (key << 32 | ~index); the 12 leading key bits are the same for every candidate
@@ -158,27 +153,30 @@ __device__ __forceinline__ uint64_t composite52(const float* row, int32_t i) {
 
 __global__ void __launch_bounds__(FIN_THREADS)
 topk_finish_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
-                   uint32_t* __restrict__ state, const int32_t* __restrict__ cand, int32_t* __restrict__ winners,
-                   int k, int sort_len, int32_t* __restrict__ idx_out) {
-  extern __shared__ int32_t s_sort[];                         // sort_len entries
+                   const uint32_t* __restrict__ state, const int32_t* __restrict__ cand,
+                   uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
+                   uint32_t* __restrict__ dev_status) {
+  __shared__ uint64_t s_comp[FIN_CACHE];
   __shared__ uint32_t s_hist[256];
-  __shared__ uint64_t s_prefix;                               // chosen leading bits of the threshold composite
-  __shared__ uint32_t s_need, s_digit, s_wpos;
-  const int head = blockIdx.x, tid = threadIdx.x;
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
+  __shared__ uint32_t s_need, s_digit, s_bucket;
+  const int head = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const int32_t* cand_h = cand + (size_t)head * (size_t)n;
-  int32_t* win_h = winners + (size_t)head * (size_t)k;
+  uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
   const uint32_t m = state[head * 8 + 4];
-  const uint32_t c_hi = state[head * 8 + 1];
-  const uint32_t need0 = state[head * 8 + 2];
+  const uint32_t need0 = min(state[head * 8 + 2], m);
+  const bool cached = m <= FIN_CACHE;
+  if (cached)
+    for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite52(row, cand_h[c]);
 
-  // ---- radix select of the need0 largest composites among the m candidates.  The 12 leading key bits are
-  //      equal for all of them; digits of 8 bits are taken from bit 52 downwards (the first covers 4 bits).
-  uint64_t thr = 0;                                           // winners are candidates with composite >= thr
+  // ---- radix select of the need0 largest composites among the m candidates; digits are taken from bit 52
+  //      downwards (4 bits first, then 8 at a time) until the chosen bucket is taken whole.
+  uint64_t thr = 0;                                           // chosen candidates: composite >= thr
   if (need0 > 0 && need0 < m) {
     if (tid == 0) { s_prefix = 0; s_need = need0; }
-    __syncthreads();
-    int hi = 52;                                              // bits [hi, 64) are decided
+    int hi = 52;
     while (hi > 0) {
       const int bits = (hi % 8) ? (hi % 8) : 8;
       const int lo = hi - bits;
@@ -186,9 +184,8 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
       __syncthreads();
       const uint64_t prefix = s_prefix;
       for (uint32_t c = tid; c < m; c += FIN_THREADS) {
-        const uint64_t comp = composite52(row, cand_h[c]);
-        const bool match = (comp >> hi) == (prefix >> hi);
-        if (match) atomicAdd(&s_hist[(uint32_t)(comp >> lo) & ((1u << bits) - 1u)], 1u);
+        const uint64_t comp = cached ? s_comp[c] : composite52(row, cand_h[c]);
+        if ((comp >> hi) == (prefix >> hi)) atomicAdd(&s_hist[(uint32_t)(comp >> lo) & ((1u << bits) - 1u)], 1u);
       }
       __syncthreads();
       if (tid < 32) {                                         // warp 0: suffix counts over the 256 digits
@@ -206,62 +203,78 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
         if (run < need && run + local >= need) {
 #pragma unroll
           for (int x = 0; x < 8; ++x) {
-            if (run < need && run + cnt[x] >= need) { s_digit = 255 - (8 * tid + x); s_wpos = need - run; }
+            if (run < need && run + cnt[x] >= need) {
+              s_digit = 255 - (8 * tid + x);
+              s_need = need - run;                            // still needed from inside the chosen digit
+              s_bucket = cnt[x];
+            }
             run += cnt[x];
           }
         }
       }
       __syncthreads();
-      if (tid == 0) {
-        s_prefix |= (uint64_t)s_digit << lo;
-        s_need = s_wpos;                                      // still needed from inside the chosen digit
-      }
+      if (tid == 0) s_prefix |= (uint64_t)s_digit << lo;
+      const bool whole = s_need == s_bucket;                  // the chosen bucket is taken entirely: done
       __syncthreads();
       hi = lo;
+      if (whole) break;
     }
-    // composites are distinct, so exactly one candidate equals the decided low 52 bits: it is the threshold
-    thr = s_prefix;
+    thr = s_prefix;                                           // undecided low bits are zero
   }
-  if (tid == 0) s_wpos = 0;
-  __syncthreads();
   if (need0 > 0) {
     for (uint32_t c = tid; c < m; c += FIN_THREADS) {
       const int32_t i = cand_h[c];
-      const bool take = (need0 >= m) || (composite52(row, i) >= thr);
-      if (take) {
-        const uint32_t pos = atomicAdd(&s_wpos, 1u);
-        if (c_hi + pos < (uint32_t)k) win_h[c_hi + pos] = i;
-      }
+      const uint64_t comp = cached ? s_comp[c] : composite52(row, i);
+      if (need0 >= m || comp >= thr) atomicOr(&bm[i >> 5], 1u << (i & 31));
     }
+  }
+  // ---- forced sink / local tokens
+  const long long n_forced = F.sink_end + (n - F.local_begin);
+  for (long long e = tid; e < n_forced; e += FIN_THREADS) {
+    const long long i = (e < F.sink_end) ? e : (F.local_begin + (e - F.sink_end));
+    atomicOr(&bm[i >> 5], 1u << (i & 31));
   }
   __syncthreads();
 
-  // ---- gather forced tokens + winners, sort ascending, write
-  const int n_sink = (int)F.sink_end;
-  const int n_loc = (int)(n - F.local_begin);
-  const int n_forced = n_sink + n_loc;
-  const int n_win = min((int)(c_hi + s_wpos), k - n_forced);
-  for (int e = tid; e < sort_len; e += FIN_THREADS) {
-    int32_t v = 0x7fffffff;
-    if (e < n_sink) v = e;
-    else if (e < n_forced) v = (int32_t)(F.local_begin + (e - n_sink));
-    else if (e < n_forced + n_win) v = win_h[e - n_forced];
-    s_sort[e] = v;
+  // ---- ascending emission: thread t owns a contiguous run of bitmap words
+  const long long words = (n + 31) / 32;
+  const long long per = (words + FIN_THREADS - 1) / FIN_THREADS;
+  const long long w0 = min((long long)tid * per, words), w1 = min(w0 + per, words);
+  uint32_t cnt = 0;
+  for (long long w = w0; w < w1; ++w) cnt += __popc(bm[w]);
+  uint32_t incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t w = s_warp[lane];
+    uint32_t wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    s_warp[lane] = wi - w;
+    if (lane == 31 && wi != (uint32_t)k) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
   }
   __syncthreads();
-  for (int size = 2; size <= sort_len; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int e = tid; e < sort_len / 2; e += FIN_THREADS) {
-        const int lo_i = 2 * e - (e & (stride - 1));
-        const int hi_i = lo_i + stride;
-        const bool up = (lo_i & size) == 0;
-        const int32_t a = s_sort[lo_i], b = s_sort[hi_i];
-        if ((a > b) == up) { s_sort[lo_i] = b; s_sort[hi_i] = a; }
-      }
-      __syncthreads();
+  uint32_t pos = s_warp[warp] + incl - cnt;
+  int32_t* out = idx_out + (size_t)head * k;
+  for (long long w = w0; w < w1; ++w) {
+    uint32_t bitsw = bm[w];
+    while (bitsw) {
+      const int b = __ffs(bitsw) - 1;
+      if (pos < (uint32_t)k) out[pos] = (int32_t)(w * 32 + b);
+      ++pos;
+      bitsw &= bitsw - 1;
     }
   }
-  for (int e = tid; e < k; e += FIN_THREADS) idx_out[(size_t)head * k + e] = s_sort[e];
+  if (tid == FIN_THREADS - 1)                                 // short selection (non-finite scores): pad with the last token
+    for (uint32_t e = pos; e < (uint32_t)k; ++e) out[e] = (int32_t)(n - 1);
 }
 
 }  // namespace
@@ -286,18 +299,15 @@ extern "C" int fathom_topk(fathom_ctx* ctx, const fathom_layout* L, const float*
   const uint32_t want = (uint32_t)(k - n_forced);
 
   // histograms and per-head state are contiguous at the start of the arena
-  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.cand - (char*)S.hist, st));
-  dim3 grid((unsigned)((n + TK_TILE - 1) / TK_TILE), (unsigned)Hq);
-  topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.hist);
+  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
+  dim3 hgrid((unsigned)((n + HIST_TILE - 1) / HIST_TILE), (unsigned)Hq);
+  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.hist);
   topk_find_bin_kernel<<<Hq, FIN_THREADS, 0, st>>>(S.hist, S.state, want, ctx->dev_status);
-  topk_filter_kernel<<<grid, TK_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.winners, k);
-  int sort_len = 2;
-  while (sort_len < k) sort_len <<= 1;
-  const size_t smem = (size_t)sort_len * sizeof(int32_t);
-  if (smem > 48 * 1024)
-    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  topk_finish_kernel<<<Hq, FIN_THREADS, smem, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.winners, k,
-                                                    sort_len, idx);
+  dim3 fgrid((unsigned)((n + FILT_TILE - 1) / FILT_TILE), (unsigned)Hq);
+  topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
+                                                     S.bitmap_words);
+  topk_finish_kernel<<<Hq, FIN_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
+                                                 S.bitmap_words, k, idx, ctx->dev_status);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
