@@ -1,124 +1,71 @@
 // fathom_build_planes: K -> channel-major bit planes + fp16 block scales (Sec. 3.2, Eq. 2).
 //
-// A 64-token block of one KV head is 64 x 128 contiguous values (32 KB in fp32), so it is fetched with
-// one bulk asynchronous copy (cp.async.bulk, global -> shared, completion on an mbarrier) into a
-// STAGES-deep ring; persistent CTAs walk contiguous runs of blocks so that loads for the next blocks
-// are in flight while the current one is quantised.  One thread owns one channel: it pulls its column
-// out of shared memory (bank = channel mod 32, conflict-free), takes the block maximum, rounds a/8 to
-// fp16 and derives the four plane bits of every code by comparing k with exact multiples of the
-// stored scale, most significant bit first:
+// Two threads own one channel of a 64-token block (32 tokens each): the 128 threads of a token half read
+// every token row as 512 contiguous bytes, keep their 32 values in registers, exchange the two half maxima
+// through shared memory, round a/8 to fp16 and derive the four plane bits of every code by comparing k
+// with exact multiples of the stored scale, most significant bit first:
 //     bit0 = k >= 0;  bit1 = k >= (bit0 ? 4 : -4) s;  bit2 = k >= thr1 + (bit1 ? 2 : -2) s;  ...
 // m * s (|m| <= 7, s an fp16 value) is exact in fp32, so the four comparisons give exactly
-// clip(floor(k / s), -8, 7) + 8 with no division.  Consecutive blocks of a CTA write consecutive
-// 8-byte words of each (channel, plane) row, which merge into full sectors in L2.
+// clip(floor(k / s), -8, 7) + 8 with no division.  A CTA walks BLOCKS_PER_CTA consecutive blocks and
+// collects their plane words and scales in shared memory, then writes every (channel, plane) row segment
+// as whole 32-byte sectors (partial-sector writes cost a fill read each).
 #include "fathom_common.cuh"
 
 namespace {
 
-constexpr int STAGES = 3;
-constexpr uint32_t WAIT_LIMIT = 1u << 24;                     // bounded spin on the load barrier
+constexpr int BP_THREADS = 2 * FATHOM_D;
+constexpr int BLOCKS_PER_CTA = 8;
+constexpr int HALF = FATHOM_BLOCK / 2;                         // tokens per thread
+constexpr int OUT_PITCH = FATHOM_NPLANES * BLOCKS_PER_CTA * 2 + 1;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Returns false when the wait gave up (the caller records it and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
-__device__ __forceinline__ float to_f32(float x) { return x; }
-__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float load_k(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load_k(const __nv_bfloat16* p) { return __bfloat162float(__ldg(p)); }
 
 template <typename T>
-__global__ void __launch_bounds__(FATHOM_D, 2)
-build_planes_kernel(const T* __restrict__ K, uint64_t* __restrict__ planes, uint16_t* __restrict__ scales,
-                    long long n, long long nb, long long plane_stride, long long scale_stride,
-                    long long total_blocks, long long chunk, uint32_t* __restrict__ dev_status) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t full[STAGES];
-  T* tiles = reinterpret_cast<T*>(smem_raw);                   // [STAGES][64][128]
-  constexpr uint32_t ROW_BYTES = FATHOM_D * sizeof(T);
-  constexpr int TILE_ELEMS = FATHOM_BLOCK * FATHOM_D;
+__global__ void __launch_bounds__(BP_THREADS)
+build_planes_kernel(const T* __restrict__ K, uint32_t* __restrict__ planes32, uint16_t* __restrict__ scales,
+                    long long n, long long nb, long long plane_stride, long long scale_stride) {
+  __shared__ float s_amax[2][2][FATHOM_D];                     // [parity of block][token half][channel]
+  __shared__ uint32_t s_out[FATHOM_D][OUT_PITCH];              // [channel][plane][block][half], padded against bank conflicts
+  __shared__ uint16_t s_scale[FATHOM_D][BLOCKS_PER_CTA];
+  const int j = threadIdx.x & (FATHOM_D - 1);                  // channel
+  const int half = threadIdx.x >> 7;                           // 0: tokens 0..31 of the block, 1: tokens 32..63
+  const int h = blockIdx.y;                                    // KV head
+  const long long b0 = (long long)blockIdx.x * BLOCKS_PER_CTA;
+  const T* Kh = K + (size_t)h * (size_t)n * FATHOM_D;
 
-  const int j = threadIdx.x;                                   // channel
-  const long long first = (long long)blockIdx.x * chunk;
-  const long long count = min(chunk, total_blocks - first);
-  if (count <= 0) return;
+  for (int bb = 0; bb < BLOCKS_PER_CTA; ++bb) {
+    const long long b = b0 + bb;
+    if (b >= nb) break;                                        // uniform over the CTA
+    const long long i0 = b * FATHOM_BLOCK + half * HALF;
+    const int valid = (int)min((long long)HALF, n - i0);       // of this thread's 32 tokens (may be <= 0)
 
-  if (j == 0) {
-    for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-
-  auto issue = [&](long long s) {                              // thread 0 only
-    const long long gb = first + s;
-    const long long h = gb / nb, b = gb % nb;
-    const uint32_t valid = (uint32_t)min((long long)FATHOM_BLOCK, n - b * FATHOM_BLOCK);
-    const int st = (int)(s % STAGES);
-    mbar_expect_tx(&full[st], valid * ROW_BYTES);
-    bulk_load(tiles + (size_t)st * TILE_ELEMS, K + ((size_t)h * (size_t)n + (size_t)b * FATHOM_BLOCK) * FATHOM_D,
-              valid * ROW_BYTES, &full[st]);
-  };
-  if (j == 0)
-    for (long long s = 0; s < min((long long)STAGES, count); ++s) issue(s);
-
-  for (long long s = 0; s < count; ++s) {
-    const long long gb = first + s;
-    const long long h = gb / nb, b = gb % nb;
-    const int valid = (int)min((long long)FATHOM_BLOCK, n - b * FATHOM_BLOCK);
-    const int st = (int)(s % STAGES);
-    if (!mbar_wait_bounded(&full[st], (uint32_t)((s / STAGES) & 1))) {
-      if (j == 0) atomicOr(dev_status, FATHOM_DEV_WAIT_EXPIRED);
-      // give the copies still in flight a bounded chance to land before this CTA's shared memory is released
-      for (int q = 0; q < STAGES; ++q) mbar_wait_bounded(&full[q], (uint32_t)(((s + q) / STAGES) & 1));
-      return;
-    }
-    const T* tile = tiles + (size_t)st * TILE_ELEMS;
-    float v[FATHOM_BLOCK];
+    float v[HALF];
+    if (valid >= HALF) {
 #pragma unroll
-    for (int i = 0; i < FATHOM_BLOCK; ++i) v[i] = to_f32(tile[i * FATHOM_D + j]);
-    __syncthreads();                                           // every thread has its column: the stage is free
-    if (j == 0 && s + STAGES < count) issue(s + STAGES);
-    if (valid < FATHOM_BLOCK) {
+      for (int i = 0; i < HALF; ++i) v[i] = load_k(Kh + (size_t)(i0 + i) * FATHOM_D + j);
+    } else {
 #pragma unroll
-      for (int i = 0; i < FATHOM_BLOCK; ++i) v[i] = (i < valid) ? v[i] : 0.0f;
+      for (int i = 0; i < HALF; ++i) v[i] = (i < valid) ? load_k(Kh + (size_t)(i0 + i) * FATHOM_D + j) : 0.0f;
     }
-
     float a = 0.0f;
 #pragma unroll
-    for (int i = 0; i < FATHOM_BLOCK; ++i) a = fmaxf(a, fabsf(v[i]));
+    for (int i = 0; i < HALF; ++i) a = fmaxf(a, fabsf(v[i]));
+    s_amax[bb & 1][half][j] = a;
+    __syncthreads();
+    a = fmaxf(a, s_amax[bb & 1][half ^ 1][j]);
+
     const __half sh = __float2half_rn(a * 0.125f);             // a/8 is exact; one rounding to fp16
     const float sc = __half2float(sh);
     const float s2 = sc * 2.0f, s4 = sc * 4.0f;
 
-    uint32_t w[FATHOM_NPLANES][2] = {{0u, 0u}, {0u, 0u}, {0u, 0u}, {0u, 0u}};
-    const uint64_t keep = ~0ull >> (64 - valid);               // absent tail tokens carry 0 bits
+    uint32_t w[FATHOM_NPLANES] = {0u, 0u, 0u, 0u};
+    const uint32_t keep = (valid >= HALF) ? ~0u : (valid <= 0 ? 0u : (~0u >> (32 - valid)));   // absent tail tokens carry 0 bits
     if (sc > 0.0f) {
 #pragma unroll
-      for (int i = 0; i < FATHOM_BLOCK; ++i) {
+      for (int i = 0; i < HALF; ++i) {
         const float k = v[i];
-        const uint32_t m = 1u << (i & 31);
+        const uint32_t m = 1u << i;
         const bool c0 = k >= 0.0f;
         float thr = c0 ? s4 : -s4;
         const bool c1 = k >= thr;
@@ -126,25 +73,47 @@ build_planes_kernel(const T* __restrict__ K, uint64_t* __restrict__ planes, uint
         const bool c2 = k >= thr;
         thr += c2 ? sc : -sc;
         const bool c3 = k >= thr;
-        if (c0) w[0][i >> 5] |= m;
-        if (c1) w[1][i >> 5] |= m;
-        if (c2) w[2][i >> 5] |= m;
-        if (c3) w[3][i >> 5] |= m;
+        if (c0) w[0] |= m;
+        if (c1) w[1] |= m;
+        if (c2) w[2] |= m;
+        if (c3) w[3] |= m;
       }
 #pragma unroll
-      for (int p = 0; p < FATHOM_NPLANES; ++p) {
-        w[p][0] &= (uint32_t)keep;
-        w[p][1] &= (uint32_t)(keep >> 32);
-      }
+      for (int p = 0; p < FATHOM_NPLANES; ++p) w[p] &= keep;
     } else {                                                   // zero scale: every code is 8 = 0b1000
-      w[0][0] = (uint32_t)keep;
-      w[0][1] = (uint32_t)(keep >> 32);
+      w[0] = keep;
     }
-    uint64_t* prow = planes + (((size_t)h * FATHOM_D + j) * FATHOM_NPLANES) * (size_t)plane_stride + b;
+    // little-endian halves of the 64-bit plane word: tokens 0..31 in the low 32 bits
 #pragma unroll
-    for (int p = 0; p < FATHOM_NPLANES; ++p)
-      prow[(size_t)p * plane_stride] = ((uint64_t)w[p][1] << 32) | w[p][0];
-    scales[((size_t)h * FATHOM_D + j) * (size_t)scale_stride + b] = __half_as_ushort(sh);
+    for (int p = 0; p < FATHOM_NPLANES; ++p) s_out[j][(p * BLOCKS_PER_CTA + bb) * 2 + half] = w[p];
+    if (half == 0) s_scale[j][bb] = __half_as_ushort(sh);
+  }
+  __syncthreads();
+
+  // ---- flush: each (channel, plane) row segment is BLOCKS_PER_CTA words = 64 contiguous bytes
+  const int nblk = (int)min((long long)BLOCKS_PER_CTA, nb - b0);
+  uint64_t* planes64 = reinterpret_cast<uint64_t*>(planes32);
+  for (int e = threadIdx.x; e < FATHOM_D * FATHOM_NPLANES * (BLOCKS_PER_CTA / 2); e += BP_THREADS) {
+    const int pair = e % (BLOCKS_PER_CTA / 2);                 // two words = one 16-byte store
+    const int p = (e / (BLOCKS_PER_CTA / 2)) % FATHOM_NPLANES;
+    const int c = e / (BLOCKS_PER_CTA / 2 * FATHOM_NPLANES);
+    const uint32_t* src = &s_out[c][(p * BLOCKS_PER_CTA + 2 * pair) * 2];
+    uint64_t* dst = planes64 + (((size_t)h * FATHOM_D + c) * FATHOM_NPLANES + p) * (size_t)plane_stride + b0 + 2 * pair;
+    if (2 * pair + 1 < nblk) {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(src[0], src[1], src[2], src[3]);
+    } else if (2 * pair < nblk) {
+      dst[0] = ((uint64_t)src[1] << 32) | src[0];
+    }
+  }
+  for (int e = threadIdx.x; e < FATHOM_D; e += BP_THREADS) {
+    uint16_t* dst = scales + ((size_t)h * FATHOM_D + e) * (size_t)scale_stride + b0;
+    if (nblk == BLOCKS_PER_CTA) {
+      const uint16_t* sp = s_scale[e];
+      *reinterpret_cast<uint4*>(dst) = make_uint4(sp[0] | ((uint32_t)sp[1] << 16), sp[2] | ((uint32_t)sp[3] << 16),
+                                                  sp[4] | ((uint32_t)sp[5] << 16), sp[6] | ((uint32_t)sp[7] << 16));
+    } else {
+      for (int x = 0; x < nblk; ++x) dst[x] = s_scale[e][x];
+    }
   }
 }
 
@@ -152,17 +121,9 @@ template <typename T>
 int launch_build(fathom_ctx* ctx, const fathom_layout* L, const T* K, uint64_t* planes, uint16_t* scales,
                  cudaStream_t st) {
   const long long nb = fathom_nblocks(L->n);
-  const long long total = nb * L->n_kv_heads;
-  int sms = 148;
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
-  const long long max_ctas = 2LL * sms;                        // two resident CTAs per SM, persistent
-  long long chunk = (total + max_ctas - 1) / max_ctas;
-  chunk = (chunk + 7) / 8 * 8;                                 // runs of >= 8 blocks: 64-byte write segments per row
-  const long long ctas = (total + chunk - 1) / chunk;
-  const size_t smem = (size_t)STAGES * FATHOM_BLOCK * FATHOM_D * sizeof(T);
-  FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(build_planes_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  build_planes_kernel<T><<<(unsigned)ctas, FATHOM_D, smem, st>>>(K, planes, scales, L->n, nb, L->plane_stride_words,
-                                                                L->scale_stride, total, chunk, ctx->dev_status);
+  dim3 grid((unsigned)((nb + BLOCKS_PER_CTA - 1) / BLOCKS_PER_CTA), (unsigned)L->n_kv_heads);
+  build_planes_kernel<T><<<grid, BP_THREADS, 0, st>>>(K, reinterpret_cast<uint32_t*>(planes), scales, L->n, nb,
+                                                      L->plane_stride_words, L->scale_stride);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
