@@ -3,9 +3,10 @@
 // Bucket select on the order-preserving integer image of the fp32 score (-0 folded onto +0):
 //   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores);
 //   2. per head, the threshold bin b* whose suffix count first reaches the number wanted;
-//   3. filter (second read): a lane owns one token, so the warp ballot of "bin above b*" IS the 32-token
-//      word of a selection bitmap, written without atomics; tokens in bin b* itself are candidates,
-//      appended with warp-aggregated atomics (ballot + popc), order irrelevant;
+//   3. filter (second read): a lane owns four consecutive tokens (one 16-byte load) and compares them with
+//      the two fp32 edges of bin b*; the warp ballots of "above b*" ARE the words of a selection bitmap
+//      (word c of a 128-token group holds tokens 4 l + c at bit l), written without atomics; tokens inside
+//      bin b* are candidates, appended with warp-aggregated atomics (ballot + popc), order irrelevant;
 //   4. per head, a radix select over the candidates on the 64-bit composite (key << 32 | ~index), which
 //      makes every element distinct and encodes "ties go to the lower token index"; the chosen
 //      candidates and the forced sink/local tokens are OR-ed into the bitmap, and the k indices are
@@ -41,15 +42,26 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const long long base = (long long)blockIdx.x * HIST_TILE;
   const long long end = min(base + HIST_TILE, n);
-#pragma unroll 4
-  for (long long i = base + (long long)threadIdx.x * 4; i < end; i += HIST_THREADS * 4) {
-    // score_stride is a multiple of 4, so the float4 stays inside the row even when it straddles n
-    const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
-    const float e[4] = {x.x, x.y, x.z, x.w};
+  // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
+  if (base >= F.sink_end && base + HIST_TILE <= F.local_begin) {        // whole tile eligible: no per-token test
+    const float4* r4 = reinterpret_cast<const float4*>(row + base);
+#pragma unroll 8
+    for (int v = threadIdx.x; v < HIST_TILE / 4; v += HIST_THREADS) {
+      const float4 x = __ldg(r4 + v);
+      atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
+      atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
+      atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
+      atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
+    }
+  } else {
+    for (long long i = base + (long long)threadIdx.x * 4; i < end; i += HIST_THREADS * 4) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
+      const float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const long long t = i + c;
-      if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
+      for (int c = 0; c < 4; ++c) {
+        const long long t = i + c;
+        if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
+      }
     }
   }
   __syncthreads();
@@ -113,37 +125,93 @@ topk_find_bin_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ s
   }
 }
 
+// fp32 value whose ordered key is `key` (the inverse of ordered_key for non-NaN patterns)
+__device__ __forceinline__ float key_to_float(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// Bitmap layout: word (t / 128) * 4 + (t % 4), bit (t % 128) / 4.
+__device__ __forceinline__ long long bitmap_word(long long t) { return (t >> 7) * 4 + (t & 3); }
+__device__ __forceinline__ uint32_t bitmap_bit(long long t) { return 1u << ((t & 127) >> 2); }
+
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_filter_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    uint32_t* __restrict__ state, int32_t* __restrict__ cand, uint32_t* __restrict__ bitmap,
                    long long bitmap_words) {
+  __shared__ uint16_t s_list[FILT_TILE];                      // candidates of this tile, as offsets from its first token
+  __shared__ uint32_t s_count, s_base;
   const int head = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_count = 0u;
+  __syncthreads();
   const uint32_t bstar = state[head * 8 + 0];
+  // bin b* is [lo, hi) in fp32 order; for finite scores "key >> 20 > b*" <=> s >= hi and "== b*" <=> lo <= s < hi.
+  // A bin edge that is not a number (beyond +-inf) compares false with everything, which is what is wanted.
+  const float lo = (bstar < FATHOM_TOPK_BINS) ? key_to_float(bstar << 20) : __uint_as_float(0x7fc00000u);
+  const float hi = (bstar + 1 < FATHOM_TOPK_BINS) ? key_to_float((bstar + 1) << 20) : __uint_as_float(0x7fc00000u);
+  const bool hi_open = !(hi == hi);                           // no bin above b*: every s >= lo is a candidate
   const float* row = scores + (size_t)head * (size_t)score_stride;
   int32_t* cand_h = cand + (size_t)head * (size_t)n;
   uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
-  const long long wbase = (long long)blockIdx.x * FILT_TILE + (long long)warp * FILT_WARP_TOKENS;
-  if (wbase >= n) return;
-  uint32_t my_word = 0u;                                      // lane i keeps the ballot of iteration i
-#pragma unroll 8
-  for (int it = 0; it < 32; ++it) {
-    const long long t = wbase + it * 32 + lane;
-    const bool elig = t < n && t >= F.sink_end && t < F.local_begin;
-    const float s = (t < n) ? __ldg(row + t) : 0.0f;
-    const uint32_t bin = ordered_key(s) >> 20;
-    const bool is_cand = elig && bin == bstar;
-    const unsigned mw = __ballot_sync(0xffffffffu, elig && bin > bstar);
-    const unsigned mc = __ballot_sync(0xffffffffu, is_cand);
-    if (lane == it) my_word = mw;
-    if (mc) {
-      uint32_t pos = 0;
-      const int leader = __ffs(mc) - 1;
-      if (lane == leader) pos = atomicAdd(&state[head * 8 + 4], (uint32_t)__popc(mc));
-      pos = __shfl_sync(0xffffffffu, pos, leader);
-      if (is_cand) cand_h[pos + __popc(mc & ((1u << lane) - 1u))] = (int32_t)t;
+  const long long tile0 = (long long)blockIdx.x * FILT_TILE;
+  const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
+  const bool all_elig = wbase >= F.sink_end && wbase + FILT_WARP_TOKENS <= F.local_begin && wbase + FILT_WARP_TOKENS <= n;
+  float4 x[FILT_WARP_TOKENS / 128];
+#pragma unroll
+  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+    const long long t0 = wbase + it * 128 + lane * 4;
+    x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  uint32_t my_word = 0u;                                      // lane w keeps word w of the warp's 32 bitmap words
+  if (all_elig) {
+#pragma unroll
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+      const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+      const float mx = fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3]));
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const unsigned mw = __ballot_sync(0xffffffffu, e[c] >= hi);
+        if (lane == it * 4 + c) my_word = mw;
+      }
+      // candidates are rare (a few per thousand tokens): append them one by one to the tile's list
+      if (mx >= lo) {                                          // divergent on purpose: only lanes that hold one
+        const long long t0 = wbase + it * 128 + lane * 4;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (e[c] >= lo && (hi_open || e[c] < hi)) s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(t0 + c - tile0);
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+      const long long t0 = wbase + it * 128 + lane * 4;
+      const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const long long t = t0 + c;
+        const bool elig = t < n && t >= F.sink_end && t < F.local_begin;
+        const bool is_cand = elig && e[c] >= lo && (hi_open || e[c] < hi);
+        const unsigned mw = __ballot_sync(0xffffffffu, elig && e[c] >= hi);
+        const unsigned mc = __ballot_sync(0xffffffffu, is_cand);
+        if (lane == it * 4 + c) my_word = mw;
+        if (mc) {
+          uint32_t pos = 0;
+          const int leader = __ffs(mc) - 1;
+          if (lane == leader) pos = atomicAdd(&s_count, (uint32_t)__popc(mc));
+          pos = __shfl_sync(0xffffffffu, pos, leader);
+          if (is_cand) s_list[pos + __popc(mc & ((1u << lane) - 1u))] = (uint16_t)(t - tile0);
+        }
+      }
     }
   }
-  bm[wbase / 32 + lane] = my_word;                            // 32 consecutive words, one coalesced store
+  if (wbase < n) bm[wbase / 32 + lane] = my_word;             // 32 consecutive words, one coalesced store
+  // one global atomic per tile reserves the slice of the head's candidate list
+  __syncthreads();
+  const uint32_t cnt = s_count;
+  if (cnt == 0u) return;
+  if (threadIdx.x == 0) s_base = atomicAdd(&state[head * 8 + 4], cnt);
+  __syncthreads();
+  const uint32_t base = s_base;
+  for (uint32_t e = threadIdx.x; e < cnt; e += FILT_THREADS) cand_h[base + e] = (int32_t)(tile0 + s_list[e]);
 }
 
 // low 52 bits of (key << 32 | ~index); the 12 leading key bits are the same for every candidate
@@ -225,23 +293,34 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
     for (uint32_t c = tid; c < m; c += FIN_THREADS) {
       const int32_t i = cand_h[c];
       const uint64_t comp = cached ? s_comp[c] : composite52(row, i);
-      if (need0 >= m || comp >= thr) atomicOr(&bm[i >> 5], 1u << (i & 31));
+      if (need0 >= m || comp >= thr) atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
     }
   }
   // ---- forced sink / local tokens
   const long long n_forced = F.sink_end + (n - F.local_begin);
   for (long long e = tid; e < n_forced; e += FIN_THREADS) {
     const long long i = (e < F.sink_end) ? e : (F.local_begin + (e - F.sink_end));
-    atomicOr(&bm[i >> 5], 1u << (i & 31));
+    atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
   }
   __syncthreads();
 
-  // ---- ascending emission: thread t owns a contiguous run of bitmap words
-  const long long words = (n + 31) / 32;
-  const long long per = (words + FIN_THREADS - 1) / FIN_THREADS;
-  const long long w0 = min((long long)tid * per, words), w1 = min(w0 + per, words);
+  // ---- ascending emission: thread t owns a contiguous run of 128-token groups (4 bitmap words each)
+  const long long groups = (n + 127) / 128;
+  const long long per = (groups + FIN_THREADS - 1) / FIN_THREADS;
+  const long long g0 = min((long long)tid * per, groups), g1 = min(g0 + per, groups);
+  const uint4* bm4 = reinterpret_cast<const uint4*>(bm);
+  constexpr int REG_GROUPS = 8;                               // groups kept in registers between count and emit
+  uint4 keep[REG_GROUPS];
   uint32_t cnt = 0;
-  for (long long w = w0; w < w1; ++w) cnt += __popc(bm[w]);
+#pragma unroll
+  for (int x = 0; x < REG_GROUPS; ++x) {
+    keep[x] = (g0 + x < g1) ? bm4[g0 + x] : make_uint4(0u, 0u, 0u, 0u);
+    cnt += __popc(keep[x].x) + __popc(keep[x].y) + __popc(keep[x].z) + __popc(keep[x].w);
+  }
+  for (long long g = g0 + REG_GROUPS; g < g1; ++g) {
+    const uint4 w = bm4[g];
+    cnt += __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
+  }
   uint32_t incl = cnt;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -264,15 +343,22 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
   __syncthreads();
   uint32_t pos = s_warp[warp] + incl - cnt;
   int32_t* out = idx_out + (size_t)head * k;
-  for (long long w = w0; w < w1; ++w) {
-    uint32_t bitsw = bm[w];
-    while (bitsw) {
-      const int b = __ffs(bitsw) - 1;
-      if (pos < (uint32_t)k) out[pos] = (int32_t)(w * 32 + b);
-      ++pos;
-      bitsw &= bitsw - 1;
+  auto emit_group = [&](long long g, const uint4 w) {
+    uint32_t any = w.x | w.y | w.z | w.w;
+    while (any) {
+      const int l = __ffs(any) - 1;
+      any &= any - 1;
+      const int32_t t = (int32_t)(g * 128 + 4 * l);
+      if ((w.x >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t; ++pos; }
+      if ((w.y >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 1; ++pos; }
+      if ((w.z >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 2; ++pos; }
+      if ((w.w >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 3; ++pos; }
     }
-  }
+  };
+#pragma unroll
+  for (int x = 0; x < REG_GROUPS; ++x)
+    if (g0 + x < g1) emit_group(g0 + x, keep[x]);
+  for (long long g = g0 + REG_GROUPS; g < g1; ++g) emit_group(g, bm4[g]);
   if (tid == FIN_THREADS - 1)                                 // short selection (non-finite scores): pad with the last token
     for (uint32_t e = pos; e < (uint32_t)k; ++e) out[e] = (int32_t)(n - 1);
 }
