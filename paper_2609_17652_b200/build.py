@@ -31,6 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    cmd += os.environ.get("FATHOM_NVCC_FLAGS", "").split()        # extra flags, e.g. "-DNDEBUG"
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]

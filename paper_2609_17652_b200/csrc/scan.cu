@@ -2,161 +2,274 @@
 //
 // A t-plane read of channel j dequantises to  a * sum_{p<t} (2 b_p - 1) 2^-(p+1)  with a = 8 s the
 // block range, so a score is a signed sum of per-(block, channel, plane) weights
-//     w[beta][j][p][h] = q_hj * a_{beta,j} * 2^-(p+1),      score = 2 * sum_{b_p = 1} w  -  sum w.
-// A CTA owns one plan (NH query heads sharing the planes that are read) and a tile of TILE_BLOCKS
-// 64-token blocks.  The active (channel, plane) rows of the plan are processed in chunks: the
-// chunk's plane words for the tile are staged in shared memory with 16-byte loads (every row is one
-// contiguous run, Sec. 3.5), the weights 2w and the bias -sum w are computed once per (block, row)
-// from the fp16 scales, and then each lane owns tokens l and l + 32 of a block and adds 2w for every
-// set bit.  Only planes p < t_j and scales of active channels are touched.
+//     w[beta][j][p][h] = q_hj * a_{beta,j} * 2^-(p+1),      score_i = sum_rows (b_i ? +w : -w).
+// One add per (token, row, head) makes the scan arithmetic-bound (Sec. 6 "Arithmetic per byte"), so the
+// kernel trades adds for table lookups: the active (channel, plane) rows of a plan are taken four at a
+// time, and for every (64-token block, group of four rows) the 16 possible signed sums are tabulated once
+// (15 adds per head) and then looked up per token with the token's four plane bits as the index.
+//
+// A CTA owns one plan (NH query heads that share the planes read) and 16 blocks (1024 tokens).  Up to 48
+// rows at a time it stages, with 16-byte loads, the rows' plane words (128 contiguous bytes per row: every
+// row is one contiguous run, Sec. 3.5) and fp16 scales (32 bytes per row) in shared memory; all these loads
+// are issued before anything waits, which is what a store in pinned host memory needs to run at link rate.
+// Then each of the four warps owns four consecutive blocks (256 tokens) and runs on its own (only
+// __syncwarp), walking the staged rows in chunks of four groups.  Per chunk a warp builds its
+//   tables     lane (group, head pair, block) takes the four staged scales, forms the weights and writes the
+//              16-entry table (8 bytes per entry = two heads); tables are 136 bytes apart so that the 32 lanes
+//              store to distinct banks;
+//   indices    lane (group, block, half) turns four 32-token row words into 32 four-bit indices with a
+//              4 x 4 bit-block transpose across the four registers (20 logic operations);
+// and then looks up: lane l owns tokens l and l + 32 of a block: one 8-byte load of the packed indices, then per
+//              head pair one 8-byte table load (all lanes hit one 128-byte table: conflict-free) and one
+//              packed add.
+// Only planes p < t_j and the scales of active channels are ever read.
 #include "fathom_common.cuh"
 
 namespace {
 
-constexpr int TILE_BLOCKS = 32;          // 2048 tokens per CTA
-constexpr int ROW_CHUNK = 32;            // active rows staged per pass
-constexpr int SCAN_THREADS = 256;
-constexpr int SCAN_WARPS = SCAN_THREADS / 32;
-constexpr int BLOCKS_PER_WARP = TILE_BLOCKS / SCAN_WARPS;   // 4
+constexpr int SCAN_WARPS = 4;
+constexpr int SCAN_THREADS = SCAN_WARPS * 32;
+constexpr int WB = 4;                                        // blocks per warp
+constexpr int TILE_BLOCKS = SCAN_WARPS * WB;                 // 1024 tokens per CTA
+constexpr int ROWS_PER_GROUP = 4;
+constexpr int GC = 4;                                        // groups per chunk
+constexpr int CHUNK_ROWS = GC * ROWS_PER_GROUP;              // 16
+constexpr int STAGE_ROWS = 3 * CHUNK_ROWS;                   // rows staged per CTA pass (a B = 48 plan in one pass)
+
+template <int NH> struct ScanCfg {
+  static constexpr int HP = NH == 1 ? 1 : NH / 2;            // head pairs (tables per block and group)
+  static constexpr int EB = NH == 1 ? 4 : 8;                 // bytes per table entry
+  static constexpr int TSTRIDE = 16 * EB + EB;               // bytes between tables (padded: 34 or 17 words)
+  static constexpr int NTAB = GC * HP * WB;                  // tables per warp and chunk
+};
+
+__device__ __forceinline__ void add2(unsigned long long& acc, unsigned long long v) {
+  asm("add.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(v));
+}
+
+// 4 x 4 bit-block transpose across four words: afterwards nibble k of word w holds, for token 4 k + w,
+// the bits of rows a, b, c, d at bit 0, 1, 2, 3.
+__device__ __forceinline__ void transpose_rows(uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+  uint32_t t;
+  t = ((a >> 1) ^ b) & 0x55555555u; b ^= t; a ^= t << 1;
+  t = ((c >> 1) ^ d) & 0x55555555u; d ^= t; c ^= t << 1;
+  t = ((a >> 2) ^ c) & 0x33333333u; c ^= t; a ^= t << 2;
+  t = ((b >> 2) ^ d) & 0x33333333u; d ^= t; b ^= t << 2;
+}
 
 template <int NH>
-struct alignas(16) Wvec { float v[NH]; };
+struct alignas(16) WarpSmem {
+  using C = ScanCfg<NH>;
+  uint32_t idx[GC][WB * 4 * 2 + 2];                          // [group][(block, token mod 4, half)] + 2 pad words: 8 nibbles each;
+                                                             // the pad spreads the four groups over different banks
+  alignas(8) unsigned char tab[C::NTAB * C::TSTRIDE];
+};
 
 template <int NH>
 __global__ void __launch_bounds__(SCAN_THREADS)
 scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
             const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
             long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
-            int G) {
+            int G, int heads_per_plan) {
+  using C = ScanCfg<NH>;
+  constexpr int HP = C::HP, EB = C::EB, TSTRIDE = C::TSTRIDE;
   __shared__ uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];      // channel of active row r
   __shared__ uint8_t row_pl[FATHOM_D * FATHOM_NPLANES];       // plane of active row r
   __shared__ int s_nrows;
+  __shared__ int warp_tot[4];
   __shared__ float s_q[NH][FATHOM_D];
-  __shared__ alignas(16) uint64_t s_words[ROW_CHUNK][TILE_BLOCKS];
-  __shared__ Wvec<NH> s_w[TILE_BLOCKS][ROW_CHUNK];            // 2 w per (block, row), all heads
-  __shared__ float s_bias[TILE_BLOCKS][NH];                   // sum of w over all active rows
+  __shared__ alignas(16) uint64_t s_words[STAGE_ROWS][TILE_BLOCKS];   // staged plane words
+  __shared__ alignas(16) uint16_t s_scale[STAGE_ROWS][TILE_BLOCKS];   // staged fp16 scales
+  __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
+  __shared__ WarpSmem<NH> s_warp[SCAN_WARPS];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int plan = blockIdx.y;
-  const int h0 = plan * NH;
+  const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
+  const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
   const int kv = h0 / G;
-  const long long blk0 = (long long)blockIdx.x * TILE_BLOCKS;
-  const int nblk = (int)min((long long)TILE_BLOCKS, nb - blk0);
 
-  // ---- active row list of this plan, ordered by channel then plane (thread 0..127 = channel)
-  if (tid < FATHOM_D) {
+  // ---- active row list of this plan, ordered by channel then plane (thread = channel)
+  {
     const int t = depth[(size_t)plan * FATHOM_D + tid];
-    // exclusive prefix of depths over channels via warp scans + a 4-entry carry
-    int incl = t;
+    int incl = t;                                             // inclusive prefix of depths over channels
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += y;
     }
-    __shared__ int warp_tot[4];
     if (lane == 31) warp_tot[warp] = incl;
-    // the four channel warps synchronise through the named barrier below
-    asm volatile("bar.sync 1, 128;");
+    for (int e = tid; e < NH * FATHOM_D; e += SCAN_THREADS) s_q[e / FATHOM_D][e % FATHOM_D] = q[(size_t)h0 * FATHOM_D + e];
+    __syncthreads();
     int base = 0;
     for (int w = 0; w < warp; ++w) base += warp_tot[w];
     const int start = base + incl - t;
     for (int p = 0; p < t; ++p) { row_ch[start + p] = (uint16_t)tid; row_pl[start + p] = (uint8_t)p; }
     if (tid == FATHOM_D - 1) s_nrows = base + incl;
+    __syncthreads();
   }
-  for (int e = tid; e < NH * FATHOM_D; e += SCAN_THREADS) s_q[e / FATHOM_D][e % FATHOM_D] = q[(size_t)h0 * FATHOM_D + e];
-  for (int e = tid; e < TILE_BLOCKS * NH; e += SCAN_THREADS) (&s_bias[0][0])[e] = 0.0f;
-  __syncthreads();
   const int nrows = s_nrows;
 
-  float acc[BLOCKS_PER_WARP][2][NH];
-#pragma unroll
-  for (int b = 0; b < BLOCKS_PER_WARP; ++b)
-#pragma unroll
-    for (int x = 0; x < 2; ++x)
-#pragma unroll
-      for (int h = 0; h < NH; ++h) acc[b][x][h] = 0.0f;
+  WarpSmem<NH>& S = s_warp[warp];
+  const long long blk0 = (long long)blockIdx.x * TILE_BLOCKS;  // first block of this CTA
+  const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
+  const int wb0 = warp * WB;                                   // first block of this warp within the tile
+  const int nblk = max(0, min(WB, nblk_cta - wb0));
 
-  const uint64_t* planes_kv = planes + (size_t)kv * FATHOM_D * FATHOM_NPLANES * (size_t)plane_stride;
-  const uint16_t* scales_kv = scales + (size_t)kv * FATHOM_D * (size_t)scale_stride;
-
-  for (int r0 = 0; r0 < nrows; r0 += ROW_CHUNK) {
-    const int rc = min(ROW_CHUNK, nrows - r0);
-    // ---- stage plane words: 16 threads x 16 B per row
-    for (int e = tid; e < rc * (TILE_BLOCKS / 2); e += SCAN_THREADS) {
-      const int r = e / (TILE_BLOCKS / 2), c = e % (TILE_BLOCKS / 2);
-      uint4 val = make_uint4(0u, 0u, 0u, 0u);
-      if (2 * c < nblk) {
-        const int j = row_ch[r0 + r], p = row_pl[r0 + r];
-        const uint64_t* src = planes_kv + ((size_t)j * FATHOM_NPLANES + p) * (size_t)plane_stride + blk0 + 2 * c;
-        val = __ldg(reinterpret_cast<const uint4*>(src));
-      }
-      *reinterpret_cast<uint4*>(&s_words[r][2 * c]) = val;
+  // lookup role: lane owns tokens lane (low word half) and lane + 32 (high half) of each of the warp's blocks
+  const int my_w = lane & 3;                                  // word of the transposed quadruple that holds my token
+  const int rot = (4 * (lane >> 2) - (EB == 8 ? 3 : 2)) & 31; // brings my nibble to the byte-offset position
+  constexpr uint32_t OFFMASK = 15u * EB;
+  unsigned long long acc2[WB][2][HP];                         // packed head pairs (NH >= 2)
+  float acc1[WB][2];                                          // NH == 1
+#pragma unroll
+  for (int b = 0; b < WB; ++b)
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      acc1[b][x] = 0.0f;
+#pragma unroll
+      for (int hp = 0; hp < HP; ++hp) acc2[b][x][hp] = 0ull;
     }
-    // ---- weights: thread handles block beta = tid / 8 and rows (tid % 8) + 8 i
+
+  const uint64_t* planes_kv = planes + (size_t)kv * FATHOM_D * FATHOM_NPLANES * (size_t)plane_stride + blk0;
+  const uint16_t* scales_kv = scales + (size_t)kv * FATHOM_D * (size_t)scale_stride + blk0;
+
+  for (int s0 = 0; s0 < nrows; s0 += STAGE_ROWS) {
+    const int sc = min(STAGE_ROWS, nrows - s0);                // rows staged in this pass
+    if (s0 > 0) __syncthreads();                               // every warp is done with the previous pass
+    // ---- stage plane words (8 x 16 B per row), scales (2 x 16 B per row) and per-row query factors
     {
-      const int beta = tid >> 3, sub = tid & 7;
-      float part[NH];
+      uint4 wv[STAGE_ROWS * 8 / SCAN_THREADS];
 #pragma unroll
-      for (int h = 0; h < NH; ++h) part[h] = 0.0f;
-      if (beta < nblk) {
-        for (int r = sub; r < rc; r += 8) {
-          const int j = row_ch[r0 + r], p = row_pl[r0 + r];
-          const float s = __half2float(__ushort_as_half(__ldg(scales_kv + (size_t)j * scale_stride + blk0 + beta)));
-          const float a_p = s * (8.0f / (float)(2 << p));     // a * 2^-(p+1), exact
-          Wvec<NH> w2;
-#pragma unroll
-          for (int h = 0; h < NH; ++h) {
-            const float w = s_q[h][j] * a_p;
-            part[h] += w;
-            w2.v[h] = 2.0f * w;
-          }
-          s_w[beta][r] = w2;
+      for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
+        const int e = tid + k * SCAN_THREADS, r = e >> 3, c = e & 7;
+        wv[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < sc && 2 * c < nblk_cta) {
+          const int j = row_ch[s0 + r], p = row_pl[s0 + r];
+          wv[k] = __ldg(reinterpret_cast<const uint4*>(planes_kv + ((size_t)j * FATHOM_NPLANES + p) * (size_t)plane_stride + 2 * c));
         }
       }
-      // fixed-order reduction of the 8 partial sums of a block (lanes 8k .. 8k+7)
-#pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        float v = part[h];
-        v += __shfl_xor_sync(0xffffffffu, v, 1);
-        v += __shfl_xor_sync(0xffffffffu, v, 2);
-        v += __shfl_xor_sync(0xffffffffu, v, 4);
-        if (sub == 0 && beta < nblk) s_bias[beta][h] += v;
+      uint4 sv = make_uint4(0u, 0u, 0u, 0u);
+      if (tid < STAGE_ROWS * 2) {
+        const int r = tid >> 1, c = tid & 1;
+        if (r < sc && 8 * c < nblk_cta)
+          sv = __ldg(reinterpret_cast<const uint4*>(scales_kv + (size_t)row_ch[s0 + r] * (size_t)scale_stride + 8 * c));
       }
+      if (tid < STAGE_ROWS) {
+        const bool valid = tid < sc;
+        const int j = valid ? row_ch[s0 + tid] : 0, p = valid ? row_pl[s0 + tid] : 0;
+        const float pw = valid ? __int_as_float((129 - p) << 23) : 0.0f;   // 8 * 2^-(p+1) = 2^(2-p), exact
+#pragma unroll
+        for (int h = 0; h < NH; ++h) s_qs[tid][h] = s_q[h][j] * pw;
+      }
+#pragma unroll
+      for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
+        const int e = tid + k * SCAN_THREADS;
+        *reinterpret_cast<uint4*>(&s_words[e >> 3][2 * (e & 7)]) = wv[k];
+      }
+      if (tid < STAGE_ROWS * 2) *reinterpret_cast<uint4*>(&s_scale[tid >> 1][8 * (tid & 1)]) = sv;
     }
     __syncthreads();
-    // ---- accumulate: warp w owns blocks w, w + 8, ...; lane owns tokens lane and lane + 32
+
+    for (int r0 = 0; r0 < sc; r0 += CHUNK_ROWS) {
+      const int rc = min(CHUNK_ROWS, sc - r0);                   // rows in this chunk
+      const int gc = (rc + ROWS_PER_GROUP - 1) / ROWS_PER_GROUP; // groups in this chunk (the last may be padded)
+
+      // ---- tables: lane = (group, head pair, block)
 #pragma unroll
-    for (int b = 0; b < BLOCKS_PER_WARP; ++b) {
-      const int beta = warp + b * SCAN_WARPS;
-      if (beta < nblk) {
-        for (int r = 0; r < rc; ++r) {
-          const uint64_t word = s_words[r][beta];
-          const Wvec<NH> w2 = s_w[beta][r];
-          const bool lo = ((uint32_t)word >> lane) & 1u;
-          const bool hi = ((uint32_t)(word >> 32) >> lane) & 1u;
+      for (int t0 = 0; t0 < C::NTAB; t0 += 32) {
+        const int t = t0 + lane;
+        const int beta = t % WB, hp = (t / WB) % HP, g = t / (WB * HP);
+        if (t < C::NTAB && g < gc) {
+          float wa[ROWS_PER_GROUP], wb[ROWS_PER_GROUP];
 #pragma unroll
-          for (int h = 0; h < NH; ++h) {
-            if (lo) acc[b][0][h] += w2.v[h];
-            if (hi) acc[b][1][h] += w2.v[h];
+          for (int x = 0; x < ROWS_PER_GROUP; ++x) {
+            const int r = r0 + g * ROWS_PER_GROUP + x;            // staged rows beyond sc carry zero factors
+            const float s = __half2float(__ushort_as_half(s_scale[r][wb0 + beta]));
+            if (NH == 1) {
+              wa[x] = s_qs[r][0] * s; wb[x] = 0.0f;
+            } else {
+              const float2 qq = *reinterpret_cast<const float2*>(&s_qs[r][2 * hp]);
+              wa[x] = qq.x * s; wb[x] = qq.y * s;
+            }
+          }
+          float ta[16], tb[16];
+          ta[0] = -((wa[0] + wa[1]) + (wa[2] + wa[3]));
+          tb[0] = -((wb[0] + wb[1]) + (wb[2] + wb[3]));
+#pragma unroll
+          for (int x = 0; x < ROWS_PER_GROUP; ++x) {
+            const float da = 2.0f * wa[x], db = 2.0f * wb[x];
+#pragma unroll
+            for (int e = 0; e < (1 << x); ++e) { ta[e + (1 << x)] = ta[e] + da; tb[e + (1 << x)] = tb[e] + db; }
+          }
+          unsigned char* tab = S.tab + t * TSTRIDE;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            if (NH == 1) reinterpret_cast<float*>(tab)[e] = ta[e];
+            else reinterpret_cast<float2*>(tab)[e] = make_float2(ta[e], tb[e]);
           }
         }
       }
+
+      // ---- indices: lane = (group, block, half)
+      {
+        const int half = lane & 1, beta = (lane >> 1) & 3, g = lane >> 3;
+        if (g < gc) {
+          const uint32_t* w32 = reinterpret_cast<const uint32_t*>(&s_words[r0 + g * ROWS_PER_GROUP][wb0 + beta]) + half;
+          uint32_t a = w32[0 * TILE_BLOCKS * 2];
+          uint32_t b = w32[1 * TILE_BLOCKS * 2];
+          uint32_t c = w32[2 * TILE_BLOCKS * 2];
+          uint32_t d = w32[3 * TILE_BLOCKS * 2];
+          transpose_rows(a, b, c, d);
+          S.idx[g][(beta * 4 + 0) * 2 + half] = a;
+          S.idx[g][(beta * 4 + 1) * 2 + half] = b;
+          S.idx[g][(beta * 4 + 2) * 2 + half] = c;
+          S.idx[g][(beta * 4 + 3) * 2 + half] = d;
+        }
+      }
+      __syncwarp();
+
+      // ---- lookup
+#pragma unroll
+      for (int b = 0; b < WB; ++b) {
+#pragma unroll
+        for (int g = 0; g < GC; ++g) {
+          if (g < gc) {
+            const uint2 nib = *reinterpret_cast<const uint2*>(&S.idx[g][(b * 4 + my_w) * 2]);
+            const uint32_t off_lo = __funnelshift_r(nib.x, nib.x, rot) & OFFMASK;
+            const uint32_t off_hi = __funnelshift_r(nib.y, nib.y, rot) & OFFMASK;
+            const unsigned char* tab = S.tab + ((g * HP) * WB + b) * TSTRIDE;
+            if (NH == 1) {
+              acc1[b][0] += *reinterpret_cast<const float*>(tab + off_lo);
+              acc1[b][1] += *reinterpret_cast<const float*>(tab + off_hi);
+            } else {
+#pragma unroll
+              for (int hp = 0; hp < HP; ++hp) {
+                add2(acc2[b][0][hp], *reinterpret_cast<const unsigned long long*>(tab + hp * (WB * TSTRIDE) + off_lo));
+                add2(acc2[b][1][hp], *reinterpret_cast<const unsigned long long*>(tab + hp * (WB * TSTRIDE) + off_hi));
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
     }
-    __syncthreads();
   }
 
-  // ---- epilogue: score = 2 sum_{bit=1} w - sum w
+  // ---- epilogue
 #pragma unroll
-  for (int b = 0; b < BLOCKS_PER_WARP; ++b) {
-    const int beta = warp + b * SCAN_WARPS;
-    if (beta < nblk) {
-      const long long tok = (blk0 + beta) * FATHOM_BLOCK + lane;
+  for (int b = 0; b < WB; ++b) {
+    if (b < nblk) {
+      const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
-        const float bias = s_bias[beta][h];
         float* row = scores + (size_t)(h0 + h) * (size_t)score_stride;
-        if (tok < n) row[tok] = acc[b][0][h] - bias;
-        if (tok + 32 < n) row[tok + 32] = acc[b][1][h] - bias;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          float v;
+          if (NH == 1) v = acc1[b][x];
+          else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
+          if (tok + 32 * x < n) row[tok + 32 * x] = v;
+        }
       }
     }
   }
@@ -164,12 +277,12 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
 
 template <int NH>
 int launch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
-                const uint8_t* depth, float* scores, cudaStream_t st) {
+                const uint8_t* depth, int heads_per_plan, float* scores, cudaStream_t st) {
   const long long nb = fathom_nblocks(L->n);
-  const int plans = L->n_q_heads / NH;
-  dim3 grid((unsigned)((nb + TILE_BLOCKS - 1) / TILE_BLOCKS), (unsigned)plans);
+  dim3 grid((unsigned)((nb + TILE_BLOCKS - 1) / TILE_BLOCKS), (unsigned)(L->n_q_heads / NH));
   scan_kernel<NH><<<grid, SCAN_THREADS, 0, st>>>(planes, scales, q, depth, scores, L->n, nb, L->plane_stride_words,
-                                                 L->scale_stride, L->score_stride, L->n_q_heads / L->n_kv_heads);
+                                                 L->scale_stride, L->score_stride, L->n_q_heads / L->n_kv_heads,
+                                                 heads_per_plan);
   return 0;
 }
 
@@ -185,10 +298,10 @@ extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64
   if (!fathom_aligned16(planes) || !fathom_aligned16(scales) || !fathom_aligned16(scores)) return FATHOM_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   switch (heads_per_plan) {
-    case 1: launch_scan<1>(L, planes, scales, q, depth, scores, st); break;
-    case 2: launch_scan<2>(L, planes, scales, q, depth, scores, st); break;
-    case 4: launch_scan<4>(L, planes, scales, q, depth, scores, st); break;
-    case 8: launch_scan<8>(L, planes, scales, q, depth, scores, st); break;
+    case 1: launch_scan<1>(L, planes, scales, q, depth, 1, scores, st); break;
+    case 2: launch_scan<2>(L, planes, scales, q, depth, 2, scores, st); break;
+    case 4: launch_scan<4>(L, planes, scales, q, depth, 4, scores, st); break;
+    case 8: launch_scan<4>(L, planes, scales, q, depth, 8, scores, st); break;   // two CTAs of four heads share a plan
     default: return FATHOM_ERR_UNSUPPORTED;
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
