@@ -43,7 +43,8 @@ typedef enum {
   FATHOM_ERR_UNSUPPORTED = -2,      /* d != 128, heads_per_plan not in {1,2,4,8}, unknown mode/dtype */
   FATHOM_ERR_ALIGNMENT = -3,        /* pointer or stride not aligned as the layout requires */
   FATHOM_ERR_SCRATCH_TOO_SMALL = -4,/* context scratch smaller than fathom_scratch_bytes() for this call */
-  FATHOM_ERR_CUDA = -5              /* a CUDA runtime call failed (see fathom_last_cuda_error) */
+  FATHOM_ERR_CUDA = -5,             /* a CUDA runtime call failed (see fathom_last_cuda_error) */
+  FATHOM_ERR_STATIC_LIMIT = -6      /* problem larger than the built-in scratch of an allocation-free entry point */
 } fathom_status;
 
 typedef enum { FATHOM_F32 = 0, FATHOM_BF16 = 1 } fathom_dtype;
@@ -145,6 +146,27 @@ int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* score
 int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* layout, const float* q,
                          const void* Krows, const void* Vrows, int row_dtype, const int32_t* idx,
                          int k, float softmax_scale, float* out, void* stream);
+
+/* ---- (5b) gather + exact attention without any allocation — the paper has no counterpart ------
+ * Same computation, arguments and results as fathom_sparse_attend, for callers that cannot obtain device
+ * memory of their own: a plug-in that is only handed buffers by its host application, a serving process
+ * whose memory pool already owns the whole GPU (cudaMalloc would fail there), or a decode loop that must
+ * not pay the device-wide synchronisation an allocation or a free can imply.  It needs no fathom_ctx and
+ * calls neither cudaMalloc nor cudaFree nor any allocating library routine: the per-chunk softmax partials
+ * live in an array that is compiled into the library (about 1 MB of device memory on every GPU that loads
+ * the library, held until the process exits).
+ *   Limit: n_q_heads * ceil(k / 128) <= FATHOM_ATTEND_STATIC_MAX_CHUNKS, otherwise FATHOM_ERR_STATIC_LIMIT
+ *   is returned and nothing is launched (32 query heads allow k <= 8192).
+ *   First use on a device: the call looks up the device address of the built-in array once per device
+ *   (cudaGetSymbolAddress, with the stream's device current — make it current before calling).  Make this
+ *   first call before any stream capture begins; later calls on that device only enqueue two kernels.
+ *   Sharing: every call on a device uses the same array, which keeps the previous call's contents.  Each
+ *   call overwrites every element it later reads, so nothing needs clearing, but two calls that may overlap
+ *   on the device (different streams, no dependency) race on it and must be ordered by the caller. */
+#define FATHOM_ATTEND_STATIC_MAX_CHUNKS 2048
+int fathom_sparse_attend_static(const fathom_layout* layout, const float* q, const void* Krows,
+                                const void* Vrows, int row_dtype, const int32_t* idx, int k,
+                                float softmax_scale, float* out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -21,7 +21,7 @@ DEV_TOPK_SHORT, DEV_WAIT_EXPIRED = 0x1, 0x2
 
 EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error",
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
-           "fathom_topk", "fathom_sparse_attend"]
+           "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static"]
 
 
 class Layout(C.Structure):
@@ -58,6 +58,7 @@ def _load() -> C.CDLL:
     lib.fathom_scan.argtypes = [vp, LP, vp, vp, vp, vp, i32, vp, vp]
     lib.fathom_topk.argtypes = [vp, LP, vp, i32, i32, i32, vp, vp]
     lib.fathom_sparse_attend.argtypes = [vp, LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
+    lib.fathom_sparse_attend_static.argtypes = [LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
     for name in EXPORTS:
         if name not in ("fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error"):
             getattr(lib, name).restype = C.c_int
@@ -150,6 +151,22 @@ class Context:
         st = C.c_uint32(0)
         self._check(lib.fathom_device_status(self._h, _stream(stream), C.byref(st)))
         return st.value
+
+
+ATTEND_STATIC_MAX_CHUNKS = 2048
+
+
+def fathom_sparse_attend_static(layout, q, Krows, Vrows, idx, k, softmax_scale, out, stream=None, row_dtype=None):
+    """Attention over the selected rows for callers that cannot allocate device memory: no context, no
+    scratch arena.  The partial results live in an array built into the library (limit:
+    n_q_heads * ceil(k / 128) <= ATTEND_STATIC_MAX_CHUNKS).  The current device must be the stream's; the
+    first call on a device looks up the array's address and should come before any stream capture; calls
+    that may overlap on the device share the array and must be ordered by the caller."""
+    rc = lib.fathom_sparse_attend_static(C.byref(layout), _ptr(q), _ptr(Krows), _ptr(Vrows),
+                                         _dtype_code(Krows) if row_dtype is None else row_dtype, _ptr(idx), k,
+                                         C.c_float(softmax_scale), _ptr(out), _stream(stream))
+    if rc != 0:
+        raise FathomError(rc)
 
 
 def fathom_scratch_bytes(layout: Layout, k: int) -> int:

@@ -93,6 +93,7 @@ const char* fathom_strerror(int status) {
     case FATHOM_ERR_ALIGNMENT: return "pointer or stride is not 16-byte aligned as the layout requires";
     case FATHOM_ERR_SCRATCH_TOO_SMALL: return "context scratch arena is smaller than fathom_scratch_bytes() for this call";
     case FATHOM_ERR_CUDA: return "a CUDA runtime call failed (see fathom_last_cuda_error)";
+    case FATHOM_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of the allocation-free entry point (n_q_heads * ceil(k / 128) > FATHOM_ATTEND_STATIC_MAX_CHUNKS)";
     default: return "unknown fathom status";
   }
 }

@@ -8,6 +8,8 @@
 // bit-reproducible.
 #include "fathom_common.cuh"
 
+#include <mutex>
+
 namespace {
 
 constexpr int AT_THREADS = FATHOM_ATTN_CHUNK;   // 128 threads: one per row, then one per channel
@@ -153,5 +155,61 @@ extern "C" int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* L, con
                                                               softmax_scale, S.partial, S.splits);
   attend_combine_kernel<<<Hq, FATHOM_D, 0, st>>>(S.partial, S.splits, out);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+// ---- allocation-free variant --------------------------------------------------------------------------
+// Scratch for callers that cannot allocate: the per-chunk (max, denominator, weighted sum) triples live in
+// this array instead of a context's arena.  In host code the name below is only a handle for the runtime,
+// not a device address, so the address is fetched once per device with cudaGetSymbolAddress and that
+// pointer is what the kernels receive.
+static __device__ __align__(256) float g_attend_static_partials[FATHOM_ATTEND_STATIC_MAX_CHUNKS * (FATHOM_D + 2)];
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+float* g_static_partials_ptr[STATIC_MAX_DEVICES];            // device address per device ordinal, null until first use
+std::mutex g_static_mutex;
+}  // namespace
+
+extern "C" int fathom_sparse_attend_static(const fathom_layout* L, const float* q, const void* Krows, const void* Vrows,
+                                           int row_dtype, const int32_t* idx, int k, float softmax_scale, float* out,
+                                           void* stream) {
+  if (!q || !Krows || !Vrows || !idx || !out) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k < 1 || k > L->n) return FATHOM_ERR_INVALID_ARG;
+  if (row_dtype != FATHOM_BF16 && row_dtype != FATHOM_F32) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(Krows) || !fathom_aligned16(Vrows)) return FATHOM_ERR_ALIGNMENT;
+  const int Hq = L->n_q_heads, G = Hq / L->n_kv_heads;
+  const int splits = (k + FATHOM_ATTN_CHUNK - 1) / FATHOM_ATTN_CHUNK;
+  if ((long long)Hq * splits > FATHOM_ATTEND_STATIC_MAX_CHUNKS) return FATHOM_ERR_STATIC_LIMIT;
+
+  // set-up, once per device, with that device current
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FATHOM_ERR_CUDA;
+  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return FATHOM_ERR_UNSUPPORTED;
+  float* partial = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_partials_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_attend_static_partials) != cudaSuccess || !p) return FATHOM_ERR_CUDA;
+      g_static_partials_ptr[dev] = static_cast<float*>(p);
+    }
+    partial = g_static_partials_ptr[dev];
+  }
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid((unsigned)splits, (unsigned)Hq);
+  if (row_dtype == FATHOM_BF16)
+    attend_partial_kernel<__nv_bfloat16><<<grid, AT_THREADS, 0, st>>>(
+        q, static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k, L->n, G,
+        softmax_scale, partial, splits);
+  else
+    attend_partial_kernel<float><<<grid, AT_THREADS, 0, st>>>(q, static_cast<const float*>(Krows),
+                                                              static_cast<const float*>(Vrows), idx, k, L->n, G,
+                                                              softmax_scale, partial, splits);
+  attend_combine_kernel<<<Hq, FATHOM_D, 0, st>>>(partial, splits, out);
+  if (cudaGetLastError() != cudaSuccess) return FATHOM_ERR_CUDA;
   return FATHOM_OK;
 }
