@@ -35,9 +35,11 @@ METRIC = "keys_scanned_per_s"
 UNIT = "keys/s"
 WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3, planes in HBM)",
                 n=1 << 20, Hkv=8, Hq=32, d=128, B=48, k=4096, heads_per_plan=4)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (captured at n = 131072 and scaled by the tokens a full launch processes); None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": None, "scan_kernel": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per unit (one token of one KV head) from the ncu captures
+# summarised under profiles/: build at n = 131072 (596.1 MB / 1,048,576 units; traffic is proportional to
+# units), scan at n = 1,048,576 and B = 48 (136.9 MB / 8,388,608 units; part of the score writes is still in
+# L2 when the kernel ends).  Multiplied by the units of a launch in the JSON line.
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.3}
 
 
 def parse_args():
