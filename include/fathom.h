@@ -159,9 +159,9 @@ int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* layout, const flo
  *   is returned and nothing is launched (32 query heads allow k <= 8192).
  *   First use on a device: the call looks up the device address of the built-in array once per device
  *   (cudaGetSymbolAddress, with the stream's device current — make it current before calling).  Make this
- *   first call before any stream capture begins; later calls on that device only enqueue two kernels.
+ *   first call before any stream capture begins; later calls on that device only enqueue one kernel.
  *   Sharing: every call on a device uses the same array, which keeps the previous call's contents.  Each
- *   call overwrites every element it later reads, so nothing needs clearing, but two calls that may overlap
+ *   call overwrites every element it later reads and re-arms its ticket counters, so nothing needs clearing, but two calls that may overlap
  *   on the device (different streams, no dependency) race on it and must be ordered by the caller. */
 #define FATHOM_ATTEND_STATIC_MAX_CHUNKS 2048
 int fathom_sparse_attend_static(const fathom_layout* layout, const float* q, const void* Krows,

@@ -1,71 +1,77 @@
 // fathom_alloc_depth: per-plan read depths (Sec. 3.3, Eq. 3 and Eq. 4; fixed-channel rule of Sec. 2).
 //
-// One CTA of 4 * 128 threads per plan; thread (j, m) owns candidate plane m = 1..4 of channel j.
-// Eq. 4 at the smallest water line that fits the budget grants exactly the min(B, 4d) candidate
-// planes with the largest priority g_j 4^-m, so each thread ranks its own candidate against the
-// other 511 (ties: lower channel, then lower plane) and is granted when its rank is below B.  All
-// arithmetic is fp64 with explicit round-to-nearest intrinsics (no fused multiply-add), so the
-// ranking is identical on every machine; no logarithm is evaluated.
+// Eq. 4 at the smallest water line that fits the budget grants exactly the min(B, 4d) candidate planes
+// (channel j, plane m = 1..4) with the largest priority g_j 4^-m, so a candidate is granted when fewer than
+// B others rank before it (ties: lower channel, then lower plane).  Four CTAs of 128 threads serve a plan:
+// every CTA computes all 128 importances (thread = channel; fp64 with explicit round-to-nearest intrinsics,
+// no fused multiply-add, so the ranking is identical on every machine; no logarithm is evaluated) and ranks
+// the 128 candidates of its own 32 channels against all 512.  Non-negative doubles order like their bit
+// patterns, so the comparisons run on 64-bit integers.
 #include "fathom_common.cuh"
 
 namespace {
 
 constexpr int NCAND = FATHOM_D * FATHOM_NPLANES;   // 512
+constexpr int CTAS_PER_PLAN = 4;
+constexpr int AD_THREADS = NCAND / CTAS_PER_PLAN;  // 128
 
-__global__ void __launch_bounds__(NCAND)
+__global__ void __launch_bounds__(AD_THREADS)
 alloc_depth_kernel(const float* __restrict__ q, const float* __restrict__ var, int mode, int budget,
                    int heads_per_plan, int G, uint8_t* __restrict__ depth) {
-  __shared__ double pri[NCAND];
-  const int plan = blockIdx.x;
+  __shared__ alignas(16) unsigned long long pri[NCAND];       // bit patterns of the (non-negative) priorities
+  const int plan = blockIdx.x / CTAS_PER_PLAN, part = blockIdx.x % CTAS_PER_PLAN;
   const int tid = threadIdx.x;
-  const int j = tid >> 2;             // channel
-  const int m = (tid & 3) + 1;        // candidate plane 1..4
   const int h0 = plan * heads_per_plan;
   const int kv = h0 / G;
   uint8_t* out = depth + (size_t)plan * FATHOM_D;
 
   if (mode == FATHOM_DEPTH_UNIFORM) {
-    if (m == 1) out[j] = (uint8_t)min(max(budget, 0), FATHOM_NPLANES);
+    if (part == 0) out[tid] = (uint8_t)min(max(budget, 0), FATHOM_NPLANES);
     return;
   }
 
-  double key;
-  if (mode == FATHOM_DEPTH_WATERFILL) {
+  {                                                           // thread = channel: its four priorities
+    const int j = tid;
     double acc = 0.0;
-    for (int h = h0; h < h0 + heads_per_plan; ++h) {
-      const double x = (double)q[(size_t)h * FATHOM_D + j];
-      acc = __dadd_rn(acc, __dmul_rn(x, x));                  // Eq. 3, heads in ascending order
+    if (mode == FATHOM_DEPTH_WATERFILL) {
+      for (int h = h0; h < h0 + heads_per_plan; ++h) {
+        const double x = (double)q[(size_t)h * FATHOM_D + j];
+        acc = __dadd_rn(acc, __dmul_rn(x, x));                // Eq. 3, heads in ascending order
+      }
+      const double g = __dmul_rn(acc, (double)var[(size_t)kv * FATHOM_D + j]);
+      pri[4 * j + 0] = (unsigned long long)__double_as_longlong(fabs(__dmul_rn(g, 0.25)));        // g_j 4^-m
+      pri[4 * j + 1] = (unsigned long long)__double_as_longlong(fabs(__dmul_rn(g, 0.0625)));
+      pri[4 * j + 2] = (unsigned long long)__double_as_longlong(fabs(__dmul_rn(g, 0.015625)));
+      pri[4 * j + 3] = (unsigned long long)__double_as_longlong(fabs(__dmul_rn(g, 0.00390625)));
+    } else {                                                  // fixed top-r channels by sum_h |q_j|
+      for (int h = h0; h < h0 + heads_per_plan; ++h)
+        acc = __dadd_rn(acc, fabs((double)q[(size_t)h * FATHOM_D + j]));
+      const unsigned long long key = (unsigned long long)__double_as_longlong(acc);
+      pri[4 * j + 0] = key; pri[4 * j + 1] = key; pri[4 * j + 2] = key; pri[4 * j + 3] = key;
     }
-    const double g = __dmul_rn(acc, (double)var[(size_t)kv * FATHOM_D + j]);
-    const double scale = (m == 1) ? 0.25 : (m == 2) ? 0.0625 : (m == 3) ? 0.015625 : 0.00390625;
-    key = __dmul_rn(g, scale);                                // g_j 4^-m
-  } else {                                                    // fixed top-r channels by sum_h |q_j|
-    double acc = 0.0;
-    for (int h = h0; h < h0 + heads_per_plan; ++h)
-      acc = __dadd_rn(acc, fabs((double)q[(size_t)h * FATHOM_D + j]));
-    key = acc;
   }
-  pri[tid] = key;
   __syncthreads();
 
-  bool granted;
+  const int id = part * AD_THREADS + tid;                     // my candidate: channel id / 4, plane id % 4 + 1
+  const unsigned long long key = pri[id];
+  int rank = 0;
   if (mode == FATHOM_DEPTH_WATERFILL) {
-    int rank = 0;
-    for (int o = 0; o < NCAND; ++o) {
-      const double p = pri[o];
-      rank += (p > key) || (p == key && o < tid);
+#pragma unroll 8
+    for (int o = 0; o < NCAND; o += 2) {
+      const ulonglong2 p = *reinterpret_cast<const ulonglong2*>(&pri[o]);
+      rank += (p.x > key) || (p.x == key && o < id);
+      rank += (p.y > key) || (p.y == key && o + 1 < id);
     }
-    granted = rank < budget;
-  } else {
-    int rank = 0;                                             // rank channels only (candidate m = 1 of each)
+  } else {                                                    // rank channels only (one key per channel)
+#pragma unroll 8
     for (int o = 0; o < NCAND; o += 4) {
-      const double p = pri[o];
-      rank += (p > key) || (p == key && o < (tid & ~3));
+      const unsigned long long p = pri[o];
+      rank += (p > key) || (p == key && o < (id & ~3));
     }
-    granted = rank < budget;                                  // all four planes of a chosen channel
   }
+  const bool granted = rank < budget;                         // fixed mode: all four planes of a chosen channel
   const unsigned ball = __ballot_sync(0xffffffffu, granted);
-  if (m == 1) out[j] = (uint8_t)__popc((ball >> (threadIdx.x & 31)) & 0xFu);
+  if ((id & 3) == 0) out[id >> 2] = (uint8_t)__popc((ball >> (tid & 31)) & 0xFu);
 }
 
 }  // namespace
@@ -83,7 +89,7 @@ extern "C" int fathom_alloc_depth(fathom_ctx* ctx, const fathom_layout* L, const
   const int G = L->n_q_heads / L->n_kv_heads;
   if (heads_per_plan < 1 || G % heads_per_plan != 0) return FATHOM_ERR_INVALID_ARG;
   const int plans = L->n_q_heads / heads_per_plan;
-  alloc_depth_kernel<<<plans, NCAND, 0, static_cast<cudaStream_t>(stream)>>>(q, var, mode, budget, heads_per_plan, G, depth);
+  alloc_depth_kernel<<<plans * CTAS_PER_PLAN, AD_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(q, var, mode, budget, heads_per_plan, G, depth);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

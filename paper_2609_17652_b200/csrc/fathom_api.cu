@@ -59,8 +59,8 @@ int fathom_create(fathom_ctx** out, int device, size_t scratch_bytes) {
   c->scratch_bytes = scratch_bytes;
   c->dev_status = nullptr;
   c->last_cuda = cudaSuccess;
-  cudaError_t e = cudaMalloc(&c->dev_status, 256);
-  if (e == cudaSuccess) e = cudaMemset(c->dev_status, 0, 256);
+  cudaError_t e = cudaMalloc(&c->dev_status, FATHOM_CTL_BYTES);
+  if (e == cudaSuccess) e = cudaMemset(c->dev_status, 0, FATHOM_CTL_BYTES);
   if (e == cudaSuccess && scratch_bytes > 0) e = cudaMalloc(&c->scratch, scratch_bytes);
   if (e != cudaSuccess) {
     if (c->dev_status) cudaFree(c->dev_status);

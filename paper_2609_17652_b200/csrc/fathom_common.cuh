@@ -11,12 +11,15 @@
 #define FATHOM_D 128            // channels per head (Sec. 1: Qwen3-8B head size)
 #define FATHOM_BLOCK 64         // tokens per scale block (Sec. 3.2)
 #define FATHOM_NPLANES 4        // bits per code (Sec. 3.2)
+#define FATHOM_CTL_BYTES 8192   // device control block of a context (zeroed once at creation)
+#define FATHOM_CTL_TICKETS 64   // first ticket counter (word index); counters re-arm themselves
+#define FATHOM_CTL_MAX_HEADS ((FATHOM_CTL_BYTES / 4) - FATHOM_CTL_TICKETS)
 
 struct fathom_ctx {
   int device;
   void* scratch;               // device arena, 256-byte aligned
   size_t scratch_bytes;
-  uint32_t* dev_status;        // device status word
+  uint32_t* dev_status;        // device control block: word 0 = status word, words FATHOM_CTL_TICKETS.. = ticket counters
   cudaError_t last_cuda;
 };
 

@@ -3,9 +3,10 @@
 // Split-k: CTA (split, head) handles FATHOM_ATTN_CHUNK selected rows.  Logits: one thread per row reads
 // its whole K row with 16-byte loads (a row is 256 B in bf16) against q held in shared memory.  After the
 // chunk maximum and exp, each warp walks 32 rows of V with a lane owning 4 channels (one coalesced
-// 256/512-byte row per load instruction) and the four warps are summed in a fixed order.  A second kernel
-// merges the per-chunk (max, denominator, weighted sum) triples in split order, so the output is
-// bit-reproducible.
+// 256/512-byte row per load instruction) and the four warps are summed in a fixed order.  Every CTA
+// publishes its (max, denominator, weighted sum) triple and takes a ticket; the CTA that draws the last
+// ticket of a head merges all triples in split order, so the output is bit-reproducible whichever CTA
+// that is, and no second launch is needed.
 #include "fathom_common.cuh"
 
 #include <mutex>
@@ -57,7 +58,8 @@ template <typename T>
 __global__ void __launch_bounds__(AT_THREADS)
 attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, const T* __restrict__ Vrows,
                       const int32_t* __restrict__ idx, int k, long long n, int G, float softmax_scale,
-                      float* __restrict__ partial, int splits) {
+                      float* __restrict__ partial, int splits, unsigned int* __restrict__ tickets,
+                      float* __restrict__ result) {
   __shared__ float s_q[FATHOM_D];
   __shared__ float s_p[AT_THREADS];
   __shared__ int32_t s_idx[AT_THREADS];
@@ -111,22 +113,32 @@ attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, 
   float* out = partial + ((size_t)head * splits + split) * (FATHOM_D + 2);
   out[2 + tid] = ((s_acc[0][tid] + s_acc[1][tid]) + s_acc[2][tid]) + s_acc[3][tid];
   if (tid == 0) { out[0] = m; out[1] = ((s_red[0] + s_red[1]) + s_red[2]) + s_red[3]; }
-}
 
-__global__ void __launch_bounds__(FATHOM_D)
-attend_combine_kernel(const float* __restrict__ partial, int splits, float* __restrict__ out) {
-  const int head = blockIdx.x, tid = threadIdx.x;
+  // ---- publish; the CTA that draws the head's last ticket merges all chunks (and re-arms the ticket counter)
+  __shared__ bool s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int t = atomicAdd(&tickets[head], 1u);
+    s_last = (t == (unsigned int)splits - 1u);
+    if (s_last) tickets[head] = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
   const float* P = partial + (size_t)head * splits * (FATHOM_D + 2);
   float M = -INFINITY;
-  for (int s = 0; s < splits; ++s) M = fmaxf(M, P[(size_t)s * (FATHOM_D + 2)]);
+#pragma unroll 8
+  for (int s = 0; s < splits; ++s) M = fmaxf(M, __ldcg(P + (size_t)s * (FATHOM_D + 2)));
   float num = 0.0f, den = 0.0f;
+#pragma unroll 8
   for (int s = 0; s < splits; ++s) {
     const float* ps = P + (size_t)s * (FATHOM_D + 2);
-    const float w = expf(ps[0] - M);
-    den = fmaf(w, ps[1], den);
-    num = fmaf(w, ps[2 + tid], num);
+    const float w = expf(__ldcg(ps) - M);
+    den = fmaf(w, __ldcg(ps + 1), den);
+    num = fmaf(w, __ldcg(ps + 2 + tid), num);
   }
-  out[(size_t)head * FATHOM_D + tid] = num / den;
+  result[(size_t)head * FATHOM_D + tid] = num / den;
 }
 
 }  // namespace
@@ -141,19 +153,20 @@ extern "C" int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* L, con
   if (row_dtype != FATHOM_BF16 && row_dtype != FATHOM_F32) return FATHOM_ERR_UNSUPPORTED;
   if (!fathom_aligned16(Krows) || !fathom_aligned16(Vrows)) return FATHOM_ERR_ALIGNMENT;
   const int Hq = L->n_q_heads, G = Hq / L->n_kv_heads;
+  if (Hq > FATHOM_CTL_MAX_HEADS) return FATHOM_ERR_UNSUPPORTED;
   fathom_attn_scratch S = fathom_carve_attn(ctx->scratch, Hq, k);
   if (S.bytes > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  unsigned int* tickets = ctx->dev_status + FATHOM_CTL_TICKETS;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid((unsigned)S.splits, (unsigned)Hq);
   if (row_dtype == FATHOM_BF16)
     attend_partial_kernel<__nv_bfloat16><<<grid, AT_THREADS, 0, st>>>(
         q, static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k, L->n, G,
-        softmax_scale, S.partial, S.splits);
+        softmax_scale, S.partial, S.splits, tickets, out);
   else
     attend_partial_kernel<float><<<grid, AT_THREADS, 0, st>>>(q, static_cast<const float*>(Krows),
                                                               static_cast<const float*>(Vrows), idx, k, L->n, G,
-                                                              softmax_scale, S.partial, S.splits);
-  attend_combine_kernel<<<Hq, FATHOM_D, 0, st>>>(S.partial, S.splits, out);
+                                                              softmax_scale, S.partial, S.splits, tickets, out);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
@@ -164,10 +177,14 @@ extern "C" int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* L, con
 // not a device address, so the address is fetched once per device with cudaGetSymbolAddress and that
 // pointer is what the kernels receive.
 static __device__ __align__(256) float g_attend_static_partials[FATHOM_ATTEND_STATIC_MAX_CHUNKS * (FATHOM_D + 2)];
+// Ticket counters of the merge step, one per query head; zero when the library is loaded and re-armed by
+// the merging CTA of every call, so they never need clearing either.
+static __device__ __align__(256) unsigned int g_attend_static_tickets[FATHOM_ATTEND_STATIC_MAX_CHUNKS];
 
 namespace {
 constexpr int STATIC_MAX_DEVICES = 64;
 float* g_static_partials_ptr[STATIC_MAX_DEVICES];            // device address per device ordinal, null until first use
+unsigned int* g_static_tickets_ptr[STATIC_MAX_DEVICES];
 std::mutex g_static_mutex;
 }  // namespace
 
@@ -189,14 +206,18 @@ extern "C" int fathom_sparse_attend_static(const fathom_layout* L, const float* 
   if (cudaGetDevice(&dev) != cudaSuccess) return FATHOM_ERR_CUDA;
   if (dev < 0 || dev >= STATIC_MAX_DEVICES) return FATHOM_ERR_UNSUPPORTED;
   float* partial = nullptr;
+  unsigned int* tickets = nullptr;
   {
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_partials_ptr[dev]) {
-      void* p = nullptr;
+      void *p = nullptr, *t = nullptr;
       if (cudaGetSymbolAddress(&p, g_attend_static_partials) != cudaSuccess || !p) return FATHOM_ERR_CUDA;
+      if (cudaGetSymbolAddress(&t, g_attend_static_tickets) != cudaSuccess || !t) return FATHOM_ERR_CUDA;
+      g_static_tickets_ptr[dev] = static_cast<unsigned int*>(t);
       g_static_partials_ptr[dev] = static_cast<float*>(p);
     }
     partial = g_static_partials_ptr[dev];
+    tickets = g_static_tickets_ptr[dev];
   }
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -204,12 +225,11 @@ extern "C" int fathom_sparse_attend_static(const fathom_layout* L, const float* 
   if (row_dtype == FATHOM_BF16)
     attend_partial_kernel<__nv_bfloat16><<<grid, AT_THREADS, 0, st>>>(
         q, static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k, L->n, G,
-        softmax_scale, partial, splits);
+        softmax_scale, partial, splits, tickets, out);
   else
     attend_partial_kernel<float><<<grid, AT_THREADS, 0, st>>>(q, static_cast<const float*>(Krows),
                                                               static_cast<const float*>(Vrows), idx, k, L->n, G,
-                                                              softmax_scale, partial, splits);
-  attend_combine_kernel<<<Hq, FATHOM_D, 0, st>>>(partial, splits, out);
+                                                              softmax_scale, partial, splits, tickets, out);
   if (cudaGetLastError() != cudaSuccess) return FATHOM_ERR_CUDA;
   return FATHOM_OK;
 }
