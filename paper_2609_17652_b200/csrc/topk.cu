@@ -219,17 +219,47 @@ __device__ __forceinline__ uint64_t composite52(const float* row, int32_t i) {
   return ((((uint64_t)ordered_key(row[i])) << 32) | (uint32_t)(~(uint32_t)i)) & ((1ull << 52) - 1ull);
 }
 
+// Exclusive prefix over the block of one value per thread (warp shuffles + one shared array of 32 warp totals).
+// Returns the exclusive prefix; *total receives the block sum.  Two __syncthreads.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t w = s_warp[lane];
+    uint32_t wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    s_warp[lane] = wi - w;
+    if (lane == 31) s_warp[32] = wi;
+  }
+  __syncthreads();
+  *total = s_warp[32];
+  return s_warp[warp] + incl - v;
+}
+
 __global__ void __launch_bounds__(FIN_THREADS)
 topk_finish_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    const uint32_t* __restrict__ state, const int32_t* __restrict__ cand,
                    uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
                    uint32_t* __restrict__ dev_status) {
+  constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
+  constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   __shared__ uint64_t s_comp[FIN_CACHE];
-  __shared__ uint32_t s_hist[256];
-  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_hist[DIGITS];
+  __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
-  __shared__ uint32_t s_need, s_digit, s_bucket;
-  const int head = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ uint32_t s_need, s_bucket;
+  const int head = blockIdx.x, tid = threadIdx.x;
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const int32_t* cand_h = cand + (size_t)head * (size_t)n;
   uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
@@ -239,53 +269,44 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
   if (cached)
     for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite52(row, cand_h[c]);
 
-  // ---- radix select of the need0 largest composites among the m candidates; digits are taken from bit 52
-  //      downwards (4 bits first, then 8 at a time) until the chosen bucket is taken whole.
+  // ---- radix select of the need0 largest composites among the m candidates: 11-bit digits from bit 52
+  //      downwards (the last digit is 8 bits) until the chosen bucket is taken whole.
   uint64_t thr = 0;                                           // chosen candidates: composite >= thr
   if (need0 > 0 && need0 < m) {
     if (tid == 0) { s_prefix = 0; s_need = need0; }
     int hi = 52;
     while (hi > 0) {
-      const int bits = (hi % 8) ? (hi % 8) : 8;
+      const int bits = min(DIGIT_BITS, hi);
       const int lo = hi - bits;
-      if (tid < 256) s_hist[tid] = 0u;
+      for (int d = tid; d < DIGITS; d += FIN_THREADS) s_hist[d] = 0u;
       __syncthreads();
       const uint64_t prefix = s_prefix;
+      const uint32_t need = s_need;
       for (uint32_t c = tid; c < m; c += FIN_THREADS) {
         const uint64_t comp = cached ? s_comp[c] : composite52(row, cand_h[c]);
         if ((comp >> hi) == (prefix >> hi)) atomicAdd(&s_hist[(uint32_t)(comp >> lo) & ((1u << bits) - 1u)], 1u);
       }
       __syncthreads();
-      if (tid < 32) {                                         // warp 0: suffix counts over the 256 digits
-        uint32_t cnt[8], local = 0;
+      // thread t owns digits DIGITS-1-DPT*t .. (descending): the block prefix is a suffix count
+      uint32_t cnt[DPT], local = 0;
 #pragma unroll
-        for (int x = 0; x < 8; ++x) { cnt[x] = s_hist[255 - (8 * tid + x)]; local += cnt[x]; }
-        uint32_t incl = local;
+      for (int x = 0; x < DPT; ++x) { cnt[x] = s_hist[DIGITS - 1 - (DPT * tid + x)]; local += cnt[x]; }
+      uint32_t total;
+      uint32_t run = block_exclusive_scan(local, s_warp, &total);
+      if (run < need && run + local >= need) {
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-          if (tid >= o) incl += y;
-        }
-        const uint32_t need = s_need;
-        uint32_t run = incl - local;
-        if (run < need && run + local >= need) {
-#pragma unroll
-          for (int x = 0; x < 8; ++x) {
-            if (run < need && run + cnt[x] >= need) {
-              s_digit = 255 - (8 * tid + x);
-              s_need = need - run;                            // still needed from inside the chosen digit
-              s_bucket = cnt[x];
-            }
-            run += cnt[x];
+        for (int x = 0; x < DPT; ++x) {
+          if (run < need && run + cnt[x] >= need) {
+            s_prefix = prefix | ((uint64_t)(DIGITS - 1 - (DPT * tid + x)) << lo);
+            s_need = need - run;                              // still needed from inside the chosen digit
+            s_bucket = cnt[x];
           }
+          run += cnt[x];
         }
       }
       __syncthreads();
-      if (tid == 0) s_prefix |= (uint64_t)s_digit << lo;
-      const bool whole = s_need == s_bucket;                  // the chosen bucket is taken entirely: done
-      __syncthreads();
       hi = lo;
-      if (whole) break;
+      if (s_need == s_bucket) break;                          // the chosen bucket is taken entirely: done
     }
     thr = s_prefix;                                           // undecided low bits are zero
   }
@@ -304,63 +325,46 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
   }
   __syncthreads();
 
-  // ---- ascending emission: thread t owns a contiguous run of 128-token groups (4 bitmap words each)
+  // ---- ascending emission.  128-token groups (4 bitmap words each) are dealt to threads round-robin in
+  //      rounds of FIN_THREADS groups, so every load of a warp is 512 contiguous bytes; within a round the
+  //      thread order is the token order, and the rounds follow one another.
   const long long groups = (n + 127) / 128;
-  const long long per = (groups + FIN_THREADS - 1) / FIN_THREADS;
-  const long long g0 = min((long long)tid * per, groups), g1 = min(g0 + per, groups);
   const uint4* bm4 = reinterpret_cast<const uint4*>(bm);
-  constexpr int REG_GROUPS = 8;                               // groups kept in registers between count and emit
-  uint4 keep[REG_GROUPS];
-  uint32_t cnt = 0;
-#pragma unroll
-  for (int x = 0; x < REG_GROUPS; ++x) {
-    keep[x] = (g0 + x < g1) ? bm4[g0 + x] : make_uint4(0u, 0u, 0u, 0u);
-    cnt += __popc(keep[x].x) + __popc(keep[x].y) + __popc(keep[x].z) + __popc(keep[x].w);
-  }
-  for (long long g = g0 + REG_GROUPS; g < g1; ++g) {
-    const uint4 w = bm4[g];
-    cnt += __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
-  }
-  uint32_t incl = cnt;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const uint32_t w = s_warp[lane];
-    uint32_t wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    s_warp[lane] = wi - w;
-    if (lane == 31 && wi != (uint32_t)k) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
-  }
-  __syncthreads();
-  uint32_t pos = s_warp[warp] + incl - cnt;
   int32_t* out = idx_out + (size_t)head * k;
-  auto emit_group = [&](long long g, const uint4 w) {
-    uint32_t any = w.x | w.y | w.z | w.w;
-    while (any) {
-      const int l = __ffs(any) - 1;
-      any &= any - 1;
-      const int32_t t = (int32_t)(g * 128 + 4 * l);
-      if ((w.x >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t; ++pos; }
-      if ((w.y >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 1; ++pos; }
-      if ((w.z >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 2; ++pos; }
-      if ((w.w >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 3; ++pos; }
-    }
-  };
+  uint32_t base = 0;
+  constexpr int ROUNDS_AT_ONCE = 8;
+  for (long long g0 = 0; g0 < groups; g0 += (long long)ROUNDS_AT_ONCE * FIN_THREADS) {
+    uint4 w[ROUNDS_AT_ONCE];
+    uint32_t cnt[ROUNDS_AT_ONCE];
 #pragma unroll
-  for (int x = 0; x < REG_GROUPS; ++x)
-    if (g0 + x < g1) emit_group(g0 + x, keep[x]);
-  for (long long g = g0 + REG_GROUPS; g < g1; ++g) emit_group(g, bm4[g]);
-  if (tid == FIN_THREADS - 1)                                 // short selection (non-finite scores): pad with the last token
-    for (uint32_t e = pos; e < (uint32_t)k; ++e) out[e] = (int32_t)(n - 1);
+    for (int x = 0; x < ROUNDS_AT_ONCE; ++x) {
+      const long long g = g0 + (long long)x * FIN_THREADS + tid;
+      w[x] = (g < groups) ? bm4[g] : make_uint4(0u, 0u, 0u, 0u);
+      cnt[x] = __popc(w[x].x) + __popc(w[x].y) + __popc(w[x].z) + __popc(w[x].w);
+    }
+#pragma unroll
+    for (int x = 0; x < ROUNDS_AT_ONCE; ++x) {
+      if (g0 + (long long)x * FIN_THREADS >= groups) break;   // uniform
+      uint32_t total;
+      uint32_t pos = base + block_exclusive_scan(cnt[x], s_warp, &total);
+      base += total;
+      const long long g = g0 + (long long)x * FIN_THREADS + tid;
+      uint32_t any = w[x].x | w[x].y | w[x].z | w[x].w;
+      while (any) {
+        const int l = __ffs(any) - 1;
+        any &= any - 1;
+        const int32_t t = (int32_t)(g * 128 + 4 * l);
+        if ((w[x].x >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t; ++pos; }
+        if ((w[x].y >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 1; ++pos; }
+        if ((w[x].z >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 2; ++pos; }
+        if ((w[x].w >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 3; ++pos; }
+      }
+    }
+  }
+  if (base != (uint32_t)k && tid == 0) {                      // short (non-finite scores) or long selection
+    atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+    for (uint32_t e = base; e < (uint32_t)k; ++e) out[e] = (int32_t)(n - 1);   // pad with the last token
+  }
 }
 
 }  // namespace
