@@ -66,7 +66,7 @@ struct alignas(16) WarpSmem {
 };
 
 template <int NH>
-__global__ void __launch_bounds__(SCAN_THREADS)
+__global__ void __launch_bounds__(SCAN_THREADS, 8)              // 64 registers: occupancy matters more than spills here
 scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
             const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
             long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
