@@ -190,3 +190,32 @@ def test_determinism_two_runs_same_bytes():
     b = run_gpu(L, 48, 256, 4)
     for key in ("planes", "depth", "scores", "idx", "out"):
         assert np.array_equal(a[key], b[key]), key
+
+
+def test_multi_session_batch_with_host_resident_planes():
+    """A small stand-in for the agentic multi-session batch: several sessions of ragged, log-uniform lengths,
+    two independently seeded layers each, planes read zero-copy from pinned host memory."""
+    from workloads.synth import session_lengths
+    lengths = session_lengths(4, lo=1000, hi=20000, seed=3)
+    assert len(set(n % 64 for n in lengths)) > 1                       # not forced to multiples of 64
+    for s, n in enumerate(lengths):
+        for layer in range(2):
+            L = make_layer(n, Hkv=2, Hq=8, seed=12, session=s, layer=layer, device="cuda")
+            check_all(L, B=48, k=min(256, n), hpp=4, host_planes=True)
+
+
+def test_non_finite_scores_raise_the_short_flag():
+    from paper_2609_17652_b200 import binding as fb
+    n, Hq, k = 5000, 2, 64
+    lay = fb.make_layout(1, Hq, n)
+    s = torch.randn(Hq, lay.score_stride, device="cuda")
+    s[1, :n - 10] = float("nan")                                        # head 1 has only 10 finite scores
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    ctx.fathom_topk(lay, s, k, 0, 0, idx)
+    assert ctx.fathom_device_status() & fb.DEV_TOPK_SHORT
+    got = idx.cpu().numpy()
+    assert np.array_equal(got[0], O.topk(s[:1, :n].cpu().numpy().astype(np.float64), k)[0])   # the finite head is unaffected
+    assert np.all((got[1] >= 0) & (got[1] < n))                         # padded with a valid index, never out of range
+    assert ctx.fathom_device_status() == 0                              # reading the word clears it
+    ctx.close()
