@@ -374,3 +374,30 @@ def exact_scores(q, Krows) -> np.ndarray:
     Hkv = Krows.shape[0]
     G = Hq // Hkv
     return np.stack([np.asarray(Krows[h // G], dtype=np.float64) @ q[h] for h in range(Hq)])
+
+
+# --------------------------------------------------------------------------
+# O6  union of a group's winners  (Sec. 1: the union of the G heads' winners is fetched once per KV head;
+#     Sec. 4 "Offload harness": "the gather of the union of the selected rows")
+# --------------------------------------------------------------------------
+def gather_union(idx: np.ndarray, G: int, Krows, Vrows):
+    """O6: per KV head kv, the ascending list u of distinct tokens picked by its G query heads, the rows
+    K[kv][u], V[kv][u], and every pick rewritten as its position in u.
+    Returns (ulists [list of arrays], K_stage [list], V_stage [list], idx_local [Hq][k] int32)."""
+    idx = np.asarray(idx)
+    Hq, k = idx.shape
+    Hkv = Hq // G
+    ulists, Ks, Vs = [], [], []
+    idx_local = np.empty((Hq, k), dtype=np.int32)
+    for kv in range(Hkv):
+        picks = set()
+        for h in range(kv * G, (kv + 1) * G):
+            picks |= set(int(t) for t in idx[h])
+        u = np.array(sorted(picks), dtype=np.int64)
+        pos = {int(t): p for p, t in enumerate(u)}
+        for h in range(kv * G, (kv + 1) * G):
+            idx_local[h] = [pos[int(t)] for t in idx[h]]
+        ulists.append(u)
+        Ks.append(np.asarray(Krows[kv])[u])
+        Vs.append(np.asarray(Vrows[kv])[u])
+    return ulists, Ks, Vs, idx_local

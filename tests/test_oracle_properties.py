@@ -329,3 +329,31 @@ def test_needles_are_selected_at_B48():
     s = O.scan(planes, scales, L.q.numpy(), dep, 4096, 1)
     idx = O.topk(s, 64)
     assert set(L.needles[0].tolist()) <= set(idx[0].tolist())
+
+
+# ---------------------------------------------------------------- O6 union of winners
+def test_union_of_winners_properties():
+    r = np.random.default_rng(9)
+    Hkv, G, n, k, d = 3, 4, 500, 60, 8
+    Kr = r.standard_normal((Hkv, n, d)).astype(np.float32)
+    Vr = r.standard_normal((Hkv, n, d)).astype(np.float32)
+    q = r.standard_normal((Hkv * G, d)).astype(np.float32)
+    idx = np.stack([np.sort(r.permutation(n)[:k]) for _ in range(Hkv * G)]).astype(np.int32)
+    idx[1] = idx[0]                                           # two heads with identical picks
+    ul, Ks, Vs, loc = O.gather_union(idx, G, Kr, Vr)
+    for kv in range(Hkv):
+        u = ul[kv]
+        assert np.all(np.diff(u) > 0) and k <= len(u) <= G * k             # ascending, distinct, bounded
+        assert np.array_equal(u, np.unique(idx[kv * G:(kv + 1) * G]))       # library routine on the definition
+        for h in range(kv * G, (kv + 1) * G):
+            assert np.array_equal(u[loc[h]], idx[h])                        # positions map back to the picks
+        assert np.array_equal(Ks[kv], Kr[kv][u]) and np.array_equal(Vs[kv], Vr[kv][u])
+    assert len(ul[0]) <= 3 * k                                              # the duplicate head adds nothing
+    # attention over the staged rows with the local indices is the attention over the original rows
+    a = O.sparse_attend(q, Kr, Vr, idx, 0.3)
+    cap = max(len(u) for u in ul)
+    Kst = np.zeros((Hkv, cap, d), np.float32); Vst = np.zeros((Hkv, cap, d), np.float32)
+    for kv in range(Hkv):
+        Kst[kv, :len(ul[kv])] = Ks[kv]; Vst[kv, :len(ul[kv])] = Vs[kv]
+    b = O.sparse_attend(q, Kst, Vst, loc, 0.3)
+    assert np.array_equal(a, b)
