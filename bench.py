@@ -264,6 +264,8 @@ def run_ours(args):
     # ---- planes in pinned host memory, read zero-copy by the scan kernel over the host link
     if rank == 0 and not args.no_host_resident:
         result["host_resident_scan"] = host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, plane_bytes_read)
+        result["host_resident_row_fetch"] = row_fetch_leg(ctx, lay, L, idx, k, G, stream,
+                                                          result["host_resident_scan"]["link_peak_gbs"])
 
     # ---- end to end through the C ABI from HOST buffers: H2D of the step's inputs and D2H of its result are timed
     if not args.no_e2e:
@@ -308,6 +310,33 @@ def host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, p
     return {"scan_ms": round(t, 4), "bytes_over_link": plane_bytes_read, "gbs": round(gbs, 2),
             "link_peak_gbs": round(link_gbs, 2), "frac_of_measured_link": round(gbs / link_gbs, 4),
             "link_probe": "1 GiB pinned->device copy, best of 10"}
+
+
+def row_fetch_leg(ctx, lay, L, idx, k, G, stream, link_gbs):
+    """K/V rows in pinned host memory: the union of each group's winners is fetched once over the host link."""
+    hK = torch.empty(L.Krows.shape, dtype=L.Krows.dtype, pin_memory=True); hK.copy_(L.Krows)
+    hV = torch.empty(L.Vrows.shape, dtype=L.Vrows.dtype, pin_memory=True); hV.copy_(L.Vrows)
+    dev = L.Krows.device
+    Kst = torch.empty((L.Hkv, G * k, L.d), dtype=L.Krows.dtype, device=dev)
+    Vst = torch.empty_like(Kst)
+    loc = torch.empty((L.Hq, k), dtype=torch.int32, device=dev)
+    cnt = torch.zeros((L.Hkv,), dtype=torch.int32, device=dev)
+    ts = []
+    for it in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        ctx.fathom_gather_union(lay, idx, k, hK, hV, Kst, Vst, loc, cnt, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            ts.append(a.elapsed_time(b))
+    t = statistics.median(ts)
+    rows = int(cnt.sum().item())
+    nbytes = rows * L.d * 2 * L.Krows.element_size()
+    gbs = nbytes / (t * 1e-3) / 1e9
+    del hK, hV
+    return {"ms": round(t, 4), "distinct_rows": rows, "picks": int(L.Hq * k), "bytes_over_link": nbytes,
+            "gbs": round(gbs, 2), "frac_of_measured_link": round(gbs / link_gbs, 4)}
 
 
 def e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step):

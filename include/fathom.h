@@ -147,6 +147,24 @@ int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* layout, const flo
                          const void* Krows, const void* Vrows, int row_dtype, const int32_t* idx,
                          int k, float softmax_scale, float* out, void* stream);
 
+/* ---- (6) union of a group's winners, fetched once — Sec. 1 and Sec. 4 "Offload harness" ---------
+ * The G query heads of a KV head mostly pick overlapping tokens; the offloaded decode step fetches the
+ * distinct rows of each KV head once (at most G * k of them) and runs attention on the fetched copy.
+ * For every KV head this call forms the ascending list of distinct tokens in idx[kv*G .. kv*G+G-1][*],
+ * copies their K and V rows into the staging buffers in that order, and rewrites every pick as its position
+ * in the staged rows.  Attention over (K_stage, V_stage, idx_local) with a layout whose n is G * k gives
+ * bit for bit what attention over (Krows, Vrows, idx) gives.
+ *   idx          in   [Hq][k] int32 (each list without repeats, e.g. from fathom_topk)
+ *   Krows, Vrows in   [Hkv][n][d] FATHOM_BF16 or FATHOM_F32, device memory or device-addressable pinned host
+ *                     memory (then each distinct row crosses the host link exactly once), 16-byte aligned
+ *   K_stage, V_stage out [Hkv][G * k][d] same dtype, device; rows beyond union_count[kv] are not written
+ *   idx_local    out  [Hq][k] int32, positions in [0, union_count[kv])
+ *   union_count  out  [Hkv] int32
+ * Uses the context scratch (fathom_scratch_bytes). */
+int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int32_t* idx, int k,
+                        const void* Krows, const void* Vrows, int row_dtype, void* K_stage, void* V_stage,
+                        int32_t* idx_local, int32_t* union_count, void* stream);
+
 /* ---- (5b) gather + exact attention without any allocation — the paper has no counterpart ------
  * Same computation, arguments and results as fathom_sparse_attend, for callers that cannot obtain device
  * memory of their own: a plug-in that is only handed buffers by its host application, a serving process

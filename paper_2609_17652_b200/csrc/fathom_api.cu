@@ -43,7 +43,9 @@ size_t fathom_scratch_bytes(const fathom_layout* L, int k) {
   if (fathom_check_layout(L) != FATHOM_OK || k < 1) return 0;
   size_t a = fathom_carve_topk(nullptr, L->n_q_heads, L->n, k).bytes;
   size_t b = fathom_carve_attn(nullptr, L->n_q_heads, k).bytes;
-  return a > b ? a : b;
+  size_t c = fathom_union_scratch_bytes(L->n_kv_heads, L->n, (L->n_q_heads / L->n_kv_heads) * k);
+  size_t m = a > b ? a : b;
+  return m > c ? m : c;
 }
 
 int fathom_create(fathom_ctx** out, int device, size_t scratch_bytes) {

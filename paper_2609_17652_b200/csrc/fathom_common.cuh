@@ -60,3 +60,4 @@ struct fathom_attn_scratch {
 };
 fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k);
 fathom_attn_scratch fathom_carve_attn(void* base, int Hq, int k);
+size_t fathom_union_scratch_bytes(int Hkv, long long n, int capacity);   // bitmap + word ranks + union list

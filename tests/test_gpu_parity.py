@@ -219,3 +219,49 @@ def test_non_finite_scores_raise_the_short_flag():
     assert np.all((got[1] >= 0) & (got[1] < n))                         # padded with a valid index, never out of range
     assert ctx.fathom_device_status() == 0                              # reading the word clears it
     ctx.close()
+
+
+@pytest.mark.parametrize("rows_on_host,dtype", [(False, torch.bfloat16), (True, torch.bfloat16), (False, torch.float32)])
+def test_union_of_winners_fetched_once(rows_on_host, dtype):
+    """fathom_gather_union against the oracle (bit-exact lists, counts, positions and staged rows), and attention
+    over the staged rows against attention over the original rows (identical)."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hkv, Hq, k, G = 9000, 2, 8, 300, 4
+    L = make_layer(n, Hkv, Hq, seed=21, device="cuda")
+    g = run_gpu(L, 48, k, G)                                            # real top-k lists (heads of a group overlap)
+    idx = torch.from_numpy(g["idx"]).cuda()
+    Kr = L.Krows if dtype == torch.bfloat16 else L.K
+    Vr = L.Vrows if dtype == torch.bfloat16 else L.Vrows.float()
+    if rows_on_host:
+        hK = torch.empty(Kr.shape, dtype=dtype, pin_memory=True); hK.copy_(Kr)
+        hV = torch.empty(Vr.shape, dtype=dtype, pin_memory=True); hV.copy_(Vr)
+        Ksrc, Vsrc = hK, hV
+    else:
+        Ksrc, Vsrc = Kr, Vr
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    cap = G * k
+    Kst = torch.full((Hkv, cap, 128), 7.0, dtype=dtype, device="cuda")
+    Vst = torch.full((Hkv, cap, 128), 7.0, dtype=dtype, device="cuda")
+    loc = torch.full((Hq, k), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((Hkv,), -1, dtype=torch.int32, device="cuda")
+    ctx.fathom_gather_union(lay, idx, k, Ksrc, Vsrc, Kst, Vst, loc, cnt, row_dtype=fb.BF16 if dtype == torch.bfloat16 else fb.F32)
+    # attention over the staged rows (layout with n = G * k) vs attention over the original rows
+    lay2 = fb.make_layout(Hkv, Hq, cap)
+    o_direct = torch.zeros((Hq, 128), device="cuda"); o_staged = torch.zeros((Hq, 128), device="cuda")
+    ctx.fathom_sparse_attend(lay, L.q, Kr, Vr, idx, k, 1 / math.sqrt(128), o_direct)
+    torch.cuda.synchronize()
+    ctx.fathom_sparse_attend(lay2, L.q, Kst, Vst, loc, k, 1 / math.sqrt(128), o_staged)
+    torch.cuda.synchronize()
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+    ul, Ks, Vs, loc_ref = O.gather_union(g["idx"], G, Kr.float().cpu().numpy(), Vr.float().cpu().numpy())
+    assert np.array_equal(cnt.cpu().numpy(), [len(u) for u in ul])
+    assert np.array_equal(loc.cpu().numpy(), loc_ref)
+    for kv in range(Hkv):
+        c = len(ul[kv])
+        assert c < cap                                                  # the group's picks do overlap
+        assert np.array_equal(Kst[kv, :c].float().cpu().numpy(), Ks[kv])
+        assert np.array_equal(Vst[kv, :c].float().cpu().numpy(), Vs[kv])
+        assert np.all(Kst[kv, c:].float().cpu().numpy() == 7.0)         # rows past the union are untouched
+    assert np.array_equal(o_direct.cpu().numpy(), o_staged.cpu().numpy())
