@@ -100,7 +100,11 @@ int fathom_version(void);
  *   K       in   [Hkv][n][d], token-major, k_dtype FATHOM_F32 or FATHOM_BF16, 16-byte aligned
  *   planes  out  [Hkv][d][4][plane_stride_words] uint64; words beta >= nb of a row are not written
  *   scales  out  [Hkv][d][scale_stride] fp16 bit patterns; elements beta >= nb are not written
- * A prefix of t planes of a channel is its t-bit mid-rise quantiser with the same block scale. */
+ * A prefix of t planes of a channel is its t-bit mid-rise quantiser with the same block scale.
+ * Appending keys (the paper does not cover it): new tokens can raise the maximum of the last, partly filled
+ * block, so that block must be re-quantised; earlier blocks never change.  Call this function on the tail only:
+ * per KV head, pass K, planes and scales advanced to block b0 = 8 * (old_block_count / 8) (a multiple of 8 keeps
+ * all three pointers 16-byte aligned), n = new_n - 64 * b0, n_kv_heads = 1 and the store's own strides. */
 int fathom_build_planes(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype,
                         uint64_t* planes, uint16_t* scales, void* stream);
 

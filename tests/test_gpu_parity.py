@@ -265,3 +265,35 @@ def test_union_of_winners_fetched_once(rows_on_host, dtype):
         assert np.array_equal(Vst[kv, :c].float().cpu().numpy(), Vs[kv])
         assert np.all(Kst[kv, c:].float().cpu().numpy() == 7.0)         # rows past the union are untouched
     assert np.array_equal(o_direct.cpu().numpy(), o_staged.cpu().numpy())
+
+
+def test_appending_keys_rebuilds_only_the_tail():
+    """Incremental append (the paper is silent; a serving stack needs it): new keys can raise the maximum of the
+    last, partly filled block, so that block is re-quantised.  Rebuilding from a block index that is a multiple of
+    8 keeps every pointer 16-byte aligned, and the result equals a build of the whole sequence."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, n1, n2 = 2, 5000, 5300                                        # 5000 tokens, then 300 more
+    L = make_layer(n2, Hkv, 8, seed=31, device="cuda")
+    lay2 = fb.make_layout(Hkv, 8, n2)
+    ctx = fb.Context(0, 0)
+    shape_p, shape_s = (Hkv, 128, 4, lay2.plane_stride_words), (Hkv, 128, lay2.scale_stride)
+    full_p = torch.zeros(shape_p, dtype=torch.int64, device="cuda"); full_s = torch.zeros(shape_s, dtype=torch.int16, device="cuda")
+    ctx.fathom_build_planes(lay2, L.K, full_p, full_s)
+    # store built for the first n1 tokens (same strides, sized for n2) ...
+    inc_p = torch.zeros(shape_p, dtype=torch.int64, device="cuda"); inc_s = torch.zeros(shape_s, dtype=torch.int16, device="cuda")
+    lay1 = fb.make_layout(Hkv, 8, n1)
+    lay1.plane_stride_words, lay1.scale_stride = lay2.plane_stride_words, lay2.scale_stride
+    K1 = L.K[:, :n1].contiguous()
+    ctx.fathom_build_planes(lay1, K1, inc_p, inc_s)
+    # ... then the tail from block b0 = 8 * floor(floor(n1 / 64) / 8) on, one KV head at a time (a head's tokens are
+    # contiguous in K, and its plane / scale rows keep their strides)
+    b0 = (n1 // 64) // 8 * 8
+    tail = fb.make_layout(1, 1, n2 - b0 * 64)
+    tail.plane_stride_words, tail.scale_stride = lay2.plane_stride_words, lay2.scale_stride
+    for kv in range(Hkv):
+        ctx.fathom_build_planes(tail, L.K[kv, b0 * 64:].contiguous(), inc_p[kv, :, :, b0:].data_ptr(), inc_s[kv, :, b0:].data_ptr(),
+                                k_dtype=fb.F32)
+    torch.cuda.synchronize()
+    nb = (n2 + 63) // 64
+    assert torch.equal(inc_p[..., :nb], full_p[..., :nb]) and torch.equal(inc_s[..., :nb], full_s[..., :nb])
+    ctx.close()
