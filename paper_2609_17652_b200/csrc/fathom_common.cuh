@@ -50,6 +50,7 @@ struct fathom_topk_scratch {
   uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 4 candidates written
   uint32_t* bitmap;      // [Hq][bitmap_words] selection bitmap, token i at bit (i % 32) of word i / 32
   int32_t* cand;         // [Hq][n] token indices of the threshold bin
+  uint32_t* tile_count;  // [Hq][ceil(n / 8192)] selected tokens per filter tile, then their exclusive prefix
   long long bitmap_words;
   size_t bytes;
 };

@@ -1,16 +1,18 @@
 // fathom_topk: per-query-head top-k over n scores with deterministic ties (Sec. 2 "Top-k decoding").
 //
 // Bucket select on the order-preserving integer image of the fp32 score (-0 folded onto +0):
-//   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores);
-//   2. per head, the threshold bin b* whose suffix count first reaches the number wanted;
+//   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores); the CTA that
+//      finishes a head's histogram last (ticket counter) finds
+//   2. the threshold bin b* whose suffix count first reaches the number wanted;
 //   3. filter (second read): a lane owns four consecutive tokens (one 16-byte load) and compares them with
 //      the two fp32 edges of bin b*; the warp ballots of "above b*" ARE the words of a selection bitmap
 //      (word c of a 128-token group holds tokens 4 l + c at bit l), written without atomics; tokens inside
 //      bin b* are candidates, appended with warp-aggregated atomics (ballot + popc), order irrelevant;
 //   4. per head, a radix select over the candidates on the 64-bit composite (key << 32 | ~index), which
 //      makes every element distinct and encodes "ties go to the lower token index"; the chosen
-//      candidates and the forced sink/local tokens are OR-ed into the bitmap, and the k indices are
-//      emitted in ascending order by a popcount prefix sum over the bitmap words.
+//      candidates and the forced sink/local tokens are OR-ed into the bitmap and added to the per-tile
+//      counts the filter left behind, whose prefix sum gives every tile its place in the output;
+//   5. one small CTA per 8192-token tile emits its indices in ascending order (popcount prefix in the tile).
 // The selected set is unique, so neither the append order nor atomics can show in the output.
 #include "fathom_common.cuh"
 
@@ -32,10 +34,15 @@ __device__ __forceinline__ uint32_t ordered_key(float f) {
 
 struct Forced { long long sink_end, local_begin; };          // eligible tokens: sink_end <= i < local_begin
 
+__device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp);
+
 __global__ void __launch_bounds__(HIST_THREADS)
 topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
-                 uint32_t* __restrict__ hist) {
+                 uint32_t* __restrict__ hist, uint32_t* __restrict__ state, uint32_t want,
+                 uint32_t* __restrict__ dev_status) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
+  __shared__ bool s_last;
   const int head = blockIdx.y;
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) sh[b] = 0u;
   __syncthreads();
@@ -70,58 +77,56 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
     const uint32_t c = sh[b];
     if (c) atomicAdd(&g[b], c);
   }
+  // the CTA that draws the head's last ticket sees the complete histogram and finds the threshold bin
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&state[head * 8 + 5], 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  find_threshold_bin(g, state + head * 8, want, dev_status, sh);
 }
 
 // state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it,
-// [4] = candidates appended by the filter
-__global__ void __launch_bounds__(FIN_THREADS)
-topk_find_bin_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ state, uint32_t want,
-                     uint32_t* __restrict__ dev_status) {
-  __shared__ uint32_t warp_sum[32];
-  const int head = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t* h = hist + (size_t)head * FATHOM_TOPK_BINS;
-  // thread t owns bins 4095 - 4t .. 4092 - 4t (descending), so an inclusive scan over threads is a suffix count
-  uint32_t c[4], local = 0;
+// [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
+// Run by the HIST_THREADS threads of the CTA that completed the head's histogram: thread t owns bins
+// 4095 - 16 t .. 4080 - 16 t (descending), so a block prefix over threads is a suffix count over bins.
+__device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp) {
+  constexpr int BPT = FATHOM_TOPK_BINS / HIST_THREADS;        // 16 bins per thread
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (want == 0) {                                            // nothing to select: no bin is above or equal
+    if (tid == 0) { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
+    return;
+  }
+  uint32_t c[BPT], local = 0;
 #pragma unroll
-  for (int x = 0; x < 4; ++x) { c[x] = h[FATHOM_TOPK_BINS - 1 - (4 * tid + x)]; local += c[x]; }
+  for (int x = 0; x < BPT; ++x) { c[x] = __ldcg(h + (FATHOM_TOPK_BINS - 1 - (BPT * tid + x))); local += c[x]; }
   uint32_t incl = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += y;
   }
-  if (lane == 31) warp_sum[warp] = incl;
+  if (lane == 31) s_warp[warp] = incl;
   __syncthreads();
-  if (warp == 0) {
-    uint32_t w = warp_sum[lane], wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    warp_sum[lane] = wi - w;                                  // exclusive
-  }
-  __syncthreads();
-  const uint32_t above = warp_sum[warp] + incl - local;       // tokens in bins above this thread's four
-  if (want == 0) {                                            // nothing to select: no bin is above or equal
-    if (tid == 0) { state[head * 8 + 0] = FATHOM_TOPK_BINS; state[head * 8 + 1] = 0; state[head * 8 + 2] = 0; }
-    return;
-  }
+  uint32_t above = incl - local;
+  for (int w = 0; w < warp; ++w) above += s_warp[w];          // 8 warps: a short serial carry
   if (above < want && above + local >= want) {
     uint32_t run = above;
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
+    for (int x = 0; x < BPT; ++x) {
       if (run < want && run + c[x] >= want) {
-        state[head * 8 + 0] = (uint32_t)(FATHOM_TOPK_BINS - 1 - (4 * tid + x));
-        state[head * 8 + 1] = run;
-        state[head * 8 + 2] = want - run;
+        st[0] = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
+        st[1] = run;
+        st[2] = want - run;
       }
       run += c[x];
     }
   }
-  if (tid == FIN_THREADS - 1 && above + local < want) {       // fewer eligible tokens than wanted: take them all
+  if (tid == HIST_THREADS - 1 && above + local < want) {      // fewer eligible tokens than wanted: take them all
     atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
-    state[head * 8 + 0] = 0; state[head * 8 + 1] = above + local - c[3]; state[head * 8 + 2] = c[3];
+    st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1];
   }
 }
 
@@ -137,11 +142,11 @@ __device__ __forceinline__ uint32_t bitmap_bit(long long t) { return 1u << ((t &
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_filter_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    uint32_t* __restrict__ state, int32_t* __restrict__ cand, uint32_t* __restrict__ bitmap,
-                   long long bitmap_words) {
+                   long long bitmap_words, uint32_t* __restrict__ tile_count) {
   __shared__ uint16_t s_list[FILT_TILE];                      // candidates of this tile, as offsets from its first token
-  __shared__ uint32_t s_count, s_base;
+  __shared__ uint32_t s_count, s_base, s_sel;
   const int head = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) s_count = 0u;
+  if (threadIdx.x == 0) { s_count = 0u; s_sel = 0u; }
   __syncthreads();
   const uint32_t bstar = state[head * 8 + 0];
   // bin b* is [lo, hi) in fp32 order; for finite scores "key >> 20 > b*" <=> s >= hi and "== b*" <=> lo <= s < hi.
@@ -204,8 +209,15 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
     }
   }
   if (wbase < n) bm[wbase / 32 + lane] = my_word;             // 32 consecutive words, one coalesced store
+  {                                                           // tokens of this tile selected so far (bins above b*)
+    uint32_t c = __popc(my_word);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if (lane == 0 && c) atomicAdd(&s_sel, c);
+  }
   // one global atomic per tile reserves the slice of the head's candidate list
   __syncthreads();
+  if (threadIdx.x == 0) tile_count[(size_t)head * gridDim.x + blockIdx.x] = s_sel;
   const uint32_t cnt = s_count;
   if (cnt == 0u) return;
   if (threadIdx.x == 0) s_base = atomicAdd(&state[head * 8 + 4], cnt);
@@ -248,10 +260,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
 }
 
 __global__ void __launch_bounds__(FIN_THREADS)
-topk_finish_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
+topk_select_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    const uint32_t* __restrict__ state, const int32_t* __restrict__ cand,
                    uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
-                   uint32_t* __restrict__ dev_status) {
+                   uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   __shared__ uint64_t s_comp[FIN_CACHE];
@@ -263,6 +275,7 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const int32_t* cand_h = cand + (size_t)head * (size_t)n;
   uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
+  uint32_t* tc = tile_count + (size_t)head * ntiles;
   const uint32_t m = state[head * 8 + 4];
   const uint32_t need0 = min(state[head * 8 + 2], m);
   const bool cached = m <= FIN_CACHE;
@@ -314,7 +327,10 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
     for (uint32_t c = tid; c < m; c += FIN_THREADS) {
       const int32_t i = cand_h[c];
       const uint64_t comp = cached ? s_comp[c] : composite52(row, i);
-      if (need0 >= m || comp >= thr) atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
+      if (need0 >= m || comp >= thr) {
+        atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
+        atomicAdd(&tc[i / FILT_TILE], 1u);
+      }
     }
   }
   // ---- forced sink / local tokens
@@ -322,48 +338,61 @@ topk_finish_kernel(const float* __restrict__ scores, long long n, long long scor
   for (long long e = tid; e < n_forced; e += FIN_THREADS) {
     const long long i = (e < F.sink_end) ? e : (F.local_begin + (e - F.sink_end));
     atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
+    atomicAdd(&tc[i / FILT_TILE], 1u);
   }
+  __threadfence();
   __syncthreads();
 
-  // ---- ascending emission.  128-token groups (4 bitmap words each) are dealt to threads round-robin in
-  //      rounds of FIN_THREADS groups, so every load of a warp is 512 contiguous bytes; within a round the
-  //      thread order is the token order, and the rounds follow one another.
-  const long long groups = (n + 127) / 128;
-  const uint4* bm4 = reinterpret_cast<const uint4*>(bm);
-  int32_t* out = idx_out + (size_t)head * k;
+  // ---- every tile's place in the output: exclusive prefix of the tile counts, in place
   uint32_t base = 0;
-  constexpr int ROUNDS_AT_ONCE = 8;
-  for (long long g0 = 0; g0 < groups; g0 += (long long)ROUNDS_AT_ONCE * FIN_THREADS) {
-    uint4 w[ROUNDS_AT_ONCE];
-    uint32_t cnt[ROUNDS_AT_ONCE];
-#pragma unroll
-    for (int x = 0; x < ROUNDS_AT_ONCE; ++x) {
-      const long long g = g0 + (long long)x * FIN_THREADS + tid;
-      w[x] = (g < groups) ? bm4[g] : make_uint4(0u, 0u, 0u, 0u);
-      cnt[x] = __popc(w[x].x) + __popc(w[x].y) + __popc(w[x].z) + __popc(w[x].w);
-    }
-#pragma unroll
-    for (int x = 0; x < ROUNDS_AT_ONCE; ++x) {
-      if (g0 + (long long)x * FIN_THREADS >= groups) break;   // uniform
-      uint32_t total;
-      uint32_t pos = base + block_exclusive_scan(cnt[x], s_warp, &total);
-      base += total;
-      const long long g = g0 + (long long)x * FIN_THREADS + tid;
-      uint32_t any = w[x].x | w[x].y | w[x].z | w[x].w;
-      while (any) {
-        const int l = __ffs(any) - 1;
-        any &= any - 1;
-        const int32_t t = (int32_t)(g * 128 + 4 * l);
-        if ((w[x].x >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t; ++pos; }
-        if ((w[x].y >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 1; ++pos; }
-        if ((w[x].z >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 2; ++pos; }
-        if ((w[x].w >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 3; ++pos; }
-      }
-    }
+  for (int t0 = 0; t0 < ntiles; t0 += FIN_THREADS) {
+    const int t = t0 + tid;
+    const uint32_t c = (t < ntiles) ? __ldcg(tc + t) : 0u;
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan(c, s_warp, &total);
+    if (t < ntiles) tc[t] = base + ex;
+    base += total;
+    __syncthreads();
   }
-  if (base != (uint32_t)k && tid == 0) {                      // short (non-finite scores) or long selection
+  if (base != (uint32_t)k && tid == 0) {                      // short selection (non-finite scores)
     atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+    int32_t* out = idx_out + (size_t)head * k;
     for (uint32_t e = base; e < (uint32_t)k; ++e) out[e] = (int32_t)(n - 1);   // pad with the last token
+  }
+}
+
+// One CTA per (tile of FILT_TILE tokens, head): thread = group of 128 tokens (4 bitmap words, one 16-byte load).
+__global__ void __launch_bounds__(FILT_TILE / 128)
+topk_emit_kernel(const uint32_t* __restrict__ bitmap, long long bitmap_words, const uint32_t* __restrict__ tile_offset,
+                 long long n, int k, int32_t* __restrict__ idx_out) {
+  constexpr int EMIT_THREADS = FILT_TILE / 128;               // 64
+  __shared__ uint32_t s_w[EMIT_THREADS / 32];
+  const int head = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long g = (long long)blockIdx.x * EMIT_THREADS + tid;
+  const long long groups = (n + 127) / 128;
+  const uint4* bm4 = reinterpret_cast<const uint4*>(bitmap + (size_t)head * (size_t)bitmap_words);
+  const uint4 w = (g < groups) ? __ldcg(bm4 + g) : make_uint4(0u, 0u, 0u, 0u);
+  const uint32_t c = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
+  uint32_t incl = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_w[warp] = incl;
+  __syncthreads();
+  uint32_t pos = tile_offset[(size_t)head * gridDim.x + blockIdx.x] + incl - c;
+  for (int x = 0; x < warp; ++x) pos += s_w[x];
+  int32_t* out = idx_out + (size_t)head * k;
+  uint32_t any = w.x | w.y | w.z | w.w;
+  while (any) {
+    const int l = __ffs(any) - 1;
+    any &= any - 1;
+    const int32_t t = (int32_t)(g * 128 + 4 * l);
+    if ((w.x >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t; ++pos; }
+    if ((w.y >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 1; ++pos; }
+    if ((w.z >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 2; ++pos; }
+    if ((w.w >> l) & 1u) { if (pos < (uint32_t)k) out[pos] = t + 3; ++pos; }
   }
 }
 
@@ -391,13 +420,14 @@ extern "C" int fathom_topk(fathom_ctx* ctx, const fathom_layout* L, const float*
   // histograms and per-head state are contiguous at the start of the arena
   FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
   dim3 hgrid((unsigned)((n + HIST_TILE - 1) / HIST_TILE), (unsigned)Hq);
-  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.hist);
-  topk_find_bin_kernel<<<Hq, FIN_THREADS, 0, st>>>(S.hist, S.state, want, ctx->dev_status);
-  dim3 fgrid((unsigned)((n + FILT_TILE - 1) / FILT_TILE), (unsigned)Hq);
+  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.hist, S.state, want, ctx->dev_status);
+  const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
+  dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
   topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
-                                                     S.bitmap_words);
-  topk_finish_kernel<<<Hq, FIN_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
-                                                 S.bitmap_words, k, idx, ctx->dev_status);
+                                                     S.bitmap_words, S.tile_count);
+  topk_select_kernel<<<Hq, FIN_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
+                                                 S.bitmap_words, k, idx, ctx->dev_status, S.tile_count, ntiles);
+  topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
