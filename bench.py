@@ -168,6 +168,16 @@ def run_ours(args):
         else:
             ctx.fathom_sparse_attend(lay, q, Kr, Vr, idx, k, sm_scale, out, stream)
 
+    def stage_on(i, st):
+        if i == 1:
+            ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, B, hpp, depth, st)
+        elif i == 2:
+            ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, scores, st)
+        elif i == 3:
+            ctx.fathom_topk(lay, scores, k, 0, 0, idx, st)
+        else:
+            ctx.fathom_sparse_attend(lay, L.q, L.Krows, L.Vrows, idx, k, sm_scale, out, st)
+
     def step(events=None):
         for i in range(5):
             if events is not None:
@@ -258,6 +268,40 @@ def run_ours(args):
         "topk (4 kernels, 2 passes over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
         "sparse_attend": roof("sparse_attend", stage_us["sparse_attend"], "attend_*", n * Hkv),
     }
+    # the scan is bound by shared-memory table lookups and issue slots, not by HBM: also report it that way
+    groups_per_plan = [(int(r.sum()) + 3) // 4 for r in depth_h]            # groups of four active rows
+    lookups = n * sum(groups_per_plan) * max(1, hpp // 2)                    # per token, group and head pair
+    lookup_peak = 148 * 15.8 * 1.965e9                          # measured: 15.8 eight-byte lookups per clock per SM
+    result["roofline_other_kernels"]["scan"]["alt_bound"] = {
+        "bound": "shared-memory lookups", "achieved": round(lookups / (stage_us["scan"] * 1e-6) / 1e12, 3), "peak": round(lookup_peak / 1e12, 3),
+        "unit": "T lookups/s", "frac": round(lookups / (stage_us["scan"] * 1e-6) / lookup_peak, 4),
+        "note": "one 8-byte table load per token, group of four rows and head pair; peak from a micro-benchmark (DESIGN.md)"}
+
+    # ---- the decode part of the step (everything but the one-off build) replayed as one CUDA graph, median of 30
+    graph_us = None
+    try:
+        gs = torch.cuda.Stream()
+        gs.wait_stream(stream)
+        with torch.cuda.stream(gs):
+            for i in range(1, 5):
+                stage_on(i, gs)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=gs):
+                for i in range(1, 5):
+                    stage_on(i, gs)
+        torch.cuda.synchronize()
+        ts = []
+        for it in range(33):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); g.replay(); b.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(a.elapsed_time(b) * 1e3)
+        graph_us = round(statistics.median(ts), 2)
+        del g
+    except Exception as e:                                      # report, never hide
+        graph_us = "capture failed: " + repr(e)
+    result["decode_step_us_per_layer_cuda_graph"] = graph_us
     result["device_status"] = status
     result["wall_ms_per_step"] = round(1e3 * t_wall / args.steps, 4)
 
