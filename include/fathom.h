@@ -141,6 +141,19 @@ int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* pl
 int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* scores, int k,
                 int n_sink, int n_local, int32_t* idx, void* stream);
 
+/* ---- (3+4) fused scan and top-k, scores never materialised — Sec. 6 ("a fused kernel would narrow the gap") ------
+ * Gives exactly the idx that fathom_topk would give on the scores of fathom_scan (same arguments), without writing
+ * or re-reading the n * Hq scores: (a) every 16th 1024-token tile is scanned and the bin of the 12 leading score-key
+ * bits in which the sample's k-th largest score lies is found per head; at least k tokens reach that bin's lower
+ * edge, so no winner lies below it; (b) the full scan keeps only the (score, token) pairs that reach the edge;
+ * (c) the exact selection (ties to the lower token) runs on those candidates.  The threshold is a bound, not an
+ * estimate, so the result never depends on how representative the sample is - only the number of candidates does.
+ * Sequences too short to sample (fewer than 16 tiles or fewer than 2 k sampled tokens) are scanned into scratch
+ * and selected densely.  Uses the context scratch (fathom_scratch_bytes). */
+int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes, const uint16_t* scales,
+                     const float* q, const uint8_t* depth, int heads_per_plan, int k, int n_sink, int n_local,
+                     int32_t* idx, void* stream);
+
 /* ---- (5) gather + exact attention — Sec. 2 "Top-k decoding" --------------------------------
  * Per query head h with KV head h / G:  out[h] = softmax_i(softmax_scale * q_h . K[idx[h][i]]) . V[idx[h][i]]
  * over its own k selected rows (fp32 arithmetic on rows of `row_dtype`).

@@ -21,11 +21,19 @@ fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k) {
   size_t off = 0;
   s.hist = reinterpret_cast<uint32_t*>(p + off);    off += fathom_round_up((size_t)Hq * FATHOM_TOPK_BINS * 4, 256);
   s.state = reinterpret_cast<uint32_t*>(p + off);   off += fathom_round_up((size_t)Hq * 8 * 4, 256);
+  s.cand_count = reinterpret_cast<uint32_t*>(p + off); off += fathom_round_up((size_t)Hq * 4, 256);
   s.bitmap_words = (long long)((n + 1023) / 1024) * 32;                    // whole 32-word groups
   s.bitmap = reinterpret_cast<uint32_t*>(p + off);  off += fathom_round_up((size_t)Hq * (size_t)s.bitmap_words * 4, 256);
   s.cand = reinterpret_cast<int32_t*>(p + off);     off += fathom_round_up((size_t)Hq * (size_t)n * 4, 256);
   s.tile_count = reinterpret_cast<uint32_t*>(p + off); off += fathom_round_up((size_t)Hq * (size_t)((n + 8191) / 8192) * 4, 256);
-  (void)k;
+  s.cand_score = reinterpret_cast<float*>(p + off); off += fathom_round_up((size_t)Hq * (size_t)n * 4, 256);
+  {
+    const long long tile = fathom_scan_tile_tokens();
+    const int step = fathom_fused_tile_step(n, k);
+    const long long sampled = ((n + tile - 1) / tile + step - 1) / step;
+    s.sample_stride = step == 1 ? (long long)((n + 3) / 4 * 4) : sampled * tile;
+    s.sample = reinterpret_cast<float*>(p + off);   off += fathom_round_up((size_t)Hq * (size_t)s.sample_stride * 4, 256);
+  }
   s.bytes = off;
   return s;
 }

@@ -41,16 +41,38 @@ static inline int64_t fathom_nblocks(int64_t n) { return (n + FATHOM_BLOCK - 1) 
 static inline bool fathom_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t fathom_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// ---- pieces shared by scan.cu and topk.cu for the fused scan + selection (fathom_scan_topk) -------------------
+struct fathom_scan_fuse {       // extra arguments of the sampling / filtering scan variants
+  int tile_step;                // sample: scan every tile_step-th tile
+  const uint32_t* state;        // filter: [Hq][8], word 0 = threshold bin found on the sample
+  long long sink_end, local_begin;   // filter: eligible tokens are sink_end <= i < local_begin
+  float* cand_score;            // filter: [Hq][capacity] scores of the candidates
+  int32_t* cand_idx;            // filter: [Hq][capacity] their tokens
+  uint32_t* cand_count;         // filter: [Hq]
+  long long capacity;
+};
+int fathom_scan_tile_tokens();  // tokens per scan tile (the sampling granularity)
+int fathom_fused_tile_step(long long n, int k);   // 16, or 1 when the sequence is too short to sample
+int fathom_launch_scan_sample(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
+                              const uint8_t* depth, int heads_per_plan, float* sample, long long sample_stride,
+                              int tile_step, cudaStream_t st);
+int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
+                              const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st);
+
 // ---- scratch arena carving (one place, used by fathom_scratch_bytes and by the calls) --------
 #define FATHOM_TOPK_BINS 4096            // 12 leading bits of the ordered score key
 #define FATHOM_ATTN_CHUNK 128            // selected rows handled by one CTA of the partial kernel
 
 struct fathom_topk_scratch {
   uint32_t* hist;        // [Hq][FATHOM_TOPK_BINS]
-  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 4 candidates written
+  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 4 candidates written, 5 tickets
+  uint32_t* cand_count;  // [Hq] candidates collected by the filtering scan (fused path)
   uint32_t* bitmap;      // [Hq][bitmap_words] selection bitmap, token i at bit (i % 32) of word i / 32
   int32_t* cand;         // [Hq][n] token indices of the threshold bin
   uint32_t* tile_count;  // [Hq][ceil(n / 8192)] selected tokens per filter tile, then their exclusive prefix
+  float* cand_score;     // [Hq][n] scores of the fused path's candidates
+  float* sample;         // [Hq][sample_stride] scores of the sampled scan tiles (fused path)
+  long long sample_stride;
   long long bitmap_words;
   size_t bytes;
 };

@@ -57,6 +57,13 @@ __device__ __forceinline__ void transpose_rows(uint32_t& a, uint32_t& b, uint32_
   t = ((b >> 2) ^ d) & 0x33333333u; d ^= t; b ^= t << 2;
 }
 
+// fp32 value whose order-preserving integer image (see topk.cu) has `bin` as its 12 leading bits and zeros below:
+// the lower edge of that histogram bin
+__device__ __forceinline__ float bin_lower_edge(uint32_t bin) {
+  const uint32_t key = bin << 20;
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
 template <int NH>
 struct alignas(16) WarpSmem {
   using C = ScanCfg<NH>;
@@ -65,12 +72,17 @@ struct alignas(16) WarpSmem {
   alignas(8) unsigned char tab[C::NTAB * C::TSTRIDE];
 };
 
-template <int NH>
+// MODE 0: scores of every token are written (fathom_scan).
+// MODE 1: only every tile_step-th tile is scanned and its scores are written compactly (tile i of the launch at
+//         token positions 1024 i ..) - the sample from which fathom_scan_topk derives a safe threshold.
+// MODE 2: every tile is scanned, nothing is written but the tokens whose score reaches the head's threshold:
+//         (score, token) pairs appended to the head's candidate list.
+template <int NH, int MODE>
 __global__ void __launch_bounds__(SCAN_THREADS, 8)              // 64 registers: occupancy matters more than spills here
 scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
             const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
             long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
-            int G, int heads_per_plan) {
+            int G, int heads_per_plan, fathom_scan_fuse fz) {
   using C = ScanCfg<NH>;
   constexpr int HP = C::HP, EB = C::EB, TSTRIDE = C::TSTRIDE;
   __shared__ uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];      // channel of active row r
@@ -110,7 +122,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
   const int nrows = s_nrows;
 
   WarpSmem<NH>& S = s_warp[warp];
-  const long long blk0 = (long long)blockIdx.x * TILE_BLOCKS;  // first block of this CTA
+  const long long blk0 = (long long)blockIdx.x * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;  // first block of this CTA
   const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
   const int wb0 = warp * WB;                                   // first block of this warp within the tile
   const int nblk = max(0, min(WB, nblk_cta - wb0));
@@ -256,37 +268,136 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
   }
 
   // ---- epilogue
+  if (MODE != 2) {
 #pragma unroll
-  for (int b = 0; b < WB; ++b) {
-    if (b < nblk) {
-      const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;
+    for (int b = 0; b < WB; ++b) {
+      if (b < nblk) {
+        const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;                       // token scanned
+        const long long dst = MODE == 1 ? tok - blk0 * FATHOM_BLOCK + (long long)blockIdx.x * (TILE_BLOCKS * FATHOM_BLOCK) : tok;
 #pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        float* row = scores + (size_t)(h0 + h) * (size_t)score_stride;
+        for (int h = 0; h < NH; ++h) {
+          float* row = scores + (size_t)(h0 + h) * (size_t)score_stride;
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            float v;
+            if (NH == 1) v = acc1[b][x];
+            else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
+            if (tok + 32 * x < n) row[dst + 32 * x] = v;
+          }
+        }
+      }
+    }
+  } else {
+    // candidates of this warp's 256 tokens, per head, collected in the (now idle) table memory and appended to
+    // the head's global list; entry = (score bits, token)
+    constexpr int LIST = (int)(sizeof(S.tab) / sizeof(uint2)) / NH;    // entries per head
+    uint2* list = reinterpret_cast<uint2*>(S.tab);
+    uint32_t* cnt = S.idx[0];                                          // NH counters (index memory is idle too)
+    __syncwarp();
+    if (lane < NH) cnt[lane] = 0u;
+    __syncwarp();
+    float thr[NH];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) thr[h] = bin_lower_edge(fz.state[(h0 + h) * 8]);
+#pragma unroll
+    for (int b = 0; b < WB; ++b) {
+      if (b < nblk) {
+        const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-          float v;
-          if (NH == 1) v = acc1[b][x];
-          else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
-          if (tok + 32 * x < n) row[tok + 32 * x] = v;
+          const long long t = tok + 32 * x;
+          const bool elig = t < n && t >= fz.sink_end && t < fz.local_begin;
+#pragma unroll
+          for (int h = 0; h < NH; ++h) {
+            float v;
+            if (NH == 1) v = acc1[b][x];
+            else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
+            if (elig && v >= thr[h]) {
+              const uint32_t p = atomicAdd(&cnt[h], 1u);
+              if (p < (uint32_t)LIST) list[h * LIST + p] = make_uint2(__float_as_uint(v), (uint32_t)t);
+              else {                                                   // list full: straight to the global list
+                const uint32_t gp = atomicAdd(&fz.cand_count[h0 + h], 1u);
+                if ((long long)gp < fz.capacity) {
+                  fz.cand_score[(size_t)(h0 + h) * fz.capacity + gp] = v;
+                  fz.cand_idx[(size_t)(h0 + h) * fz.capacity + gp] = (int32_t)t;
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+    // one global atomic per (CTA, head): the four warps' counts are summed, the slice is reserved once
+    __shared__ uint32_t s_wcnt[SCAN_WARPS][NH], s_cbase[NH];
+    __syncwarp();
+    if (lane < NH) s_wcnt[warp][lane] = min(cnt[lane], (uint32_t)LIST);
+    __syncthreads();
+    if (tid < NH) {
+      uint32_t tot = 0;
+#pragma unroll
+      for (int w = 0; w < SCAN_WARPS; ++w) tot += s_wcnt[w][tid];
+      s_cbase[tid] = tot ? atomicAdd(&fz.cand_count[h0 + tid], tot) : 0u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+      const uint32_t c = s_wcnt[warp][h];
+      uint32_t base = s_cbase[h];
+      for (int w = 0; w < warp; ++w) base += s_wcnt[w][h];
+      for (uint32_t e = lane; e < c; e += 32) {
+        const uint2 it = list[h * LIST + e];
+        if ((long long)(base + e) < fz.capacity) {
+          fz.cand_score[(size_t)(h0 + h) * fz.capacity + base + e] = __uint_as_float(it.x);
+          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + base + e] = (int32_t)it.y;
         }
       }
     }
   }
 }
 
-template <int NH>
+template <int NH, int MODE>
 int launch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
-                const uint8_t* depth, int heads_per_plan, float* scores, cudaStream_t st) {
+                const uint8_t* depth, int heads_per_plan, float* scores, long long score_stride,
+                const fathom_scan_fuse& fz, cudaStream_t st) {
   const long long nb = fathom_nblocks(L->n);
-  dim3 grid((unsigned)((nb + TILE_BLOCKS - 1) / TILE_BLOCKS), (unsigned)(L->n_q_heads / NH));
-  scan_kernel<NH><<<grid, SCAN_THREADS, 0, st>>>(planes, scales, q, depth, scores, L->n, nb, L->plane_stride_words,
-                                                 L->scale_stride, L->score_stride, L->n_q_heads / L->n_kv_heads,
-                                                 heads_per_plan);
+  const long long ntiles = (nb + TILE_BLOCKS - 1) / TILE_BLOCKS;
+  const long long gx = MODE == 1 ? (ntiles + fz.tile_step - 1) / fz.tile_step : ntiles;
+  dim3 grid((unsigned)gx, (unsigned)(L->n_q_heads / NH));
+  scan_kernel<NH, MODE><<<grid, SCAN_THREADS, 0, st>>>(planes, scales, q, depth, scores, L->n, nb, L->plane_stride_words,
+                                                       L->scale_stride, score_stride, L->n_q_heads / L->n_kv_heads,
+                                                       heads_per_plan, fz);
   return 0;
 }
 
+template <int MODE>
+int dispatch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
+                  const uint8_t* depth, int heads_per_plan, float* scores, long long score_stride,
+                  const fathom_scan_fuse& fz, cudaStream_t st) {
+  switch (heads_per_plan) {
+    case 1: return launch_scan<1, MODE>(L, planes, scales, q, depth, 1, scores, score_stride, fz, st);
+    case 2: return launch_scan<2, MODE>(L, planes, scales, q, depth, 2, scores, score_stride, fz, st);
+    case 4: return launch_scan<4, MODE>(L, planes, scales, q, depth, 4, scores, score_stride, fz, st);
+    case 8: return launch_scan<4, MODE>(L, planes, scales, q, depth, 8, scores, score_stride, fz, st);   // two CTAs of four heads share a plan
+    default: return FATHOM_ERR_UNSUPPORTED;
+  }
+}
+
 }  // namespace
+
+int fathom_scan_tile_tokens() { return TILE_BLOCKS * FATHOM_BLOCK; }
+
+int fathom_launch_scan_sample(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
+                              const uint8_t* depth, int heads_per_plan, float* sample, long long sample_stride,
+                              int tile_step, cudaStream_t st) {
+  fathom_scan_fuse fz = {};
+  fz.tile_step = tile_step;
+  return dispatch_scan<1>(L, planes, scales, q, depth, heads_per_plan, sample, sample_stride, fz, st);
+}
+
+int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
+                              const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st) {
+  return dispatch_scan<2>(L, planes, scales, q, depth, heads_per_plan, nullptr, 0, fz, st);
+}
 
 extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64_t* planes, const uint16_t* scales,
                            const float* q, const uint8_t* depth, int heads_per_plan, float* scores, void* stream) {
@@ -296,14 +407,10 @@ extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64
   const int G = L->n_q_heads / L->n_kv_heads;
   if (heads_per_plan < 1 || G % heads_per_plan != 0) return FATHOM_ERR_INVALID_ARG;
   if (!fathom_aligned16(planes) || !fathom_aligned16(scales) || !fathom_aligned16(scores)) return FATHOM_ERR_ALIGNMENT;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  switch (heads_per_plan) {
-    case 1: launch_scan<1>(L, planes, scales, q, depth, 1, scores, st); break;
-    case 2: launch_scan<2>(L, planes, scales, q, depth, 2, scores, st); break;
-    case 4: launch_scan<4>(L, planes, scales, q, depth, 4, scores, st); break;
-    case 8: launch_scan<4>(L, planes, scales, q, depth, 8, scores, st); break;   // two CTAs of four heads share a plan
-    default: return FATHOM_ERR_UNSUPPORTED;
-  }
+  fathom_scan_fuse fz = {};
+  fz.tile_step = 1;
+  rc = dispatch_scan<0>(L, planes, scales, q, depth, heads_per_plan, scores, L->score_stride, fz, static_cast<cudaStream_t>(stream));
+  if (rc != FATHOM_OK) return rc;
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

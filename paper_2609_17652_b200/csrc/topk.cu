@@ -19,7 +19,7 @@
 namespace {
 
 constexpr int HIST_THREADS = 256;
-constexpr int HIST_TILE = 32768;                             // scores per CTA of the histogram pass
+constexpr int HIST_TILE = 32768;                             // most scores per CTA of the histogram pass
 constexpr int FILT_THREADS = 256;
 constexpr int FILT_WARP_TOKENS = 1024;                       // 32 ballots -> 32 bitmap words per warp
 constexpr int FILT_TILE = (FILT_THREADS / 32) * FILT_WARP_TOKENS;   // 8192 tokens per CTA
@@ -40,20 +40,20 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
 __global__ void __launch_bounds__(HIST_THREADS)
 topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                  uint32_t* __restrict__ hist, uint32_t* __restrict__ state, uint32_t want,
-                 uint32_t* __restrict__ dev_status) {
+                 uint32_t* __restrict__ dev_status, int tile) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ bool s_last;
   const int head = blockIdx.y;
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  const long long base = (long long)blockIdx.x * HIST_TILE;
-  const long long end = min(base + HIST_TILE, n);
+  const long long base = (long long)blockIdx.x * tile;         // tile: scores per CTA, a multiple of 1024
+  const long long end = min(base + tile, n);
   // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
-  if (base >= F.sink_end && base + HIST_TILE <= F.local_begin) {        // whole tile eligible: no per-token test
+  if (base >= F.sink_end && base + tile <= F.local_begin) {   // whole tile eligible: no per-token test
     const float4* r4 = reinterpret_cast<const float4*>(row + base);
 #pragma unroll 8
-    for (int v = threadIdx.x; v < HIST_TILE / 4; v += HIST_THREADS) {
+    for (int v = threadIdx.x; v < tile / 4; v += HIST_THREADS) {
       const float4 x = __ldg(r4 + v);
       atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
       atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
@@ -259,11 +259,17 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return s_warp[warp] + incl - v;
 }
 
+// FUSED = false: candidates are the tokens of the threshold bin (their 12 leading key bits agree), scores are read
+//                 from the dense score rows, the number needed comes from the histogram state.
+// FUSED = true : candidates are (score, token) pairs collected by the filtering scan; `want_fused` of them are needed
+//                 and the whole 64-bit composite takes part in the select.
+template <bool FUSED>
 __global__ void __launch_bounds__(FIN_THREADS)
 topk_select_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    const uint32_t* __restrict__ state, const int32_t* __restrict__ cand,
                    uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
-                   uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles) {
+                   uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
+                   const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_fused) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   __shared__ uint64_t s_comp[FIN_CACHE];
@@ -272,22 +278,37 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
   __shared__ uint32_t s_need, s_bucket;
   const int head = blockIdx.x, tid = threadIdx.x;
-  const float* row = scores + (size_t)head * (size_t)score_stride;
-  const int32_t* cand_h = cand + (size_t)head * (size_t)n;
+  // dense: scores row of the head, candidate tokens [n];  fused: candidate scores and tokens [cand_capacity]
+  const float* row = scores + (size_t)head * (size_t)(FUSED ? cand_capacity : score_stride);
+  const int32_t* cand_h = cand + (size_t)head * (size_t)(FUSED ? cand_capacity : n);
   uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
   uint32_t* tc = tile_count + (size_t)head * ntiles;
-  const uint32_t m = state[head * 8 + 4];
-  const uint32_t need0 = min(state[head * 8 + 2], m);
-  const bool cached = m <= FIN_CACHE;
+  const uint32_t m = FUSED ? (uint32_t)min((long long)cand_count[head], cand_capacity) : state[head * 8 + 4];
+  const uint32_t need0 = min(FUSED ? want_fused : state[head * 8 + 2], m);
+  constexpr int TOP = FUSED ? 64 : 52;                        // undecided bits of the composite
+  auto composite = [&](uint32_t c) -> uint64_t {
+    if (FUSED) return (((uint64_t)ordered_key(row[c])) << 32) | (uint32_t)(~(uint32_t)cand_h[c]);
+    return composite52(row, cand_h[c]);
+  };
+  // The working set is either all m candidates in global memory or a subset kept in shared memory: everything when
+  // m fits, otherwise the bucket of the first digit once it fits (what ranks above that bucket is marked at once).
+  __shared__ uint32_t s_ncache;
+  bool cached = m <= FIN_CACHE;
+  uint32_t mc = m;                                            // size of the working set
+  auto mark = [&](uint64_t comp) {                            // the token sits in the low 32 bits of every composite
+    const int32_t i = (int32_t)~(uint32_t)comp;
+    atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
+    atomicAdd(&tc[i / FILT_TILE], 1u);
+  };
   if (cached)
-    for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite52(row, cand_h[c]);
+    for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite(c);
 
-  // ---- radix select of the need0 largest composites among the m candidates: 11-bit digits from bit 52
-  //      downwards (the last digit is 8 bits) until the chosen bucket is taken whole.
+  // ---- radix select of the need0 largest composites among the m candidates: 11-bit digits from the top
+  //      undecided bit downwards (the last digit is shorter) until the chosen bucket is taken whole.
   uint64_t thr = 0;                                           // chosen candidates: composite >= thr
   if (need0 > 0 && need0 < m) {
-    if (tid == 0) { s_prefix = 0; s_need = need0; }
-    int hi = 52;
+    if (tid == 0) { s_prefix = 0; s_need = need0; s_ncache = 0u; }
+    int hi = TOP;
     while (hi > 0) {
       const int bits = min(DIGIT_BITS, hi);
       const int lo = hi - bits;
@@ -295,9 +316,21 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       __syncthreads();
       const uint64_t prefix = s_prefix;
       const uint32_t need = s_need;
-      for (uint32_t c = tid; c < m; c += FIN_THREADS) {
-        const uint64_t comp = cached ? s_comp[c] : composite52(row, cand_h[c]);
-        if ((comp >> hi) == (prefix >> hi)) atomicAdd(&s_hist[(uint32_t)(comp >> lo) & ((1u << bits) - 1u)], 1u);
+      // batches of 8 elements per thread: all loads of a batch are in flight together (one CTA serves a head, so
+      // a load per loop iteration would leave the pass latency-bound)
+      for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS * 8) {
+        uint64_t comp[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const uint32_t c = c0 + u * FIN_THREADS + tid;
+          comp[u] = c < mc ? (cached ? s_comp[c] : composite(c)) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const uint32_t c = c0 + u * FIN_THREADS + tid;
+          if (c < mc && (hi >= 64 || (comp[u] >> hi) == (prefix >> hi)))
+            atomicAdd(&s_hist[(uint32_t)(comp[u] >> lo) & ((1u << bits) - 1u)], 1u);
+        }
       }
       __syncthreads();
       // thread t owns digits DIGITS-1-DPT*t .. (descending): the block prefix is a suffix count
@@ -320,17 +353,43 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       __syncthreads();
       hi = lo;
       if (s_need == s_bucket) break;                          // the chosen bucket is taken entirely: done
+      if (!cached && s_bucket <= FIN_CACHE) {
+        // the undecided bucket fits in shared memory: pull it in, mark what ranks above it, go on from there
+        const uint64_t pfx = s_prefix;
+        for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS * 8) {
+          uint64_t comp[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t c = c0 + u * FIN_THREADS + tid;
+            comp[u] = c < mc ? composite(c) : 0ull;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t c = c0 + u * FIN_THREADS + tid;
+            const uint64_t top = hi >= 64 ? 0ull : (comp[u] >> hi), ptop = hi >= 64 ? 0ull : (pfx >> hi);
+            if (c < mc && top > ptop) mark(comp[u]);
+            const bool keep = c < mc && top == ptop;
+            const unsigned km = __ballot_sync(0xffffffffu, keep);               // warp-aggregated append
+            if (km) {
+              uint32_t pos = 0;
+              const int leader = __ffs(km) - 1;
+              if ((tid & 31) == leader) pos = atomicAdd(&s_ncache, (uint32_t)__popc(km));
+              pos = __shfl_sync(0xffffffffu, pos, leader);
+              if (keep) s_comp[pos + __popc(km & ((1u << (tid & 31)) - 1u))] = comp[u];
+            }
+          }
+        }
+        __syncthreads();
+        cached = true;
+        mc = s_ncache;
+      }
     }
     thr = s_prefix;                                           // undecided low bits are zero
   }
   if (need0 > 0) {
-    for (uint32_t c = tid; c < m; c += FIN_THREADS) {
-      const int32_t i = cand_h[c];
-      const uint64_t comp = cached ? s_comp[c] : composite52(row, i);
-      if (need0 >= m || comp >= thr) {
-        atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
-        atomicAdd(&tc[i / FILT_TILE], 1u);
-      }
+    for (uint32_t c = tid; c < mc; c += FIN_THREADS) {
+      const uint64_t comp = cached ? s_comp[c] : composite(c);
+      if (need0 >= m || comp >= thr) mark(comp);
     }
   }
   // ---- forced sink / local tokens
@@ -398,6 +457,32 @@ topk_emit_kernel(const uint32_t* __restrict__ bitmap, long long bitmap_words, co
 
 }  // namespace
 
+// Scores per histogram CTA: large tiles amortise the 4096-bin flush, but short rows still need a few hundred CTAs.
+static int hist_tile_for(long long n, int Hq) {
+  long long tile = HIST_TILE;
+  while (tile > 4096 && ((n + tile - 1) / tile) * Hq < 600) tile /= 2;
+  return (int)tile;
+}
+
+// Dense selection over score rows (the four launches of fathom_topk).
+static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, long long score_stride, int Hq, int k,
+                          Forced F, uint32_t want, const fathom_topk_scratch& S, int32_t* idx, cudaStream_t st) {
+  // histograms, per-head state and candidate counters are contiguous at the start of the arena
+  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
+  const int htile = hist_tile_for(n, Hq);
+  dim3 hgrid((unsigned)((n + htile - 1) / htile), (unsigned)Hq);
+  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, want, ctx->dev_status, htile);
+  const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
+  dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
+  topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
+                                                     S.tile_count);
+  topk_select_kernel<false><<<Hq, FIN_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
+                                                        k, idx, ctx->dev_status, S.tile_count, ntiles, nullptr, 0, 0u);
+  topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
 extern "C" int fathom_topk(fathom_ctx* ctx, const fathom_layout* L, const float* scores, int k, int n_sink,
                            int n_local, int32_t* idx, void* stream) {
   if (!ctx || !scores || !idx) return FATHOM_ERR_INVALID_ARG;
@@ -411,22 +496,86 @@ extern "C" int fathom_topk(fathom_ctx* ctx, const fathom_layout* L, const float*
   F.local_begin = (n - n_local > F.sink_end) ? (n - n_local) : F.sink_end;
   const long long n_forced = F.sink_end + (n - F.local_begin);
   if (n_forced > k) return FATHOM_ERR_INVALID_ARG;
-  const int Hq = L->n_q_heads;
+  fathom_topk_scratch S = fathom_carve_topk(ctx->scratch, L->n_q_heads, n, k);
+  if (S.bytes > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  return run_dense_topk(ctx, scores, n, L->score_stride, L->n_q_heads, k, F, (uint32_t)(k - n_forced), S, idx,
+                        static_cast<cudaStream_t>(stream));
+}
+
+// Tile step of the sample scan for (n, k): every 16th scan tile when that sample still holds at least 2 k tokens,
+// otherwise 1 (the "sample" is then the whole score array and the dense selection runs on it).
+int fathom_fused_tile_step(long long n, int k) {
+  const long long tile = fathom_scan_tile_tokens();
+  const long long ntiles = (n + tile - 1) / tile;
+  const long long sampled = (ntiles + 15) / 16;                       // tiles 0, 16, 32, ...
+  const long long last_start = (sampled - 1) * 16 * tile;             // first token of the last sampled tile (< n)
+  const long long valid = (sampled - 1) * tile + ((n - last_start) < tile ? (n - last_start) : tile);
+  return (ntiles >= 16 && valid >= 2LL * k) ? 16 : 1;
+}
+
+extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const uint64_t* planes, const uint16_t* scales,
+                                const float* q, const uint8_t* depth, int heads_per_plan, int k, int n_sink, int n_local,
+                                int32_t* idx, void* stream) {
+  if (!ctx || !planes || !scales || !q || !depth || !idx) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  const int Hq = L->n_q_heads, G = Hq / L->n_kv_heads;
+  if (heads_per_plan < 1 || G % heads_per_plan != 0) return FATHOM_ERR_INVALID_ARG;
+  if (heads_per_plan != 1 && heads_per_plan != 2 && heads_per_plan != 4 && heads_per_plan != 8) return FATHOM_ERR_UNSUPPORTED;
+  if (k < 1 || k > L->n || k > FATHOM_MAX_K || n_sink < 0 || n_local < 0) return FATHOM_ERR_INVALID_ARG;
+  if (!fathom_aligned16(planes) || !fathom_aligned16(scales)) return FATHOM_ERR_ALIGNMENT;
+  const long long n = L->n;
+  Forced F;
+  F.sink_end = n_sink < n ? n_sink : n;
+  F.local_begin = (n - n_local > F.sink_end) ? (n - n_local) : F.sink_end;
+  const long long n_forced = F.sink_end + (n - F.local_begin);
+  if (n_forced > k) return FATHOM_ERR_INVALID_ARG;
   fathom_topk_scratch S = fathom_carve_topk(ctx->scratch, Hq, n, k);
   if (S.bytes > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint32_t want = (uint32_t)(k - n_forced);
+  const int step = fathom_fused_tile_step(n, k);
+  const long long tile = fathom_scan_tile_tokens();
+  const long long ntiles_scan = (n + tile - 1) / tile;
 
-  // histograms and per-head state are contiguous at the start of the arena
+  // ---- sample: scores of every `step`-th scan tile, compact
+  rc = fathom_launch_scan_sample(L, planes, scales, q, depth, heads_per_plan, S.sample, S.sample_stride, step, st);
+  if (rc != FATHOM_OK) return rc;
+  if (step == 1)                                              // short sequence: the sample is the whole score array
+    return run_dense_topk(ctx, S.sample, n, S.sample_stride, Hq, k, F, want, S, idx, st);
+
+  // ---- threshold: the bin in which the sample's k-th largest score lies.  At least k tokens of the sample, hence
+  //      at least k - n_forced eligible tokens of the sequence, reach its lower edge: no winner can lie below it.
+  const long long sampled = (ntiles_scan + step - 1) / step;
+  const long long last_start = (sampled - 1) * step * tile;
+  const long long n_sample = (sampled - 1) * tile + ((n - last_start) < tile ? (n - last_start) : tile);
   FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
-  dim3 hgrid((unsigned)((n + HIST_TILE - 1) / HIST_TILE), (unsigned)Hq);
-  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.hist, S.state, want, ctx->dev_status);
+  Forced none;
+  none.sink_end = 0;
+  none.local_begin = n_sample;
+  const int htile = hist_tile_for(n_sample, Hq);
+  dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
+  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(S.sample, n_sample, S.sample_stride, none, S.hist, S.state, (uint32_t)k,
+                                                   ctx->dev_status, htile);
+  // ---- full scan that keeps only the tokens reaching their head's threshold
   const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
+  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.bitmap, 0, (size_t)Hq * S.bitmap_words * 4, st));
+  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.tile_count, 0, (size_t)Hq * ntiles * 4, st));
+  fathom_scan_fuse fz = {};
+  fz.tile_step = 1;
+  fz.state = S.state;
+  fz.sink_end = F.sink_end;
+  fz.local_begin = F.local_begin;
+  fz.cand_score = S.cand_score;
+  fz.cand_idx = S.cand;
+  fz.cand_count = S.cand_count;
+  fz.capacity = n;
+  rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
+  if (rc != FATHOM_OK) return rc;
+  // ---- exact selection among the candidates, then ascending emission
+  topk_select_kernel<true><<<Hq, FIN_THREADS, 0, st>>>(S.cand_score, n, 0, F, S.state, S.cand, S.bitmap, S.bitmap_words, k, idx,
+                                                       ctx->dev_status, S.tile_count, ntiles, S.cand_count, n, want);
   dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
-  topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
-                                                     S.bitmap_words, S.tile_count);
-  topk_select_kernel<<<Hq, FIN_THREADS, 0, st>>>(scores, n, L->score_stride, F, S.state, S.cand, S.bitmap,
-                                                 S.bitmap_words, k, idx, ctx->dev_status, S.tile_count, ntiles);
   topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;

@@ -1,6 +1,6 @@
 """Times (or exposes to a profiler) ONE stage of the hot path on synthetic device buffers.
 
-    python -m paper_2609_17652_b200.probe --stage scan|topk|attend|build|alloc [--n N] [--iters I] [--budget B] [--k K]
+    python -m paper_2609_17652_b200.probe --stage scan|topk|scan_topk|attend|build|alloc [--n N] [--iters I] [--budget B] [--k K]
 
 Unlike bench.py it allocates only what the chosen stage touches (random plane words and scales for the scan,
 random scores for top-k, ...), so a full-size launch fits in a few hundred MB and can be captured with ncu.
@@ -19,7 +19,7 @@ from . import binding as fb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend"])
+    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend", "scan_topk"])
     ap.add_argument("--n", type=int, default=1 << 20)
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--budget", type=int, default=48)
@@ -45,14 +45,14 @@ def main():
 
     if a.stage == "build":
         K = torch.randn(Hkv, n, d, device=dev)
-    if a.stage in ("build", "scan"):
+    if a.stage in ("build", "scan", "scan_topk"):
         planes = torch.randint(-(1 << 62), 1 << 62, (Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
         scales = torch.rand(Hkv, d, lay.scale_stride, device=dev).mul_(0.5).add_(0.01).to(torch.float16).view(torch.int16)
         if a.host_planes:
             hp = torch.empty(planes.shape, dtype=planes.dtype, pin_memory=True); hp.copy_(planes)
             hs = torch.empty(scales.shape, dtype=scales.dtype, pin_memory=True); hs.copy_(scales)
             planes, scales = hp, hs
-    if a.stage in ("scan", "topk"):
+    if a.stage in ("scan", "topk", "scan_topk"):
         scores = torch.randn(Hq, lay.score_stride, device=dev)
         idx = torch.zeros((Hq, a.k), dtype=torch.int32, device=dev)
     if a.stage == "attend":
@@ -72,6 +72,8 @@ def main():
             ctx.fathom_scan(lay, planes, scales, q, depth, hpp, scores, st)
         elif a.stage == "topk":
             ctx.fathom_topk(lay, scores, a.k, 0, 0, idx, st)
+        elif a.stage == "scan_topk":
+            ctx.fathom_scan_topk(lay, planes, scales, q, depth, hpp, a.k, 0, 0, idx, st)
         else:
             ctx.fathom_sparse_attend(lay, q, Kr, Vr, idx, a.k, 1.0 / math.sqrt(d), out, st)
 

@@ -297,3 +297,47 @@ def test_appending_keys_rebuilds_only_the_tail():
     nb = (n2 + 63) // 64
     assert torch.equal(inc_p[..., :nb], full_p[..., :nb]) and torch.equal(inc_s[..., :nb], full_s[..., :nb])
     ctx.close()
+
+
+def _fused_vs_unfused(L, B, k, hpp, mode=0, n_sink=0, n_local=0):
+    from paper_2609_17652_b200 import binding as fb
+    lay = fb.make_layout(L.Hkv, L.Hq, L.n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    dev = L.K.device
+    planes = torch.zeros((L.Hkv, 128, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
+    scales = torch.zeros((L.Hkv, 128, lay.scale_stride), dtype=torch.int16, device=dev)
+    ctx.fathom_build_planes(lay, L.K, planes, scales)
+    depth = torch.zeros((L.Hq // hpp, 128), dtype=torch.uint8, device=dev)
+    ctx.fathom_alloc_depth(lay, L.q, L.var, mode, B, hpp, depth)
+    scores = torch.zeros((L.Hq, lay.score_stride), dtype=torch.float32, device=dev)
+    want = torch.full((L.Hq, k), -1, dtype=torch.int32, device=dev)
+    got = torch.full((L.Hq, k), -2, dtype=torch.int32, device=dev)
+    ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, scores)
+    ctx.fathom_topk(lay, scores, k, n_sink, n_local, want)
+    torch.cuda.synchronize()
+    ctx.fathom_scan_topk(lay, planes, scales, L.q, depth, hpp, k, n_sink, n_local, got)
+    torch.cuda.synchronize()
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+    assert torch.equal(got, want)
+    return scores[:, :L.n].cpu().numpy(), got.cpu().numpy()
+
+
+@pytest.mark.parametrize("n,k,hpp", [(40000, 300, 4), (40000, 300, 1), (70001, 1000, 2), (9000, 64, 4), (20000, 4096, 4), (300, 300, 4)])
+def test_fused_scan_topk_equals_scan_then_topk(n, k, hpp):
+    """The fused entry point (threshold from a sampled scan, filtering scan, candidate select) must return exactly
+    the lists of fathom_scan + fathom_topk, which are themselves checked against the oracle; sampled path (n >= 16
+    tiles and >= 2 k sampled tokens) and dense fallback (short sequences) are both covered."""
+    L = make_layer(n, Hkv=2, Hq=8, seed=n + k, device="cuda")
+    s, idx = _fused_vs_unfused(L, 48, k, hpp)
+    assert np.array_equal(idx, O.topk(s.astype(np.float64), k))
+
+
+def test_fused_scan_topk_with_forced_tokens_and_degenerate_scores():
+    L = make_layer(50000, Hkv=2, Hq=8, seed=77, device="cuda")
+    _fused_vs_unfused(L, 48, 200, 4, n_sink=4, n_local=32)
+    _fused_vs_unfused(L, 16, 500, 4, mode=1)                           # fixed-channel plan
+    _fused_vs_unfused(L, 0, 100, 4)                                    # B = 0: all scores equal, every token is a candidate
+    # scores that grow along the sequence: the sampled tiles see the trend, the bound stays a bound
+    L.K[:, :, :] = L.K * torch.linspace(0.2, 3.0, L.n, device="cuda")[None, :, None]
+    _fused_vs_unfused(L, 48, 400, 4)
