@@ -401,3 +401,46 @@ def gather_union(idx: np.ndarray, G: int, Krows, Vrows):
         Ks.append(np.asarray(Krows[kv])[u])
         Vs.append(np.asarray(Vrows[kv])[u])
     return ulists, Ks, Vs, idx_local
+
+
+# --------------------------------------------------------------------------
+# O7  KLT-rotated store  (Sec. 3.5 "Basis rule"; Appendix B5 session calibration)
+# --------------------------------------------------------------------------
+def calibrate(K: np.ndarray):
+    """Per KV head: mean mu[d] and covariance C[d][d] of the session's own keys (Appendix B5: "the mean,
+    eigenbasis and eigenvalues of each layer's keys computed from the session's own prefill cache, one covariance
+    per KV head"); unbiased (n - 1), fp64.  Returns (mu [Hkv][d], C [Hkv][d][d])."""
+    K = np.asarray(K, dtype=np.float32).astype(np.float64)
+    Hkv, n, d = K.shape
+    mu = K.mean(axis=1)
+    C = np.empty((Hkv, d, d))
+    for h in range(Hkv):
+        X = K[h] - mu[h]
+        C[h] = X.T @ X / max(n - 1, 1)
+    return mu, C
+
+
+def klt_basis(C: np.ndarray):
+    """Eigenbasis V (columns = directions) and eigenvalues lambda of each covariance, largest variance first.
+    (The order of the directions does not change what is read: the depth rule ranks them by g_j anyway.)"""
+    Hkv, d, _ = C.shape
+    V = np.empty((Hkv, d, d))
+    lam = np.empty((Hkv, d))
+    for h in range(Hkv):
+        w, U = np.linalg.eigh(C[h])
+        order = np.argsort(-w, kind="stable")
+        lam[h] = np.maximum(w[order], 0.0)
+        V[h] = U[:, order]
+    return V, lam
+
+
+def rotate_keys(K: np.ndarray, mu: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """(k - mu) V per KV head (Sec. 3.5: "stores planes of (k - mu) V"), fp64."""
+    K = np.asarray(K, dtype=np.float32).astype(np.float64)
+    return np.stack([(K[h] - np.asarray(mu, dtype=np.float64)[h]) @ np.asarray(V, dtype=np.float64)[h] for h in range(K.shape[0])])
+
+
+def rotate_query(q: np.ndarray, V: np.ndarray, G: int) -> np.ndarray:
+    """q^(h) V of the head's KV head (Sec. 3.5: g_j = sum_h ((q^(h) V)_j)^2 lambda_j), fp64."""
+    q = np.asarray(q, dtype=np.float32).astype(np.float64)
+    return np.stack([q[h] @ np.asarray(V, dtype=np.float64)[h // G] for h in range(q.shape[0])])

@@ -357,3 +357,33 @@ def test_union_of_winners_properties():
         Kst[kv, :len(ul[kv])] = Ks[kv]; Vst[kv, :len(ul[kv])] = Vs[kv]
     b = O.sparse_attend(q, Kst, Vst, loc, 0.3)
     assert np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- O7 KLT-rotated store
+def test_klt_rotation_properties():
+    r = np.random.default_rng(12)
+    Hkv, G, n, d = 2, 2, 400, 16
+    A = r.standard_normal((Hkv, d, d))
+    K = (r.standard_normal((Hkv, n, d)) @ A + r.standard_normal((Hkv, 1, d)) * 3).astype(np.float32)
+    q = r.standard_normal((Hkv * G, d)).astype(np.float32)
+    mu, C = O.calibrate(K)
+    for h in range(Hkv):                                                    # library routines on the definitions
+        assert np.allclose(mu[h], K[h].astype(np.float64).mean(0), rtol=0, atol=1e-12)
+        assert np.allclose(C[h], np.cov(K[h].astype(np.float64), rowvar=False, ddof=1), rtol=1e-10, atol=1e-12)
+    V, lam = O.klt_basis(C)
+    Kr = O.rotate_keys(K, mu, V)
+    qr = O.rotate_query(q, V, G)
+    for h in range(Hkv):
+        assert np.allclose(V[h].T @ V[h], np.eye(d), atol=1e-10)             # orthonormal basis
+        assert np.all(np.diff(lam[h]) <= 1e-12)                              # largest variance first
+        cov_rot = np.cov(Kr[h], rowvar=False, ddof=1)
+        assert np.allclose(cov_rot, np.diag(lam[h]), atol=1e-8 * lam[h].max())   # rotated channels are uncorrelated,
+        assert np.allclose(Kr[h].mean(0), 0, atol=1e-10)                     # centred, with variances lambda
+    # scores are preserved up to a per-head constant: q.k = (qV).((k - mu)V) + q.mu
+    for hq in range(Hkv * G):
+        h = hq // G
+        exact = K[h].astype(np.float64) @ q[hq].astype(np.float64)
+        rot = Kr[h] @ qr[hq] + q[hq].astype(np.float64) @ mu[h]
+        assert np.allclose(exact, rot, rtol=1e-10, atol=1e-9)
+    # so the ranking, and with it the exact top-k set, is the same in both bases
+    assert np.array_equal(O.topk(O.exact_scores(q, K), 20), O.topk(np.stack([Kr[h // G] @ qr[h] for h in range(Hkv * G)]), 20))
