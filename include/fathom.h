@@ -182,6 +182,27 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
                         const void* Krows, const void* Vrows, int row_dtype, void* K_stage, void* V_stage,
                         int32_t* idx_local, int32_t* union_count, void* stream);
 
+/* ---- (7) KLT-rotated store and session calibration — Sec. 3.5 "Basis rule", Appendix B5 --------------
+ * On models without QK-norm the paper stores planes of the rotated keys (k - mu) V, V the eigenbasis of the
+ * key covariance of the KV head, and ranks channels by g_j = sum_h ((q_h V)_j)^2 lambda_j; nothing else changes
+ * (q . k = (q V) . ((k - mu) V) + q . mu, and the last term is the same for every key).  With these three calls
+ * the rest of the path is used as is: build planes from K_rot, pass q_rot to fathom_alloc_depth (with the
+ * eigenvalues as `var`) and to fathom_scan, and run attention on the original rows.
+ *   fathom_calibrate:    mean [Hkv][d] and unbiased covariance cov [Hkv][d][d] (fp32, accumulated per 8192-token
+ *                        tile in fp32 and across tiles in fp64, fixed order) of the session's own keys; the
+ *                        eigen-decomposition of the 128 x 128 covariances is the caller's (once per session).
+ *                        Uses the context scratch.
+ *   fathom_rotate_keys:  K_rot [Hkv][n][d] fp32 = (K - mean) basis, basis [Hkv][d][d] row-major with the
+ *                        directions in its columns; plain fp32 multiply-adds in a fixed order.
+ *   fathom_rotate_query: q_rot [Hq][d] = q basis[h / G].
+ * K is [Hkv][n][d], FATHOM_F32 or FATHOM_BF16, 16-byte aligned, like basis, cov and K_rot. */
+int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype, float* mean,
+                     float* cov, void* stream);
+int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype,
+                       const float* mean, const float* basis, float* K_rot, void* stream);
+int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* layout, const float* q, const float* basis,
+                        float* q_rot, void* stream);
+
 /* ---- (5b) gather + exact attention without any allocation — the paper has no counterpart ------
  * Same computation, arguments and results as fathom_sparse_attend, for callers that cannot obtain device
  * memory of their own: a plug-in that is only handed buffers by its host application, a serving process

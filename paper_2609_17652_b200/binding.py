@@ -22,7 +22,7 @@ DEV_TOPK_SHORT, DEV_WAIT_EXPIRED = 0x1, 0x2
 EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error",
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
-           "fathom_scan_topk"]
+           "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query"]
 
 
 class Layout(C.Structure):
@@ -59,6 +59,9 @@ def _load() -> C.CDLL:
     lib.fathom_scan.argtypes = [vp, LP, vp, vp, vp, vp, i32, vp, vp]
     lib.fathom_topk.argtypes = [vp, LP, vp, i32, i32, i32, vp, vp]
     lib.fathom_sparse_attend.argtypes = [vp, LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
+    lib.fathom_calibrate.argtypes = [vp, LP, vp, i32, vp, vp, vp]
+    lib.fathom_rotate_keys.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp]
+    lib.fathom_rotate_query.argtypes = [vp, LP, vp, vp, vp, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_sparse_attend_static.argtypes = [LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
@@ -149,6 +152,16 @@ class Context:
         self._check(lib.fathom_sparse_attend(self._h, C.byref(layout), _ptr(q), _ptr(Krows), _ptr(Vrows),
                                              _dtype_code(Krows) if row_dtype is None else row_dtype, _ptr(idx), k,
                                              C.c_float(softmax_scale), _ptr(out), _stream(stream)))
+
+    def fathom_calibrate(self, layout, K, mean, cov, stream=None):
+        self._check(lib.fathom_calibrate(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(cov), _stream(stream)))
+
+    def fathom_rotate_keys(self, layout, K, mean, basis, K_rot, stream=None):
+        self._check(lib.fathom_rotate_keys(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(basis),
+                                           _ptr(K_rot), _stream(stream)))
+
+    def fathom_rotate_query(self, layout, q, basis, q_rot, stream=None):
+        self._check(lib.fathom_rotate_query(self._h, C.byref(layout), _ptr(q), _ptr(basis), _ptr(q_rot), _stream(stream)))
 
     def fathom_scan_topk(self, layout, planes, scales, q, depth, heads_per_plan, k, n_sink, n_local, idx, stream=None):
         self._check(lib.fathom_scan_topk(self._h, C.byref(layout), _ptr(planes), _ptr(scales), _ptr(q), _ptr(depth),

@@ -83,4 +83,5 @@ struct fathom_attn_scratch {
 };
 fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k);
 fathom_attn_scratch fathom_carve_attn(void* base, int Hq, int k);
-size_t fathom_union_scratch_bytes(int Hkv, long long n, int capacity);   // bitmap + word ranks + union list
+size_t fathom_union_scratch_bytes(int Hkv, long long n, int capacity);
+size_t fathom_calib_scratch_bytes(int Hkv, long long n);                  // partial means and covariances   // bitmap + word ranks + union list

@@ -1,0 +1,246 @@
+// KLT-rotated store (Sec. 3.5 "Basis rule") and session calibration (Appendix B5).
+//
+//   fathom_calibrate      mean and covariance of a session's own keys, one covariance per KV head;
+//   fathom_rotate_keys    K' = (K - mu) V, the keys whose planes the rotated variant stores;
+//   fathom_rotate_query   q' = q V, from which g_j = sum_h (q'_hj)^2 lambda_j is formed by fathom_alloc_depth
+//                         (eigenvalues passed as `var`).
+// The eigen-decomposition of the 128 x 128 covariances is left to the caller (once per session and KV head).
+//
+// Rotation and covariance are the same register-tiled product  C[i][j] += P[t][i] * Q[t][j]  over a shared-memory
+// panel: 256 threads, each an 8 x 8 block of the 128 x 128 result (columns split 4 + 4 so that the 16-byte panel
+// loads of neighbouring lanes are contiguous).  They run in plain fp32 FMAs in a fixed order: the rotated keys feed
+// a quantiser whose codes must not depend on the machine, which rules out tf32; a tensor-core version would need a
+// three-way split of the operands.
+#include "fathom_common.cuh"
+
+namespace {
+
+constexpr int KT_THREADS = 256;
+constexpr int PANEL = FATHOM_D + 4;                          // floats per panel row (16-byte aligned, staggers banks)
+constexpr int COV_ROWS = 8192;                               // rows per CTA of the covariance pass
+constexpr int MEAN_ROWS = 1024;                              // rows per CTA of the mean pass
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// acc[i][j] += sum_t P[t][8 ty + i] * Q[t][cols(tx, j)],  cols = 4 tx + j (j < 4), 64 + 4 tx + (j - 4) (j >= 4)
+__device__ __forceinline__ void panel_product(const float* __restrict__ P, const float* __restrict__ Q, int T, int ty, int tx,
+                                              float (&acc)[8][8]) {
+#pragma unroll 4
+  for (int t = 0; t < T; ++t) {
+    const float4 a0 = *reinterpret_cast<const float4*>(P + t * PANEL + 8 * ty);
+    const float4 a1 = *reinterpret_cast<const float4*>(P + t * PANEL + 8 * ty + 4);
+    const float4 b0 = *reinterpret_cast<const float4*>(Q + t * PANEL + 4 * tx);
+    const float4 b1 = *reinterpret_cast<const float4*>(Q + t * PANEL + 64 + 4 * tx);
+    const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+  }
+}
+
+// ---- K' = (K - mu) V : one CTA per 128 tokens of one KV head -------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(KT_THREADS)
+rotate_keys_kernel(const T* __restrict__ K, const float* __restrict__ mean, const float* __restrict__ basis,
+                   float* __restrict__ K_rot, long long n) {
+  extern __shared__ __align__(16) float sm[];
+  float* As = sm;                                             // [c][row]: the token tile, transposed, mean removed
+  float* Bs = sm + FATHOM_D * PANEL;                          // [c][j]  : the basis
+  const int kv = blockIdx.y, tid = threadIdx.x;
+  const long long r0 = (long long)blockIdx.x * FATHOM_D;
+  const T* Kh = K + ((size_t)kv * (size_t)n + (size_t)r0) * FATHOM_D;
+  const float* V = basis + (size_t)kv * FATHOM_D * FATHOM_D;
+  const float* mu = mean + (size_t)kv * FATHOM_D;
+  for (int e = tid; e < FATHOM_D * (FATHOM_D / 4); e += KT_THREADS) {        // basis rows, 16 bytes a piece
+    const int c = e / (FATHOM_D / 4), j4 = e % (FATHOM_D / 4);
+    *reinterpret_cast<float4*>(Bs + c * PANEL + 4 * j4) = __ldg(reinterpret_cast<const float4*>(V + c * FATHOM_D) + j4);
+  }
+  // token tile: lane = row (so the transposed stores of a warp are conflict-free), 4 channels per step
+  for (int e = tid; e < FATHOM_D * (FATHOM_D / 4); e += KT_THREADS) {
+    const int row = e % FATHOM_D, c4 = e / FATHOM_D;
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (r0 + row < n) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x) v[x] = to_f32(Kh[(size_t)row * FATHOM_D + 4 * c4 + x]) - mu[4 * c4 + x];
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x) As[(4 * c4 + x) * PANEL + row] = v[x];
+  }
+  __syncthreads();
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+  panel_product(As, Bs, FATHOM_D, ty, tx, acc);
+  float* out = K_rot + ((size_t)kv * (size_t)n + (size_t)r0) * FATHOM_D;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = 8 * ty + i;
+    if (r0 + row < n) {
+      *reinterpret_cast<float4*>(out + (size_t)row * FATHOM_D + 4 * tx) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+      *reinterpret_cast<float4*>(out + (size_t)row * FATHOM_D + 64 + 4 * tx) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+    }
+  }
+}
+
+// ---- q' = q V ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(FATHOM_D)
+rotate_query_kernel(const float* __restrict__ q, const float* __restrict__ basis, float* __restrict__ q_rot, int G) {
+  __shared__ float s_q[FATHOM_D];
+  const int h = blockIdx.x, j = threadIdx.x;
+  const float* V = basis + (size_t)(h / G) * FATHOM_D * FATHOM_D;
+  s_q[j] = q[(size_t)h * FATHOM_D + j];
+  __syncthreads();
+  float acc = 0.0f;
+#pragma unroll 8
+  for (int c = 0; c < FATHOM_D; ++c) acc = fmaf(s_q[c], __ldg(V + c * FATHOM_D + j), acc);
+  q_rot[(size_t)h * FATHOM_D + j] = acc;
+}
+
+// ---- calibration ------------------------------------------------------------------------------------------------
+// (1) partial column sums of MEAN_ROWS tokens; (2) their fp64 sum in tile order -> mean;
+// (3) partial (K - mu)^T (K - mu) of COV_ROWS tokens; (4) their fp64 sum in tile order / (n - 1) -> covariance.
+template <typename T>
+__global__ void __launch_bounds__(KT_THREADS)
+mean_partial_kernel(const T* __restrict__ K, long long n, float* __restrict__ partial, int tiles) {
+  __shared__ float s_part[2][FATHOM_D];
+  const int kv = blockIdx.y, tid = threadIdx.x, c = tid & (FATHOM_D - 1), half = tid >> 7;
+  const long long r0 = (long long)blockIdx.x * MEAN_ROWS;
+  const long long r1 = min(r0 + MEAN_ROWS, n);
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
+  float s = 0.0f;
+  for (long long r = r0 + half; r < r1; r += 2) s += to_f32(Kh[(size_t)r * FATHOM_D + c]);
+  s_part[half][c] = s;
+  __syncthreads();
+  if (half == 0) partial[((size_t)kv * tiles + blockIdx.x) * FATHOM_D + c] = s_part[0][c] + s_part[1][c];
+}
+
+__global__ void __launch_bounds__(FATHOM_D)
+mean_final_kernel(const float* __restrict__ partial, int tiles, long long n, float* __restrict__ mean) {
+  const int kv = blockIdx.x, c = threadIdx.x;
+  double s = 0.0;
+  for (int t = 0; t < tiles; ++t) s += (double)partial[((size_t)kv * tiles + t) * FATHOM_D + c];
+  mean[(size_t)kv * FATHOM_D + c] = (float)(s / (double)n);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(KT_THREADS)
+cov_partial_kernel(const T* __restrict__ K, long long n, const float* __restrict__ mean, float* __restrict__ partial, int tiles) {
+  extern __shared__ __align__(16) float sm[];
+  float* Xs = sm;                                             // [row][c], mean removed, 128 rows at a time
+  const int kv = blockIdx.y, tid = threadIdx.x;
+  const long long t0 = (long long)blockIdx.x * COV_ROWS;
+  const long long t1 = min(t0 + COV_ROWS, n);
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
+  const float* mu = mean + (size_t)kv * FATHOM_D;
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+  for (long long r0 = t0; r0 < t1; r0 += FATHOM_D) {
+    __syncthreads();
+    for (int e = tid; e < FATHOM_D * (FATHOM_D / 4); e += KT_THREADS) {      // consecutive threads = consecutive channels
+      const int row = e / (FATHOM_D / 4), c4 = e % (FATHOM_D / 4);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r0 + row < t1) {
+        const T* src = Kh + (size_t)(r0 + row) * FATHOM_D + 4 * c4;
+        v = make_float4(to_f32(src[0]) - mu[4 * c4], to_f32(src[1]) - mu[4 * c4 + 1], to_f32(src[2]) - mu[4 * c4 + 2],
+                        to_f32(src[3]) - mu[4 * c4 + 3]);
+      }
+      *reinterpret_cast<float4*>(Xs + row * PANEL + 4 * c4) = v;
+    }
+    __syncthreads();
+    panel_product(Xs, Xs, FATHOM_D, ty, tx, acc);            // rows past the end are zero and add nothing
+  }
+  float* out = partial + ((size_t)kv * tiles + blockIdx.x) * FATHOM_D * FATHOM_D;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = 8 * ty + i;
+    *reinterpret_cast<float4*>(out + row * FATHOM_D + 4 * tx) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    *reinterpret_cast<float4*>(out + row * FATHOM_D + 64 + 4 * tx) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+  }
+}
+
+__global__ void __launch_bounds__(FATHOM_D)
+cov_final_kernel(const float* __restrict__ partial, int tiles, long long n, float* __restrict__ cov) {
+  const int kv = blockIdx.y, i = blockIdx.x, j = threadIdx.x;
+  double s = 0.0;
+  for (int t = 0; t < tiles; ++t) s += (double)partial[(((size_t)kv * tiles + t) * FATHOM_D + i) * FATHOM_D + j];
+  cov[((size_t)kv * FATHOM_D + i) * FATHOM_D + j] = (float)(s / (double)(n > 1 ? n - 1 : 1));
+}
+
+}  // namespace
+
+size_t fathom_calib_scratch_bytes(int Hkv, long long n) {
+  const size_t mt = (size_t)((n + MEAN_ROWS - 1) / MEAN_ROWS), ct = (size_t)((n + COV_ROWS - 1) / COV_ROWS);
+  return fathom_round_up((size_t)Hkv * mt * FATHOM_D * 4, 256) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256);
+}
+
+extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* mean, float* cov,
+                                void* stream) {
+  if (!ctx || !K || !mean || !cov) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k_dtype != FATHOM_F32 && k_dtype != FATHOM_BF16) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(K) || !fathom_aligned16(cov)) return FATHOM_ERR_ALIGNMENT;
+  const int Hkv = L->n_kv_heads;
+  const long long n = L->n;
+  if (fathom_calib_scratch_bytes(Hkv, n) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  const int mt = (int)((n + MEAN_ROWS - 1) / MEAN_ROWS), ct = (int)((n + COV_ROWS - 1) / COV_ROWS);
+  float* pmean = static_cast<float*>(ctx->scratch);
+  float* pcov = reinterpret_cast<float*>(static_cast<char*>(ctx->scratch) + fathom_round_up((size_t)Hkv * mt * FATHOM_D * 4, 256));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);
+  if (k_dtype == FATHOM_F32) {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    mean_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, pmean, mt);
+    mean_final_kernel<<<Hkv, FATHOM_D, 0, st>>>(pmean, mt, n, mean);
+    cov_partial_kernel<float><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const float*>(K), n, mean, pcov, ct);
+  } else {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    mean_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, pmean, mt);
+    mean_final_kernel<<<Hkv, FATHOM_D, 0, st>>>(pmean, mt, n, mean);
+    cov_partial_kernel<__nv_bfloat16><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(K), n, mean, pcov, ct);
+  }
+  cov_final_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, ct, n, cov);
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+extern "C" int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
+                                  const float* basis, float* K_rot, void* stream) {
+  if (!ctx || !K || !mean || !basis || !K_rot) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k_dtype != FATHOM_F32 && k_dtype != FATHOM_BF16) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(K) || !fathom_aligned16(basis) || !fathom_aligned16(K_rot)) return FATHOM_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t smem = (size_t)2 * FATHOM_D * PANEL * sizeof(float);
+  dim3 grid((unsigned)((L->n + FATHOM_D - 1) / FATHOM_D), (unsigned)L->n_kv_heads);
+  if (k_dtype == FATHOM_F32) {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(rotate_keys_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    rotate_keys_kernel<float><<<grid, KT_THREADS, smem, st>>>(static_cast<const float*>(K), mean, basis, K_rot, L->n);
+  } else {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(rotate_keys_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    rotate_keys_kernel<__nv_bfloat16><<<grid, KT_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(K), mean, basis, K_rot, L->n);
+  }
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+extern "C" int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* L, const float* q, const float* basis, float* q_rot,
+                                   void* stream) {
+  if (!ctx || !q || !basis || !q_rot) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  rotate_query_kernel<<<L->n_q_heads, FATHOM_D, 0, static_cast<cudaStream_t>(stream)>>>(q, basis, q_rot, L->n_q_heads / L->n_kv_heads);
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}

@@ -341,3 +341,42 @@ def test_fused_scan_topk_with_forced_tokens_and_degenerate_scores():
     # scores that grow along the sequence: the sampled tiles see the trend, the bound stays a bound
     L.K[:, :, :] = L.K * torch.linspace(0.2, 3.0, L.n, device="cuda")[None, :, None]
     _fused_vs_unfused(L, 48, 400, 4)
+
+
+@pytest.mark.parametrize("n", [5000, 8192 + 77])
+def test_klt_rotated_store(n):
+    """Session calibration, rotation of keys and queries against the oracle, and the rotated variant end to end:
+    planes of (K - mu) V, importance from q V and the eigenvalues, same scan / top-k / attention."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq, G, k = 2, 8, 4, 128
+    L = make_layer(n, Hkv, Hq, seed=41, device="cuda")
+    mix = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda"))[0]          # correlate the channels
+    K = (torch.bmm(L.K, mix) + 0.5).contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    mean = torch.zeros((Hkv, 128), device="cuda"); cov = torch.zeros((Hkv, 128, 128), device="cuda")
+    ctx.fathom_calibrate(lay, K, mean, cov)
+    torch.cuda.synchronize()
+    Kh = K.cpu().numpy()
+    mu_ref, C_ref = O.calibrate(Kh)
+    assert np.allclose(mean.cpu().numpy(), mu_ref, rtol=1e-5, atol=1e-5)
+    scale = np.abs(C_ref).max(axis=(1, 2), keepdims=True)
+    assert np.all(np.abs(cov.cpu().numpy() - C_ref) <= 2e-5 * scale)
+    # basis from the oracle's eigen-decomposition of the GPU's own statistics (stage isolation)
+    V_ref, lam_ref = O.klt_basis(cov.cpu().numpy().astype(np.float64))
+    V = torch.from_numpy(V_ref.astype(np.float32)).cuda().contiguous()
+    lam = torch.from_numpy(lam_ref.astype(np.float32)).cuda().contiguous()
+    K_rot = torch.full((Hkv, n, 128), float("nan"), device="cuda"); q_rot = torch.zeros((Hq, 128), device="cuda")
+    ctx.fathom_rotate_keys(lay, K, mean, V, K_rot)
+    ctx.fathom_rotate_query(lay, L.q, V, q_rot)
+    torch.cuda.synchronize()
+    Kr_ref = O.rotate_keys(Kh, mean.cpu().numpy(), V.cpu().numpy())
+    rown = np.linalg.norm(Kr_ref, axis=2, keepdims=True)
+    assert np.all(np.abs(K_rot.cpu().numpy() - Kr_ref) <= 1e-5 * rown + 1e-6)
+    qr_ref = O.rotate_query(L.q.cpu().numpy(), V.cpu().numpy(), G)
+    assert np.allclose(q_rot.cpu().numpy(), qr_ref, rtol=1e-5, atol=1e-5)
+    ctx.close()
+    # the rest of the path on the rotated store, checked stage by stage against the oracle
+    L.K, L.q, L.var = K_rot, q_rot, lam
+    g, ref = check_all(L, B=48, k=k, hpp=G)
+    assert np.all(g["depth"].sum(1) == 48)
