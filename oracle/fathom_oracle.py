@@ -1,7 +1,7 @@
 """CPU oracle for the Fathom decode-step hot path (TEST INFRASTRUCTURE ONLY).
 
 This module is the slow, plain restatement of what the five calls of the
-library compute, written from the paper's definitions in numpy / fp64.  It is
+library compute (and of the calibration-time steps around them), written from the paper's definitions in numpy / fp64.  It is
 imported only by the tests, by the smoke check and by the benchmark's
 `cpu_baseline` / `--impl reference` legs.  It shares no code with the CUDA
 path and never imports the product package; the product never imports it.
@@ -444,3 +444,61 @@ def rotate_query(q: np.ndarray, V: np.ndarray, G: int) -> np.ndarray:
     """q^(h) V of the head's KV head (Sec. 3.5: g_j = sum_h ((q^(h) V)_j)^2 lambda_j), fp64."""
     q = np.asarray(q, dtype=np.float32).astype(np.float64)
     return np.stack([q[h] @ np.asarray(V, dtype=np.float64)[h // G] for h in range(q.shape[0])])
+
+
+# --------------------------------------------------------------------------
+# O8  per-channel key statistics  (Sec. 3.3: Var(k_j) in the importance g_j; Appendix B5: taken from the
+#     session's own keys)
+# --------------------------------------------------------------------------
+def channel_variance(K: np.ndarray):
+    """Per (KV head, channel): mean and unbiased sample variance  sum_i (k_ij - mean_j)^2 / (n - 1)  of the
+    session's keys, written out as the definition in fp64 (Appendix A prints n - 1 values).
+    Returns (mean [Hkv][d], var [Hkv][d])."""
+    K = np.asarray(K, dtype=np.float32).astype(np.float64)
+    Hkv, n, d = K.shape
+    mean = np.empty((Hkv, d))
+    var = np.empty((Hkv, d))
+    for h in range(Hkv):
+        for j in range(d):
+            col = K[h, :, j]
+            m = col.sum() / n
+            mean[h, j] = m
+            dev = col - m
+            var[h, j] = (dev * dev).sum() / max(n - 1, 1)
+    return mean, var
+
+
+# --------------------------------------------------------------------------
+# O9  per-layer budgets  (Sec. 3.4 "Per-layer budgets")
+# --------------------------------------------------------------------------
+def plan_layer_budgets(err: np.ndarray, levels, target_mean: float) -> np.ndarray:
+    """Greedy per-layer plan: budgets B_l from the ascending list `levels` (the paper's range is 24..128) at a
+    target mean.  err[l][i] is the measured error of layer l at budget levels[i].  Every layer starts at the
+    lowest level; each step raises one layer by one level, namely the layer with the largest error drop per added
+    bit  (err[l][i] - err[l][i+1]) / (levels[i+1] - levels[i]),  ties to the lower layer; a step is admissible
+    while the sum of budgets stays <= target_mean * L; the plan is final when no step is admissible.
+    (The paper fixes neither the start nor the step; this reading moves bits one level at a time from the floor.)
+    Returns the level INDEX per layer."""
+    err = np.asarray(err, dtype=np.float64)
+    levels = [int(b) for b in levels]
+    L, nlev = err.shape
+    assert nlev == len(levels) and all(levels[i] < levels[i + 1] for i in range(nlev - 1))
+    cur = np.zeros(L, dtype=np.int64)
+    total = L * levels[0]
+    cap = float(target_mean) * L
+    while True:
+        best, best_gain = -1, 0.0
+        for l in range(L):
+            i = int(cur[l])
+            if i + 1 >= nlev:
+                continue
+            step = levels[i + 1] - levels[i]
+            if total + step > cap:
+                continue
+            gain = (err[l, i] - err[l, i + 1]) / step
+            if best < 0 or gain > best_gain:
+                best, best_gain = l, gain
+        if best < 0:
+            return cur
+        total += levels[int(cur[best]) + 1] - levels[int(cur[best])]
+        cur[best] += 1

@@ -387,3 +387,69 @@ def test_klt_rotation_properties():
         assert np.allclose(exact, rot, rtol=1e-10, atol=1e-9)
     # so the ranking, and with it the exact top-k set, is the same in both bases
     assert np.array_equal(O.topk(O.exact_scores(q, K), 20), O.topk(np.stack([Kr[h // G] @ qr[h] for h in range(Hkv * G)]), 20))
+
+
+# ---------------------------------------------------------------- O8 per-channel statistics
+def test_channel_variance_matches_the_worked_example_closed_forms_and_the_covariance_diagonal():
+    import json, os
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "appendix_a_worked_example.json")))
+    K = np.asarray(g["K"], dtype=np.float32)[None]                           # six keys, four channels
+    _, var = O.channel_variance(K)
+    assert np.allclose(var[0], g["var_printed"], atol=6e-4)                  # Appendix A prints n - 1 variances to 3 decimals
+    # closed form: the integers 0 .. n-1 have mean (n - 1)/2 and unbiased variance n (n + 1) / 12
+    n = 1000
+    ramp = np.arange(n, dtype=np.float32)[None, :, None] * np.ones((1, 1, 3), np.float32)
+    ramp[0, :, 1] += 5.0                                                      # a shift moves the mean only
+    ramp[0, :, 2] *= -2.0                                                     # a scale multiplies the variance by its square
+    mean, var = O.channel_variance(ramp)
+    assert np.allclose(mean[0], [(n - 1) / 2, (n - 1) / 2 + 5, -(n - 1)], rtol=1e-13)
+    assert np.allclose(var[0], [n * (n + 1) / 12, n * (n + 1) / 12, 4 * n * (n + 1) / 12], rtol=1e-13)
+    # library routine and the diagonal of the session covariance (a different code path)
+    K = rng_keys(3, 2, 777, 9)
+    mean, var = O.channel_variance(K)
+    mu, C = O.calibrate(K)
+    for h in range(2):
+        assert np.allclose(var[h], np.var(K[h].astype(np.float64), axis=0, ddof=1), rtol=1e-12)
+        assert np.allclose(var[h], np.diag(C[h]), rtol=1e-12)
+        assert np.allclose(mean[h], mu[h], rtol=0, atol=1e-13)
+    # a single key has no spread
+    _, v1 = O.channel_variance(K[:, :1])
+    assert np.all(v1 == 0)
+
+
+# ---------------------------------------------------------------- O9 per-layer budgets
+def test_layer_budget_plan_hand_example():
+    levels = [24, 32, 40, 48]
+    #            24    32    40    48
+    err = [[1.00, 0.50, 0.40, 0.39],     # layer 0: big first drop
+           [1.00, 0.90, 0.30, 0.29],     # layer 1: the drop comes late
+           [0.20, 0.19, 0.18, 0.17]]     # layer 2: flat
+    # mean 32 -> 24 bits to hand out in steps of 8: layer 0 (0.50/8); then layers 0 and 1 both offer 0.10/8 and the
+    # tie goes to layer 0; then layer 1 (0.10/8 against layer 0's 0.01/8)
+    assert list(O.plan_layer_budgets(err, levels, 32)) == [2, 1, 0]
+    # mean 40 -> 48 bits = 6 steps: continue 1 (0.60/8), then 0 (0.01/8) == 1 (0.01/8) == 2 (0.01/8) -> lower layer 0, then 1
+    assert list(O.plan_layer_budgets(err, levels, 40)) == [3, 3, 0]
+    # the floor and the ceiling
+    assert list(O.plan_layer_budgets(err, levels, 24)) == [0, 0, 0]
+    assert list(O.plan_layer_budgets(err, levels, 48)) == [3, 3, 3]
+    assert list(O.plan_layer_budgets(err, levels, 1000)) == [3, 3, 3]
+    # a target between two sums is never exceeded: mean 30 allows 18 extra bits = two steps
+    assert list(O.plan_layer_budgets(err, levels, 30)) == [2, 0, 0]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_layer_budget_plan_is_optimal_for_convex_error_curves(seed):
+    """Marginal analysis: with evenly spaced levels and error curves that fall with diminishing returns, moving bits
+    one level at a time to the steepest layer minimises the summed error among all plans of the same total."""
+    r = np.random.default_rng(seed)
+    L, nlev = 4, 5
+    levels = [24 + 8 * i for i in range(nlev)]
+    drops = -np.sort(-r.uniform(0.01, 1.0, size=(L, nlev - 1)), axis=1)       # decreasing drops = convex curve
+    err = np.concatenate([np.full((L, 1), 5.0), 5.0 - np.cumsum(drops, axis=1)], axis=1)
+    for steps in range(0, L * (nlev - 1) + 1, 3):
+        target = (L * levels[0] + 8 * steps) / L
+        plan = O.plan_layer_budgets(err, levels, target)
+        assert plan.sum() == steps
+        best = min(sum(err[l, c[l]] for l in range(L))
+                   for c in itertools.product(range(nlev), repeat=L) if sum(c) == steps)
+        assert abs(sum(err[l, plan[l]] for l in range(L)) - best) < 1e-12
