@@ -188,8 +188,9 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
  * (q . k = (q V) . ((k - mu) V) + q . mu, and the last term is the same for every key).  With these three calls
  * the rest of the path is used as is: build planes from K_rot, pass q_rot to fathom_alloc_depth (with the
  * eigenvalues as `var`) and to fathom_scan, and run attention on the original rows.
- *   fathom_calibrate:    mean [Hkv][d] and unbiased covariance cov [Hkv][d][d] (fp32, accumulated per 8192-token
- *                        tile in fp32 and across tiles in fp64, fixed order) of the session's own keys; the
+ *   fathom_calibrate:    mean [Hkv][d] (as fathom_channel_variance computes it) and unbiased covariance
+ *                        cov [Hkv][d][d] (fp32, accumulated per 8192-token tile in fp32 and across tiles in fp64,
+ *                        fixed order) of the session's own keys; the
  *                        eigen-decomposition of the 128 x 128 covariances is the caller's (once per session).
  *                        Uses the context scratch.
  *   fathom_rotate_keys:  K_rot [Hkv][n][d] fp32 = (K - mean) basis, basis [Hkv][d][d] row-major with the
@@ -202,6 +203,26 @@ int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* layout, const void*
                        const float* mean, const float* basis, float* K_rot, void* stream);
 int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* layout, const float* q, const float* basis,
                         float* q_rot, void* stream);
+
+/* ---- (8) per-channel key statistics — Sec. 3.3 (the Var(k_j) of g_j), Appendix B5 (from the session's own keys)
+ * mean [Hkv][d] and var [Hkv][d] (device, fp32): mean and unbiased (n - 1) sample variance of every channel of
+ * K [Hkv][n][d] (device, FATHOM_F32 or FATHOM_BF16, 16-byte aligned).  One pass over the keys; per 1024-token
+ * tile fp32 sums of the keys shifted by the tile's first key, merged across tiles in fp64 in tile order
+ * (deterministic).  var feeds fathom_alloc_depth for the raw store.  n = 1 gives var = 0.  Uses the context scratch
+ * (FATHOM_ERR_SCRATCH_TOO_SMALL if the context was created for a smaller layout). */
+int fathom_channel_variance(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype, float* mean,
+                            float* var, void* stream);
+
+/* ---- (9) per-layer budgets — Sec. 3.4 "Per-layer budgets" --------------------------------------------------
+ * HOST function, no GPU work: the greedy plan that assigns each of n_layers layers one of n_levels budgets
+ * (levels[], strictly ascending bits, e.g. 24 .. 128) at a target mean.  err [n_layers][n_levels] (host, row-major)
+ * is the caller's measured error of layer l at budget levels[i].  Every layer starts at levels[0]; each step raises
+ * one layer by one level, the layer with the largest error drop per added bit (ties: lower layer), while the sum of
+ * budgets stays <= target_mean * n_layers.  level_index [n_layers] (host) receives the chosen level per layer; pass
+ * levels[level_index[l]] as `budget` to fathom_alloc_depth for layer l.  The paper fixes neither start nor step size;
+ * this is the reading taken.  FATHOM_ERR_INVALID_ARG on NULL, non-ascending levels or NaN errors. */
+int fathom_plan_layer_budgets(const double* err, int n_layers, int n_levels, const int* levels, double target_mean,
+                              int* level_index);
 
 /* ---- (5b) gather + exact attention without any allocation — the paper has no counterpart ------
  * Same computation, arguments and results as fathom_sparse_attend, for callers that cannot obtain device

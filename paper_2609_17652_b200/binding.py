@@ -22,7 +22,8 @@ DEV_TOPK_SHORT, DEV_WAIT_EXPIRED = 0x1, 0x2
 EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_strerror", "fathom_last_cuda_error",
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
-           "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query"]
+           "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
+           "fathom_channel_variance", "fathom_plan_layer_budgets"]
 
 
 class Layout(C.Structure):
@@ -62,6 +63,8 @@ def _load() -> C.CDLL:
     lib.fathom_calibrate.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_rotate_keys.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp]
     lib.fathom_rotate_query.argtypes = [vp, LP, vp, vp, vp, vp]
+    lib.fathom_channel_variance.argtypes = [vp, LP, vp, i32, vp, vp, vp]
+    lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_sparse_attend_static.argtypes = [LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
@@ -156,6 +159,9 @@ class Context:
     def fathom_calibrate(self, layout, K, mean, cov, stream=None):
         self._check(lib.fathom_calibrate(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(cov), _stream(stream)))
 
+    def fathom_channel_variance(self, layout, K, mean, var, stream=None):
+        self._check(lib.fathom_channel_variance(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(var), _stream(stream)))
+
     def fathom_rotate_keys(self, layout, K, mean, basis, K_rot, stream=None):
         self._check(lib.fathom_rotate_keys(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(basis),
                                            _ptr(K_rot), _stream(stream)))
@@ -193,6 +199,19 @@ def fathom_sparse_attend_static(layout, q, Krows, Vrows, idx, k, softmax_scale, 
                                          C.c_float(softmax_scale), _ptr(out), _stream(stream))
     if rc != 0:
         raise FathomError(rc)
+
+
+def fathom_plan_layer_budgets(err, levels, target_mean: float):
+    """Host-side greedy per-layer plan: err [L][n_levels] (any nested sequence of floats), levels ascending ints.
+    Returns the chosen level index per layer (marshalling only: the plan is computed inside the library)."""
+    L, nlev = len(err), len(levels)
+    flat = (C.c_double * (L * nlev))(*[float(x) for row in err for x in row])
+    lev = (C.c_int * nlev)(*[int(b) for b in levels])
+    out = (C.c_int * L)()
+    rc = lib.fathom_plan_layer_budgets(flat, L, nlev, lev, C.c_double(target_mean), out)
+    if rc != 0:
+        raise FathomError(rc)
+    return list(out)
 
 
 def fathom_scratch_bytes(layout: Layout, k: int) -> int:

@@ -1,5 +1,6 @@
 // KLT-rotated store (Sec. 3.5 "Basis rule") and session calibration (Appendix B5).
 //
+//   fathom_channel_variance  per-channel mean and variance of a session's keys (the raw store's Var(k_j));
 //   fathom_calibrate      mean and covariance of a session's own keys, one covariance per KV head;
 //   fathom_rotate_keys    K' = (K - mu) V, the keys whose planes the rotated variant stores;
 //   fathom_rotate_query   q' = q V, from which g_j = sum_h (q'_hj)^2 lambda_j is formed by fathom_alloc_depth
@@ -103,31 +104,8 @@ rotate_query_kernel(const float* __restrict__ q, const float* __restrict__ basis
 }
 
 // ---- calibration ------------------------------------------------------------------------------------------------
-// (1) partial column sums of MEAN_ROWS tokens; (2) their fp64 sum in tile order -> mean;
-// (3) partial (K - mu)^T (K - mu) of COV_ROWS tokens; (4) their fp64 sum in tile order / (n - 1) -> covariance.
-template <typename T>
-__global__ void __launch_bounds__(KT_THREADS)
-mean_partial_kernel(const T* __restrict__ K, long long n, float* __restrict__ partial, int tiles) {
-  __shared__ float s_part[2][FATHOM_D];
-  const int kv = blockIdx.y, tid = threadIdx.x, c = tid & (FATHOM_D - 1), half = tid >> 7;
-  const long long r0 = (long long)blockIdx.x * MEAN_ROWS;
-  const long long r1 = min(r0 + MEAN_ROWS, n);
-  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
-  float s = 0.0f;
-  for (long long r = r0 + half; r < r1; r += 2) s += to_f32(Kh[(size_t)r * FATHOM_D + c]);
-  s_part[half][c] = s;
-  __syncthreads();
-  if (half == 0) partial[((size_t)kv * tiles + blockIdx.x) * FATHOM_D + c] = s_part[0][c] + s_part[1][c];
-}
-
-__global__ void __launch_bounds__(FATHOM_D)
-mean_final_kernel(const float* __restrict__ partial, int tiles, long long n, float* __restrict__ mean) {
-  const int kv = blockIdx.x, c = threadIdx.x;
-  double s = 0.0;
-  for (int t = 0; t < tiles; ++t) s += (double)partial[((size_t)kv * tiles + t) * FATHOM_D + c];
-  mean[(size_t)kv * FATHOM_D + c] = (float)(s / (double)n);
-}
-
+// (1) the mean from the one-pass statistics kernels below; (2) partial (K - mu)^T (K - mu) of COV_ROWS tokens;
+// (3) their fp64 sum in tile order / (n - 1) -> covariance.
 template <typename T>
 __global__ void __launch_bounds__(KT_THREADS)
 cov_partial_kernel(const T* __restrict__ K, long long n, const float* __restrict__ mean, float* __restrict__ partial, int tiles) {
@@ -172,15 +150,134 @@ __global__ void __launch_bounds__(FATHOM_D)
 cov_final_kernel(const float* __restrict__ partial, int tiles, long long n, float* __restrict__ cov) {
   const int kv = blockIdx.y, i = blockIdx.x, j = threadIdx.x;
   double s = 0.0;
+#pragma unroll 8
   for (int t = 0; t < tiles; ++t) s += (double)partial[(((size_t)kv * tiles + t) * FATHOM_D + i) * FATHOM_D + j];
   cov[((size_t)kv * FATHOM_D + i) * FATHOM_D + j] = (float)(s / (double)(n > 1 ? n - 1 : 1));
 }
 
+// ---- per-channel mean and variance (the Var(k_j) of the importance g_j) -----------------------------------------
+// One pass over the keys.  A CTA takes MEAN_ROWS tokens of one KV head and, per channel, the sums of (x - s) and
+// (x - s)^2 with s the tile's first key (a shift inside the data keeps the squares free of cancellation); the
+// final kernel merges the tiles in fp64 in tile order: mean_t = s + S1/n_t, M2_t = S2 - S1^2/n_t,
+// M2 = sum M2_t + sum n_t (mean_t - mean)^2.
+__device__ __forceinline__ float4 load4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                     __uint_as_float(u.y & 0xffff0000u));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(KT_THREADS)
+var_partial_kernel(const T* __restrict__ K, long long n, float* __restrict__ partial, int tiles) {
+  __shared__ float4 s_sum[8][32], s_sq[8][32];
+  const int kv = blockIdx.y, tid = threadIdx.x, cq = tid & 31, rl = tid >> 5;   // warp = row lane, lane = 4 channels
+  const long long r0 = (long long)blockIdx.x * MEAN_ROWS;
+  const long long r1 = min(r0 + MEAN_ROWS, n);
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D + 4 * cq;
+  const float4 sh = load4(Kh + (size_t)r0 * FATHOM_D);
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll 8
+  for (long long r = r0 + rl; r < r1; r += 8) {
+    const float4 x = load4(Kh + (size_t)r * FATHOM_D);
+    const float dx = x.x - sh.x, dy = x.y - sh.y, dz = x.z - sh.z, dw = x.w - sh.w;
+    a.x += dx; a.y += dy; a.z += dz; a.w += dw;
+    b.x = fmaf(dx, dx, b.x); b.y = fmaf(dy, dy, b.y); b.z = fmaf(dz, dz, b.z); b.w = fmaf(dw, dw, b.w);
+  }
+  s_sum[rl][cq] = a;
+  s_sq[rl][cq] = b;
+  __syncthreads();
+  if (rl == 0) {
+#pragma unroll
+    for (int w = 1; w < 8; ++w) {                                // row lanes in a fixed order
+      const float4 u = s_sum[w][cq], v = s_sq[w][cq];
+      a.x += u.x; a.y += u.y; a.z += u.z; a.w += u.w;
+      b.x += v.x; b.y += v.y; b.z += v.z; b.w += v.w;
+    }
+    float* out = partial + ((size_t)kv * tiles + blockIdx.x) * 3 * FATHOM_D + 4 * cq;
+    *reinterpret_cast<float4*>(out) = sh;
+    *reinterpret_cast<float4*>(out + FATHOM_D) = a;
+    *reinterpret_cast<float4*>(out + 2 * FATHOM_D) = b;
+  }
+}
+
+// 1024 threads per KV head: thread (channel, lane) merges tiles lane, lane + 8, ... and the eight lanes are then
+// combined in lane order, so the result does not depend on scheduling.
+constexpr int VF_LANES = 8;
+__global__ void __launch_bounds__(FATHOM_D * VF_LANES)
+var_final_kernel(const float* __restrict__ partial, int tiles, long long n, float* __restrict__ mean, float* __restrict__ var) {
+  __shared__ double s_acc[VF_LANES][FATHOM_D];
+  __shared__ double s_mu[FATHOM_D];
+  const int kv = blockIdx.x, c = threadIdx.x & (FATHOM_D - 1), tl = threadIdx.x >> 7;
+  const float* P = partial + (size_t)kv * tiles * 3 * FATHOM_D + c;
+  double total = 0.0;
+#pragma unroll 4
+  for (int t = tl; t < tiles; t += VF_LANES) {
+    const double nt = (double)min((long long)MEAN_ROWS, n - (long long)t * MEAN_ROWS);
+    total += nt * (double)P[(size_t)t * 3 * FATHOM_D] + (double)P[(size_t)t * 3 * FATHOM_D + FATHOM_D];
+  }
+  s_acc[tl][c] = total;
+  __syncthreads();
+  if (tl == 0) {
+    double sum = 0.0;
+#pragma unroll
+    for (int w = 0; w < VF_LANES; ++w) sum += s_acc[w][c];
+    s_mu[c] = sum / (double)n;
+  }
+  __syncthreads();
+  const double mu = s_mu[c];
+  double m2 = 0.0;
+#pragma unroll 4
+  for (int t = tl; t < tiles; t += VF_LANES) {
+    const double nt = (double)min((long long)MEAN_ROWS, n - (long long)t * MEAN_ROWS);
+    const double s1 = (double)P[(size_t)t * 3 * FATHOM_D + FATHOM_D], s2 = (double)P[(size_t)t * 3 * FATHOM_D + 2 * FATHOM_D];
+    const double dm = (double)P[(size_t)t * 3 * FATHOM_D] + s1 / nt - mu;
+    m2 += (s2 - s1 * s1 / nt) + nt * dm * dm;
+  }
+  __syncthreads();
+  s_acc[tl][c] = m2;
+  __syncthreads();
+  if (tl == 0) {
+    double sum = 0.0;
+#pragma unroll
+    for (int w = 0; w < VF_LANES; ++w) sum += s_acc[w][c];
+    mean[(size_t)kv * FATHOM_D + c] = (float)mu;
+    var[(size_t)kv * FATHOM_D + c] = (float)(sum > 0.0 ? sum / (double)(n > 1 ? n - 1 : 1) : 0.0);
+  }
+}
+
 }  // namespace
 
+static size_t stats_partial_bytes(int Hkv, long long n) {
+  return fathom_round_up((size_t)Hkv * (size_t)((n + MEAN_ROWS - 1) / MEAN_ROWS) * 3 * FATHOM_D * 4, 256);
+}
+
 size_t fathom_calib_scratch_bytes(int Hkv, long long n) {
-  const size_t mt = (size_t)((n + MEAN_ROWS - 1) / MEAN_ROWS), ct = (size_t)((n + COV_ROWS - 1) / COV_ROWS);
-  return fathom_round_up((size_t)Hkv * mt * FATHOM_D * 4, 256) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256);
+  const size_t ct = (size_t)((n + COV_ROWS - 1) / COV_ROWS);
+  return stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256) +
+         fathom_round_up((size_t)Hkv * FATHOM_D * 4, 256);
+}
+
+extern "C" int fathom_channel_variance(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* mean, float* var,
+                                       void* stream) {
+  if (!ctx || !K || !mean || !var) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k_dtype != FATHOM_F32 && k_dtype != FATHOM_BF16) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(K)) return FATHOM_ERR_ALIGNMENT;
+  const int Hkv = L->n_kv_heads;
+  const long long n = L->n;
+  if (fathom_calib_scratch_bytes(Hkv, n) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  const int mt = (int)((n + MEAN_ROWS - 1) / MEAN_ROWS);
+  float* part = static_cast<float*>(ctx->scratch);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (k_dtype == FATHOM_F32)
+    var_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, part, mt);
+  else
+    var_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, part, mt);
+  var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var);
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
 }
 
 extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* mean, float* cov,
@@ -194,19 +291,21 @@ extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const v
   const long long n = L->n;
   if (fathom_calib_scratch_bytes(Hkv, n) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
   const int mt = (int)((n + MEAN_ROWS - 1) / MEAN_ROWS), ct = (int)((n + COV_ROWS - 1) / COV_ROWS);
-  float* pmean = static_cast<float*>(ctx->scratch);
-  float* pcov = reinterpret_cast<float*>(static_cast<char*>(ctx->scratch) + fathom_round_up((size_t)Hkv * mt * FATHOM_D * 4, 256));
+  char* base = static_cast<char*>(ctx->scratch);
+  float* part = reinterpret_cast<float*>(base);
+  float* pcov = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n));
+  float* var_tmp = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);
   if (k_dtype == FATHOM_F32) {
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    mean_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, pmean, mt);
-    mean_final_kernel<<<Hkv, FATHOM_D, 0, st>>>(pmean, mt, n, mean);
+    var_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, part, mt);
+    var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
     cov_partial_kernel<float><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const float*>(K), n, mean, pcov, ct);
   } else {
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    mean_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, pmean, mt);
-    mean_final_kernel<<<Hkv, FATHOM_D, 0, st>>>(pmean, mt, n, mean);
+    var_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, part, mt);
+    var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
     cov_partial_kernel<__nv_bfloat16><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(K), n, mean, pcov, ct);
   }
   cov_final_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, ct, n, cov);

@@ -1,6 +1,6 @@
 """Times (or exposes to a profiler) ONE stage of the hot path on synthetic device buffers.
 
-    python -m paper_2609_17652_b200.probe --stage scan|topk|scan_topk|attend|build|alloc|rotate|calibrate [--n N] [--iters I] [--budget B] [--k K]
+    python -m paper_2609_17652_b200.probe --stage scan|topk|scan_topk|attend|build|alloc|rotate|calibrate|variance [--n N] [--iters I] [--budget B] [--k K]
 
 Unlike bench.py it allocates only what the chosen stage touches (random plane words and scales for the scan,
 random scores for top-k, ...), so a full-size launch fits in a few hundred MB and can be captured with ncu.
@@ -19,7 +19,7 @@ from . import binding as fb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "calibrate"])
+    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "calibrate", "variance"])
     ap.add_argument("--n", type=int, default=1 << 20)
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--budget", type=int, default=48)
@@ -43,9 +43,9 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     st = torch.cuda.current_stream()
 
-    if a.stage in ("build", "rotate", "calibrate"):
+    if a.stage in ("build", "rotate", "calibrate", "variance"):
         K = torch.randn(Hkv, n, d, device=dev)
-    if a.stage in ("rotate", "calibrate"):
+    if a.stage in ("rotate", "calibrate", "variance"):
         mean = torch.zeros(Hkv, d, device=dev)
         cov = torch.zeros(Hkv, d, d, device=dev)
         basis = torch.linalg.qr(torch.randn(Hkv, d, d, device=dev))[0].contiguous()
@@ -81,6 +81,8 @@ def main():
             ctx.fathom_rotate_keys(lay, K, mean, basis, K_rot, st)
         elif a.stage == "calibrate":
             ctx.fathom_calibrate(lay, K, mean, cov, st)
+        elif a.stage == "variance":
+            ctx.fathom_channel_variance(lay, K, mean, cov[:, 0], st)
         elif a.stage == "scan_topk":
             ctx.fathom_scan_topk(lay, planes, scales, q, depth, hpp, a.k, 0, 0, idx, st)
         else:

@@ -62,3 +62,34 @@ def test_scratch_bytes_and_host_side_rejection(fb):
     assert fb.lib.fathom_alloc_depth(None, C.byref(lay), 16, 16, 0, 48, 4, 16, None) == -1
     assert fb.lib.fathom_sparse_attend(None, C.byref(lay), 16, 16, 16, 1, 16, 10, C.c_float(1.0), 16, None) == -1
     assert fb.lib.fathom_destroy(None) == 0
+
+
+def test_layer_budget_plan_host_function_matches_the_oracle(fb):
+    """fathom_plan_layer_budgets is host code: compared here, level by level, with the oracle's greedy plan on random
+    error tables (convex and not), uneven level spacing, ties and targets between two sums."""
+    import numpy as np
+    from oracle import fathom_oracle as O
+    r = np.random.default_rng(5)
+    for trial in range(60):
+        L = int(r.integers(1, 40)); nlev = int(r.integers(1, 9))
+        levels = np.cumsum(r.integers(1, 17, size=nlev)) + 16
+        err = r.uniform(0, 1, size=(L, nlev))
+        if trial % 3 == 0:
+            err = -np.sort(-err, axis=1)                   # falling curves
+        if trial % 4 == 0:
+            err = np.round(err, 1)                         # many ties
+        target = float(r.uniform(levels[0] - 1, levels[-1] + 1))
+        got = fb.fathom_plan_layer_budgets(err.tolist(), levels.tolist(), target)
+        ref = O.plan_layer_budgets(err, levels, target)
+        assert got == list(ref), (trial, L, nlev, target)
+        assert sum(levels[i] for i in got) <= max(target, levels[0]) * L + 1e-9
+    # the paper's range at its two means: 36 layers, levels 24 .. 128 in steps of 8
+    levels = list(range(24, 129, 8))
+    err = np.exp(-np.outer(r.uniform(0.01, 0.06, 36), levels))
+    for mean in (48, 64):
+        got = fb.fathom_plan_layer_budgets(err.tolist(), levels, mean)
+        assert got == list(O.plan_layer_budgets(err, levels, mean))
+        assert sum(levels[i] for i in got) == mean * 36
+    assert fb.lib.fathom_plan_layer_budgets(None, 1, 1, None, C.c_double(1.0), None) == -1
+    bad = (C.c_int * 2)(32, 32); e = (C.c_double * 2)(1.0, 0.5); out = (C.c_int * 1)()
+    assert fb.lib.fathom_plan_layer_budgets(e, 1, 2, bad, C.c_double(40.0), out) == -1

@@ -380,3 +380,30 @@ def test_klt_rotated_store(n):
     L.K, L.q, L.var = K_rot, q_rot, lam
     g, ref = check_all(L, B=48, k=k, hpp=G)
     assert np.all(g["depth"].sum(1) == 48)
+
+
+@pytest.mark.parametrize("n,dtype", [(1, torch.float32), (777, torch.float32), (1024, torch.float32), (40000 + 13, torch.float32),
+                                     (9000, torch.bfloat16)])
+def test_channel_variance_kernel(n, dtype):
+    """Per-channel mean and unbiased variance of the session's keys against the oracle's written-out definition,
+    with a large common offset (the case a one-pass sum of squares gets wrong), several tiles and a ragged tail;
+    then the depths planned from the kernel's variances equal those from the oracle's."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq = 2, 8
+    L = make_layer(max(n, 64), Hkv, Hq, seed=77, device="cuda")
+    K = (L.K[:, :n] + 40.0).to(dtype).contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, 1))
+    mean = torch.full((Hkv, 128), float("nan"), device="cuda"); var = torch.full((Hkv, 128), float("nan"), device="cuda")
+    ctx.fathom_channel_variance(lay, K, mean, var)
+    ctx.fathom_channel_variance(lay, K, mean, var)                             # scratch reuse
+    torch.cuda.synchronize()
+    mu_ref, var_ref = O.channel_variance(K.float().cpu().numpy())
+    sd = np.sqrt(var_ref)
+    assert np.all(np.abs(mean.cpu().numpy() - mu_ref) <= 1e-6 * np.abs(mu_ref) + 1e-5 * sd)
+    assert np.all(np.abs(var.cpu().numpy() - var_ref) <= 1e-5 * var_ref)
+    if n > 1:
+        d_gpu = O.alloc_depth(L.q.cpu().numpy(), var.cpu().numpy(), "waterfill", 48, 4)
+        d_ref = O.alloc_depth(L.q.cpu().numpy(), var_ref.astype(np.float32), "waterfill", 48, 4)
+        assert np.mean(d_gpu != d_ref) < 0.01                                  # equal up to near-ties in g_j
+    ctx.close()
