@@ -136,18 +136,27 @@ int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* pl
  * index, -0 equal to +0.  Requires 1 <= k <= n, forced count <= k, k <= FATHOM_MAX_K.
  *   scores  in   [Hq][score_stride] fp32 (finite)
  *   idx     out  [Hq][k] int32, ascending token indices
- * Uses the context scratch (fathom_scratch_bytes). */
+ * Uses the context scratch (fathom_scratch_bytes).
+ * Long rows (at least 64 chunks of 1024 scores, k - forced >= 256) are read once: a histogram of every 16th chunk
+ * gives an estimated threshold bin (and a bound: the bin of the sample's own (k - forced)-th largest score), one pass
+ * collects the tokens above the estimate, and the exact selection runs among them.  If any head collected fewer than
+ * it needs, a second collection above the bound, enqueued behind the first, runs instead; the decision is taken on
+ * the device and the result is the same either way.  Shorter rows take two passes (histogram of all scores, filter).
+ * Environment: FATHOM_TOPK_PATH=two_pass (read once) always takes the two-pass selection. */
 #define FATHOM_MAX_K 16384
 int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* scores, int k,
                 int n_sink, int n_local, int32_t* idx, void* stream);
 
 /* ---- (3+4) fused scan and top-k, scores never materialised — Sec. 6 ("a fused kernel would narrow the gap") ------
  * Gives exactly the idx that fathom_topk would give on the scores of fathom_scan (same arguments), without writing
- * or re-reading the n * Hq scores: (a) every 16th 1024-token tile is scanned and the bin of the 12 leading score-key
- * bits in which the sample's k-th largest score lies is found per head; at least k tokens reach that bin's lower
- * edge, so no winner lies below it; (b) the full scan keeps only the (score, token) pairs that reach the edge;
- * (c) the exact selection (ties to the lower token) runs on those candidates.  The threshold is a bound, not an
- * estimate, so the result never depends on how representative the sample is - only the number of candidates does.
+ * or re-reading the n * Hq scores: (a) every 16th 1024-token tile is scanned and histogrammed per head (12 leading
+ * score-key bits); (b) the full scan keeps only the (score, token) pairs that reach a threshold bin's lower edge;
+ * (c) the exact selection (ties to the lower token) runs on those candidates and writes idx.  Two thresholds come
+ * from the sample: a BOUND (the bin of the sample's k-th largest score: at least k tokens reach it, so no winner lies
+ * below) and an ESTIMATE (the bin of the rank that k tokens of the whole sequence are expected to reach, plus four
+ * standard deviations: ~6 times fewer candidates).  The scan runs with the estimate; if any head then holds fewer
+ * candidates than it needs, a second scan with the bound, enqueued behind the first, does the work instead - the
+ * decision is taken on the device, and the result never depends on how representative the sample is.
  * Sequences too short to sample (fewer than 16 tiles or fewer than 2 k sampled tokens) are scanned into scratch
  * and selected densely.  Uses the context scratch (fathom_scratch_bytes). */
 int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes, const uint16_t* scales,

@@ -22,6 +22,7 @@ fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k) {
   s.hist = reinterpret_cast<uint32_t*>(p + off);    off += fathom_round_up((size_t)Hq * FATHOM_TOPK_BINS * 4, 256);
   s.state = reinterpret_cast<uint32_t*>(p + off);   off += fathom_round_up((size_t)Hq * 8 * 4, 256);
   s.cand_count = reinterpret_cast<uint32_t*>(p + off); off += fathom_round_up((size_t)Hq * 4, 256);
+  s.cand_count2 = reinterpret_cast<uint32_t*>(p + off); off += fathom_round_up((size_t)Hq * 4, 256);
   s.bitmap_words = (long long)((n + 1023) / 1024) * 32;                    // whole 32-word groups
   s.bitmap = reinterpret_cast<uint32_t*>(p + off);  off += fathom_round_up((size_t)Hq * (size_t)s.bitmap_words * 4, 256);
   s.cand = reinterpret_cast<int32_t*>(p + off);     off += fathom_round_up((size_t)Hq * (size_t)n * 4, 256);

@@ -42,9 +42,29 @@ static inline bool fathom_aligned16(const void* p) { return (reinterpret_cast<ui
 static inline size_t fathom_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- pieces shared by scan.cu and topk.cu for the fused scan + selection (fathom_scan_topk) -------------------
+// A launch that belongs to one of two alternative continuations decides on the device whether it runs.  A first
+// attempt collects, per head, the tokens above an ESTIMATED threshold; it goes on only if every head collected at
+// least `want` of them.  Otherwise the second attempt, enqueued behind it with a threshold that is a guaranteed
+// bound, does the work.  The host enqueues both and never synchronises.
+struct fathom_gate {
+  const uint32_t* counts;       // [heads] candidates the first attempt collected per head
+  uint32_t want;
+  int heads;
+  int mode;                     // 0: always run, 1: only if every head collected enough, 2: only if some head did not
+};
+// Called by every thread of the CTA at the top of a gated kernel.
+__device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g) {
+  if (g.mode == 0) return true;
+  bool ok = true;
+  for (int h = threadIdx.x; h < g.heads; h += blockDim.x) ok = ok && (__ldcg(g.counts + h) >= g.want);
+  const bool all_ok = __syncthreads_and(ok) != 0;
+  return g.mode == 1 ? all_ok : !all_ok;
+}
+
 struct fathom_scan_fuse {       // extra arguments of the sampling / filtering scan variants
   int tile_step;                // sample: scan every tile_step-th tile
   const uint32_t* state;        // filter: [Hq][8], word 0 = threshold bin found on the sample
+  fathom_gate gate;             // filter: whether this launch runs at all
   long long sink_end, local_begin;   // filter: eligible tokens are sink_end <= i < local_begin
   float* cand_score;            // filter: [Hq][capacity] scores of the candidates
   int32_t* cand_idx;            // filter: [Hq][capacity] their tokens
@@ -65,8 +85,10 @@ int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, co
 
 struct fathom_topk_scratch {
   uint32_t* hist;        // [Hq][FATHOM_TOPK_BINS]
-  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 4 candidates written, 5 tickets
-  uint32_t* cand_count;  // [Hq] candidates collected by the filtering scan (fused path)
+  uint32_t* state;       // [Hq][8]: 0 threshold bin, 1 count above it, 2 needed from it, 3 bound bin (sampled paths),
+                         //          4 candidates written, 5 tickets
+  uint32_t* cand_count;  // [Hq] candidates collected above an estimated threshold (single-pass top-k, fused path)
+  uint32_t* cand_count2; // [Hq] candidates of the second attempt (threshold that is a bound, not an estimate)
   uint32_t* bitmap;      // [Hq][bitmap_words] selection bitmap, token i at bit (i % 32) of word i / 32
   int32_t* cand;         // [Hq][n] token indices of the threshold bin
   uint32_t* tile_count;  // [Hq][ceil(n / 8192)] selected tokens per filter tile, then their exclusive prefix

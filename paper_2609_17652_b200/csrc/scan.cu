@@ -60,6 +60,8 @@ __device__ __forceinline__ void transpose_rows(uint32_t& a, uint32_t& b, uint32_
 // fp32 value whose order-preserving integer image (see topk.cu) has `bin` as its 12 leading bits and zeros below:
 // the lower edge of that histogram bin
 __device__ __forceinline__ float bin_lower_edge(uint32_t bin) {
+  if (bin >= FATHOM_TOPK_BINS) return __uint_as_float(0x7fc00000u);   // past the last bin: nothing reaches it (NaN compares false)
+  if (bin <= 7u) return -INFINITY;                                    // bins below -inf's hold no finite score: everything reaches them
   const uint32_t key = bin << 20;
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
@@ -95,6 +97,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
   __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
   __shared__ WarpSmem<NH> s_warp[SCAN_WARPS];
 
+  if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA

@@ -16,6 +16,10 @@
 // The selected set is unique, so neither the append order nor atomics can show in the output.
 #include "fathom_common.cuh"
 
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+
 namespace {
 
 constexpr int HIST_THREADS = 256;
@@ -34,40 +38,48 @@ __device__ __forceinline__ uint32_t ordered_key(float f) {
 
 struct Forced { long long sink_end, local_begin; };          // eligible tokens: sink_end <= i < local_begin
 
-__device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
-                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp);
+using Gate = fathom_gate;
 
+__device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, bool bound_slot);
+
+// A CTA histograms `reps` tiles of `tile` scores that start cta_stride tokens apart (cta_stride = tile, reps = 1 for a
+// full pass; a multiple of the tile when only every m-th tile is histogrammed to estimate a threshold, in which case
+// dev_status is NULL: a short sample is no error).
 __global__ void __launch_bounds__(HIST_THREADS)
 topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                  uint32_t* __restrict__ hist, uint32_t* __restrict__ state, uint32_t want,
-                 uint32_t* __restrict__ dev_status, int tile) {
+                 uint32_t* __restrict__ dev_status, int tile, long long cta_stride, int reps, uint32_t want_bound) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ bool s_last;
   const int head = blockIdx.y;
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  const long long base = (long long)blockIdx.x * tile;         // tile: scores per CTA, a multiple of 1024
-  const long long end = min(base + tile, n);
-  // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
-  if (base >= F.sink_end && base + tile <= F.local_begin) {   // whole tile eligible: no per-token test
-    const float4* r4 = reinterpret_cast<const float4*>(row + base);
+  for (int rep = 0; rep < reps; ++rep) {
+    const long long base = ((long long)blockIdx.x * reps + rep) * cta_stride;   // tile: scores per tile, a multiple of 1024
+    if (base >= n) break;
+    const long long end = min(base + tile, n);
+    // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
+    if (base >= F.sink_end && base + tile <= F.local_begin) {   // whole tile eligible: no per-token test
+      const float4* r4 = reinterpret_cast<const float4*>(row + base);
 #pragma unroll 8
-    for (int v = threadIdx.x; v < tile / 4; v += HIST_THREADS) {
-      const float4 x = __ldg(r4 + v);
-      atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
-      atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
-      atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
-      atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
-    }
-  } else {
-    for (long long i = base + (long long)threadIdx.x * 4; i < end; i += HIST_THREADS * 4) {
-      const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
-      const float e[4] = {x.x, x.y, x.z, x.w};
+      for (int v = threadIdx.x; v < tile / 4; v += HIST_THREADS) {
+        const float4 x = __ldg(r4 + v);
+        atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
+      }
+    } else {
+      for (long long i = base + (long long)threadIdx.x * 4; i < end; i += HIST_THREADS * 4) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(row + i));
+        const float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const long long t = i + c;
-        if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
+        for (int c = 0; c < 4; ++c) {
+          const long long t = i + c;
+          if (t >= F.sink_end && t < F.local_begin) atomicAdd(&sh[ordered_key(e[c]) >> 20], 1u);
+        }
       }
     }
   }
@@ -84,19 +96,28 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  find_threshold_bin(g, state + head * 8, want, dev_status, sh);
+  find_threshold_bin(g, state + head * 8, want, dev_status, sh, false);
+  if (want_bound) {                                           // sampled histogram: also the bin that is a bound (word 3)
+    __syncthreads();
+    find_threshold_bin(g, state + head * 8, want_bound, nullptr, sh, true);
+  }
 }
 
 // state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it,
 // [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
 // Run by the HIST_THREADS threads of the CTA that completed the head's histogram: thread t owns bins
 // 4095 - 16 t .. 4080 - 16 t (descending), so a block prefix over threads is a suffix count over bins.
+// bound_slot: only the bin is wanted and goes to word 3 (a histogram of a sample: the bin of the sample's
+// want-th largest eligible score is reached by at least `want` eligible tokens of the whole row).
 __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
-                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp) {
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, bool bound_slot) {
   constexpr int BPT = FATHOM_TOPK_BINS / HIST_THREADS;        // 16 bins per thread
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (want == 0) {                                            // nothing to select: no bin is above or equal
-    if (tid == 0) { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
+    if (tid == 0) {
+      if (bound_slot) st[3] = FATHOM_TOPK_BINS;
+      else { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
+    }
     return;
   }
   uint32_t c[BPT], local = 0;
@@ -117,16 +138,17 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
 #pragma unroll
     for (int x = 0; x < BPT; ++x) {
       if (run < want && run + c[x] >= want) {
-        st[0] = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
-        st[1] = run;
-        st[2] = want - run;
+        const uint32_t bin = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
+        if (bound_slot) st[3] = bin;
+        else { st[0] = bin; st[1] = run; st[2] = want - run; }
       }
       run += c[x];
     }
   }
   if (tid == HIST_THREADS - 1 && above + local < want) {      // fewer eligible tokens than wanted: take them all
-    atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
-    st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1];
+    if (dev_status) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+    if (bound_slot) st[3] = 0;
+    else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; }
   }
 }
 
@@ -226,6 +248,61 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
   for (uint32_t e = threadIdx.x; e < cnt; e += FILT_THREADS) cand_h[base + e] = (int32_t)(tile0 + s_list[e]);
 }
 
+// Collection pass of the sampled paths: every eligible token whose score reaches the lower edge of the head's
+// threshold bin is appended to the head's candidate list as a (score, token) pair.  state_word 0: the bin estimated
+// from a histogram of every 16th chunk (first attempt); 3: the bin that is a bound (second attempt, gated).
+__global__ void __launch_bounds__(FILT_THREADS)
+topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
+                    const uint32_t* __restrict__ state, int state_word, float* __restrict__ cand_score,
+                    int32_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_count, Gate gate) {
+  __shared__ uint16_t s_list[FILT_TILE];
+  __shared__ uint32_t s_count, s_base;
+  if (!fathom_gate_open(gate)) return;
+  const int head = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_count = 0u;
+  __syncthreads();
+  const uint32_t bstar = state[head * 8 + state_word];
+  // lower edge of the bin; the bins below -inf's (no finite score lies there) stand for "every score", a bin past the
+  // last for "none" (a comparison with NaN is false)
+  const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
+  const float* row = scores + (size_t)head * (size_t)score_stride;
+  const long long tile0 = (long long)blockIdx.x * FILT_TILE;
+  const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
+  const bool all_elig = wbase >= F.sink_end && wbase + FILT_WARP_TOKENS <= F.local_begin && wbase + FILT_WARP_TOKENS <= n;
+  float4 x[FILT_WARP_TOKENS / 128];
+#pragma unroll
+  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+    const long long t0 = wbase + it * 128 + lane * 4;
+    x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+    const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+    if (fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])) >= lo) {  // divergent on purpose: candidates are rare
+      const long long t0 = wbase + it * 128 + lane * 4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const long long t = t0 + c;
+        if (e[c] >= lo && (all_elig || (t < n && t >= F.sink_end && t < F.local_begin)))
+          s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(t - tile0);
+      }
+    }
+  }
+  __syncthreads();
+  const uint32_t cnt = s_count;
+  if (cnt == 0u) return;
+  if (threadIdx.x == 0) s_base = atomicAdd(&cand_count[head], cnt);
+  __syncthreads();
+  const uint32_t base = s_base;
+  float* cs = cand_score + (size_t)head * (size_t)n;
+  int32_t* ci = cand_idx + (size_t)head * (size_t)n;
+  for (uint32_t e = threadIdx.x; e < cnt; e += FILT_THREADS) {
+    const long long t = tile0 + s_list[e];
+    cs[base + e] = row[t];
+    ci[base + e] = (int32_t)t;
+  }
+}
+
 // low 52 bits of (key << 32 | ~index); the 12 leading key bits are the same for every candidate
 __device__ __forceinline__ uint64_t composite52(const float* row, int32_t i) {
   return ((((uint64_t)ordered_key(row[i])) << 32) | (uint32_t)(~(uint32_t)i)) & ((1ull << 52) - 1ull);
@@ -259,49 +336,66 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return s_warp[warp] + incl - v;
 }
 
-// FUSED = false: candidates are the tokens of the threshold bin (their 12 leading key bits agree), scores are read
-//                 from the dense score rows, the number needed comes from the histogram state.
-// FUSED = true : candidates are (score, token) pairs collected by the filtering scan; `want_fused` of them are needed
-//                 and the whole 64-bit composite takes part in the select.
-template <bool FUSED>
+// DIRECT = false: candidates are the tokens of the threshold bin (their 12 leading key bits agree), scores are read
+//                  from the dense score rows, the number needed comes from the histogram state; the chosen tokens are
+//                  OR-ed into the bitmap the filter started, and topk_emit_kernel writes the indices.
+// DIRECT = true : candidates are (score, token) pairs collected above a threshold; `want_direct` of them are needed,
+//                  the whole 64-bit composite takes part in the select, and the kernel itself writes the head's k
+//                  indices in ascending order: the chosen tokens are gathered in shared memory, distributed over
+//                  SORT_BUCKETS equal token ranges (counting sort), and ranked inside their range by comparison.
+constexpr int SORT_BUCKETS = 4096;
+template <bool DIRECT>
 __global__ void __launch_bounds__(FIN_THREADS)
 topk_select_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                    const uint32_t* __restrict__ state, const int32_t* __restrict__ cand,
                    uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
-                   const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_fused) {
+                   const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
+                   Gate gate) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
+  if (!fathom_gate_open(gate)) return;
   __shared__ uint64_t s_comp[FIN_CACHE];
   __shared__ uint32_t s_hist[DIGITS];
   __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
-  __shared__ uint32_t s_need, s_bucket;
+  __shared__ uint32_t s_need, s_bucket, s_ntok;
+  extern __shared__ __align__(16) unsigned char s_dyn[];      // DIRECT: range counters, chosen tokens, tokens by range
+  uint32_t* s_range = reinterpret_cast<uint32_t*>(s_dyn);                       // [SORT_BUCKETS]
+  int32_t* s_tok = reinterpret_cast<int32_t*>(s_range + SORT_BUCKETS);          // [k]
+  int32_t* s_sorted = s_tok + k;                                                // [k]
   const int head = blockIdx.x, tid = threadIdx.x;
-  // dense: scores row of the head, candidate tokens [n];  fused: candidate scores and tokens [cand_capacity]
-  const float* row = scores + (size_t)head * (size_t)(FUSED ? cand_capacity : score_stride);
-  const int32_t* cand_h = cand + (size_t)head * (size_t)(FUSED ? cand_capacity : n);
-  uint32_t* bm = bitmap + (size_t)head * (size_t)bitmap_words;
-  uint32_t* tc = tile_count + (size_t)head * ntiles;
-  const uint32_t m = FUSED ? (uint32_t)min((long long)cand_count[head], cand_capacity) : state[head * 8 + 4];
-  const uint32_t need0 = min(FUSED ? want_fused : state[head * 8 + 2], m);
-  constexpr int TOP = FUSED ? 64 : 52;                        // undecided bits of the composite
+  // dense: scores row of the head, candidate tokens [n];  direct: candidate scores and tokens [cand_capacity]
+  const float* row = scores + (size_t)head * (size_t)(DIRECT ? cand_capacity : score_stride);
+  const int32_t* cand_h = cand + (size_t)head * (size_t)(DIRECT ? cand_capacity : n);
+  uint32_t* bm = DIRECT ? nullptr : bitmap + (size_t)head * (size_t)bitmap_words;
+  uint32_t* tc = DIRECT ? nullptr : tile_count + (size_t)head * ntiles;
+  const uint32_t m = DIRECT ? (uint32_t)min((long long)cand_count[head], cand_capacity) : state[head * 8 + 4];
+  const uint32_t need0 = min(DIRECT ? want_direct : state[head * 8 + 2], m);
+  constexpr int TOP = DIRECT ? 64 : 52;                       // undecided bits of the composite
   auto composite = [&](uint32_t c) -> uint64_t {
-    if (FUSED) return (((uint64_t)ordered_key(row[c])) << 32) | (uint32_t)(~(uint32_t)cand_h[c]);
+    if (DIRECT) return (((uint64_t)ordered_key(row[c])) << 32) | (uint32_t)(~(uint32_t)cand_h[c]);
     return composite52(row, cand_h[c]);
   };
   // The working set is either all m candidates in global memory or a subset kept in shared memory: everything when
-  // m fits, otherwise the bucket of the first digit once it fits (what ranks above that bucket is marked at once).
+  // m fits, otherwise the bucket of the first digit once it fits (what ranks above that bucket is taken at once).
   __shared__ uint32_t s_ncache;
   bool cached = m <= FIN_CACHE;
   uint32_t mc = m;                                            // size of the working set
   auto mark = [&](uint64_t comp) {                            // the token sits in the low 32 bits of every composite
     const int32_t i = (int32_t)~(uint32_t)comp;
-    atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
-    atomicAdd(&tc[i / FILT_TILE], 1u);
+    if (DIRECT) {
+      const uint32_t p = atomicAdd(&s_ntok, 1u);
+      if (p < (uint32_t)k) s_tok[p] = i;
+    } else {
+      atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
+      atomicAdd(&tc[i / FILT_TILE], 1u);
+    }
   };
+  if (tid == 0) s_ntok = 0u;
   if (cached)
     for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite(c);
+  __syncthreads();
 
   // ---- radix select of the need0 largest composites among the m candidates: 11-bit digits from the top
   //      undecided bit downwards (the last digit is shorter) until the chosen bucket is taken whole.
@@ -354,7 +448,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       hi = lo;
       if (s_need == s_bucket) break;                          // the chosen bucket is taken entirely: done
       if (!cached && s_bucket <= FIN_CACHE) {
-        // the undecided bucket fits in shared memory: pull it in, mark what ranks above it, go on from there
+        // the undecided bucket fits in shared memory: pull it in, take what ranks above it, go on from there
         const uint64_t pfx = s_prefix;
         for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS * 8) {
           uint64_t comp[8];
@@ -392,6 +486,50 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       if (need0 >= m || comp >= thr) mark(comp);
     }
   }
+
+  if (DIRECT) {
+    // ---- ascending output: sink tokens, the chosen tokens in token order, local tokens
+    for (int d = tid; d < SORT_BUCKETS; d += FIN_THREADS) s_range[d] = 0u;
+    __syncthreads();
+    const uint32_t cnt = min(s_ntok, (uint32_t)k);            // = need0
+    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) atomicAdd(&s_range[(uint32_t)s_tok[e] >> bucket_shift], 1u);
+    __syncthreads();
+    {                                                         // exclusive prefix over the ranges, in place
+      constexpr int RPT = SORT_BUCKETS / FIN_THREADS;
+      uint32_t c[RPT], local = 0;
+#pragma unroll
+      for (int x = 0; x < RPT; ++x) { c[x] = s_range[RPT * tid + x]; local += c[x]; }
+      uint32_t total;
+      uint32_t run = block_exclusive_scan(local, s_warp, &total);
+#pragma unroll
+      for (int x = 0; x < RPT; ++x) { s_range[RPT * tid + x] = run; run += c[x]; }
+    }
+    __syncthreads();
+    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) {       // afterwards s_range[r] is the END of range r
+      const int32_t t = s_tok[e];
+      s_sorted[atomicAdd(&s_range[(uint32_t)t >> bucket_shift], 1u)] = t;
+    }
+    __syncthreads();
+    int32_t* out = idx_out + (size_t)head * k;
+    const uint32_t n_sink = (uint32_t)F.sink_end, n_loc = (uint32_t)(n - F.local_begin);
+    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) {
+      const int32_t t = s_sorted[e];
+      const uint32_t r = (uint32_t)t >> bucket_shift;
+      const uint32_t beg = r ? s_range[r - 1] : 0u, end = s_range[r];
+      uint32_t rank = 0;
+      for (uint32_t j = beg; j < end; ++j) rank += s_sorted[j] < t;
+      out[n_sink + beg + rank] = t;
+    }
+    for (uint32_t e = tid; e < n_sink; e += FIN_THREADS) out[e] = (int32_t)e;
+    for (uint32_t e = tid; e < n_loc; e += FIN_THREADS) out[n_sink + cnt + e] = (int32_t)(F.local_begin + e);
+    const uint32_t filled = n_sink + cnt + n_loc;
+    if (filled != (uint32_t)k) {                              // short selection (non-finite scores)
+      if (tid == 0) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+      for (uint32_t e = filled + tid; e < (uint32_t)k; e += FIN_THREADS) out[e] = (int32_t)(n - 1);   // pad with the last token
+    }
+    return;
+  }
+
   // ---- forced sink / local tokens
   const long long n_forced = F.sink_end + (n - F.local_begin);
   for (long long e = tid; e < n_forced; e += FIN_THREADS) {
@@ -464,21 +602,83 @@ static int hist_tile_for(long long n, int Hq) {
   return (int)tile;
 }
 
-// Dense selection over score rows (the four launches of fathom_topk).
+// Rank in a sample of n_sample of n tokens whose score is, with a margin of four standard deviations of the
+// sampling count, low enough that `want` tokens of the whole sequence reach it.
+static uint32_t estimate_rank(uint32_t want, long long n_sample, long long n) {
+  const double expect = (double)want * (double)n_sample / (double)n;
+  return (uint32_t)(expect + 4.0 * sqrt(expect) + 16.0);
+}
+
+static bool force_two_pass() {
+  static const bool v = [] { const char* e = getenv("FATHOM_TOPK_PATH"); return e && strcmp(e, "two_pass") == 0; }();
+  return v;
+}
+
+// log2 of the token range per counting-sort bucket of the direct select: the smallest that maps n tokens to SORT_BUCKETS
+static int bucket_shift_for(long long n) {
+  int s = 0;
+  while (((n - 1) >> s) >= SORT_BUCKETS) ++s;
+  return s;
+}
+
+static size_t direct_select_smem(int k) { return (size_t)SORT_BUCKETS * 4 + (size_t)2 * k * 4; }
+
+// The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
+// and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
+// gate_mode 0: a single attempt whose threshold is a bound (candidates counted in S.cand_count).
+static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, Forced F, uint32_t want, const fathom_topk_scratch& S,
+                                int32_t* idx, int gate_mode, cudaStream_t st) {
+  static bool attr_set[64] = {};
+  if (ctx->device >= 0 && ctx->device < 64 && !attr_set[ctx->device]) {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)direct_select_smem(FATHOM_MAX_K)));
+    attr_set[ctx->device] = true;
+  }
+  Gate g = {S.cand_count, want, Hq, gate_mode};
+  topk_select_kernel<true><<<Hq, FIN_THREADS, direct_select_smem(k), st>>>(
+      S.cand_score, n, 0, F, S.state, S.cand, nullptr, 0, k, idx, ctx->dev_status, nullptr, 0,
+      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g);
+  return FATHOM_OK;
+}
+
 static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, long long score_stride, int Hq, int k,
                           Forced F, uint32_t want, const fathom_topk_scratch& S, int32_t* idx, cudaStream_t st) {
-  // histograms, per-head state and candidate counters are contiguous at the start of the arena
+  // histograms, per-head states and candidate counters are contiguous at the start of the arena
   FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
-  const int htile = hist_tile_for(n, Hq);
-  dim3 hgrid((unsigned)((n + htile - 1) / htile), (unsigned)Hq);
-  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, want, ctx->dev_status, htile);
   const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
   dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
-  topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
-                                                     S.tile_count);
-  topk_select_kernel<false><<<Hq, FIN_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
-                                                        k, idx, ctx->dev_status, S.tile_count, ntiles, nullptr, 0, 0u);
-  topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
+  Gate always = {nullptr, 0u, 0, 0};
+  // Single pass when the row is long enough to estimate the threshold from every 16th 1024-score chunk.
+  const long long chunks = (n + 1023) / 1024, sampled = (chunks + 15) / 16;
+  const long long n_sample = sampled * 1024 <= n ? sampled * 1024 : n;       // upper bound on the sampled scores
+  const uint32_t rank = estimate_rank(want, n_sample, n);
+  const bool single = !force_two_pass() && want >= 256 && chunks >= 64 && (long long)rank * 8 <= n_sample;
+  if (!single) {
+    // two passes: histogram of all scores and threshold bin, filter, select within the bin, ascending emission
+    const int htile = hist_tile_for(n, Hq);
+    dim3 hgrid((unsigned)((n + htile - 1) / htile), (unsigned)Hq);
+    topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, want, ctx->dev_status, htile,
+                                                     (long long)htile, 1, 0u);
+    topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
+                                                       S.tile_count);
+    topk_select_kernel<false><<<Hq, FIN_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
+                                                          k, idx, ctx->dev_status, S.tile_count, ntiles, nullptr, 0, 0u, 0, always);
+    topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
+  } else {
+    const int reps = sampled >= 64 ? 8 : 1;                            // sampled chunks per CTA
+    dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
+    topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
+                                                     reps, want);
+    topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
+                                                        always);
+    int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 1, st);
+    if (rc != FATHOM_OK) return rc;
+    Gate short_of = {S.cand_count, want, Hq, 2};
+    topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 3, S.cand_score, S.cand, S.cand_count2,
+                                                        short_of);
+    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 2, st);
+    if (rc != FATHOM_OK) return rc;
+  }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
@@ -544,8 +744,10 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   if (step == 1)                                              // short sequence: the sample is the whole score array
     return run_dense_topk(ctx, S.sample, n, S.sample_stride, Hq, k, F, want, S, idx, st);
 
-  // ---- threshold: the bin in which the sample's k-th largest score lies.  At least k tokens of the sample, hence
-  //      at least k - n_forced eligible tokens of the sequence, reach its lower edge: no winner can lie below it.
+  // ---- thresholds from a histogram of the sample.  Bound: the bin in which the sample's k-th largest score lies; at
+  //      least k tokens of the sample, hence at least k - n_forced eligible tokens of the sequence, reach its lower
+  //      edge, so no winner can lie below it.  Estimate: the bin of the rank that `want` tokens of the whole sequence
+  //      are expected to reach (plus four standard deviations); far fewer candidates, but no guarantee.
   const long long sampled = (ntiles_scan + step - 1) / step;
   const long long last_start = (sampled - 1) * step * tile;
   const long long n_sample = (sampled - 1) * tile + ((n - last_start) < tile ? (n - last_start) : tile);
@@ -553,14 +755,14 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   Forced none;
   none.sink_end = 0;
   none.local_begin = n_sample;
+  const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)n_forced;
+  const bool two_attempts = !force_two_pass() && want >= 256 && (long long)rank * 2 <= k;
   const int htile = hist_tile_for(n_sample, Hq);
   dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
-  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(S.sample, n_sample, S.sample_stride, none, S.hist, S.state, (uint32_t)k,
-                                                   ctx->dev_status, htile);
-  // ---- full scan that keeps only the tokens reaching their head's threshold
-  const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
-  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.bitmap, 0, (size_t)Hq * S.bitmap_words * 4, st));
-  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.tile_count, 0, (size_t)Hq * ntiles * 4, st));
+  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(S.sample, n_sample, S.sample_stride, none, S.hist, S.state,
+                                                   two_attempts ? rank : (uint32_t)k, two_attempts ? nullptr : ctx->dev_status,
+                                                   htile, (long long)htile, 1, two_attempts ? (uint32_t)k : 0u);
+  // ---- full scan that keeps only the tokens reaching their head's threshold, then the exact selection among them
   fathom_scan_fuse fz = {};
   fz.tile_step = 1;
   fz.state = S.state;
@@ -570,13 +772,20 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   fz.cand_idx = S.cand;
   fz.cand_count = S.cand_count;
   fz.capacity = n;
+  fz.gate = fathom_gate{nullptr, 0u, 0, 0};
   rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
   if (rc != FATHOM_OK) return rc;
-  // ---- exact selection among the candidates, then ascending emission
-  topk_select_kernel<true><<<Hq, FIN_THREADS, 0, st>>>(S.cand_score, n, 0, F, S.state, S.cand, S.bitmap, S.bitmap_words, k, idx,
-                                                       ctx->dev_status, S.tile_count, ntiles, S.cand_count, n, want);
-  dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
-  topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
+  rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, two_attempts ? 1 : 0, st);
+  if (rc != FATHOM_OK) return rc;
+  if (two_attempts) {                                         // stands by: runs only if some head's estimate was too high
+    fz.state = S.state + 3;
+    fz.cand_count = S.cand_count2;
+    fz.gate = fathom_gate{S.cand_count, want, Hq, 2};
+    rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
+    if (rc != FATHOM_OK) return rc;
+    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 2, st);
+    if (rc != FATHOM_OK) return rc;
+  }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

@@ -407,3 +407,38 @@ def test_channel_variance_kernel(n, dtype):
         d_ref = O.alloc_depth(L.q.cpu().numpy(), var_ref.astype(np.float32), "waterfill", 48, 4)
         assert np.mean(d_gpu != d_ref) < 0.01                                  # equal up to near-ties in g_j
     ctx.close()
+
+
+@pytest.mark.parametrize("n_sink,n_local", [(0, 0), (4, 32)])
+def test_topk_single_pass_and_its_exact_fallback(n_sink, n_local):
+    """Long rows take the single-pass path (threshold estimated from every 16th 1024-score chunk, candidates
+    collected in one read, exact selection among them).  Rows built so that the estimate is right, far too high
+    (only the sampled chunks hold high scores: too few candidates -> the exact two-pass path must take over on
+    the device), far too low (sampled chunks hold the lowest scores: nearly every token is a candidate) and
+    degenerate (all equal, heavy ties) must all give the oracle's selection."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hq, k = 200_000 + 37, 6, 3000
+    lay = fb.make_layout(1, Hq, n)
+    r = np.random.default_rng(21)
+    s = np.zeros((Hq, lay.score_stride), dtype=np.float32)
+    pos = np.arange(n)
+    sampled = (pos // 1024) % 16 == 0
+    s[0, :n] = r.standard_normal(n)                                              # estimate about right
+    s[1, :n] = np.where(sampled, 10.0, -10.0) + r.standard_normal(n)             # estimate far too high
+    s[2, :n] = np.where(sampled, -10.0, 10.0) + r.standard_normal(n)             # estimate far too low
+    s[3, :n] = 2.5                                                                # all equal
+    s[4, :n] = np.round(r.standard_normal(n), 1)                                  # heavy ties
+    s[5, :n] = r.standard_normal(n) * np.where(pos < n // 2, 0.1, 3.0)            # spread changes along the row
+    sc = torch.from_numpy(s).cuda()
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    want = O.topk(s[:, :n].astype(np.float64), k, n_sink, n_local)
+    for rows in ([0, 3, 4, 5], [0, 1, 2, 3, 4, 5]):          # without and with a head that forces the fall-back
+        sub = sc[rows].contiguous()
+        lay_sub = fb.make_layout(1, len(rows), n)
+        out = torch.full((len(rows), k), -1, dtype=torch.int32, device="cuda")
+        for _ in range(2):                                   # scratch reuse
+            ctx.fathom_topk(lay_sub, sub, k, n_sink, n_local, out)
+        assert np.array_equal(out.cpu().numpy(), want[rows])
+        assert ctx.fathom_device_status() == 0
+    ctx.close()
