@@ -158,7 +158,9 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     stage_names = ["build_planes", "alloc_depth", "scan", "topk", "sparse_attend"]
-    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 4, "sparse_attend": 1}
+    topk_passes = fb.fathom_topk_passes(lay, k)                 # 1: sampled estimate + one collection pass; 2: histogram + filter
+    # single pass: sample histogram, collection, selection + the gated second collection and selection; two passes: 4 kernels
+    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 5 if topk_passes == 1 else 4, "sparse_attend": 1}
 
     def stage(i, K=L.K, Kr=L.Krows, Vr=L.Vrows, q=L.q, var=L.var, pl=planes, sc=scales):
         if i == 0:
@@ -219,7 +221,7 @@ def run_ours(args):
     alg_bytes = {
         "build_planes": n * Hkv * (d * 4 + 68.0),
         "scan": plane_bytes_read + 4.0 * Hq * n,
-        "topk": 2 * 4.0 * Hq * n,
+        "topk": topk_passes * 4.0 * Hq * n,
         "sparse_attend": Hq * k * d * 2 * 2.0,
     }
     peak, peak_src = measured_peaks()
@@ -269,7 +271,7 @@ def run_ours(args):
     result["roofline"] = roof("build_planes", stage_us["build_planes"], "build_planes_kernel", n * Hkv)
     result["roofline_other_kernels"] = {
         "scan": roof("scan", stage_us["scan"], "scan_kernel", n * Hkv),
-        "topk (4 kernels, 2 passes over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
+        f"topk ({topk_passes} pass{'es' if topk_passes > 1 else ''} over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
         "sparse_attend": roof("sparse_attend", stage_us["sparse_attend"], "attend_*", n * Hkv),
     }
     # the scan is bound by shared-memory table lookups and issue slots, not by HBM: also report it that way
@@ -306,6 +308,20 @@ def run_ours(args):
     except Exception as e:                                      # report, never hide
         graph_us = "capture failed: " + repr(e)
     result["decode_step_us_per_layer_cuda_graph"] = graph_us
+
+    # ---- the same decode step with scan and selection fused (scores never written): alloc, scan_topk, attend
+    def fused_on(st):
+        ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, B, hpp, depth, st)
+        ctx.fathom_scan_topk(lay, planes, scales, L.q, depth, hpp, k, 0, 0, idx, st)
+        ctx.fathom_sparse_attend(lay, L.q, L.Krows, L.Vrows, idx, k, sm_scale, out, st)
+    ts = []
+    for it in range(33):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); fused_on(stream); b.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            ts.append(a.elapsed_time(b) * 1e3)
+    result["decode_step_fused_us_per_layer"] = round(statistics.median(ts), 2)
     result["device_status"] = status
     result["wall_ms_per_step"] = round(1e3 * t_wall / args.steps, 4)
 

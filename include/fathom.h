@@ -146,6 +146,9 @@ int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* pl
 #define FATHOM_MAX_K 16384
 int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* scores, int k,
                 int n_sink, int n_local, int32_t* idx, void* stream);
+/* How many times fathom_topk reads the scores for these arguments (host only, no GPU work): 1 or 2, or a negative
+ * status for arguments fathom_topk would reject. */
+int fathom_topk_passes(const fathom_layout* layout, int k, int n_sink, int n_local);
 
 /* ---- (3+4) fused scan and top-k, scores never materialised — Sec. 6 ("a fused kernel would narrow the gap") ------
  * Gives exactly the idx that fathom_topk would give on the scores of fathom_scan (same arguments), without writing

@@ -23,7 +23,7 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
-           "fathom_channel_variance", "fathom_plan_layer_budgets"]
+           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes"]
 
 
 class Layout(C.Structure):
@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
     lib.fathom_rotate_query.argtypes = [vp, LP, vp, vp, vp, vp]
     lib.fathom_channel_variance.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
+    lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_sparse_attend_static.argtypes = [LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
@@ -212,6 +213,13 @@ def fathom_plan_layer_budgets(err, levels, target_mean: float):
     if rc != 0:
         raise FathomError(rc)
     return list(out)
+
+
+def fathom_topk_passes(layout: Layout, k: int, n_sink: int = 0, n_local: int = 0) -> int:
+    rc = int(lib.fathom_topk_passes(C.byref(layout), k, n_sink, n_local))
+    if rc < 0:
+        raise FathomError(rc)
+    return rc
 
 
 def fathom_scratch_bytes(layout: Layout, k: int) -> int:

@@ -28,7 +28,7 @@ constexpr int FILT_THREADS = 256;
 constexpr int FILT_WARP_TOKENS = 1024;                       // 32 ballots -> 32 bitmap words per warp
 constexpr int FILT_TILE = (FILT_THREADS / 32) * FILT_WARP_TOKENS;   // 8192 tokens per CTA
 constexpr int FIN_THREADS = 1024;
-constexpr int FIN_CACHE = 4096;                              // candidate composites kept in shared memory
+constexpr int FIN_CACHE = 8192;                              // candidate composites kept in shared memory (dynamic, 64 KB)
 
 __device__ __forceinline__ uint32_t ordered_key(float f) {
   uint32_t u = __float_as_uint(f);
@@ -41,7 +41,7 @@ struct Forced { long long sink_end, local_begin; };          // eligible tokens:
 using Gate = fathom_gate;
 
 __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
-                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, bool bound_slot);
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, uint32_t want_bound);
 
 // A CTA histograms `reps` tiles of `tile` scores that start cta_stride tokens apart (cta_stride = tile, reps = 1 for a
 // full pass; a multiple of the tile when only every m-th tile is histogrammed to estimate a threshold, in which case
@@ -56,11 +56,27 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += HIST_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  for (int rep = 0; rep < reps; ++rep) {
-    const long long base = ((long long)blockIdx.x * reps + rep) * cta_stride;   // tile: scores per tile, a multiple of 1024
-    if (base >= n) break;
+  // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
+  const long long first = (long long)blockIdx.x * reps * cta_stride;
+  if (reps > 1) {
+    // sampled tiles (those that lie wholly inside the row), walked as one index space so that the loads of different
+    // tiles are in flight together.  Forced tokens are not told apart here: the caller asks for a bound rank that
+    // allows for all of them.
+    const int per_tile = tile / 4, pt_shift = 31 - __clz(per_tile);   // tile is a power of two
+#pragma unroll 8
+    for (int v = threadIdx.x; v < reps * per_tile; v += HIST_THREADS) {
+      const long long tb = first + (long long)(v >> pt_shift) * cta_stride;
+      if (tb + tile <= n) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(row + tb) + (v & (per_tile - 1)));
+        atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
+        atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
+      }
+    }
+  } else {
+    const long long base = first;
     const long long end = min(base + tile, n);
-    // score_stride is a multiple of 4, so a float4 stays inside the row even when it straddles n
     if (base >= F.sink_end && base + tile <= F.local_begin) {   // whole tile eligible: no per-token test
       const float4* r4 = reinterpret_cast<const float4*>(row + base);
 #pragma unroll 8
@@ -96,30 +112,19 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  find_threshold_bin(g, state + head * 8, want, dev_status, sh, false);
-  if (want_bound) {                                           // sampled histogram: also the bin that is a bound (word 3)
-    __syncthreads();
-    find_threshold_bin(g, state + head * 8, want_bound, nullptr, sh, true);
-  }
+  find_threshold_bin(g, state + head * 8, want, dev_status, sh, want_bound);
 }
 
-// state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it,
-// [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
+// state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it, [3] = bound bin
+// of a sampled histogram, [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
 // Run by the HIST_THREADS threads of the CTA that completed the head's histogram: thread t owns bins
 // 4095 - 16 t .. 4080 - 16 t (descending), so a block prefix over threads is a suffix count over bins.
-// bound_slot: only the bin is wanted and goes to word 3 (a histogram of a sample: the bin of the sample's
-// want-th largest eligible score is reached by at least `want` eligible tokens of the whole row).
+// want: rank whose bin goes to words 0..2.  want_bound (0 = none): rank whose bin alone goes to word 3 (histogram of
+// a sample: the bin of the sample's want_bound-th largest score is reached by at least that many tokens of the row).
 __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
-                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, bool bound_slot) {
+                                   uint32_t* __restrict__ dev_status, uint32_t* s_warp, uint32_t want_bound) {
   constexpr int BPT = FATHOM_TOPK_BINS / HIST_THREADS;        // 16 bins per thread
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (want == 0) {                                            // nothing to select: no bin is above or equal
-    if (tid == 0) {
-      if (bound_slot) st[3] = FATHOM_TOPK_BINS;
-      else { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
-    }
-    return;
-  }
   uint32_t c[BPT], local = 0;
 #pragma unroll
   for (int x = 0; x < BPT; ++x) { c[x] = __ldcg(h + (FATHOM_TOPK_BINS - 1 - (BPT * tid + x))); local += c[x]; }
@@ -133,23 +138,34 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
   __syncthreads();
   uint32_t above = incl - local;
   for (int w = 0; w < warp; ++w) above += s_warp[w];          // 8 warps: a short serial carry
-  if (above < want && above + local >= want) {
-    uint32_t run = above;
-#pragma unroll
-    for (int x = 0; x < BPT; ++x) {
-      if (run < want && run + c[x] >= want) {
-        const uint32_t bin = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
-        if (bound_slot) st[3] = bin;
-        else { st[0] = bin; st[1] = run; st[2] = want - run; }
+  auto search = [&](uint32_t rank, bool bound_slot) {
+    if (rank == 0) {                                          // nothing to select: no bin is above or equal
+      if (tid == 0) {
+        if (bound_slot) st[3] = FATHOM_TOPK_BINS;
+        else { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
       }
-      run += c[x];
+      return;
     }
-  }
-  if (tid == HIST_THREADS - 1 && above + local < want) {      // fewer eligible tokens than wanted: take them all
-    if (dev_status) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
-    if (bound_slot) st[3] = 0;
-    else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; }
-  }
+    if (above < rank && above + local >= rank) {
+      uint32_t run = above;
+#pragma unroll
+      for (int x = 0; x < BPT; ++x) {
+        if (run < rank && run + c[x] >= rank) {
+          const uint32_t bin = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
+          if (bound_slot) st[3] = bin;
+          else { st[0] = bin; st[1] = run; st[2] = rank - run; }
+        }
+        run += c[x];
+      }
+    }
+    if (tid == HIST_THREADS - 1 && above + local < rank) {    // fewer tokens than wanted: take them all
+      if (!bound_slot && dev_status) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+      if (bound_slot) st[3] = 0;
+      else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; }
+    }
+  };
+  search(want, false);
+  if (want_bound) search(want_bound, true);
 }
 
 // fp32 value whose ordered key is `key` (the inverse of ordered_key for non-NaN patterns)
@@ -355,13 +371,13 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   if (!fathom_gate_open(gate)) return;
-  __shared__ uint64_t s_comp[FIN_CACHE];
   __shared__ uint32_t s_hist[DIGITS];
   __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
   __shared__ uint32_t s_need, s_bucket, s_ntok;
-  extern __shared__ __align__(16) unsigned char s_dyn[];      // DIRECT: range counters, chosen tokens, tokens by range
-  uint32_t* s_range = reinterpret_cast<uint32_t*>(s_dyn);                       // [SORT_BUCKETS]
+  extern __shared__ __align__(16) unsigned char s_dyn[];      // composite cache; DIRECT: + range counters, chosen tokens, tokens by range
+  uint64_t* s_comp = reinterpret_cast<uint64_t*>(s_dyn);                        // [FIN_CACHE]
+  uint32_t* s_range = reinterpret_cast<uint32_t*>(s_comp + FIN_CACHE);          // [SORT_BUCKETS]
   int32_t* s_tok = reinterpret_cast<int32_t*>(s_range + SORT_BUCKETS);          // [k]
   int32_t* s_sorted = s_tok + k;                                                // [k]
   const int head = blockIdx.x, tid = threadIdx.x;
@@ -382,12 +398,19 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   __shared__ uint32_t s_ncache;
   bool cached = m <= FIN_CACHE;
   uint32_t mc = m;                                            // size of the working set
-  auto mark = [&](uint64_t comp) {                            // the token sits in the low 32 bits of every composite
+  // Called by all 32 lanes of a warp together; `take` says whether this lane's composite is chosen.
+  auto mark = [&](bool take, uint64_t comp) {                 // the token sits in the low 32 bits of every composite
     const int32_t i = (int32_t)~(uint32_t)comp;
-    if (DIRECT) {
-      const uint32_t p = atomicAdd(&s_ntok, 1u);
-      if (p < (uint32_t)k) s_tok[p] = i;
-    } else {
+    if (DIRECT) {                                             // warp-aggregated append to the list of chosen tokens
+      const unsigned tm = __ballot_sync(0xffffffffu, take);
+      if (tm) {
+        uint32_t pos = 0;
+        const int leader = __ffs(tm) - 1;
+        if ((tid & 31) == leader) pos = atomicAdd(&s_ntok, (uint32_t)__popc(tm));
+        pos = __shfl_sync(0xffffffffu, pos, leader) + __popc(tm & ((1u << (tid & 31)) - 1u));
+        if (take && pos < (uint32_t)k) s_tok[pos] = i;
+      }
+    } else if (take) {
       atomicOr(&bm[bitmap_word(i)], bitmap_bit(i));
       atomicAdd(&tc[i / FILT_TILE], 1u);
     }
@@ -461,7 +484,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
           for (int u = 0; u < 8; ++u) {
             const uint32_t c = c0 + u * FIN_THREADS + tid;
             const uint64_t top = hi >= 64 ? 0ull : (comp[u] >> hi), ptop = hi >= 64 ? 0ull : (pfx >> hi);
-            if (c < mc && top > ptop) mark(comp[u]);
+            mark(c < mc && top > ptop, comp[u]);
             const bool keep = c < mc && top == ptop;
             const unsigned km = __ballot_sync(0xffffffffu, keep);               // warp-aggregated append
             if (km) {
@@ -481,9 +504,10 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     thr = s_prefix;                                           // undecided low bits are zero
   }
   if (need0 > 0) {
-    for (uint32_t c = tid; c < mc; c += FIN_THREADS) {
-      const uint64_t comp = cached ? s_comp[c] : composite(c);
-      if (need0 >= m || comp >= thr) mark(comp);
+    for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS) {       // uniform trip count: mark is a warp-wide call
+      const uint32_t c = c0 + tid;
+      const uint64_t comp = c < mc ? (cached ? s_comp[c] : composite(c)) : 0ull;
+      mark(c < mc && (need0 >= m || comp >= thr), comp);
     }
   }
 
@@ -614,6 +638,15 @@ static bool force_two_pass() {
   return v;
 }
 
+// Whether a row of n scores is selected in a single pass (and with which estimated sample rank).
+static bool single_pass_plan(long long n, int k, uint32_t want, uint32_t* rank_out) {
+  const long long chunks = n / 1024, sampled = (chunks + 15) / 16;           // whole chunks; chunks 0, 16, 32, .. are sampled
+  const long long n_sample = sampled * 1024;
+  const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)(k - want);
+  *rank_out = rank;
+  return !force_two_pass() && want >= 256 && chunks >= 64 && (long long)rank * 8 <= n_sample && (long long)k * 2 <= n_sample;
+}
+
 // log2 of the token range per counting-sort bucket of the direct select: the smallest that maps n tokens to SORT_BUCKETS
 static int bucket_shift_for(long long n) {
   int s = 0;
@@ -621,7 +654,8 @@ static int bucket_shift_for(long long n) {
   return s;
 }
 
-static size_t direct_select_smem(int k) { return (size_t)SORT_BUCKETS * 4 + (size_t)2 * k * 4; }
+static size_t select_cache_smem() { return (size_t)FIN_CACHE * 8; }
+static size_t direct_select_smem(int k) { return select_cache_smem() + (size_t)SORT_BUCKETS * 4 + (size_t)2 * k * 4; }
 
 // The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
 // and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
@@ -649,10 +683,9 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
   dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
   Gate always = {nullptr, 0u, 0, 0};
   // Single pass when the row is long enough to estimate the threshold from every 16th 1024-score chunk.
-  const long long chunks = (n + 1023) / 1024, sampled = (chunks + 15) / 16;
-  const long long n_sample = sampled * 1024 <= n ? sampled * 1024 : n;       // upper bound on the sampled scores
-  const uint32_t rank = estimate_rank(want, n_sample, n);
-  const bool single = !force_two_pass() && want >= 256 && chunks >= 64 && (long long)rank * 8 <= n_sample;
+  const long long chunks = n / 1024, sampled = (chunks + 15) / 16;           // whole chunks; chunks 0, 16, 32, .. are sampled
+  uint32_t rank = 0;
+  const bool single = single_pass_plan(n, k, want, &rank);
   if (!single) {
     // two passes: histogram of all scores and threshold bin, filter, select within the bin, ascending emission
     const int htile = hist_tile_for(n, Hq);
@@ -661,14 +694,23 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
                                                      (long long)htile, 1, 0u);
     topk_filter_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
                                                        S.tile_count);
-    topk_select_kernel<false><<<Hq, FIN_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap, S.bitmap_words,
-                                                          k, idx, ctx->dev_status, S.tile_count, ntiles, nullptr, 0, 0u, 0, always);
+    static bool attr_set[64] = {};
+    if (ctx->device >= 0 && ctx->device < 64 && !attr_set[ctx->device]) {
+      FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)select_cache_smem()));
+      attr_set[ctx->device] = true;
+    }
+    topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
+                                                                            S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
+                                                                            ntiles, nullptr, 0, 0u, 0, always);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
-    const int reps = sampled >= 64 ? 8 : 1;                            // sampled chunks per CTA
+    // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
+    // reach the bound bin, hence at least k - forced = want eligible ones
+    const int reps = 8;                                                // sampled chunks per CTA
     dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
     topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
-                                                     reps, want);
+                                                     reps, (uint32_t)k);
     topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
                                                         always);
     int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 1, st);
@@ -700,6 +742,17 @@ extern "C" int fathom_topk(fathom_ctx* ctx, const fathom_layout* L, const float*
   if (S.bytes > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
   return run_dense_topk(ctx, scores, n, L->score_stride, L->n_q_heads, k, F, (uint32_t)(k - n_forced), S, idx,
                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fathom_topk_passes(const fathom_layout* L, int k, int n_sink, int n_local) {
+  if (fathom_check_layout(L) != FATHOM_OK || k < 1 || k > L->n || n_sink < 0 || n_local < 0) return FATHOM_ERR_INVALID_ARG;
+  const long long n = L->n;
+  const long long sink_end = n_sink < n ? n_sink : n;
+  const long long local_begin = (n - n_local > sink_end) ? (n - n_local) : sink_end;
+  const long long n_forced = sink_end + (n - local_begin);
+  if (n_forced > k) return FATHOM_ERR_INVALID_ARG;
+  uint32_t rank;
+  return single_pass_plan(n, k, (uint32_t)(k - n_forced), &rank) ? 1 : 2;
 }
 
 // Tile step of the sample scan for (n, k): every 16th scan tile when that sample still holds at least 2 k tokens,
