@@ -55,6 +55,8 @@ size_t fathom_scratch_bytes(const fathom_layout* L, int k) {
   size_t b = fathom_carve_attn(nullptr, L->n_q_heads, k).bytes;
   size_t c = fathom_union_scratch_bytes(L->n_kv_heads, L->n, (L->n_q_heads / L->n_kv_heads) * k);
   size_t e = fathom_calib_scratch_bytes(L->n_kv_heads, L->n);
+  size_t r = fathom_rotate_tc_scratch_bytes(L->n_kv_heads);
+  if (r > e) e = r;
   size_t m = a > b ? a : b;
   m = m > c ? m : c;
   return m > e ? m : e;

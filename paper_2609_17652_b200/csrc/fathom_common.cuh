@@ -106,4 +106,7 @@ struct fathom_attn_scratch {
 fathom_topk_scratch fathom_carve_topk(void* base, int Hq, int64_t n, int k);
 fathom_attn_scratch fathom_carve_attn(void* base, int Hq, int k);
 size_t fathom_union_scratch_bytes(int Hkv, long long n, int capacity);
+size_t fathom_rotate_tc_scratch_bytes(int Hkv);                            // split, transposed basis of the tensor-core rotation
+int fathom_launch_rotate_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
+                            const float* basis, float* K_rot, void* scratch, cudaStream_t st);
 size_t fathom_calib_scratch_bytes(int Hkv, long long n);                  // partial means and covariances   // bitmap + word ranks + union list

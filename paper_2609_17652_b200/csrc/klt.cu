@@ -14,6 +14,9 @@
 // three-way split of the operands.
 #include "fathom_common.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 namespace {
 
 constexpr int KT_THREADS = 256;
@@ -321,6 +324,12 @@ extern "C" int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* L, const
   if (k_dtype != FATHOM_F32 && k_dtype != FATHOM_BF16) return FATHOM_ERR_UNSUPPORTED;
   if (!fathom_aligned16(K) || !fathom_aligned16(basis) || !fathom_aligned16(K_rot)) return FATHOM_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // tensor cores (tf32 operands split in two, three products) unless FATHOM_ROTATE_PATH=simt asks for the plain fp32 kernel
+  const char* path = getenv("FATHOM_ROTATE_PATH");
+  if (!(path && strcmp(path, "simt") == 0)) {
+    if (fathom_rotate_tc_scratch_bytes(L->n_kv_heads) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+    return fathom_launch_rotate_tc(ctx, L, K, k_dtype, mean, basis, K_rot, ctx->scratch, st);
+  }
   const size_t smem = (size_t)2 * FATHOM_D * PANEL * sizeof(float);
   dim3 grid((unsigned)((L->n + FATHOM_D - 1) / FATHOM_D), (unsigned)L->n_kv_heads);
   if (k_dtype == FATHOM_F32) {
