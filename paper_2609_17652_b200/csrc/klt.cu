@@ -255,9 +255,16 @@ static size_t stats_partial_bytes(int Hkv, long long n) {
   return fathom_round_up((size_t)Hkv * (size_t)((n + MEAN_ROWS - 1) / MEAN_ROWS) * 3 * FATHOM_D * 4, 256);
 }
 
-size_t fathom_calib_scratch_bytes(int Hkv, long long n) {
+// covariance partial slots per head: 8192-token tiles of the plain kernel, or the CTAs of the tensor-core kernel
+// (at most one per SM over all heads; 256 bounds the SM count)
+static size_t cov_partial_slots(int Hkv, long long n) {
   const size_t ct = (size_t)((n + COV_ROWS - 1) / COV_ROWS);
-  return stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256) +
+  const size_t tc = (size_t)(256 / Hkv > 0 ? 256 / Hkv : 1);
+  return ct > tc ? ct : tc;
+}
+
+size_t fathom_calib_scratch_bytes(int Hkv, long long n) {
+  return stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * cov_partial_slots(Hkv, n) * FATHOM_D * FATHOM_D * 4, 256) +
          fathom_round_up((size_t)Hkv * FATHOM_D * 4, 256);
 }
 
@@ -293,25 +300,40 @@ extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const v
   const int Hkv = L->n_kv_heads;
   const long long n = L->n;
   if (fathom_calib_scratch_bytes(Hkv, n) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
-  const int mt = (int)((n + MEAN_ROWS - 1) / MEAN_ROWS), ct = (int)((n + COV_ROWS - 1) / COV_ROWS);
+  const int mt = (int)((n + MEAN_ROWS - 1) / MEAN_ROWS);
+  const size_t cov_bytes = fathom_round_up((size_t)Hkv * cov_partial_slots(Hkv, n) * FATHOM_D * FATHOM_D * 4, 256);
   char* base = static_cast<char*>(ctx->scratch);
   float* part = reinterpret_cast<float*>(base);
   float* pcov = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n));
-  float* var_tmp = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * ct * FATHOM_D * FATHOM_D * 4, 256));
+  float* var_tmp = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n) + cov_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);
-  if (k_dtype == FATHOM_F32) {
-    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  // (1) mean
+  if (k_dtype == FATHOM_F32)
     var_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, part, mt);
-    var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
-    cov_partial_kernel<float><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const float*>(K), n, mean, pcov, ct);
-  } else {
-    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  else
     var_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, part, mt);
-    var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
-    cov_partial_kernel<__nv_bfloat16><<<dim3(ct, Hkv), KT_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(K), n, mean, pcov, ct);
+  var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
+  // (2) covariance partials: tensor cores (tf32 operands split in two) unless FATHOM_CALIBRATE_PATH=simt
+  const char* path = getenv("FATHOM_CALIBRATE_PATH");
+  int slots;
+  if (!(path && strcmp(path, "simt") == 0)) {
+    slots = fathom_cov_tc_ctas_per_head(Hkv);
+    if ((size_t)slots > cov_partial_slots(Hkv, n)) slots = (int)cov_partial_slots(Hkv, n);
+    rc = fathom_launch_cov_tc(ctx, L, K, k_dtype, mean, pcov, slots, st);
+    if (rc != FATHOM_OK) return rc;
+  } else {
+    slots = (int)((n + COV_ROWS - 1) / COV_ROWS);
+    const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);
+    if (k_dtype == FATHOM_F32) {
+      FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      cov_partial_kernel<float><<<dim3(slots, Hkv), KT_THREADS, smem, st>>>(static_cast<const float*>(K), n, mean, pcov, slots);
+    } else {
+      FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      cov_partial_kernel<__nv_bfloat16><<<dim3(slots, Hkv), KT_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(K), n, mean, pcov, slots);
+    }
   }
-  cov_final_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, ct, n, cov);
+  // (3) partials summed in fp64 in slot order
+  cov_final_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, slots, n, cov);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

@@ -10,9 +10,10 @@
 // tile ahead), subtract the mean, split, and store head and tail into shared memory in the K-major 128-byte-swizzled
 // layout the MMA descriptors describe; one thread then issues the 4 x 3 MMAs of the chunk (M = 128 tokens, N = 128
 // rotated channels, K = 8) and commits them to the mbarrier that frees the chunk buffer (two buffers).  The split
-// basis (transposed, K-major) stays in shared memory for the whole tile range.  After the fourth chunk the 128 x 128
-// fp32 accumulator is read back with tcgen05.ld (warp w: lanes 32 (w mod 4).., columns 64 (w div 4)..), staged per
-// warp in shared memory and written to global memory in 128-byte rows.
+// basis (transposed, K-major) stays in shared memory for the whole tile range.  Two 128 x 128 fp32 accumulators
+// alternate: while the tensor cores work on tile t, the accumulator of tile t - 1 is read back with tcgen05.ld (warp
+// w: lanes 32 (w mod 4).., columns 64 (w div 4)..), staged per warp in shared memory and written to global memory in
+// 128-byte rows.
 //
 // Every wait on an mbarrier is bounded; a wait that runs out sets FATHOM_DEV_WAIT_EXPIRED in the context status and
 // the CTA stops waiting, finishes its loops, frees its tensor memory and returns.
@@ -26,7 +27,7 @@ constexpr int KC = 32;                                       // channels per chu
 constexpr int NCHUNK = FATHOM_D / KC;                        // 4
 constexpr int SLAB = TILE_M * KC * 4;                        // 16 KB: 128 rows of 128 bytes
 constexpr int UMMA_K = 8;                                    // tf32 elements per MMA along K (32 bytes)
-constexpr uint32_t TMEM_COLS = 128;                          // fp32 accumulator columns
+constexpr uint32_t TMEM_COLS = 256;                          // two fp32 accumulators of 128 columns
 constexpr uint32_t WAIT_TRIES = 1u << 22;
 
 // shared-memory map (bytes from a 1024-byte aligned base)
@@ -36,7 +37,7 @@ constexpr int OFF_XH = OFF_VL + NCHUNK * SLAB;               // 2 slabs: key hea
 constexpr int OFF_XL = OFF_XH + 2 * SLAB;                    // 2 slabs: key tail
 constexpr int OFF_STAGE = OFF_XL + 2 * SLAB;                 // 8 warps x 32 x 32 floats
 constexpr int OFF_MU = OFF_STAGE + 8 * 32 * 32 * 4;          // 128 floats
-constexpr int OFF_BAR = OFF_MU + FATHOM_D * 4;               // 3 mbarriers + tensor-memory base
+constexpr int OFF_BAR = OFF_MU + FATHOM_D * 4;               // 4 mbarriers + tensor-memory base
 constexpr int TC_SMEM = OFF_BAR + 64 + 1024;                 // + slack for the manual 1024-byte alignment
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -106,7 +107,8 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
   float* s_mu = reinterpret_cast<float*>(sm + OFF_MU);
   float* s_stage = reinterpret_cast<float*>(sm + OFF_STAGE);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + OFF_BAR + 32);
-  const uint32_t bar_empty0 = sm_base + OFF_BAR, bar_empty1 = sm_base + OFF_BAR + 8, bar_acc = sm_base + OFF_BAR + 16;
+  const uint32_t bar_empty0 = sm_base + OFF_BAR, bar_empty1 = sm_base + OFF_BAR + 8, bar_acc0 = sm_base + OFF_BAR + 16,
+                 bar_acc1 = sm_base + OFF_BAR + 24;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   // contiguous range of tiles of this CTA over the (KV head, tile) space
@@ -115,7 +117,8 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
   if (tid == 0) {
     mbar_init(bar_empty0, 1);
     mbar_init(bar_empty1, 1);
-    mbar_init(bar_acc, 1);
+    mbar_init(bar_acc0, 1);
+    mbar_init(bar_acc1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {                                            // one warp owns the tensor-memory allocation
@@ -129,28 +132,76 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
 
   // the thread's share of a chunk: four 16-byte pieces, rows row0 + 32 i, piece c4 of the row
   const int c4 = tid & 7, row0 = tid >> 3;
+  const int x_off = slab_offset(row0, c4);
   float4 xr[NCHUNK][4];                                       // one tile ahead, in registers
-  auto load_tile = [&](long long g, int kc) {
-    const long long kv = g / tiles_per_head, r0 = (g % tiles_per_head) * TILE_M;
-    const T* Kh = K + ((size_t)kv * (size_t)n) * FATHOM_D + kc * KC + c4 * 4;
+  // rows r_first + row0 + 32 i of the head whose keys start at Kh (nullptr: no such tile, zeros)
+  auto load_tile = [&](const T* Kh, long long r_first, int kc) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const long long r = r0 + row0 + 32 * i;
-      xr[kc][i] = (g < g1 && r < n) ? load_row4<T>(Kh + (size_t)r * FATHOM_D) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const long long r = r_first + row0 + 32 * i;
+      xr[kc][i] = (Kh != nullptr && r < n) ? load_row4<T>(Kh + (size_t)r * FATHOM_D + kc * KC + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
+  auto head_keys = [&](long long kv) { return K + (size_t)kv * (size_t)n * FATHOM_D; };
   if (g0 < g1) {
 #pragma unroll
-    for (int kc = 0; kc < NCHUNK; ++kc) load_tile(g0, kc);
+    for (int kc = 0; kc < NCHUNK; ++kc) load_tile(head_keys(g0 / tiles_per_head), (g0 % tiles_per_head) * TILE_M, kc);
   }
 
   bool alive = true;                                          // false once a bounded wait ran out
   uint32_t q = 0, tcount = 0;                                 // chunks and tiles handled so far (mbarrier phases)
   long long cur_kv = -1;
+
+  // accumulator `acc` (tile number t, rows r0.. of head kv) -> registers -> per-warp staging -> 128-byte rows in global
+  // memory.  It runs one tile late, while the tensor cores work on the next tile in the other accumulator.
+  auto epilogue = [&](long long kv, long long r0, uint32_t t) {
+    const uint32_t acc = t & 1u;
+    if (alive && !mbar_wait(acc ? bar_acc1 : bar_acc0, (t >> 1) & 1u)) alive = false;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int lq = warp & 3, cb = (warp >> 2) * 64;
+    float4* st4 = reinterpret_cast<float4*>(s_stage + warp * 1024);     // 32 rows of 8 16-byte pieces, piece f of row r at f ^ (r & 7)
+    float* out = K_rot + ((size_t)kv * (size_t)n + (size_t)r0 + lq * 32) * FATHOM_D + cb;
+    const int rows_valid = (int)min((long long)32, n - r0 - lq * 32);  // rows of this warp inside the sequence (may be <= 0)
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      uint32_t r[32];
+      const uint32_t taddr = tmem_d + ((uint32_t)(lq * 32) << 16) + acc * 128u + (uint32_t)(cb + p * 32);
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+          "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+            "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+            "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+            "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+          : "r"(taddr) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      __syncwarp();
+#pragma unroll
+      for (int f = 0; f < 8; ++f)                                        // lane = row: its 32 columns as eight pieces
+        st4[lane * 8 + (f ^ (lane & 7))] = make_float4(__uint_as_float(r[4 * f]), __uint_as_float(r[4 * f + 1]),
+                                                        __uint_as_float(r[4 * f + 2]), __uint_as_float(r[4 * f + 3]));
+      __syncwarp();
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {                                   // four rows of 128 bytes per store instruction
+        const int rr = it * 4 + (lane >> 3), f = lane & 7;
+        if (rr < rows_valid)
+          *reinterpret_cast<float4*>(out + (size_t)rr * FATHOM_D + p * 32 + f * 4) = st4[rr * 8 + (f ^ (rr & 7))];
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");   // a later MMA overwrites this accumulator
+  };
+
+  long long prev_kv = -1, prev_r0 = 0;                        // tile whose epilogue is still due
+  long long kv = g0 / tiles_per_head, tile_in_head = g0 % tiles_per_head;
   for (long long g = g0; g < g1; ++g, ++tcount) {
-    const long long kv = g / tiles_per_head, r0 = (g % tiles_per_head) * TILE_M;
+    const long long r0 = tile_in_head * TILE_M;
+    long long kv_next = kv, tile_next = tile_in_head + 1;     // the tile after this one (fetched while this one is handled)
+    if (tile_next == tiles_per_head) { tile_next = 0; ++kv_next; }
+    const T* K_next = (g + 1 < g1) ? head_keys(kv_next) : nullptr;
+    const long long r_next = tile_next * TILE_M;
     if (kv != cur_kv) {                                       // new head: its split basis and mean into shared memory
-      __syncthreads();                                        // the previous tile's epilogue waited for all MMAs: nobody reads the old ones
+      if (prev_kv >= 0) { epilogue(prev_kv, prev_r0, tcount - 1); prev_kv = -1; }   // also waits for every MMA issued so far
+      __syncthreads();                                        // nobody reads the old basis any more
       const float4* gh = reinterpret_cast<const float4*>(vh_t + (size_t)kv * FATHOM_D * FATHOM_D);
       const float4* gl = reinterpret_cast<const float4*>(vl_t + (size_t)kv * FATHOM_D * FATHOM_D);
       for (int e = tid; e < FATHOM_D * (FATHOM_D / 4); e += TC_THREADS) {
@@ -163,6 +214,7 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
       cur_kv = kv;
       __syncthreads();
     }
+    const uint32_t acc_col = tmem_d + (tcount & 1u) * 128u;
 #pragma unroll
     for (int kc = 0; kc < NCHUNK; ++kc, ++q) {
       const int buf = q & 1;
@@ -174,15 +226,12 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
         const float4 x = xr[kc][i];
         const float a0 = x.x - mu.x, a1 = x.y - mu.y, a2 = x.z - mu.z, a3 = x.w - mu.w;
         const float h0 = tf32_head(a0), h1 = tf32_head(a1), h2 = tf32_head(a2), h3 = tf32_head(a3);
-        const int row = row0 + 32 * i;
-        const bool real = r0 + row < n;                       // rows past the end stay zero (the mean is not subtracted)
-        const int off = buf * SLAB + slab_offset(row, c4);
-        *reinterpret_cast<float4*>(sm + OFF_XH + off) = real ? make_float4(h0, h1, h2, h3) : make_float4(0.f, 0.f, 0.f, 0.f);
-        *reinterpret_cast<float4*>(sm + OFF_XL + off) =
-            real ? make_float4(tf32_head(a0 - h0), tf32_head(a1 - h1), tf32_head(a2 - h2), tf32_head(a3 - h3))
-                 : make_float4(0.f, 0.f, 0.f, 0.f);
+        const int off = buf * SLAB + x_off + i * 4096;        // row0 + 32 i: four 8-row groups further, same place in the group
+        // (rows past the end of the sequence give rows of the accumulator that are never written out)
+        *reinterpret_cast<float4*>(sm + OFF_XH + off) = make_float4(h0, h1, h2, h3);
+        *reinterpret_cast<float4*>(sm + OFF_XL + off) = make_float4(tf32_head(a0 - h0), tf32_head(a1 - h1), tf32_head(a2 - h2), tf32_head(a3 - h3));
       }
-      load_tile(g + 1, kc);                                   // the registers are free: fetch the next tile's chunk
+      load_tile(K_next, r_next, kc);                          // the registers are free: fetch the next tile's chunk
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncthreads();
@@ -193,24 +242,154 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
 #pragma unroll
         for (int ks = 0; ks < KC / UMMA_K; ++ks) {
           const uint32_t ko = ks * UMMA_K * 4;                // bytes along K inside the swizzled row
-          umma_tf32(tmem_d, umma_desc(xl + ko), umma_desc(vh + ko), (kc | ks) ? 1u : 0u);
-          umma_tf32(tmem_d, umma_desc(xh + ko), umma_desc(vl + ko), 1u);
-          umma_tf32(tmem_d, umma_desc(xh + ko), umma_desc(vh + ko), 1u);
+          umma_tf32(acc_col, umma_desc(xl + ko), umma_desc(vh + ko), (kc | ks) ? 1u : 0u);
+          umma_tf32(acc_col, umma_desc(xh + ko), umma_desc(vl + ko), 1u);
+          umma_tf32(acc_col, umma_desc(xh + ko), umma_desc(vh + ko), 1u);
         }
         umma_commit(bar_empty);
-        if (kc == NCHUNK - 1) umma_commit(bar_acc);
+        if (kc == NCHUNK - 1) umma_commit((tcount & 1u) ? bar_acc1 : bar_acc0);
       }
     }
-    // ---- epilogue: accumulator -> registers -> per-warp staging -> 128-byte rows in global memory
-    if (alive && !mbar_wait(bar_acc, tcount & 1)) alive = false;
+    if (prev_kv >= 0) epilogue(prev_kv, prev_r0, tcount - 1);  // the previous tile, while this one's MMAs run
+    prev_kv = kv;
+    prev_r0 = r0;
+    kv = kv_next;
+    tile_in_head = tile_next;
+  }
+  if (prev_kv >= 0) epilogue(prev_kv, prev_r0, tcount - 1);
+
+  // ---- all MMAs issued by this CTA are complete (their commits were waited for) unless a wait ran out
+  if (!alive && dev_status) atomicOr(dev_status, FATHOM_DEV_WAIT_EXPIRED);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    {
-      const int lq = warp & 3, cb = (warp >> 2) * 64;
-      float* st = s_stage + warp * 1024;
-      float* out = K_rot + ((size_t)kv * (size_t)n + (size_t)r0 + lq * 32) * FATHOM_D + cb;
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---- covariance partials on the tensor cores: C = sum_t (x_t - mu)(x_t - mu)^T ----------------------------------------
+// D[i][j] += sum_t A[i][t] B[j][t] with A = B = (X - mu)^T, i.e. M = N = 128 channels and K = tokens.  X is stored token
+// by token with the channels contiguous, which is the MN-major operand form: a slab holds 64 tokens x 32 channels in
+// rows of 128 bytes (row = token; swizzled in 32-byte pieces over groups of four rows, the only form MN-major tf32
+// operands take), four slabs side by side cover the 128 channels (leading offset = slab size), eight token rows
+// (1024 bytes) are one K step.  Head and tail of the split keys serve as both operands:
+// xh xh^T + xh xl^T + xl xh^T.  A CTA accumulates a contiguous token range of one KV head in tensor memory and writes
+// one 128 x 128 partial at the end; the partials are summed in fp64 by the caller's reduction kernel.
+constexpr int CV_TOK = 64;                                   // tokens per stage
+constexpr int CV_SLAB = CV_TOK * 128;                        // 8 KB: 64 token rows of 128 bytes (32 channels)
+constexpr int CV_PART = NCHUNK * CV_SLAB;                    // 32 KB: head (or tail) of one stage, 128 channels
+constexpr int CV_OFF_STAGE = 4 * CV_PART;                    // two stages x (head, tail), then the epilogue staging
+constexpr int CV_OFF_MU = CV_OFF_STAGE + 8 * 32 * 32 * 4;
+constexpr int CV_OFF_BAR = CV_OFF_MU + FATHOM_D * 4;
+constexpr int CV_SMEM = CV_OFF_BAR + 64 + 1024;
+// MN-major operands of 32-bit elements take the 128-byte swizzle with a 32-byte base: rows of 128 bytes (32 channels) in
+// groups of FOUR, and inside a group the 32-byte piece p of row r sits at position p ^ (r & 3).
+__device__ __forceinline__ int slab_offset_mn(int row, int c4) { return row * 128 + (((((c4 >> 1) ^ (row & 3)) << 1) | (c4 & 1)) << 4); }
+// descriptor: leading offset = bytes between 32-channel slabs, stride offset = bytes between 4-token groups, layout type 1
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(CV_SLAB >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (1ull << 61);
+}
+constexpr uint32_t UMMA_IDESC_MN = UMMA_IDESC | (1u << 15) | (1u << 16);   // A and B MN-major
+__device__ __forceinline__ void umma_tf32_mn(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+      :: "r"(tmem_d), "l"(a), "l"(b), "r"(UMMA_IDESC_MN), "r"(accumulate), "r"(0u) : "memory");
+}
+
+template <typename T>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, float* __restrict__ partial, long long n,
+                      uint32_t* __restrict__ dev_status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const uint32_t sm_base = smem_u32(sm);
+  float* s_mu = reinterpret_cast<float*>(sm + CV_OFF_MU);
+  float* s_stage = reinterpret_cast<float*>(sm + CV_OFF_STAGE);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + CV_OFF_BAR + 32);
+  const uint32_t bar_empty0 = sm_base + CV_OFF_BAR, bar_empty1 = sm_base + CV_OFF_BAR + 8, bar_acc = sm_base + CV_OFF_BAR + 16;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, kv = blockIdx.y;
+  // this CTA's tokens: stages of 64 tokens, split evenly over the CTAs of the head
+  const long long stages_total = (n + CV_TOK - 1) / CV_TOK;
+  const long long s0 = stages_total * blockIdx.x / gridDim.x, s1 = stages_total * (blockIdx.x + 1) / gridDim.x;
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
+
+  if (tid == 0) {
+    mbar_init(bar_empty0, 1);
+    mbar_init(bar_empty1, 1);
+    mbar_init(bar_acc, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(s_tmem)), "r"(128u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid < FATHOM_D) s_mu[tid] = mean[(size_t)kv * FATHOM_D + tid];
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = *s_tmem;
+
+  // the thread's share of a stage: eight 16-byte pieces; piece f = tid + 256 i is token f / 32, channels 4 (f % 32)..
+  const int q4 = tid & 31, kc = q4 >> 3, c4 = q4 & 7, tok0 = tid >> 5;      // token tok0 + 8 i
+  const int x_off = kc * CV_SLAB + slab_offset_mn(tok0, c4);                 // + 1024 i (tokens 8 apart: eight rows further)
+  const float4 mu = *reinterpret_cast<const float4*>(s_mu + 4 * q4);
+  float4 xr[8];
+  auto load_stage = [&](long long st) {
 #pragma unroll
-      for (int p = 0; p < 2; ++p) {
-        uint32_t r[32];
+    for (int i = 0; i < 8; ++i) {
+      const long long t = st * CV_TOK + tok0 + 8 * i;
+      xr[i] = (st < s1 && t < n) ? load_row4<T>(Kh + (size_t)t * FATHOM_D + 4 * q4) : make_float4(mu.x, mu.y, mu.z, mu.w);
+    }
+  };
+  load_stage(s0);
+  bool alive = true;
+  uint32_t q = 0;
+  for (long long st = s0; st < s1; ++st, ++q) {
+    const int buf = q & 1;
+    const uint32_t bar_empty = buf ? bar_empty1 : bar_empty0;
+    if (q >= 2 && alive && !mbar_wait(bar_empty, ((q >> 1) - 1) & 1)) alive = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {                             // tokens past the end were loaded as the mean: they add nothing
+      const float a0 = xr[i].x - mu.x, a1 = xr[i].y - mu.y, a2 = xr[i].z - mu.z, a3 = xr[i].w - mu.w;
+      const float h0 = tf32_head(a0), h1 = tf32_head(a1), h2 = tf32_head(a2), h3 = tf32_head(a3);
+      const int off = buf * 2 * CV_PART + x_off + i * 1024;
+      *reinterpret_cast<float4*>(sm + off) = make_float4(h0, h1, h2, h3);
+      *reinterpret_cast<float4*>(sm + off + CV_PART) = make_float4(tf32_head(a0 - h0), tf32_head(a1 - h1), tf32_head(a2 - h2), tf32_head(a3 - h3));
+    }
+    load_stage(st + 1);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t xh = sm_base + buf * 2 * CV_PART, xl = xh + CV_PART;
+#pragma unroll
+      for (int ks = 0; ks < CV_TOK / UMMA_K; ++ks) {          // eight tokens per MMA = one 1024-byte group of rows
+        const uint64_t dh = umma_desc_mn(xh + ks * 1024), dl = umma_desc_mn(xl + ks * 1024);
+        umma_tf32_mn(tmem_d, dl, dh, (q | (uint32_t)ks) ? 1u : 0u);
+        umma_tf32_mn(tmem_d, dh, dl, 1u);
+        umma_tf32_mn(tmem_d, dh, dh, 1u);
+      }
+      umma_commit(bar_empty);
+      if (st == s1 - 1) umma_commit(bar_acc);
+    }
+  }
+  // ---- the partial: accumulator -> registers -> staging -> global memory (zeros if the CTA had no tokens)
+  float* out_base = partial + ((size_t)kv * gridDim.x + blockIdx.x) * FATHOM_D * FATHOM_D;
+  if (s0 < s1) {
+    if (alive && !mbar_wait(bar_acc, 0)) alive = false;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  }
+  {
+    const int lq = warp & 3, cb = (warp >> 2) * 64;
+    float4* st4 = reinterpret_cast<float4*>(s_stage + warp * 1024);
+    float* out = out_base + (size_t)(lq * 32) * FATHOM_D + cb;
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      uint32_t r[32];
+      if (s0 < s1) {
         const uint32_t taddr = tmem_d + ((uint32_t)(lq * 32) << 16) + (uint32_t)(cb + p * 32);
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -221,25 +400,29 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
               "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
             : "r"(taddr) : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        __syncwarp();
+      } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) st[lane * 32 + (c ^ lane)] = __uint_as_float(r[c]);   // lane = row of the warp's 32
-        __syncwarp();
-#pragma unroll 8
-        for (int rr = 0; rr < 32; ++rr)
-          if (r0 + lq * 32 + rr < n) out[(size_t)rr * FATHOM_D + p * 32 + lane] = st[rr * 32 + (lane ^ rr)];
+        for (int c = 0; c < 32; ++c) r[c] = 0u;
+      }
+      __syncwarp();
+#pragma unroll
+      for (int f = 0; f < 8; ++f)
+        st4[lane * 8 + (f ^ (lane & 7))] = make_float4(__uint_as_float(r[4 * f]), __uint_as_float(r[4 * f + 1]),
+                                                        __uint_as_float(r[4 * f + 2]), __uint_as_float(r[4 * f + 3]));
+      __syncwarp();
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int rr = it * 4 + (lane >> 3), f = lane & 7;
+        *reinterpret_cast<float4*>(out + (size_t)rr * FATHOM_D + p * 32 + f * 4) = st4[rr * 8 + (f ^ (rr & 7))];
       }
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");   // the next tile's first MMA overwrites the accumulator
   }
-
-  // ---- all MMAs issued by this CTA are complete (their commits were waited for) unless a wait ran out
   if (!alive && dev_status) atomicOr(dev_status, FATHOM_DEV_WAIT_EXPIRED);
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 0) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(128u) : "memory");
   }
 }
 
@@ -268,6 +451,30 @@ int fathom_launch_rotate_tc(fathom_ctx* ctx, const fathom_layout* L, const void*
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(rotate_keys_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM));
     rotate_keys_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, TC_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), mean, vh_t, vl_t,
                                                                              K_rot, n, tiles_per_head, total, ctx->dev_status);
+  }
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+// CTAs per KV head of the tensor-core covariance pass (one 128 x 128 partial each)
+int fathom_cov_tc_ctas_per_head(int Hkv) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int c = sms / (Hkv > 0 ? Hkv : 1);
+  return c < 1 ? 1 : c;
+}
+
+// Enqueues the covariance partials [Hkv][ctas][128][128] of (K - mean); returns the number of partials per head.
+int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean, float* partial,
+                         int ctas_per_head, cudaStream_t st) {
+  dim3 grid((unsigned)ctas_per_head, (unsigned)L->n_kv_heads);
+  if (k_dtype == FATHOM_F32) {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, CV_SMEM));
+    cov_partial_tc_kernel<float><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const float*>(K), mean, partial, L->n, ctx->dev_status);
+  } else {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, CV_SMEM));
+    cov_partial_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), mean, partial, L->n,
+                                                                             ctx->dev_status);
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
