@@ -249,6 +249,21 @@ var_final_kernel(const float* __restrict__ partial, int tiles, long long n, floa
   }
 }
 
+// reduction of the tensor-core partials [kv][t][2][d][d]: cov = sum_t (P1 + P2 + P2^T) / (n - 1), fp64, slot order
+__global__ void __launch_bounds__(FATHOM_D)
+cov_final_tc_kernel(const float* __restrict__ partial, int slots, long long n, float* __restrict__ cov) {
+  const int kv = blockIdx.y, i = blockIdx.x, j = threadIdx.x;
+  const float* P = partial + (size_t)kv * slots * 2 * FATHOM_D * FATHOM_D;
+  double s = 0.0;
+#pragma unroll 4
+  for (int t = 0; t < slots; ++t) {
+    const float* p1 = P + (size_t)t * 2 * FATHOM_D * FATHOM_D;
+    const float* p2 = p1 + FATHOM_D * FATHOM_D;
+    s += (double)p1[i * FATHOM_D + j] + ((double)p2[i * FATHOM_D + j] + (double)p2[j * FATHOM_D + i]);
+  }
+  cov[((size_t)kv * FATHOM_D + i) * FATHOM_D + j] = (float)(s / (double)(n > 1 ? n - 1 : 1));
+}
+
 }  // namespace
 
 static size_t stats_partial_bytes(int Hkv, long long n) {
@@ -259,7 +274,7 @@ static size_t stats_partial_bytes(int Hkv, long long n) {
 // (at most one per SM over all heads; 256 bounds the SM count)
 static size_t cov_partial_slots(int Hkv, long long n) {
   const size_t ct = (size_t)((n + COV_ROWS - 1) / COV_ROWS);
-  const size_t tc = (size_t)(256 / Hkv > 0 ? 256 / Hkv : 1);
+  const size_t tc = 2 * (size_t)(256 / Hkv > 0 ? 256 / Hkv : 1);   // two matrices per CTA
   return ct > tc ? ct : tc;
 }
 
@@ -318,9 +333,12 @@ extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const v
   int slots;
   if (!(path && strcmp(path, "simt") == 0)) {
     slots = fathom_cov_tc_ctas_per_head(Hkv);
-    if ((size_t)slots > cov_partial_slots(Hkv, n)) slots = (int)cov_partial_slots(Hkv, n);
+    if ((size_t)slots * 2 > cov_partial_slots(Hkv, n)) slots = (int)(cov_partial_slots(Hkv, n) / 2);
     rc = fathom_launch_cov_tc(ctx, L, K, k_dtype, mean, pcov, slots, st);
     if (rc != FATHOM_OK) return rc;
+    cov_final_tc_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, slots, n, cov);
+    FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+    return FATHOM_OK;
   } else {
     slots = (int)((n + COV_ROWS - 1) / COV_ROWS);
     const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);

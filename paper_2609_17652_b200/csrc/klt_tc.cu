@@ -322,7 +322,7 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(s_tmem)), "r"(128u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(s_tmem)), "r"(256u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid < FATHOM_D) s_mu[tid] = mean[(size_t)kv * FATHOM_D + tid];
@@ -368,29 +368,30 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
 #pragma unroll
       for (int ks = 0; ks < CV_TOK / UMMA_K; ++ks) {          // eight tokens per MMA = one 1024-byte group of rows
         const uint64_t dh = umma_desc_mn(xh + ks * 1024), dl = umma_desc_mn(xl + ks * 1024);
-        umma_tf32_mn(tmem_d, dl, dh, (q | (uint32_t)ks) ? 1u : 0u);
-        umma_tf32_mn(tmem_d, dh, dl, 1u);
-        umma_tf32_mn(tmem_d, dh, dh, 1u);
+        const uint32_t accumulate = (q | (uint32_t)ks) ? 1u : 0u;
+        umma_tf32_mn(tmem_d, dh, dh, accumulate);             // first accumulator:  sum xh xh^T
+        umma_tf32_mn(tmem_d + 128u, dh, dl, accumulate);      // second accumulator: sum xh xl^T (its transpose is xl xh^T)
       }
       umma_commit(bar_empty);
       if (st == s1 - 1) umma_commit(bar_acc);
     }
   }
   // ---- the partial: accumulator -> registers -> staging -> global memory (zeros if the CTA had no tokens)
-  float* out_base = partial + ((size_t)kv * gridDim.x + blockIdx.x) * FATHOM_D * FATHOM_D;
+  float* out_base = partial + ((size_t)kv * gridDim.x + blockIdx.x) * 2 * FATHOM_D * FATHOM_D;   // two matrices per CTA
   if (s0 < s1) {
     if (alive && !mbar_wait(bar_acc, 0)) alive = false;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
-  {
+#pragma unroll 1
+  for (int which = 0; which < 2; ++which) {
     const int lq = warp & 3, cb = (warp >> 2) * 64;
     float4* st4 = reinterpret_cast<float4*>(s_stage + warp * 1024);
-    float* out = out_base + (size_t)(lq * 32) * FATHOM_D + cb;
+    float* out = out_base + (size_t)which * FATHOM_D * FATHOM_D + (size_t)(lq * 32) * FATHOM_D + cb;
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
       uint32_t r[32];
       if (s0 < s1) {
-        const uint32_t taddr = tmem_d + ((uint32_t)(lq * 32) << 16) + (uint32_t)(cb + p * 32);
+        const uint32_t taddr = tmem_d + ((uint32_t)(lq * 32) << 16) + (uint32_t)(which * 128 + cb + p * 32);
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
@@ -422,7 +423,7 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
   __syncthreads();
   if (warp == 0) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(128u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(256u) : "memory");
   }
 }
 
@@ -464,7 +465,7 @@ int fathom_cov_tc_ctas_per_head(int Hkv) {
   return c < 1 ? 1 : c;
 }
 
-// Enqueues the covariance partials [Hkv][ctas][128][128] of (K - mean); returns the number of partials per head.
+// Enqueues the covariance partials [Hkv][ctas][2][128][128] of (K - mean): sum xh xh^T and sum xh xl^T per CTA.
 int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean, float* partial,
                          int ctas_per_head, cudaStream_t st) {
   dim3 grid((unsigned)ctas_per_head, (unsigned)L->n_kv_heads);
