@@ -54,6 +54,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-host-resident", action="store_true", help="skip the pinned-host-planes scan leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-session-kernels", action="store_true", help="skip the once-per-session statistics / rotation kernels")
     ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
     ap.add_argument("--ref-sample-tokens", type=int, default=65536)
     ap.add_argument("--config4", action="store_true",
@@ -331,6 +332,10 @@ def run_ours(args):
         result["host_resident_row_fetch"] = row_fetch_leg(ctx, lay, L, idx, k, G, stream,
                                                           result["host_resident_scan"]["link_peak_gbs"])
 
+    # ---- once-per-session kernels of the raw and the KLT-rotated store (not part of the step): statistics, rotation
+    if rank == 0 and not args.no_session_kernels:
+        result["session_kernels"] = session_kernels_leg(ctx, lay, L, stream, peak)
+
     # ---- end to end through the C ABI from HOST buffers: H2D of the step's inputs and D2H of its result are timed
     if not args.no_e2e:
         result["e2e"] = e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step)
@@ -344,6 +349,53 @@ def run_ours(args):
         print(json.dumps(result))
     ctx.close()
     fdist.shutdown()
+
+
+def session_kernels_leg(ctx, lay, L, stream, hbm_peak):
+    """Times fathom_channel_variance, fathom_calibrate and fathom_rotate_keys on the bench's keys (L2 flushed before
+    each launch) and reports them against the HBM peak and, for the two contractions, the tf32 tensor peak
+    (measured bf16 peak x the nominal tf32 : bf16 ratio 1.1 : 2.25)."""
+    Hkv, n, d = L.K.shape
+    dev = L.K.device
+    mean = torch.zeros((Hkv, d), device=dev); var = torch.zeros((Hkv, d), device=dev)
+    cov = torch.zeros((Hkv, d, d), device=dev)
+    basis = torch.linalg.qr(torch.randn(Hkv, d, d, device=dev))[0].contiguous()
+    K_rot = torch.empty((Hkv, n, d), device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    calls = {
+        "channel_variance": lambda: ctx.fathom_channel_variance(lay, L.K, mean, var, stream),
+        "calibrate": lambda: ctx.fathom_calibrate(lay, L.K, mean, cov, stream),
+        "rotate_keys": lambda: ctx.fathom_rotate_keys(lay, L.K, mean, basis, K_rot, stream),
+    }
+    kbytes = float(L.K.numel() * L.K.element_size())
+    alg_bytes = {"channel_variance": kbytes, "calibrate": 2 * kbytes, "rotate_keys": kbytes + 4.0 * K_rot.numel()}
+    products = {"calibrate": 2, "rotate_keys": 3}                  # tf32 products per multiply of the split operands
+    tf32_peak = None
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            tf32_peak = float(json.load(f)["bf16_tflops"]) * 1.1 / 2.25
+    out = {}
+    for nm, fn in calls.items():
+        ts = []
+        for it in range(8):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(a.elapsed_time(b) * 1e3)
+        t_us = statistics.median(ts)
+        gbs = alg_bytes[nm] / (t_us * 1e-6) / 1e9
+        r = {"us": round(t_us, 1), "algorithmic_bytes": alg_bytes[nm], "achieved_gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / hbm_peak, 4)}
+        if nm in products:
+            tf = products[nm] * 2.0 * n * Hkv * d * d / (t_us * 1e-6) / 1e12
+            r.update({"tensor_tflops_tf32": round(tf, 1), "tf32_peak_tflops": round(tf32_peak, 1) if tf32_peak else None,
+                      "frac_of_tf32_peak": round(tf / tf32_peak, 4) if tf32_peak else None})
+        out[nm] = r
+    out["note"] = ("once per session, not in the timed step; calibrate reads the keys twice (statistics pass, covariance pass); "
+                   "the contractions run as tcgen05.mma on tf32 operands split in head and tail")
+    return out
 
 
 def host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, plane_bytes_read):

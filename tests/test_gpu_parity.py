@@ -442,3 +442,39 @@ def test_topk_single_pass_and_its_exact_fallback(n_sink, n_local):
         assert np.array_equal(out.cpu().numpy(), want[rows])
         assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("n,dtype", [(1, torch.float32), (100, torch.float32), (128, torch.float32), (64 * 75 + 1, torch.bfloat16),
+                                     (20000, torch.float32)])
+@pytest.mark.parametrize("path", ["tensor", "simt"])
+def test_rotation_and_covariance_kernels_both_paths(n, dtype, path, monkeypatch):
+    """fathom_calibrate and fathom_rotate_keys on the tensor cores (split tf32 operands) and as plain fp32 kernels,
+    each against the oracle, over tiny, ragged and multi-tile sequences, fp32 and bf16 keys, three KV heads (the
+    tile ranges of the persistent CTAs then straddle heads)."""
+    from paper_2609_17652_b200 import binding as fb
+    if path == "simt":
+        monkeypatch.setenv("FATHOM_ROTATE_PATH", "simt"); monkeypatch.setenv("FATHOM_CALIBRATE_PATH", "simt")
+    Hkv, Hq = 3, 6
+    g = torch.Generator(device="cuda"); g.manual_seed(1000 + n)
+    mix = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda", generator=g))[0]
+    sig = torch.exp(torch.rand(Hkv, 1, 128, device="cuda", generator=g) * 3.0 - 2.0)
+    K = (torch.bmm(torch.randn(Hkv, n, 128, device="cuda", generator=g) * sig, mix) + 1.5).to(dtype).contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, 1))
+    mean = torch.full((Hkv, 128), float("nan"), device="cuda"); cov = torch.full((Hkv, 128, 128), float("nan"), device="cuda")
+    ctx.fathom_calibrate(lay, K, mean, cov)
+    Kh = K.float().cpu().numpy()
+    mu_ref, C_ref = O.calibrate(Kh)
+    assert np.allclose(mean.cpu().numpy(), mu_ref, rtol=1e-5, atol=1e-5)
+    scale = np.maximum(np.abs(C_ref).max(axis=(1, 2), keepdims=True), 1e-30)
+    assert np.all(np.abs(cov.cpu().numpy() - C_ref) <= 2e-5 * scale)
+    V = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda", generator=g))[0].contiguous()
+    K_rot = torch.full((Hkv, n, 128), float("nan"), device="cuda")
+    ctx.fathom_rotate_keys(lay, K, mean, V, K_rot)
+    ctx.fathom_rotate_keys(lay, K, mean, V, K_rot)                               # scratch reuse
+    torch.cuda.synchronize()
+    Kr_ref = O.rotate_keys(Kh, mean.cpu().numpy(), V.cpu().numpy())
+    rown = np.linalg.norm(Kr_ref, axis=2, keepdims=True)
+    assert np.all(np.abs(K_rot.cpu().numpy() - Kr_ref) <= 1e-5 * rown + 1e-6)
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
