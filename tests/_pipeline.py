@@ -24,6 +24,7 @@ def run_gpu(L, B, k, hpp, mode=0, n_sink=0, n_local=0, ctx=None, rows_dtype=torc
     out["planes"] = planes[..., :nb].cpu().numpy().view(np.uint64)
     out["scales"] = scales[..., :nb].cpu().numpy().view(np.float16)
     out["planes_pad"] = planes[..., nb:].cpu().numpy()
+    out["planes_t"], out["scales_t"] = planes, scales            # device tensors, for calls made after this one
     if host_planes:
         hp = torch.empty(planes.shape, dtype=planes.dtype, pin_memory=True); hp.copy_(planes)
         hs = torch.empty(scales.shape, dtype=scales.dtype, pin_memory=True); hs.copy_(scales)

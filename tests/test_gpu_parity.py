@@ -478,3 +478,30 @@ def test_rotation_and_covariance_kernels_both_paths(n, dtype, path, monkeypatch)
     assert np.all(np.abs(K_rot.cpu().numpy() - Kr_ref) <= 1e-5 * rown + 1e-6)
     assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+def test_topk_at_the_largest_k_on_every_path():
+    """k = FATHOM_MAX_K (16384): the direct select then holds 2 x 16384 tokens, the composite cache and the range
+    counters in shared memory at once.  Single-pass and two-pass selection and the fused scan + selection."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hkv, Hq, k = 540_000 + 11, 1, 2, 16384
+    assert fb.fathom_topk_passes(fb.make_layout(Hkv, Hq, n), k) == 1
+    L = make_layer(n, Hkv, Hq, seed=33, device="cuda")
+    g = run_gpu(L, 48, k, 2, stages=("scan", "topk"))
+    ref = O.topk(g["scores"].astype(np.float64), k)
+    assert np.array_equal(g["idx"], ref)
+    # forced sink / local tokens together with the largest k, on the scores just computed
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    sc = torch.zeros((Hq, lay.score_stride), device="cuda"); sc[:, :n] = torch.from_numpy(g["scores"]).cuda()
+    idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    ctx.fathom_topk(lay, sc, k, 4, 32, idx)
+    assert np.array_equal(idx.cpu().numpy(), O.topk(g["scores"].astype(np.float64), k, 4, 32))
+    # fused: same selection without the score array
+    planes, scales = g["planes_t"], g["scales_t"]
+    depth = torch.from_numpy(g["depth"]).cuda()
+    idx2 = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    ctx.fathom_scan_topk(lay, planes, scales, L.q, depth, 2, k, 0, 0, idx2)
+    assert np.array_equal(idx2.cpu().numpy(), ref)
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
