@@ -61,6 +61,7 @@ def parse_args():
                     help="instead of the default line: the 16-session agentic batch (planes in pinned host memory), "
                          "one decode step over --layers independently seeded layers")
     ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--lanes", type=int, default=4, help="config 4: stream lanes over which the sessions are spread")
     return ap.parse_args()
 
 
@@ -504,11 +505,11 @@ def run_config4(args):
     lengths = session_lengths(16, 65536, 1048576, seed=0)
     nmax = max(lengths)
     lay_max = fb.make_layout(Hkv, Hq, nmax, d)
-    # two lanes (context + stream + work buffers): while one session's top-k and attention run, the next session's
-    # scan already pulls its planes over the host link
+    # stream lanes (context + stream + work buffers each): while one session's top-k and attention run, the next
+    # sessions' scans already pull their planes over the host link
     stream = torch.cuda.current_stream()
     lanes = []
-    for li in range(2):
+    for li in range(max(1, args.lanes)):
         lanes.append({"ctx": fb.Context(0, fb.fathom_scratch_bytes(lay_max, k)),
                       "stream": stream if li == 0 else torch.cuda.Stream(),
                       "depth": torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev),
@@ -544,19 +545,22 @@ def run_config4(args):
         ts = []
         for it in range(4):                                      # the decode step of this layer over the 16 sessions
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            fork, join = torch.cuda.Event(), torch.cuda.Event()
+            fork = torch.cuda.Event()
             a.record(stream)
             fork.record(stream)
-            lanes[1]["stream"].wait_event(fork)
+            for W in lanes[1:]:
+                W["stream"].wait_event(fork)
             for s_i, S in enumerate(sess):
-                W = lanes[s_i % 2]
+                W = lanes[s_i % len(lanes)]
                 lay, st, c = S["lay"], W["stream"], W["ctx"]
                 c.fathom_alloc_depth(lay, S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, W["depth"], st)
                 c.fathom_scan(lay, S["hp"], S["hs"], S["q"], W["depth"], hpp, W["scores"], st)
                 c.fathom_topk(lay, W["scores"], k, 0, 0, W["idx"], st)
                 c.fathom_sparse_attend(lay, S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
-            join.record(lanes[1]["stream"])
-            stream.wait_event(join)
+            for W in lanes[1:]:
+                join = torch.cuda.Event()
+                join.record(W["stream"])
+                stream.wait_event(join)
             b.record(stream)
             torch.cuda.synchronize()
             if it:
@@ -568,7 +572,9 @@ def run_config4(args):
                 ctx.fathom_alloc_depth(S["lay"], S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, depth, stream)
                 torch.cuda.synchronize()
                 bytes_link += sum(bits_per_token(r) for r in depth.cpu().numpy()) / 8.0 * S["n"] * (hpp / (Hq // Hkv))
-    status = lanes[0]["ctx"].fathom_device_status() | lanes[1]["ctx"].fathom_device_status(lanes[1]["stream"])
+    status = 0
+    for W in lanes:
+        status |= W["ctx"].fathom_device_status(W["stream"])
     total_tokens = sum(lengths)
     ms = statistics.mean(layer_ms)
     print(json.dumps({
@@ -577,7 +583,7 @@ def run_config4(args):
         "dtype": "u64 bit planes + f32 accumulate", "data": "synthetic",
         "config": {"workload": "agentic multi-session batch (config 4): 16 sessions, planes in pinned host memory",
                    "session_tokens": lengths, "total_tokens": total_tokens, "kv_heads": Hkv, "q_heads": Hq, "budget_bits": B,
-                   "k": k, "layers_measured": args.layers, "layers_of_the_model": 36},
+                   "k": k, "layers_measured": args.layers, "layers_of_the_model": 36, "stream_lanes": len(lanes)},
         "bytes_over_link_per_layer": bytes_link, "host_link_gbs": round(bytes_link / (ms * 1e-3) / 1e9, 2),
         "device_status": status}))
     for W in lanes:

@@ -40,6 +40,7 @@ struct Forced { long long sink_end, local_begin; };          // eligible tokens:
 
 using Gate = fathom_gate;
 
+template <int THREADS, bool IN_GLOBAL>
 __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
                                    uint32_t* __restrict__ dev_status, uint32_t* s_warp, uint32_t want_bound);
 
@@ -112,22 +113,28 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  find_threshold_bin(g, state + head * 8, want, dev_status, sh, want_bound);
+  find_threshold_bin<HIST_THREADS, true>(g, state + head * 8, want, dev_status, sh, want_bound);
 }
 
 // state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it, [3] = bound bin
 // of a sampled histogram, [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
-// Run by the HIST_THREADS threads of the CTA that completed the head's histogram: thread t owns bins
-// 4095 - 16 t .. 4080 - 16 t (descending), so a block prefix over threads is a suffix count over bins.
+// Run by all THREADS threads of a CTA that sees the head's complete histogram h (in global memory: the CTA that
+// finished it last; or in shared memory): thread t owns bins 4095 - BPT t .. (descending), so a block prefix over
+// threads is a suffix count over bins.  s_warp: at least THREADS / 32 words of shared memory.
 // want: rank whose bin goes to words 0..2.  want_bound (0 = none): rank whose bin alone goes to word 3 (histogram of
 // a sample: the bin of the sample's want_bound-th largest score is reached by at least that many tokens of the row).
+template <int THREADS, bool IN_GLOBAL>
 __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __restrict__ st, uint32_t want,
                                    uint32_t* __restrict__ dev_status, uint32_t* s_warp, uint32_t want_bound) {
-  constexpr int BPT = FATHOM_TOPK_BINS / HIST_THREADS;        // 16 bins per thread
+  constexpr int BPT = FATHOM_TOPK_BINS / THREADS;             // bins per thread
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t c[BPT], local = 0;
 #pragma unroll
-  for (int x = 0; x < BPT; ++x) { c[x] = __ldcg(h + (FATHOM_TOPK_BINS - 1 - (BPT * tid + x))); local += c[x]; }
+  for (int x = 0; x < BPT; ++x) {                             // a histogram other CTAs added to is read past the L1
+    const uint32_t* p = h + (FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
+    c[x] = IN_GLOBAL ? __ldcg(p) : *p;
+    local += c[x];
+  }
   uint32_t incl = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -137,7 +144,7 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
   if (lane == 31) s_warp[warp] = incl;
   __syncthreads();
   uint32_t above = incl - local;
-  for (int w = 0; w < warp; ++w) above += s_warp[w];          // 8 warps: a short serial carry
+  for (int w = 0; w < warp; ++w) above += s_warp[w];          // a short serial carry over the warps before this one
   auto search = [&](uint32_t rank, bool bound_slot) {
     if (rank == 0) {                                          // nothing to select: no bin is above or equal
       if (tid == 0) {
@@ -158,7 +165,7 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
         run += c[x];
       }
     }
-    if (tid == HIST_THREADS - 1 && above + local < rank) {    // fewer tokens than wanted: take them all
+    if (tid == THREADS - 1 && above + local < rank) {         // fewer tokens than wanted: take them all
       if (!bound_slot && dev_status) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
       if (bound_slot) st[3] = 0;
       else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; }
@@ -166,6 +173,31 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
   };
   search(want, false);
   if (want_bound) search(want_bound, true);
+}
+
+// Histogram of a head's sample (every 16th whole chunk of 1024 scores) by ONE CTA, which then finds the estimated and
+// the bound bin itself: no global histogram, no flush, no ticket.  For rows of up to a few million scores.
+constexpr int SAMPLE_THREADS = 1024;
+__global__ void __launch_bounds__(SAMPLE_THREADS)
+topk_sample_kernel(const float* __restrict__ scores, long long n, long long score_stride, uint32_t* __restrict__ state,
+                   uint32_t want, uint32_t want_bound) {
+  __shared__ uint32_t sh[FATHOM_TOPK_BINS];
+  __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
+  const int head = blockIdx.x;
+  for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) sh[b] = 0u;
+  __syncthreads();
+  const float* row = scores + (size_t)head * (size_t)score_stride;
+  const long long sampled = (n / 1024 + 15) / 16;             // chunks 0, 16, 32, .. that lie wholly inside the row
+#pragma unroll 8
+  for (long long v = threadIdx.x; v < sampled * 256; v += SAMPLE_THREADS) {
+    const float4 x = __ldg(reinterpret_cast<const float4*>(row + (v >> 8) * 16384) + (v & 255));
+    atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
+    atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
+    atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
+    atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
+  }
+  __syncthreads();
+  find_threshold_bin<SAMPLE_THREADS, false>(sh, state + head * 8, want, nullptr, s_warp, want_bound);
 }
 
 // fp32 value whose ordered key is `key` (the inverse of ordered_key for non-NaN patterns)
@@ -677,8 +709,6 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
 
 static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, long long score_stride, int Hq, int k,
                           Forced F, uint32_t want, const fathom_topk_scratch& S, int32_t* idx, cudaStream_t st) {
-  // histograms, per-head states and candidate counters are contiguous at the start of the arena
-  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
   const int ntiles = (int)((n + FILT_TILE - 1) / FILT_TILE);
   dim3 fgrid((unsigned)ntiles, (unsigned)Hq);
   Gate always = {nullptr, 0u, 0, 0};
@@ -686,6 +716,10 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
   const long long chunks = n / 1024, sampled = (chunks + 15) / 16;           // whole chunks; chunks 0, 16, 32, .. are sampled
   uint32_t rank = 0;
   const bool single = single_pass_plan(n, k, want, &rank);
+  // histograms, per-head states and candidate counters are contiguous at the start of the arena; the one-CTA sample
+  // kernel keeps its histogram in shared memory, so only the states and counters need clearing then
+  if (single && sampled <= 256) FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.state, 0, (char*)S.bitmap - (char*)S.state, st));
+  else FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
   if (!single) {
     // two passes: histogram of all scores and threshold bin, filter, select within the bin, ascending emission
     const int htile = hist_tile_for(n, Hq);
@@ -707,10 +741,14 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
     // reach the bound bin, hence at least k - forced = want eligible ones
-    const int reps = 8;                                                // sampled chunks per CTA
-    dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
-    topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
-                                                     reps, (uint32_t)k);
+    if (sampled <= 256) {                                              // up to 4M scores per row: one CTA per head
+      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, n, score_stride, S.state, rank, (uint32_t)k);
+    } else {
+      const int reps = 8;                                              // sampled chunks per CTA
+      dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
+      topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
+                                                       reps, (uint32_t)k);
+    }
     topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
                                                         always);
     int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 1, st);
