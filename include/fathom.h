@@ -138,10 +138,11 @@ int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* pl
  *   idx     out  [Hq][k] int32, ascending token indices
  * Uses the context scratch (fathom_scratch_bytes).
  * Long rows (at least 64 chunks of 1024 scores, k - forced >= 256) are read once: a histogram of every 16th chunk
- * gives an estimated threshold bin (and a bound: the bin of the sample's own (k - forced)-th largest score), one pass
- * collects the tokens above the estimate, and the exact selection runs among them.  If any head collected fewer than
- * it needs, a second collection above the bound, enqueued behind the first, runs instead; the decision is taken on
- * the device and the result is the same either way.  Shorter rows take two passes (histogram of all scores, filter).
+ * gives an estimated threshold bin (and a bound: the bin of the sample's own k-th largest score), one pass collects
+ * the tokens above the estimate, and the exact selection runs among them, head by head.  A head that collected fewer
+ * than it needs is served instead by a second launch, enqueued behind the first, in which the head's CTA collects
+ * above the bound and selects; the decision is taken on the device and the result is the same either way.  Shorter
+ * rows take two passes (histogram of all scores, filter).
  * Environment: FATHOM_TOPK_PATH=two_pass (read once) always takes the two-pass selection. */
 #define FATHOM_MAX_K 16384
 int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* scores, int k,

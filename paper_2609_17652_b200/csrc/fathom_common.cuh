@@ -50,11 +50,16 @@ struct fathom_gate {
   const uint32_t* counts;       // [heads] candidates the first attempt collected per head
   uint32_t want;
   int heads;
-  int mode;                     // 0: always run, 1: only if every head collected enough, 2: only if some head did not
+  int mode;                     // 0: always run; 1: only if every head collected enough; 2: only if some head did not;
+                                // 3 / 4: the CTA's own head (given by the kernel) collected enough / did not
 };
-// Called by every thread of the CTA at the top of a gated kernel.
-__device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g) {
+// Called by every thread of the CTA at the top of a gated kernel; `head` is used by the per-head modes only.
+__device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g, int head = 0) {
   if (g.mode == 0) return true;
+  if (g.mode >= 3) {
+    const bool ok = __ldcg(g.counts + head) >= g.want;
+    return g.mode == 3 ? ok : !ok;
+  }
   bool ok = true;
   for (int h = threadIdx.x; h < g.heads; h += blockDim.x) ok = ok && (__ldcg(g.counts + h) >= g.want);
   const bool all_ok = __syncthreads_and(ok) != 0;

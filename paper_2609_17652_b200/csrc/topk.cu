@@ -399,10 +399,11 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    uint32_t* __restrict__ bitmap, long long bitmap_words, int k, int32_t* __restrict__ idx_out,
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
                    const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
-                   Gate gate) {
+                   Gate gate, const float* __restrict__ collect_scores, long long collect_stride, float* __restrict__ collect_score_out,
+                   int32_t* __restrict__ collect_idx_out) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
-  if (!fathom_gate_open(gate)) return;
+  if (!fathom_gate_open(gate, blockIdx.x)) return;
   __shared__ uint32_t s_hist[DIGITS];
   __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
@@ -414,11 +415,54 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   int32_t* s_sorted = s_tok + k;                                                // [k]
   const int head = blockIdx.x, tid = threadIdx.x;
   // dense: scores row of the head, candidate tokens [n];  direct: candidate scores and tokens [cand_capacity]
-  const float* row = scores + (size_t)head * (size_t)(DIRECT ? cand_capacity : score_stride);
-  const int32_t* cand_h = cand + (size_t)head * (size_t)(DIRECT ? cand_capacity : n);
+  // (when the CTA collects its own candidates they are read back through the pointers they were written through)
+  const bool own_list = DIRECT && collect_scores != nullptr;
+  const float* row = (own_list ? collect_score_out : scores) + (size_t)head * (size_t)(DIRECT ? cand_capacity : score_stride);
+  const int32_t* cand_h = (own_list ? collect_idx_out : cand) + (size_t)head * (size_t)(DIRECT ? cand_capacity : n);
   uint32_t* bm = DIRECT ? nullptr : bitmap + (size_t)head * (size_t)bitmap_words;
   uint32_t* tc = DIRECT ? nullptr : tile_count + (size_t)head * ntiles;
-  const uint32_t m = DIRECT ? (uint32_t)min((long long)cand_count[head], cand_capacity) : state[head * 8 + 4];
+  // Second attempt of the single-pass top-k for this head alone (its estimate was too high): the CTA itself collects
+  // the head's tokens above the BOUND bin (state word 3) from the score row, replacing the head's candidate list.
+  __shared__ uint32_t s_collected;
+  if (DIRECT && collect_scores != nullptr) {
+    if (tid == 0) s_collected = 0u;
+    __syncthreads();
+    const uint32_t bstar = state[head * 8 + 3];
+    const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
+    const float* srow = collect_scores + (size_t)head * (size_t)collect_stride;
+    float* cs = collect_score_out + (size_t)head * (size_t)cand_capacity;
+    int32_t* ci = collect_idx_out + (size_t)head * (size_t)cand_capacity;
+    for (long long base = 0; base < n; base += (long long)FIN_THREADS * 4 * 4) {   // uniform trip count: ballots inside
+      float4 x[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const long long i = base + ((long long)u * FIN_THREADS + tid) * 4;
+        x[u] = i < n ? __ldg(reinterpret_cast<const float4*>(srow + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const long long i = base + ((long long)u * FIN_THREADS + tid) * 4;
+        const float e[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const long long t = i + c;
+          const bool take = t < n && t >= F.sink_end && t < F.local_begin && e[c] >= lo;
+          const unsigned tm = __ballot_sync(0xffffffffu, take);
+          if (tm) {
+            uint32_t pos = 0;
+            const int leader = __ffs(tm) - 1;
+            if ((tid & 31) == leader) pos = atomicAdd(&s_collected, (uint32_t)__popc(tm));
+            pos = __shfl_sync(0xffffffffu, pos, leader) + __popc(tm & ((1u << (tid & 31)) - 1u));
+            if (take && (long long)pos < cand_capacity) { cs[pos] = e[c]; ci[pos] = (int32_t)t; }
+          }
+        }
+      }
+    }
+    __threadfence_block();
+    __syncthreads();
+  }
+  const uint32_t m = DIRECT ? (uint32_t)min((long long)(collect_scores != nullptr ? s_collected : cand_count[head]), cand_capacity)
+                            : state[head * 8 + 4];
   const uint32_t need0 = min(DIRECT ? want_direct : state[head * 8 + 2], m);
   constexpr int TOP = DIRECT ? 64 : 52;                       // undecided bits of the composite
   auto composite = [&](uint32_t c) -> uint64_t {
@@ -691,9 +735,11 @@ static size_t direct_select_smem(int k) { return select_cache_smem() + (size_t)S
 
 // The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
 // and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
-// gate_mode 0: a single attempt whose threshold is a bound (candidates counted in S.cand_count).
+// gate_mode 0: a single attempt whose threshold is a bound (candidates counted in S.cand_count); 1 / 2: first and second
+// attempt of the fused path (all heads together, second list counted in S.cand_count2); 3 / 4: first and second attempt
+// of the single-pass top-k, head by head - the second collects the head's candidates itself from `scores`.
 static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, Forced F, uint32_t want, const fathom_topk_scratch& S,
-                                int32_t* idx, int gate_mode, cudaStream_t st) {
+                                int32_t* idx, int gate_mode, cudaStream_t st, const float* scores = nullptr, long long score_stride = 0) {
   static bool attr_set[64] = {};
   if (ctx->device >= 0 && ctx->device < 64 && !attr_set[ctx->device]) {
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -703,7 +749,8 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
   Gate g = {S.cand_count, want, Hq, gate_mode};
   topk_select_kernel<true><<<Hq, FIN_THREADS, direct_select_smem(k), st>>>(
       S.cand_score, n, 0, F, S.state, S.cand, nullptr, 0, k, idx, ctx->dev_status, nullptr, 0,
-      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g);
+      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g, gate_mode == 4 ? scores : nullptr,
+      score_stride, S.cand_score, S.cand);
   return FATHOM_OK;
 }
 
@@ -736,7 +783,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     }
     topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
                                                                             S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
-                                                                            ntiles, nullptr, 0, 0u, 0, always);
+                                                                            ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
@@ -751,12 +798,10 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     }
     topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
                                                         always);
-    int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 1, st);
+    int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 3, st);
     if (rc != FATHOM_OK) return rc;
-    Gate short_of = {S.cand_count, want, Hq, 2};
-    topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 3, S.cand_score, S.cand, S.cand_count2,
-                                                        short_of);
-    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 2, st);
+    // stands by: a head whose estimate was too high collects above the bound bin and selects, in one CTA
+    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 4, st, scores, score_stride);
     if (rc != FATHOM_OK) return rc;
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
