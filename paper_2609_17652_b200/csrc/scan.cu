@@ -92,6 +92,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
   __shared__ int s_nrows;
   __shared__ int warp_tot[4];
   __shared__ float s_q[NH][FATHOM_D];
+  __shared__ float s_thr[NH];                                 // MODE 2: score a token must reach, per head
   __shared__ alignas(16) uint64_t s_words[STAGE_ROWS][TILE_BLOCKS];   // staged plane words
   __shared__ alignas(16) uint16_t s_scale[STAGE_ROWS][TILE_BLOCKS];   // staged fp16 scales
   __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
@@ -114,6 +115,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
     }
     if (lane == 31) warp_tot[warp] = incl;
     for (int e = tid; e < NH * FATHOM_D; e += SCAN_THREADS) s_q[e / FATHOM_D][e % FATHOM_D] = q[(size_t)h0 * FATHOM_D + e];
+    if (MODE == 2 && tid < NH) s_thr[tid] = bin_lower_edge(fz.state[(h0 + tid) * 8]);   // fetched now, needed in the epilogue
     __syncthreads();
     int base = 0;
     for (int w = 0; w < warp; ++w) base += warp_tot[w];
@@ -301,7 +303,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
     __syncwarp();
     float thr[NH];
 #pragma unroll
-    for (int h = 0; h < NH; ++h) thr[h] = bin_lower_edge(fz.state[(h0 + h) * 8]);
+    for (int h = 0; h < NH; ++h) thr[h] = s_thr[h];
 #pragma unroll
     for (int b = 0; b < WB; ++b) {
       if (b < nblk) {

@@ -179,18 +179,19 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
 // the bound bin itself: no global histogram, no flush, no ticket.  For rows of up to a few million scores.
 constexpr int SAMPLE_THREADS = 1024;
 __global__ void __launch_bounds__(SAMPLE_THREADS)
-topk_sample_kernel(const float* __restrict__ scores, long long n, long long score_stride, uint32_t* __restrict__ state,
-                   uint32_t want, uint32_t want_bound) {
+topk_sample_kernel(const float* __restrict__ scores, long long sampled, long long chunk_stride, long long score_stride,
+                   uint32_t* __restrict__ state, uint32_t want, uint32_t want_bound) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
   const int head = blockIdx.x;
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  const long long sampled = (n / 1024 + 15) / 16;             // chunks 0, 16, 32, .. that lie wholly inside the row
+  // `sampled` whole chunks of 1024 scores, chunk_stride scores apart (16384: every 16th chunk of a score row; 1024: a
+  // compact array of sampled scores)
 #pragma unroll 8
   for (long long v = threadIdx.x; v < sampled * 256; v += SAMPLE_THREADS) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(row + (v >> 8) * 16384) + (v & 255));
+    const float4 x = __ldg(reinterpret_cast<const float4*>(row + (v >> 8) * chunk_stride) + (v & 255));
     atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
@@ -789,7 +790,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
     // reach the bound bin, hence at least k - forced = want eligible ones
     if (sampled <= 256) {                                              // up to 4M scores per row: one CTA per head
-      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, n, score_stride, S.state, rank, (uint32_t)k);
+      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k);
     } else {
       const int reps = 8;                                              // sampled chunks per CTA
       dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
@@ -893,11 +894,16 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   none.local_begin = n_sample;
   const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)n_forced;
   const bool two_attempts = !force_two_pass() && want >= 256 && (long long)rank * 2 <= k;
-  const int htile = hist_tile_for(n_sample, Hq);
-  dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
-  topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(S.sample, n_sample, S.sample_stride, none, S.hist, S.state,
-                                                   two_attempts ? rank : (uint32_t)k, two_attempts ? nullptr : ctx->dev_status,
-                                                   htile, (long long)htile, 1, two_attempts ? (uint32_t)k : 0u);
+  if (n_sample % 1024 == 0 && n_sample / 1024 <= 256) {        // whole chunks, up to 4M tokens: one CTA per head, shared memory only
+    topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(S.sample, n_sample / 1024, 1024LL, S.sample_stride, S.state,
+                                                      two_attempts ? rank : (uint32_t)k, two_attempts ? (uint32_t)k : 0u);
+  } else {
+    const int htile = hist_tile_for(n_sample, Hq);
+    dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
+    topk_hist_kernel<<<hgrid, HIST_THREADS, 0, st>>>(S.sample, n_sample, S.sample_stride, none, S.hist, S.state,
+                                                     two_attempts ? rank : (uint32_t)k, two_attempts ? nullptr : ctx->dev_status,
+                                                     htile, (long long)htile, 1, two_attempts ? (uint32_t)k : 0u);
+  }
   // ---- full scan that keeps only the tokens reaching their head's threshold, then the exact selection among them
   fathom_scan_fuse fz = {};
   fz.tile_step = 1;
