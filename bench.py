@@ -285,7 +285,8 @@ def run_ours(args):
         "unit": "T lookups/s", "frac": round(lookups / (stage_us["scan"] * 1e-6) / lookup_peak, 4),
         "note": "one 8-byte table load per token, group of four rows and head pair; peak = 148 SMs x 15.8 lookups per clock (micro-benchmark of 8-byte shared-memory loads) x 1.965 GHz"}
 
-    # ---- the decode part of the step (everything but the one-off build) replayed as one CUDA graph, median of 30
+    # ---- the decode part of the step (everything but the one-off build) replayed as one CUDA graph: ten replays back
+    #      to back per sample (a single replay would include the idle time before the graph launch arrives), median of 10
     graph_us = None
     try:
         gs = torch.cuda.Stream()
@@ -299,12 +300,15 @@ def run_ours(args):
                     stage_on(i, gs)
         torch.cuda.synchronize()
         ts = []
-        for it in range(33):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); g.replay(); b.record(stream)
+        for it in range(13):                                        # ten replays back to back per sample, as the layers
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)   # of a model would follow each other
+            a.record(stream)
+            for _ in range(10):
+                g.replay()
+            b.record(stream)
             torch.cuda.synchronize()
             if it >= 3:
-                ts.append(a.elapsed_time(b) * 1e3)
+                ts.append(a.elapsed_time(b) * 1e3 / 10.0)
         graph_us = round(statistics.median(ts), 2)
         del g
     except Exception as e:                                      # report, never hide

@@ -307,7 +307,9 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   __shared__ uint16_t s_list[FILT_TILE];
   __shared__ uint32_t s_count, s_base;
   if (!fathom_gate_open(gate)) return;
-  const int head = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // heads and tiles are walked from the last to the first: what the scan wrote last is the likeliest to be in L2 still
+  const int head = gridDim.y - 1 - blockIdx.y, tile = gridDim.x - 1 - blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) s_count = 0u;
   __syncthreads();
   const uint32_t bstar = state[head * 8 + state_word];
@@ -315,7 +317,7 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   // last for "none" (a comparison with NaN is false)
   const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
   const float* row = scores + (size_t)head * (size_t)score_stride;
-  const long long tile0 = (long long)blockIdx.x * FILT_TILE;
+  const long long tile0 = (long long)tile * FILT_TILE;
   const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
   const bool all_elig = wbase >= F.sink_end && wbase + FILT_WARP_TOKENS <= F.local_begin && wbase + FILT_WARP_TOKENS <= n;
   float4 x[FILT_WARP_TOKENS / 128];
