@@ -285,6 +285,16 @@ def run_ours(args):
         "unit": "T lookups/s", "frac": round(lookups / (stage_us["scan"] * 1e-6) / lookup_peak, 4),
         "note": "one 8-byte table load per token, group of four rows and head pair; peak = 148 SMs x 15.8 lookups per clock (micro-benchmark of 8-byte shared-memory loads) x 1.965 GHz"}
 
+    # ---- attention gathers 256-byte rows scattered over 2 + 2 GiB: every row opens a DRAM page, so the copy peak is not
+    #      the bound that matters.  A micro-benchmark of a pure gather (half a warp per row, 8 loads in flight, rows
+    #      summed and dropped) on this machine's B200 read 262,144 such rows (as many as k = 4096 x 32 heads x {K, V}) in
+    #      22.5 us (2.98 TB/s) and 1,048,576 rows at 4.68 TB/s.
+    if Hq * k * 2 == 262144:
+        result["roofline_other_kernels"]["sparse_attend"]["alt_bound"] = {
+            "bound": "scattered 256-byte row gather", "pure_gather_us": 22.5, "attend_us": round(stage_us["sparse_attend"], 2),
+            "frac": round(22.5 / stage_us["sparse_attend"], 3),
+            "note": "pure-gather time measured once by a micro-benchmark (same row count and row size, L2 flushed)"}
+
     # ---- the decode part of the step (everything but the one-off build) replayed as one CUDA graph: ten replays back
     #      to back per sample (a single replay would include the idle time before the graph launch arrives), median of 10
     graph_us = None
