@@ -1,9 +1,8 @@
 // fathom_sparse_attend: gather of the selected K/V rows + exact softmax attention (Sec. 2 "Top-k decoding").
 //
-// Split-k: CTA (split, head) handles FATHOM_ATTN_CHUNK selected rows.  Logits: one thread per row reads
-// its whole K row with 16-byte loads (a row is 256 B in bf16) against q held in shared memory.  After the
-// chunk maximum and exp, each warp walks 32 rows of V with a lane owning 4 channels (one coalesced
-// 256/512-byte row per load instruction) and the four warps are summed in a fixed order.  Every CTA
+// Split-k: CTA (split, head) handles FATHOM_ATTN_CHUNK selected rows.  Logits and the weighted V sum both give half a warp to a row (a row is
+// 256 B in bf16: 16 lanes x 16 bytes, one fully coalesced row per half-warp and load instruction), 16 rows per
+// half-warp with eight in flight; the partial sums are combined in a fixed order.  Every CTA
 // publishes its (max, denominator, weighted sum) triple and takes a ticket; the CTA that draws the last
 // ticket of a head merges all triples in split order, so the output is bit-reproducible whichever CTA
 // that is, and no second launch is needed.
@@ -44,6 +43,35 @@ __device__ __forceinline__ float dot_row(const float* row, const float* sq) {
   }
   return acc;
 }
+// eight consecutive channels of a row, as loaded (converted to fp32 only when used, to keep many rows in flight)
+struct Raw8h { uint4 x; };
+struct Raw8f { float4 a, b; };
+__device__ __forceinline__ Raw8h load_raw(const __nv_bfloat16* p) { Raw8h r; r.x = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
+__device__ __forceinline__ Raw8f load_raw(const float* p) {
+  Raw8f r; r.a = __ldg(reinterpret_cast<const float4*>(p)); r.b = __ldg(reinterpret_cast<const float4*>(p) + 1); return r;
+}
+__device__ __forceinline__ void unpack(const Raw8h& r, float v[8]) {
+  const uint32_t w[4] = {r.x.x, r.x.y, r.x.z, r.x.w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) { v[2 * c] = __uint_as_float(w[c] << 16); v[2 * c + 1] = __uint_as_float(w[c] & 0xffff0000u); }
+}
+__device__ __forceinline__ void unpack(const Raw8f& r, float v[8]) {
+  v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w; v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
+}
+template <typename T> struct RawOf;
+template <> struct RawOf<__nv_bfloat16> { using type = Raw8h; };
+template <> struct RawOf<float> { using type = Raw8f; };
+// eight consecutive channels of a row (one 16-byte load in bf16, two in fp32)
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float v[8]) {
+  const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) { v[2 * c] = __uint_as_float(w[c] << 16); v[2 * c + 1] = __uint_as_float(w[c] & 0xffff0000u); }
+}
+__device__ __forceinline__ void load8(const float* p, float v[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
 __device__ __forceinline__ void load4(const __nv_bfloat16* p, float v[4]) {
   const uint2 x = __ldg(reinterpret_cast<const uint2*>(p));
   v[0] = __uint_as_float(x.x << 16); v[1] = __uint_as_float(x.x & 0xffff0000u);
@@ -64,7 +92,7 @@ attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, 
   __shared__ float s_p[AT_THREADS];
   __shared__ int32_t s_idx[AT_THREADS];
   __shared__ float s_red[AT_WARPS];
-  __shared__ float s_acc[AT_WARPS][FATHOM_D];
+  __shared__ float s_acc[AT_THREADS / 16][FATHOM_D];          // one partial sum per half-warp
   const int split = blockIdx.x, head = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kv = head / G;
   const T* Kh = Krows + (size_t)kv * (size_t)n * FATHOM_D;
@@ -80,8 +108,35 @@ attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, 
   s_idx[tid] = row;
   __syncthreads();
 
-  float e = -INFINITY;
-  if (valid) e = dot_row(Kh + (size_t)row * FATHOM_D, s_q) * softmax_scale;
+  // Half a warp per row (16 lanes x 8 channels = one fully coalesced row per load instruction), 16 rows per half-warp.
+  // All 16 K rows of the half-warp are requested at once; its 16 V rows are requested as soon as the K rows have been
+  // used, so that they arrive while the chunk maximum and the exponentials are computed.
+  using Raw = typename RawOf<T>::type;
+  const int hw = tid >> 4, l16 = tid & 15;
+  Raw raw[16];
+#pragma unroll
+  for (int u = 0; u < 16; ++u) raw[u] = load_raw(Kh + (size_t)s_idx[hw * 16 + u] * FATHOM_D + l16 * 8);
+  {
+    float qv[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) qv[c] = s_q[l16 * 8 + c];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      float x[8];
+      unpack(raw[u], x);
+      float part = 0.0f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) part = fmaf(x[c], qv[c], part);
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);   // fixed butterfly order
+      if (l16 == 0) s_p[hw * 16 + u] = part;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 16; ++u) raw[u] = load_raw(Vh + (size_t)s_idx[hw * 16 + u] * FATHOM_D + l16 * 8);
+  __syncthreads();
+  const float e = valid ? s_p[tid] * softmax_scale : -INFINITY;
+  __syncthreads();                                           // s_p is reused for the probabilities below
   float m = e;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -96,22 +151,24 @@ attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, 
   __syncthreads();                                           // s_red reads done, s_p visible
   if (lane == 0) s_red[warp] = l;
 
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  const int rows_here = min(AT_THREADS, k - split * AT_THREADS);
-  const int r_end = min(rows_here, (warp + 1) * 32);
-#pragma unroll 8
-  for (int r = warp * 32; r < r_end; ++r) {
-    float v[4];
-    load4(Vh + (size_t)s_idx[r] * FATHOM_D + 4 * lane, v);
-    const float pr = s_p[r];
+  // weighted V sum (lane = 8 channels); the eight half-warps are summed in a fixed order
+  {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < 4; ++c) acc[c] = fmaf(pr, v[c], acc[c]);
+    for (int u = 0; u < 16; ++u) {
+      float x[8];
+      unpack(raw[u], x);
+      const float pr = s_p[hw * 16 + u];                       // rows past k carry probability 0
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[c] = fmaf(pr, x[c], acc[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) s_acc[hw][l16 * 8 + c] = acc[c];
   }
-#pragma unroll
-  for (int c = 0; c < 4; ++c) s_acc[warp][4 * lane + c] = acc[c];
   __syncthreads();
   float* out = partial + ((size_t)head * splits + split) * (FATHOM_D + 2);
-  out[2 + tid] = ((s_acc[0][tid] + s_acc[1][tid]) + s_acc[2][tid]) + s_acc[3][tid];
+  out[2 + tid] = (((s_acc[0][tid] + s_acc[1][tid]) + (s_acc[2][tid] + s_acc[3][tid])) +
+                  ((s_acc[4][tid] + s_acc[5][tid]) + (s_acc[6][tid] + s_acc[7][tid])));
   if (tid == 0) { out[0] = m; out[1] = ((s_red[0] + s_red[1]) + s_red[2]) + s_red[3]; }
 
   // ---- publish; the CTA that draws the head's last ticket merges all chunks (and re-arms the ticket counter)
