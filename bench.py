@@ -161,8 +161,8 @@ def run_ours(args):
 
     stage_names = ["build_planes", "alloc_depth", "scan", "topk", "sparse_attend"]
     topk_passes = fb.fathom_topk_passes(lay, k)                 # 1: sampled estimate + one collection pass; 2: histogram + filter
-    # single pass: sample histogram, collection, selection, the gated per-head second attempt; two passes: also 4 kernels
-    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 4, "sparse_attend": 1}
+    # single pass: sample histogram, collection, selection (3 kernels); two passes: histogram, filter, select, emit (4)
+    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 3 if topk_passes == 1 else 4, "sparse_attend": 1}
 
     def stage(i, K=L.K, Kr=L.Krows, Vr=L.Vrows, q=L.q, var=L.var, pl=planes, sc=scales):
         if i == 0:

@@ -180,10 +180,15 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
 constexpr int SAMPLE_THREADS = 1024;
 __global__ void __launch_bounds__(SAMPLE_THREADS)
 topk_sample_kernel(const float* __restrict__ scores, long long sampled, long long chunk_stride, long long score_stride,
-                   uint32_t* __restrict__ state, uint32_t want, uint32_t want_bound) {
+                   uint32_t* __restrict__ state, uint32_t want, uint32_t want_bound, uint32_t* __restrict__ cand_count,
+                   uint32_t* __restrict__ cand_count2) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
   const int head = blockIdx.x;
+  if (threadIdx.x == 0) {                                     // the collection that follows counts from zero
+    cand_count[head] = 0u;
+    if (cand_count2) cand_count2[head] = 0u;
+  }
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) sh[b] = 0u;
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
@@ -419,7 +424,8 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   const int head = blockIdx.x, tid = threadIdx.x;
   // dense: scores row of the head, candidate tokens [n];  direct: candidate scores and tokens [cand_capacity]
   // (when the CTA collects its own candidates they are read back through the pointers they were written through)
-  const bool own_list = DIRECT && collect_scores != nullptr;
+  const bool own_list = DIRECT && collect_scores != nullptr &&
+                        (gate.mode != 5 || __ldcg(gate.counts + head) < gate.want);   // the same for every thread of the CTA
   const float* row = (own_list ? collect_score_out : scores) + (size_t)head * (size_t)(DIRECT ? cand_capacity : score_stride);
   const int32_t* cand_h = (own_list ? collect_idx_out : cand) + (size_t)head * (size_t)(DIRECT ? cand_capacity : n);
   uint32_t* bm = DIRECT ? nullptr : bitmap + (size_t)head * (size_t)bitmap_words;
@@ -427,7 +433,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   // Second attempt of the single-pass top-k for this head alone (its estimate was too high): the CTA itself collects
   // the head's tokens above the BOUND bin (state word 3) from the score row, replacing the head's candidate list.
   __shared__ uint32_t s_collected;
-  if (DIRECT && collect_scores != nullptr) {
+  if (own_list) {
     if (tid == 0) s_collected = 0u;
     __syncthreads();
     const uint32_t bstar = state[head * 8 + 3];
@@ -464,7 +470,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     __threadfence_block();
     __syncthreads();
   }
-  const uint32_t m = DIRECT ? (uint32_t)min((long long)(collect_scores != nullptr ? s_collected : cand_count[head]), cand_capacity)
+  const uint32_t m = DIRECT ? (uint32_t)min((long long)(own_list ? s_collected : cand_count[head]), cand_capacity)
                             : state[head * 8 + 4];
   const uint32_t need0 = min(DIRECT ? want_direct : state[head * 8 + 2], m);
   constexpr int TOP = DIRECT ? 64 : 52;                       // undecided bits of the composite
@@ -739,8 +745,8 @@ static size_t direct_select_smem(int k) { return select_cache_smem() + (size_t)S
 // The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
 // and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
 // gate_mode 0: a single attempt whose threshold is a bound (candidates counted in S.cand_count); 1 / 2: first and second
-// attempt of the fused path (all heads together, second list counted in S.cand_count2); 3 / 4: first and second attempt
-// of the single-pass top-k, head by head - the second collects the head's candidates itself from `scores`.
+// attempt of the fused path (all heads together, second list counted in S.cand_count2); 5: the single-pass top-k, head
+// by head in one launch - a head that collected too few collects again itself, above the bound bin, from `scores`.
 static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, Forced F, uint32_t want, const fathom_topk_scratch& S,
                                 int32_t* idx, int gate_mode, cudaStream_t st, const float* scores = nullptr, long long score_stride = 0) {
   static bool attr_set[64] = {};
@@ -752,7 +758,7 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
   Gate g = {S.cand_count, want, Hq, gate_mode};
   topk_select_kernel<true><<<Hq, FIN_THREADS, direct_select_smem(k), st>>>(
       S.cand_score, n, 0, F, S.state, S.cand, nullptr, 0, k, idx, ctx->dev_status, nullptr, 0,
-      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g, gate_mode == 4 ? scores : nullptr,
+      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g, gate_mode >= 4 ? scores : nullptr,
       score_stride, S.cand_score, S.cand);
   return FATHOM_OK;
 }
@@ -767,9 +773,9 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
   uint32_t rank = 0;
   const bool single = single_pass_plan(n, k, want, &rank);
   // histograms, per-head states and candidate counters are contiguous at the start of the arena; the one-CTA sample
-  // kernel keeps its histogram in shared memory, so only the states and counters need clearing then
-  if (single && sampled <= 256) FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.state, 0, (char*)S.bitmap - (char*)S.state, st));
-  else FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
+  // kernel keeps its histogram in shared memory
+  // (the sample kernel writes every state word that path reads and clears the candidate counter: nothing to clear then)
+  if (!(single && sampled <= 256)) FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
   if (!single) {
     // two passes: histogram of all scores and threshold bin, filter, select within the bin, ascending emission
     const int htile = hist_tile_for(n, Hq);
@@ -792,7 +798,8 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
     // reach the bound bin, hence at least k - forced = want eligible ones
     if (sampled <= 256) {                                              // up to 4M scores per row: one CTA per head
-      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k);
+      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k,
+                                                        S.cand_count, nullptr);
     } else {
       const int reps = 8;                                              // sampled chunks per CTA
       dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
@@ -801,10 +808,9 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     }
     topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
                                                         always);
-    int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 3, st);
-    if (rc != FATHOM_OK) return rc;
-    // stands by: a head whose estimate was too high collects above the bound bin and selects, in one CTA
-    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 4, st, scores, score_stride);
+    // one launch serves both outcomes: a head whose estimate was low enough selects among its collected candidates; a
+    // head that fell short collects above the bound bin itself (one CTA streaming its row) and selects among those
+    int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 5, st, scores, score_stride);
     if (rc != FATHOM_OK) return rc;
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
@@ -890,15 +896,17 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   const long long sampled = (ntiles_scan + step - 1) / step;
   const long long last_start = (sampled - 1) * step * tile;
   const long long n_sample = (sampled - 1) * tile + ((n - last_start) < tile ? (n - last_start) : tile);
-  FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
+  const bool one_cta_sample = n_sample % 1024 == 0 && n_sample / 1024 <= 256;   // whole chunks, up to 4M tokens
+  if (!one_cta_sample) FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
   Forced none;
   none.sink_end = 0;
   none.local_begin = n_sample;
   const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)n_forced;
   const bool two_attempts = !force_two_pass() && want >= 256 && (long long)rank * 2 <= k;
-  if (n_sample % 1024 == 0 && n_sample / 1024 <= 256) {        // whole chunks, up to 4M tokens: one CTA per head, shared memory only
+  if (one_cta_sample) {                                       // one CTA per head, histogram in shared memory only
     topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(S.sample, n_sample / 1024, 1024LL, S.sample_stride, S.state,
-                                                      two_attempts ? rank : (uint32_t)k, two_attempts ? (uint32_t)k : 0u);
+                                                      two_attempts ? rank : (uint32_t)k, two_attempts ? (uint32_t)k : 0u, S.cand_count,
+                                                      S.cand_count2);
   } else {
     const int htile = hist_tile_for(n_sample, Hq);
     dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
