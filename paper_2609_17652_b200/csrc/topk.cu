@@ -185,6 +185,9 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
   const int head = blockIdx.x;
+  // the collection kernel may be launched as a programmatic dependent: let it start at once, it loads its scores while
+  // this kernel runs and waits for this kernel's results only before it compares
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {                                     // the collection that follows counts from zero
     cand_count[head] = 0u;
     if (cand_count2) cand_count2[head] = 0u;
@@ -307,7 +310,7 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
 // from a histogram of every 16th chunk (first attempt); 3: the bin that is a bound (second attempt, gated).
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
-                    const uint32_t* __restrict__ state, int state_word, float* __restrict__ cand_score,
+                    const uint32_t* state, int state_word, float* __restrict__ cand_score,
                     int32_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_count, Gate gate) {
   __shared__ uint16_t s_list[FILT_TILE];
   __shared__ uint32_t s_count, s_base;
@@ -316,11 +319,6 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   const int head = gridDim.y - 1 - blockIdx.y, tile = gridDim.x - 1 - blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) s_count = 0u;
-  __syncthreads();
-  const uint32_t bstar = state[head * 8 + state_word];
-  // lower edge of the bin; the bins below -inf's (no finite score lies there) stand for "every score", a bin past the
-  // last for "none" (a comparison with NaN is false)
-  const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const long long tile0 = (long long)tile * FILT_TILE;
   const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
@@ -331,6 +329,14 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
     const long long t0 = wbase + it * 128 + lane * 4;
     x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  // The scores were complete before the sample kernel started; its threshold and cleared counters are needed from
+  // here on (a no-op unless this kernel was launched as a programmatic dependent of the sample kernel).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  __syncthreads();
+  const uint32_t bstar = __ldcg(state + head * 8 + state_word);
+  // lower edge of the bin; the bins below -inf's (no finite score lies there) stand for "every score", a bin past the
+  // last for "none" (a comparison with NaN is false)
+  const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
 #pragma unroll
   for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
     const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
@@ -806,8 +812,25 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
                                                        reps, (uint32_t)k);
     }
-    topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
-                                                        always);
+    if (sampled <= 256) {
+      // programmatic dependent launch: the collection's CTAs become resident and load their scores while the 32 CTAs of
+      // the sample kernel work; they wait for its completion (griddepcontrol.wait) before they read the threshold
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = fgrid;
+      cfg.blockDim = dim3(FILT_THREADS);
+      cfg.dynamicSmemBytes = 0;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      FATHOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, topk_collect_kernel, scores, n, score_stride, F, (const uint32_t*)S.state, 0,
+                                              S.cand_score, S.cand, S.cand_count, always));
+    } else {
+      topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
+                                                          always);
+    }
     // one launch serves both outcomes: a head whose estimate was low enough selects among its collected candidates; a
     // head that fell short collects above the bound bin itself (one CTA streaming its row) and selects among those
     int rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 5, st, scores, score_stride);
