@@ -515,8 +515,28 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   //      undecided bit downwards (the last digit is shorter) until the chosen bucket is taken whole.
   uint64_t thr = 0;                                           // chosen candidates: composite >= thr
   if (need0 > 0 && need0 < m) {
-    if (tid == 0) { s_prefix = 0; s_need = need0; s_ncache = 0u; }
     int hi = TOP;
+    uint64_t common = 0;                                      // leading bits shared by every candidate
+    if (cached) {
+      // All candidates lie in a narrow band of scores, so their leading bits agree: a digit taken there would put
+      // every candidate in one histogram bin (thousands of atomics on one address).  Start below the highest bit in
+      // which any two composites differ.
+      const uint64_t first = s_comp[0];
+      uint64_t diff = 0;
+      for (uint32_t c = tid; c < m; c += FIN_THREADS) diff |= s_comp[c] ^ first;
+      uint32_t dlo = __reduce_or_sync(0xffffffffu, (uint32_t)diff), dhi = __reduce_or_sync(0xffffffffu, (uint32_t)(diff >> 32));
+      if ((tid & 31) == 0) { s_hist[2 * (tid >> 5)] = dlo; s_hist[2 * (tid >> 5) + 1] = dhi; }
+      __syncthreads();
+      dlo = 0; dhi = 0;
+#pragma unroll 8
+      for (int w = 0; w < FIN_THREADS / 32; ++w) { dlo |= s_hist[2 * w]; dhi |= s_hist[2 * w + 1]; }
+      diff = ((uint64_t)dhi << 32) | dlo;
+      hi = 64 - __clzll((long long)diff);                     // diff != 0: composites are distinct and m > 1
+      if (hi > TOP) hi = TOP;
+      common = hi >= 64 ? 0ull : (first >> hi) << hi;
+      __syncthreads();                                        // s_hist is reused by the passes
+    }
+    if (tid == 0) { s_prefix = common; s_need = need0; s_ncache = 0u; }
     while (hi > 0) {
       const int bits = min(DIGIT_BITS, hi);
       const int lo = hi - bits;
@@ -595,10 +615,41 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     thr = s_prefix;                                           // undecided low bits are zero
   }
   if (need0 > 0) {
-    for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS) {       // uniform trip count: mark is a warp-wide call
-      const uint32_t c = c0 + tid;
-      const uint64_t comp = c < mc ? (cached ? s_comp[c] : composite(c)) : 0ull;
-      mark(c < mc && (need0 >= m || comp >= thr), comp);
+    if (DIRECT && cached) {
+      // chosen tokens -> list: the warp counts its chosen candidates over all its rounds first and reserves their
+      // places with ONE atomic (an atomic per round would serialise the rounds on its return value)
+      constexpr int ROUNDS = FIN_CACHE / FIN_THREADS;          // 8: a cached working set has at most that many rounds
+      uint32_t before = 0, mine = 0;                          // chosen by lower lanes / by this lane, over the rounds
+      unsigned takes = 0;
+#pragma unroll
+      for (int r = 0; r < ROUNDS; ++r) {
+        const uint32_t c = r * FIN_THREADS + tid;
+        const bool take = c < mc && (need0 >= m || s_comp[c] >= thr);
+        const unsigned tm = __ballot_sync(0xffffffffu, take);
+        before += __popc(tm & ((1u << (tid & 31)) - 1u));
+        mine += take;
+        takes |= (unsigned)take << r;
+      }
+      // lane's first place = warp base + (chosen by lower lanes in all rounds) + ... : order inside the warp's slice is
+      // lane-major, any order will do (the list is sorted afterwards)
+      uint32_t warp_total = before + mine;                    // at lane 31: the warp's total
+      warp_total = __shfl_sync(0xffffffffu, warp_total, 31);
+      uint32_t base = 0;
+      if ((tid & 31) == 0 && warp_total) base = atomicAdd(&s_ntok, warp_total);
+      base = __shfl_sync(0xffffffffu, base, 0) + before;
+#pragma unroll
+      for (int r = 0; r < ROUNDS; ++r) {
+        if ((takes >> r) & 1u) {
+          if (base < (uint32_t)k) s_tok[base] = (int32_t)~(uint32_t)s_comp[r * FIN_THREADS + tid];
+          ++base;
+        }
+      }
+    } else {
+      for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS) {     // uniform trip count: mark is a warp-wide call
+        const uint32_t c = c0 + tid;
+        const uint64_t comp = c < mc ? (cached ? s_comp[c] : composite(c)) : 0ull;
+        mark(c < mc && (need0 >= m || comp >= thr), comp);
+      }
     }
   }
 
