@@ -141,3 +141,41 @@ def test_config5_budget_sweep_at_1M():
     assert all(a["attn_rel_err_mean"] >= b["attn_rel_err_mean"] for a, b in zip(wf, wf[1:]))
     assert wf[-1]["attn_rel_err_max"] < 1e-3 and rows[7]["attn_rel_err_max"] < 1e-3
     assert abs(rows[6]["bits_per_token"] - 68) < 1e-9 and abs(rows[7]["bits_per_token"] - 136) < 1e-9
+
+
+def test_topk_on_rows_longer_than_the_one_cta_sample_covers():
+    """Rows of more than 4M scores take the sample histogram in many CTAs (global histogram, last-ticket threshold
+    search) and a plain launch of the collection pass; the selection must still be the oracle's."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hq, k = 4_400_000 + 5, 2, 8192
+    lay = fb.make_layout(1, Hq, n)
+    assert fb.fathom_topk_passes(lay, k) == 1
+    g = torch.Generator(device="cuda"); g.manual_seed(77)
+    sc = torch.zeros((Hq, lay.score_stride), device="cuda")
+    sc[:, :n] = torch.randn((Hq, n), device="cuda", generator=g)
+    sc[1, :n] *= torch.linspace(0.5, 2.0, n, device="cuda")          # spread grows along the row
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    for n_sink, n_local in ((0, 0), (4, 32)):
+        ctx.fathom_topk(lay, sc, k, n_sink, n_local, idx)
+        want = O.topk(sc[:, :n].cpu().numpy().astype(np.float64), k, n_sink, n_local)
+        assert np.array_equal(idx.cpu().numpy(), want)
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+
+
+def test_fused_scan_topk_on_a_sequence_longer_than_the_one_cta_sample_covers():
+    """n > 4M tokens: the fused path's sample is histogrammed by many CTAs; same selection as scan + top-k."""
+    from paper_2609_17652_b200 import binding as fb
+    from tests._pipeline import run_gpu
+    n, Hkv, Hq, k = 4_300_000 + 3, 1, 2, 4096
+    L = make_layer(n, Hkv, Hq, seed=5, device="cuda", want_rows=False)
+    g = run_gpu(L, 48, k, 2, stages=("scan", "topk"))
+    assert np.array_equal(g["idx"], O.topk(g["scores"].astype(np.float64), k))
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    idx = torch.empty((Hq, k), dtype=torch.int32, device="cuda")
+    ctx.fathom_scan_topk(lay, g["planes_t"], g["scales_t"], L.q, torch.from_numpy(g["depth"]).cuda(), 2, k, 0, 0, idx)
+    assert np.array_equal(idx.cpu().numpy(), g["idx"])
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
