@@ -383,7 +383,7 @@ def session_kernels_leg(ctx, lay, L, stream, hbm_peak):
         "rotate_keys": lambda: ctx.fathom_rotate_keys(lay, L.K, mean, basis, K_rot, stream),
     }
     kbytes = float(L.K.numel() * L.K.element_size())
-    alg_bytes = {"channel_variance": kbytes, "calibrate": 2 * kbytes, "rotate_keys": kbytes + 4.0 * K_rot.numel()}
+    alg_bytes = {"channel_variance": kbytes, "calibrate": kbytes, "rotate_keys": kbytes + 4.0 * K_rot.numel()}
     products = {"calibrate": 2, "rotate_keys": 3}                  # tf32 products per multiply of the split operands
     tf32_peak = None
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -408,8 +408,8 @@ def session_kernels_leg(ctx, lay, L, stream, hbm_peak):
             r.update({"tensor_tflops_tf32": round(tf, 1), "tf32_peak_tflops": round(tf32_peak, 1) if tf32_peak else None,
                       "frac_of_tf32_peak": round(tf / tf32_peak, 4) if tf32_peak else None})
         out[nm] = r
-    out["note"] = ("once per session, not in the timed step; calibrate reads the keys twice (statistics pass, covariance pass); "
-                   "the contractions run as tcgen05.mma on tf32 operands split in head and tail")
+    out["note"] = ("once per session, not in the timed step; calibrate reads the keys once (covariance and sums of keys centred "
+                   "on a shift); the contractions run as tcgen05.mma on tf32 operands split in head and tail")
     return out
 
 

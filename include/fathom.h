@@ -201,13 +201,16 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
  * (q . k = (q V) . ((k - mu) V) + q . mu, and the last term is the same for every key).  With these three calls
  * the rest of the path is used as is: build planes from K_rot, pass q_rot to fathom_alloc_depth (with the
  * eigenvalues as `var`) and to fathom_scan, and run attention on the original rows.
- *   fathom_calibrate:    mean [Hkv][d] (as fathom_channel_variance computes it) and unbiased covariance
- *                        cov [Hkv][d][d] (fp32, accumulated per 8192-token tile in fp32 and across tiles in fp64,
- *                        fixed order) of the session's own keys; the
- *                        eigen-decomposition of the 128 x 128 covariances is the caller's (once per session).
- *                        Uses the context scratch.
+ *   fathom_calibrate:    mean [Hkv][d] and unbiased covariance cov [Hkv][d][d] (fp32) of the session's own keys in ONE
+ *                        read of the keys: the keys are centred on a shift (the mean of the head's first 256 keys),
+ *                        sum (x - shift)(x - shift)^T is accumulated on the tensor cores (tf32 operands split in head
+ *                        and tail, fp32 accumulation per CTA) together with the per-channel sums S, and a reduction
+ *                        in fp64 gives mean = shift + S / n, cov = (sum - S S^T / n) / (n - 1); fixed order throughout.
+ *                        The eigen-decomposition of the 128 x 128 covariances is the caller's (once per session).
+ *                        Uses the context scratch.  FATHOM_CALIBRATE_PATH=simt: two passes in plain fp32 FMAs.
  *   fathom_rotate_keys:  K_rot [Hkv][n][d] fp32 = (K - mean) basis, basis [Hkv][d][d] row-major with the
- *                        directions in its columns; plain fp32 multiply-adds in a fixed order.
+ *                        directions in its columns; tensor cores, tf32 operands split in head and tail (three
+ *                        products, fp32 accumulation, fixed order); FATHOM_ROTATE_PATH=simt: plain fp32 FMAs.
  *   fathom_rotate_query: q_rot [Hq][d] = q basis[h / G].
  * K is [Hkv][n][d], FATHOM_F32 or FATHOM_BF16, 16-byte aligned, like basis, cov and K_rot. */
 int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype, float* mean,

@@ -249,10 +249,20 @@ var_final_kernel(const float* __restrict__ partial, int tiles, long long n, floa
   }
 }
 
-// reduction of the tensor-core partials [kv][t][2][d][d]: cov = sum_t (P1 + P2 + P2^T) / (n - 1), fp64, slot order
+// reduction of the tensor-core partials (fp64, slot order): S = sum_t sums[kv][t], mean = shift + S / n,
+// cov = (sum_t (P1 + P2 + P2^T) - S S^T / n) / (n - 1)  with the partials [kv][t][2][d][d] of the shifted keys
 __global__ void __launch_bounds__(FATHOM_D)
-cov_final_tc_kernel(const float* __restrict__ partial, int slots, long long n, float* __restrict__ cov) {
+cov_final_tc_kernel(const float* __restrict__ partial, const float* __restrict__ partial_sum, const float* __restrict__ shift,
+                    int slots, long long n, float* __restrict__ mean, float* __restrict__ cov) {
+  __shared__ double s_S[FATHOM_D];
   const int kv = blockIdx.y, i = blockIdx.x, j = threadIdx.x;
+  {
+    double t = 0.0;
+    for (int u = 0; u < slots; ++u) t += (double)partial_sum[((size_t)kv * slots + u) * FATHOM_D + j];
+    s_S[j] = t;
+    if (i == 0) mean[(size_t)kv * FATHOM_D + j] = (float)((double)shift[(size_t)kv * FATHOM_D + j] + t / (double)n);
+  }
+  __syncthreads();
   const float* P = partial + (size_t)kv * slots * 2 * FATHOM_D * FATHOM_D;
   double s = 0.0;
 #pragma unroll 4
@@ -261,6 +271,7 @@ cov_final_tc_kernel(const float* __restrict__ partial, int slots, long long n, f
     const float* p2 = p1 + FATHOM_D * FATHOM_D;
     s += (double)p1[i * FATHOM_D + j] + ((double)p2[i * FATHOM_D + j] + (double)p2[j * FATHOM_D + i]);
   }
+  s -= s_S[i] * s_S[j] / (double)n;
   cov[((size_t)kv * FATHOM_D + i) * FATHOM_D + j] = (float)(s / (double)(n > 1 ? n - 1 : 1));
 }
 
@@ -278,9 +289,12 @@ static size_t cov_partial_slots(int Hkv, long long n) {
   return ct > tc ? ct : tc;
 }
 
+// per-CTA channel sums of the tensor-core covariance pass: at most 256 CTAs over all heads
+static size_t cov_sums_bytes() { return (size_t)256 * FATHOM_D * 4; }
+
 size_t fathom_calib_scratch_bytes(int Hkv, long long n) {
   return stats_partial_bytes(Hkv, n) + fathom_round_up((size_t)Hkv * cov_partial_slots(Hkv, n) * FATHOM_D * FATHOM_D * 4, 256) +
-         fathom_round_up((size_t)Hkv * FATHOM_D * 4, 256);
+         fathom_round_up((size_t)Hkv * FATHOM_D * 4, 256) + cov_sums_bytes();
 }
 
 extern "C" int fathom_channel_variance(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* mean, float* var,
@@ -322,24 +336,27 @@ extern "C" int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* L, const v
   float* pcov = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n));
   float* var_tmp = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n) + cov_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // (1) mean
+  const char* path = getenv("FATHOM_CALIBRATE_PATH");
+  if (!(path && strcmp(path, "simt") == 0)) {
+    // tensor cores, ONE read of the keys: covariance and per-channel sums of the keys centred on a shift
+    int slots = fathom_cov_tc_ctas_per_head(Hkv);
+    if ((size_t)slots * 2 > cov_partial_slots(Hkv, n)) slots = (int)(cov_partial_slots(Hkv, n) / 2);
+    float* psum = reinterpret_cast<float*>(base + stats_partial_bytes(Hkv, n) + cov_bytes + fathom_round_up((size_t)Hkv * FATHOM_D * 4, 256));   // [Hkv][slots][d]
+    rc = fathom_launch_cov_tc(ctx, L, K, k_dtype, var_tmp, pcov, psum, slots, st);
+    if (rc != FATHOM_OK) return rc;
+    cov_final_tc_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, psum, var_tmp, slots, n, mean, cov);
+    FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+    return FATHOM_OK;
+  }
+  // plain fp32 kernels: (1) mean
   if (k_dtype == FATHOM_F32)
     var_partial_kernel<float><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const float*>(K), n, part, mt);
   else
     var_partial_kernel<__nv_bfloat16><<<dim3(mt, Hkv), KT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(K), n, part, mt);
   var_final_kernel<<<Hkv, FATHOM_D * VF_LANES, 0, st>>>(part, mt, n, mean, var_tmp);
-  // (2) covariance partials: tensor cores (tf32 operands split in two) unless FATHOM_CALIBRATE_PATH=simt
-  const char* path = getenv("FATHOM_CALIBRATE_PATH");
+  // (2) covariance partials
   int slots;
-  if (!(path && strcmp(path, "simt") == 0)) {
-    slots = fathom_cov_tc_ctas_per_head(Hkv);
-    if ((size_t)slots * 2 > cov_partial_slots(Hkv, n)) slots = (int)(cov_partial_slots(Hkv, n) / 2);
-    rc = fathom_launch_cov_tc(ctx, L, K, k_dtype, mean, pcov, slots, st);
-    if (rc != FATHOM_OK) return rc;
-    cov_final_tc_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(pcov, slots, n, cov);
-    FATHOM_CUDA_TRY(ctx, cudaGetLastError());
-    return FATHOM_OK;
-  } else {
+  {
     slots = (int)((n + COV_ROWS - 1) / COV_ROWS);
     const size_t smem = (size_t)FATHOM_D * PANEL * sizeof(float);
     if (k_dtype == FATHOM_F32) {

@@ -298,10 +298,25 @@ __device__ __forceinline__ void umma_tf32_mn(uint32_t tmem_d, uint64_t a, uint64
       :: "r"(tmem_d), "l"(a), "l"(b), "r"(UMMA_IDESC_MN), "r"(accumulate), "r"(0u) : "memory");
 }
 
+// shift[kv][c] = mean of channel c over the head's first min(n, 256) keys (any value near the data would do)
+template <typename T>
+__global__ void __launch_bounds__(FATHOM_D)
+cov_shift_kernel(const T* __restrict__ K, long long n, float* __restrict__ shift) {
+  const int kv = blockIdx.x, c = threadIdx.x;
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
+  const int rows = (int)min((long long)256, n);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int r = 0; r < rows; r += 4)
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (r + u < rows) acc[u] += (float)Kh[(size_t)(r + u) * FATHOM_D + c];
+  shift[(size_t)kv * FATHOM_D + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)rows;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, float* __restrict__ partial, long long n,
-                      uint32_t* __restrict__ dev_status) {
+cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ shift, float* __restrict__ partial,
+                      float* __restrict__ partial_sum, long long n, uint32_t* __restrict__ dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sm_base = smem_u32(sm);
@@ -325,7 +340,7 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(s_tmem)), "r"(256u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid < FATHOM_D) s_mu[tid] = mean[(size_t)kv * FATHOM_D + tid];
+  if (tid < FATHOM_D) s_mu[tid] = shift[(size_t)kv * FATHOM_D + tid];
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -346,13 +361,15 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
   load_stage(s0);
   bool alive = true;
   uint32_t q = 0;
+  float4 sum4 = make_float4(0.f, 0.f, 0.f, 0.f);              // sum of (x - shift) over this thread's tokens, 4 channels
   for (long long st = s0; st < s1; ++st, ++q) {
     const int buf = q & 1;
     const uint32_t bar_empty = buf ? bar_empty1 : bar_empty0;
     if (q >= 2 && alive && !mbar_wait(bar_empty, ((q >> 1) - 1) & 1)) alive = false;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {                             // tokens past the end were loaded as the mean: they add nothing
+    for (int i = 0; i < 8; ++i) {                             // tokens past the end were loaded as the shift: they add nothing
       const float a0 = xr[i].x - mu.x, a1 = xr[i].y - mu.y, a2 = xr[i].z - mu.z, a3 = xr[i].w - mu.w;
+      sum4.x += a0; sum4.y += a1; sum4.z += a2; sum4.w += a3;
       const float h0 = tf32_head(a0), h1 = tf32_head(a1), h2 = tf32_head(a2), h3 = tf32_head(a3);
       const int off = buf * 2 * CV_PART + x_off + i * 1024;
       *reinterpret_cast<float4*>(sm + off) = make_float4(h0, h1, h2, h3);
@@ -375,6 +392,19 @@ cov_partial_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, f
       umma_commit(bar_empty);
       if (st == s1 - 1) umma_commit(bar_acc);
     }
+  }
+  // ---- per-channel sums of (x - shift): the eight threads of a channel quad (one per warp) are added in warp order
+  {
+    float4* red = reinterpret_cast<float4*>(s_stage);         // [8 warps][32 quads]
+    red[warp * 32 + q4] = sum4;
+    __syncthreads();
+    if (warp == 0) {
+      float4 t = red[q4];
+#pragma unroll
+      for (int w = 1; w < 8; ++w) { const float4 u = red[w * 32 + q4]; t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w; }
+      *reinterpret_cast<float4*>(partial_sum + ((size_t)kv * gridDim.x + blockIdx.x) * FATHOM_D + 4 * q4) = t;
+    }
+    __syncthreads();                                          // the staging area is reused by the epilogue below
   }
   // ---- the partial: accumulator -> registers -> staging -> global memory (zeros if the CTA had no tokens)
   float* out_base = partial + ((size_t)kv * gridDim.x + blockIdx.x) * 2 * FATHOM_D * FATHOM_D;   // two matrices per CTA
@@ -465,17 +495,21 @@ int fathom_cov_tc_ctas_per_head(int Hkv) {
   return c < 1 ? 1 : c;
 }
 
-// Enqueues the covariance partials [Hkv][ctas][2][128][128] of (K - mean): sum xh xh^T and sum xh xl^T per CTA.
-int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean, float* partial,
-                         int ctas_per_head, cudaStream_t st) {
+// Enqueues the shift, the covariance partials [Hkv][ctas][2][128][128] (sum xh xh^T and sum xh xl^T of the shifted
+// keys, per CTA) and the per-channel sums [Hkv][ctas][128].
+int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* shift, float* partial,
+                         float* partial_sum, int ctas_per_head, cudaStream_t st) {
   dim3 grid((unsigned)ctas_per_head, (unsigned)L->n_kv_heads);
   if (k_dtype == FATHOM_F32) {
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, CV_SMEM));
-    cov_partial_tc_kernel<float><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const float*>(K), mean, partial, L->n, ctx->dev_status);
+    cov_shift_kernel<float><<<L->n_kv_heads, FATHOM_D, 0, st>>>(static_cast<const float*>(K), L->n, shift);
+    cov_partial_tc_kernel<float><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const float*>(K), shift, partial, partial_sum, L->n,
+                                                                     ctx->dev_status);
   } else {
     FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(cov_partial_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, CV_SMEM));
-    cov_partial_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), mean, partial, L->n,
-                                                                             ctx->dev_status);
+    cov_shift_kernel<__nv_bfloat16><<<L->n_kv_heads, FATHOM_D, 0, st>>>(static_cast<const __nv_bfloat16*>(K), L->n, shift);
+    cov_partial_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), shift, partial,
+                                                                             partial_sum, L->n, ctx->dev_status);
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
