@@ -219,6 +219,16 @@ int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* layout, const void*
                        const float* mean, const float* basis, float* K_rot, void* stream);
 int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* layout, const float* q, const float* basis,
                         float* q_rot, void* stream);
+/* The rotated store in one call: planes and scales (layout and meaning as fathom_build_planes) of the rotated keys
+ * (K - mean) basis, bit for bit what fathom_rotate_keys (tensor-core path) followed by fathom_build_planes produce,
+ * without the [Hkv][n][d] fp32 array of rotated keys in between: the accumulator of the rotation is quantised in the
+ * kernel's epilogue (block maximum, fp16 scale, plane bits by comparison with multiples of the stored scale, plane
+ * words by warp ballots), 256 tokens = one 32-byte sector of every (channel, plane) row at a time.  It trades time
+ * for memory: the warp-collective quantiser in the epilogue makes it slower than the two calls (4.2 ms against
+ * 1.8 + 0.8 ms at n = 1M, 8 KV heads), but n * Hkv * 512 bytes of intermediate storage are not needed.  Arguments as
+ * fathom_rotate_keys and fathom_build_planes; uses the context scratch. */
+int fathom_build_planes_rotated(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype,
+                                const float* mean, const float* basis, uint64_t* planes, uint16_t* scales, void* stream);
 
 /* ---- (8) per-channel key statistics — Sec. 3.3 (the Var(k_j) of g_j), Appendix B5 (from the session's own keys)
  * mean [Hkv][d] and var [Hkv][d] (device, fp32): mean and unbiased (n - 1) sample variance of every channel of

@@ -23,7 +23,7 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
-           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes"]
+           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated"]
 
 
 class Layout(C.Structure):
@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
     lib.fathom_channel_variance.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
     lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
+    lib.fathom_build_planes_rotated.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_sparse_attend_static.argtypes = [LP, vp, vp, vp, i32, vp, i32, C.c_float, vp, vp]
@@ -166,6 +167,10 @@ class Context:
     def fathom_rotate_keys(self, layout, K, mean, basis, K_rot, stream=None):
         self._check(lib.fathom_rotate_keys(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(basis),
                                            _ptr(K_rot), _stream(stream)))
+
+    def fathom_build_planes_rotated(self, layout, K, mean, basis, planes, scales, stream=None):
+        self._check(lib.fathom_build_planes_rotated(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(basis),
+                                                    _ptr(planes), _ptr(scales), _stream(stream)))
 
     def fathom_rotate_query(self, layout, q, basis, q_rot, stream=None):
         self._check(lib.fathom_rotate_query(self._h, C.byref(layout), _ptr(q), _ptr(basis), _ptr(q_rot), _stream(stream)))

@@ -115,6 +115,8 @@ size_t fathom_union_scratch_bytes(int Hkv, long long n, int capacity);
 size_t fathom_rotate_tc_scratch_bytes(int Hkv);                            // split, transposed basis of the tensor-core rotation
 int fathom_launch_rotate_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
                             const float* basis, float* K_rot, void* scratch, cudaStream_t st);
+int fathom_launch_rotate_build_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
+                                  const float* basis, uint64_t* planes, uint16_t* scales, void* scratch, cudaStream_t st);
 int fathom_cov_tc_ctas_per_head(int Hkv);                                  // CTAs (= partials) per head of the tensor-core covariance
 int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, float* shift, float* partial,
                          float* partial_sum, int ctas_per_head, cudaStream_t st);

@@ -409,3 +409,14 @@ extern "C" int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* L, cons
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }
+
+extern "C" int fathom_build_planes_rotated(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
+                                           const float* basis, uint64_t* planes, uint16_t* scales, void* stream) {
+  if (!ctx || !K || !mean || !basis || !planes || !scales) return FATHOM_ERR_INVALID_ARG;
+  int rc = fathom_check_layout(L);
+  if (rc != FATHOM_OK) return rc;
+  if (k_dtype != FATHOM_F32 && k_dtype != FATHOM_BF16) return FATHOM_ERR_UNSUPPORTED;
+  if (!fathom_aligned16(K) || !fathom_aligned16(basis) || !fathom_aligned16(planes) || !fathom_aligned16(scales)) return FATHOM_ERR_ALIGNMENT;
+  if (fathom_rotate_tc_scratch_bytes(L->n_kv_heads) > ctx->scratch_bytes) return FATHOM_ERR_SCRATCH_TOO_SMALL;
+  return fathom_launch_rotate_build_tc(ctx, L, K, k_dtype, mean, basis, planes, scales, ctx->scratch, static_cast<cudaStream_t>(stream));
+}

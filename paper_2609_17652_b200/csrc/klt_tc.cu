@@ -268,6 +268,238 @@ rotate_keys_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, c
   }
 }
 
+// ---- rotation fused with the plane builder: planes and scales of (K - mu) V without ever storing the rotated keys ----
+// Same tile pipeline and the same sequence of MMAs as rotate_keys_tc_kernel (so every accumulator value is bit for bit
+// the rotated key that kernel would store), but the epilogue quantises instead of storing: a CTA takes 256 tokens at a
+// time (two tiles, one per accumulator = four 64-token blocks), and per block and channel forms a = max |k'| (one
+// redux per channel over the warp's 32 tokens, the two halves of a block meet in shared memory), the fp16 scale a/8,
+// the four plane bits of every code by the plane builder's comparisons with exact multiples of the stored scale, and
+// the plane words by warp ballots.  The four blocks' words of a (channel, plane) row are one 32-byte sector, written whole.
+constexpr int FB_PITCH = FATHOM_NPLANES * 4 * 2 + 1;         // words per channel in the staging: [plane][block][half], padded
+constexpr int FB_OFF_OUT = OFF_XL + 2 * SLAB;                // 128 x FB_PITCH words
+constexpr int FB_OFF_SCALE = FB_OFF_OUT + FATHOM_D * FB_PITCH * 4;          // 128 x 4 fp16
+constexpr int FB_OFF_AMAX = FB_OFF_SCALE + FATHOM_D * 4 * 2;                // [2 blocks][2 halves][128] floats
+constexpr int FB_OFF_MU = FB_OFF_AMAX + 2 * 2 * FATHOM_D * 4;
+constexpr int FB_OFF_BAR = FB_OFF_MU + FATHOM_D * 4;
+constexpr int FB_SMEM = FB_OFF_BAR + 64 + 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+rotate_build_tc_kernel(const T* __restrict__ K, const float* __restrict__ mean, const float* __restrict__ vh_t,
+                       const float* __restrict__ vl_t, uint32_t* __restrict__ planes32, uint16_t* __restrict__ scales,
+                       long long n, long long plane_stride, long long scale_stride, uint32_t* __restrict__ dev_status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const uint32_t sm_base = smem_u32(sm);
+  float* s_mu = reinterpret_cast<float*>(sm + FB_OFF_MU);
+  uint32_t* s_out = reinterpret_cast<uint32_t*>(sm + FB_OFF_OUT);
+  uint16_t* s_scale = reinterpret_cast<uint16_t*>(sm + FB_OFF_SCALE);
+  float* s_amax = reinterpret_cast<float*>(sm + FB_OFF_AMAX);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm + FB_OFF_BAR + 32);
+  const uint32_t bar_empty0 = sm_base + FB_OFF_BAR, bar_empty1 = sm_base + FB_OFF_BAR + 8, bar_acc0 = sm_base + FB_OFF_BAR + 16,
+                 bar_acc1 = sm_base + FB_OFF_BAR + 24;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, kv = blockIdx.y;
+  const long long nb = (n + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
+  const long long supers = (n + 255) / 256;                   // 256-token units of this head
+  const long long u0 = supers * blockIdx.x / gridDim.x, u1 = supers * (blockIdx.x + 1) / gridDim.x;
+  const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
+
+  if (tid == 0) {
+    mbar_init(bar_empty0, 1);
+    mbar_init(bar_empty1, 1);
+    mbar_init(bar_acc0, 1);
+    mbar_init(bar_acc1, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  {                                                           // the head's split basis and mean
+    const float4* gh = reinterpret_cast<const float4*>(vh_t + (size_t)kv * FATHOM_D * FATHOM_D);
+    const float4* gl = reinterpret_cast<const float4*>(vl_t + (size_t)kv * FATHOM_D * FATHOM_D);
+    for (int e = tid; e < FATHOM_D * (FATHOM_D / 4); e += TC_THREADS) {
+      const int j = e >> 5, f = e & 31, kc = f >> 3, p = f & 7;
+      const int off = kc * SLAB + slab_offset(j, p);
+      *reinterpret_cast<float4*>(sm + OFF_VH + off) = __ldg(gh + e);
+      *reinterpret_cast<float4*>(sm + OFF_VL + off) = __ldg(gl + e);
+    }
+    if (tid < FATHOM_D) s_mu[tid] = mean[(size_t)kv * FATHOM_D + tid];
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = *s_tmem;
+
+  const int c4 = tid & 7, row0 = tid >> 3;
+  const int x_off = slab_offset(row0, c4);
+  float4 xr[NCHUNK][4];                                       // one 128-token tile ahead, in registers
+  const long long tile_end = u1 * 2;                          // tiles of this CTA: [2 u0, 2 u1)
+  auto load_tile = [&](long long tile, int kc) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const long long r = tile * TILE_M + row0 + 32 * i;
+      xr[kc][i] = (tile < tile_end && r < n) ? load_row4<T>(Kh + (size_t)r * FATHOM_D + kc * KC + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  if (u0 < u1) {
+#pragma unroll
+    for (int kc = 0; kc < NCHUNK; ++kc) load_tile(2 * u0, kc);
+  }
+
+  bool alive = true;
+  uint32_t q = 0, ucount = 0;
+  for (long long u = u0; u < u1; ++u, ++ucount) {
+    // ---- both tiles of the unit: chunks -> shared memory -> MMAs into accumulator 0 / 1
+#pragma unroll
+    for (int sub = 0; sub < 2; ++sub) {
+      const long long tile = 2 * u + sub;
+      const uint32_t acc_col = tmem_d + (uint32_t)sub * 128u;
+#pragma unroll
+      for (int kc = 0; kc < NCHUNK; ++kc, ++q) {
+        const int buf = q & 1;
+        const uint32_t bar_empty = buf ? bar_empty1 : bar_empty0;
+        if (q >= 2 && alive && !mbar_wait(bar_empty, ((q >> 1) - 1) & 1)) alive = false;
+        const float4 mu = *reinterpret_cast<const float4*>(s_mu + kc * KC + c4 * 4);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 x = xr[kc][i];
+          const float a0 = x.x - mu.x, a1 = x.y - mu.y, a2 = x.z - mu.z, a3 = x.w - mu.w;
+          const float h0 = tf32_head(a0), h1 = tf32_head(a1), h2 = tf32_head(a2), h3 = tf32_head(a3);
+          const int off = buf * SLAB + x_off + i * 4096;
+          *reinterpret_cast<float4*>(sm + OFF_XH + off) = make_float4(h0, h1, h2, h3);
+          *reinterpret_cast<float4*>(sm + OFF_XL + off) = make_float4(tf32_head(a0 - h0), tf32_head(a1 - h1), tf32_head(a2 - h2), tf32_head(a3 - h3));
+        }
+        load_tile(tile + 1, kc);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t xh = sm_base + OFF_XH + buf * SLAB, xl = sm_base + OFF_XL + buf * SLAB;
+          const uint32_t vh = sm_base + OFF_VH + kc * SLAB, vl = sm_base + OFF_VL + kc * SLAB;
+#pragma unroll
+          for (int ks = 0; ks < KC / UMMA_K; ++ks) {
+            const uint32_t ko = ks * UMMA_K * 4;
+            umma_tf32(acc_col, umma_desc(xl + ko), umma_desc(vh + ko), (kc | ks) ? 1u : 0u);
+            umma_tf32(acc_col, umma_desc(xh + ko), umma_desc(vl + ko), 1u);
+            umma_tf32(acc_col, umma_desc(xh + ko), umma_desc(vh + ko), 1u);
+          }
+          umma_commit(bar_empty);
+          if (kc == NCHUNK - 1) umma_commit(sub ? bar_acc1 : bar_acc0);
+        }
+      }
+    }
+    // ---- quantising epilogue, tile by tile.  Warp w: tokens 32 (w & 3) .. + 31 of the tile, channels 64 (w >> 2) .. + 63.
+    const int lq = warp & 3, blk = lq >> 1, half = lq & 1, cb = (warp >> 2) * 64;
+#pragma unroll 1
+    for (int sub = 0; sub < 2; ++sub) {
+      if (alive && !mbar_wait(sub ? bar_acc1 : bar_acc0, ucount & 1)) alive = false;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const long long tok = (2 * u + sub) * TILE_M + lq * 32 + lane;          // this lane's token
+      const bool present = tok < n;
+      const uint32_t keep = __ballot_sync(0xffffffffu, present);             // absent tail tokens carry 0 bits
+      uint32_t r[2][32];
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        const uint32_t taddr = tmem_d + ((uint32_t)(lq * 32) << 16) + (uint32_t)sub * 128u + (uint32_t)(cb + p * 32);
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+            : "=r"(r[p][0]), "=r"(r[p][1]), "=r"(r[p][2]), "=r"(r[p][3]), "=r"(r[p][4]), "=r"(r[p][5]), "=r"(r[p][6]), "=r"(r[p][7]),
+              "=r"(r[p][8]), "=r"(r[p][9]), "=r"(r[p][10]), "=r"(r[p][11]), "=r"(r[p][12]), "=r"(r[p][13]), "=r"(r[p][14]),
+              "=r"(r[p][15]), "=r"(r[p][16]), "=r"(r[p][17]), "=r"(r[p][18]), "=r"(r[p][19]), "=r"(r[p][20]), "=r"(r[p][21]),
+              "=r"(r[p][22]), "=r"(r[p][23]), "=r"(r[p][24]), "=r"(r[p][25]), "=r"(r[p][26]), "=r"(r[p][27]), "=r"(r[p][28]),
+              "=r"(r[p][29]), "=r"(r[p][30]), "=r"(r[p][31])
+            : "r"(taddr) : "memory");
+      }
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // block maximum per channel: |k'| of non-negative floats orders like its bit pattern, so one integer redux per
+      // channel gives the warp's maximum; lane c keeps channel c's
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        uint32_t mine = 0u;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          if (!present) r[p][c] = 0u;                         // an absent token counts as 0 everywhere
+          const uint32_t m = __reduce_max_sync(0xffffffffu, r[p][c] & 0x7fffffffu);
+          if (lane == c) mine = m;
+        }
+        s_amax[(blk * 2 + half) * FATHOM_D + cb + p * 32 + lane] = __uint_as_float(mine);
+      }
+      __syncthreads();                                        // the two halves of every block have met
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        const int ch = cb + p * 32 + lane;                    // the channel whose scale and plane words this lane keeps
+        const float a = fmaxf(s_amax[(blk * 2 + 0) * FATHOM_D + ch], s_amax[(blk * 2 + 1) * FATHOM_D + ch]);
+        const __half sh = __float2half_rn(a * 0.125f);        // a/8 is exact; one rounding to fp16
+        const float my_sc = __half2float(sh);
+        uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float sc = __shfl_sync(0xffffffffu, my_sc, c);               // scale of channel cb + 32 p + c
+          const float k = __uint_as_float(r[p][c]);
+          const float s2 = sc * 2.0f, s4 = sc * 4.0f;
+          const bool c0 = k >= 0.0f;
+          float thr = c0 ? s4 : -s4;
+          const bool c1 = k >= thr;
+          thr += c1 ? s2 : -s2;
+          const bool c2 = k >= thr;
+          thr += c2 ? sc : -sc;
+          const bool c3 = k >= thr;
+          const uint32_t b0 = __ballot_sync(0xffffffffu, c0), b1 = __ballot_sync(0xffffffffu, c1);
+          const uint32_t b2 = __ballot_sync(0xffffffffu, c2), b3 = __ballot_sync(0xffffffffu, c3);
+          if (lane == c) { w0 = b0; w1 = b1; w2 = b2; w3 = b3; }
+        }
+        if (my_sc > 0.0f) { w0 &= keep; w1 &= keep; w2 &= keep; w3 &= keep; }
+        else { w0 = keep; w1 = 0u; w2 = 0u; w3 = 0u; }        // zero scale: every code is 8 = 0b1000
+        const int bu = 2 * sub + blk;                         // block within the 256-token unit
+        uint32_t* o = s_out + ch * FB_PITCH;
+        o[(0 * 4 + bu) * 2 + half] = w0;
+        o[(1 * 4 + bu) * 2 + half] = w1;
+        o[(2 * 4 + bu) * 2 + half] = w2;
+        o[(3 * 4 + bu) * 2 + half] = w3;
+        if (half == 0) s_scale[ch * 4 + bu] = __half_as_ushort(sh);
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();                                        // s_amax is reused by the next tile
+    }
+    // ---- flush: the unit's four blocks of every (channel, plane) row are 32 contiguous bytes
+    {
+      const long long b0 = 4 * u;
+      const int nblk = (int)min((long long)4, nb - b0);
+      uint64_t* planes64 = reinterpret_cast<uint64_t*>(planes32);
+      for (int e = tid; e < FATHOM_D * FATHOM_NPLANES; e += TC_THREADS) {
+        const int ch = e >> 2, p = e & 3;
+        const uint32_t* src = s_out + ch * FB_PITCH + p * 8;
+        uint64_t* dst = planes64 + (((size_t)kv * FATHOM_D + ch) * FATHOM_NPLANES + p) * (size_t)plane_stride + b0;
+#pragma unroll
+        for (int pair = 0; pair < 2; ++pair) {
+          if (2 * pair + 1 < nblk) {
+            *reinterpret_cast<uint4*>(dst + 2 * pair) = make_uint4(src[4 * pair], src[4 * pair + 1], src[4 * pair + 2], src[4 * pair + 3]);
+          } else if (2 * pair < nblk) {
+            dst[2 * pair] = ((uint64_t)src[4 * pair + 1] << 32) | src[4 * pair];
+          }
+        }
+      }
+      if (tid < FATHOM_D) {
+        uint16_t* dst = scales + ((size_t)kv * FATHOM_D + tid) * (size_t)scale_stride + b0;
+        for (int x = 0; x < nblk; ++x) dst[x] = s_scale[tid * 4 + x];
+      }
+    }
+    __syncthreads();                                          // the staging is rewritten by the next unit
+  }
+
+  if (!alive && dev_status) atomicOr(dev_status, FATHOM_DEV_WAIT_EXPIRED);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // ---- covariance partials on the tensor cores: C = sum_t (x_t - mu)(x_t - mu)^T ----------------------------------------
 // D[i][j] += sum_t A[i][t] B[j][t] with A = B = (X - mu)^T, i.e. M = N = 128 channels and K = tokens.  X is stored token
 // by token with the channels contiguous, which is the MN-major operand form: a slab holds 64 tokens x 32 channels in
@@ -510,6 +742,36 @@ int fathom_launch_cov_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K,
     cov_shift_kernel<__nv_bfloat16><<<L->n_kv_heads, FATHOM_D, 0, st>>>(static_cast<const __nv_bfloat16*>(K), L->n, shift);
     cov_partial_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, CV_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), shift, partial,
                                                                              partial_sum, L->n, ctx->dev_status);
+  }
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+// Enqueues the fused rotation + plane builder; scratch holds the split, transposed basis (fathom_rotate_tc_scratch_bytes).
+int fathom_launch_rotate_build_tc(fathom_ctx* ctx, const fathom_layout* L, const void* K, int k_dtype, const float* mean,
+                                  const float* basis, uint64_t* planes, uint16_t* scales, void* scratch, cudaStream_t st) {
+  const int Hkv = L->n_kv_heads;
+  const long long n = L->n;
+  float* vh_t = static_cast<float*>(scratch);
+  float* vl_t = vh_t + (size_t)Hkv * FATHOM_D * FATHOM_D;
+  split_basis_kernel<<<dim3(FATHOM_D, Hkv), FATHOM_D, 0, st>>>(basis, vh_t, vl_t);
+  int dev = 0, sms = 0;
+  FATHOM_CUDA_TRY(ctx, cudaGetDevice(&dev));
+  FATHOM_CUDA_TRY(ctx, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const long long supers = (n + 255) / 256;
+  long long per_head = sms / Hkv > 0 ? sms / Hkv : 1;
+  if (per_head > supers) per_head = supers;
+  dim3 grid((unsigned)per_head, (unsigned)Hkv);
+  uint32_t* p32 = reinterpret_cast<uint32_t*>(planes);
+  if (k_dtype == FATHOM_F32) {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(rotate_build_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM));
+    rotate_build_tc_kernel<float><<<grid, TC_THREADS, FB_SMEM, st>>>(static_cast<const float*>(K), mean, vh_t, vl_t, p32, scales, n,
+                                                                      L->plane_stride_words, L->scale_stride, ctx->dev_status);
+  } else {
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(rotate_build_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM));
+    rotate_build_tc_kernel<__nv_bfloat16><<<grid, TC_THREADS, FB_SMEM, st>>>(static_cast<const __nv_bfloat16*>(K), mean, vh_t, vl_t, p32,
+                                                                              scales, n, L->plane_stride_words, L->scale_stride,
+                                                                              ctx->dev_status);
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;

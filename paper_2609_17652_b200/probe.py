@@ -1,6 +1,6 @@
 """Times (or exposes to a profiler) ONE stage of the hot path on synthetic device buffers.
 
-    python -m paper_2609_17652_b200.probe --stage scan|topk|scan_topk|attend|build|alloc|rotate|calibrate|variance [--n N] [--iters I] [--budget B] [--k K]
+    python -m paper_2609_17652_b200.probe --stage scan|topk|scan_topk|attend|build|alloc|rotate|rotate_build|calibrate|variance [--n N] [--iters I] [--budget B] [--k K]
 
 Unlike bench.py it allocates only what the chosen stage touches (random plane words and scales for the scan,
 random scores for top-k, ...), so a full-size launch fits in a few hundred MB and can be captured with ncu.
@@ -19,7 +19,7 @@ from . import binding as fb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "calibrate", "variance"])
+    ap.add_argument("--stage", required=True, choices=["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "rotate_build", "calibrate", "variance"])
     ap.add_argument("--n", type=int, default=1 << 20)
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--budget", type=int, default=48)
@@ -43,14 +43,14 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     st = torch.cuda.current_stream()
 
-    if a.stage in ("build", "rotate", "calibrate", "variance"):
+    if a.stage in ("build", "rotate", "rotate_build", "calibrate", "variance"):
         K = torch.randn(Hkv, n, d, device=dev)
-    if a.stage in ("rotate", "calibrate", "variance"):
+    if a.stage in ("rotate", "rotate_build", "calibrate", "variance"):
         mean = torch.zeros(Hkv, d, device=dev)
         cov = torch.zeros(Hkv, d, d, device=dev)
         basis = torch.linalg.qr(torch.randn(Hkv, d, d, device=dev))[0].contiguous()
         K_rot = torch.empty(Hkv, n, d, device=dev) if a.stage == "rotate" else None
-    if a.stage in ("build", "scan", "scan_topk"):
+    if a.stage in ("build", "rotate_build", "scan", "scan_topk"):
         planes = torch.randint(-(1 << 62), 1 << 62, (Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
         scales = torch.rand(Hkv, d, lay.scale_stride, device=dev).mul_(0.5).add_(0.01).to(torch.float16).view(torch.int16)
         if a.host_planes:
@@ -79,6 +79,8 @@ def main():
             ctx.fathom_topk(lay, scores, a.k, 0, 0, idx, st)
         elif a.stage == "rotate":
             ctx.fathom_rotate_keys(lay, K, mean, basis, K_rot, st)
+        elif a.stage == "rotate_build":
+            ctx.fathom_build_planes_rotated(lay, K, mean, basis, planes, scales, st)
         elif a.stage == "calibrate":
             ctx.fathom_calibrate(lay, K, mean, cov, st)
         elif a.stage == "variance":

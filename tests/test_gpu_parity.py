@@ -505,3 +505,38 @@ def test_topk_at_the_largest_k_on_every_path():
     assert np.array_equal(idx2.cpu().numpy(), ref)
     assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("n,dtype", [(1, torch.float32), (100, torch.float32), (257, torch.float32), (5000, torch.bfloat16),
+                                     (8192 + 77, torch.float32), (70000, torch.float32)])
+def test_rotated_store_in_one_call_equals_rotate_then_build(n, dtype):
+    """fathom_build_planes_rotated gives bit for bit the planes and scales of fathom_rotate_keys followed by
+    fathom_build_planes (both of which are checked against the oracle elsewhere), for tiny, ragged and multi-unit
+    sequences, three KV heads, fp32 and bf16 keys; a channel of constant keys exercises the zero scale."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq = 3, 6
+    g = torch.Generator(device="cuda"); g.manual_seed(2000 + n)
+    mix = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda", generator=g))[0]
+    sig = torch.exp(torch.rand(Hkv, 1, 128, device="cuda", generator=g) * 3.0 - 2.0)
+    K = (torch.bmm(torch.randn(Hkv, n, 128, device="cuda", generator=g) * sig, mix) + 0.75).to(dtype).contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, 1))
+    mean = K.float().mean(dim=1).contiguous()
+    V = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda", generator=g))[0].contiguous()
+    V[1] = torch.eye(128, device="cuda"); K[1, :, 5] = 3.0; mean[1, 5] = 3.0       # rotated channel 5 of head 1 is all zero
+    K_rot = torch.empty((Hkv, n, 128), device="cuda")
+    ctx.fathom_rotate_keys(lay, K, mean, V, K_rot)
+    nb = (n + 63) // 64
+    p_ref = torch.full((Hkv, 128, 4, lay.plane_stride_words), -1, dtype=torch.int64, device="cuda")
+    s_ref = torch.full((Hkv, 128, lay.scale_stride), -1, dtype=torch.int16, device="cuda")
+    ctx.fathom_build_planes(lay, K_rot, p_ref, s_ref)
+    p_one = torch.full_like(p_ref, -1); s_one = torch.full_like(s_ref, -1)
+    ctx.fathom_build_planes_rotated(lay, K, mean, V, p_one, s_one)
+    ctx.fathom_build_planes_rotated(lay, K, mean, V, p_one, s_one)                 # scratch reuse
+    torch.cuda.synchronize()
+    assert torch.equal(p_one[..., :nb], p_ref[..., :nb])
+    assert torch.equal(s_one[..., :nb], s_ref[..., :nb])
+    assert torch.all(p_one[..., nb:] == -1) and torch.all(s_one[..., nb:] == -1)   # padding untouched
+    assert torch.all(s_one[1, 5, :nb] == 0) and torch.all(p_one[1, 5, 1:, :nb] == 0)
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
