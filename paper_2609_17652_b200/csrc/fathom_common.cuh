@@ -69,7 +69,8 @@ __device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g, int head 
 
 struct fathom_scan_fuse {       // extra arguments of the sampling / filtering scan variants
   int tile_step;                // sample: scan every tile_step-th tile
-  const uint32_t* state;        // filter: [Hq][8], word 0 = threshold bin found on the sample
+  const uint32_t* state;        // filter: [Hq][8] (pointer already offset to the word to read): a threshold bin, or,
+  int state_is_score;           //         if state_is_score, the fp32 bits of the score a candidate must reach
   fathom_gate gate;             // filter: whether this launch runs at all
   long long sink_end, local_begin;   // filter: eligible tokens are sink_end <= i < local_begin
   float* cand_score;            // filter: [Hq][capacity] scores of the candidates

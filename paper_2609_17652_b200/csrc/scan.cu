@@ -115,7 +115,8 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
     }
     if (lane == 31) warp_tot[warp] = incl;
     for (int e = tid; e < NH * FATHOM_D; e += SCAN_THREADS) s_q[e / FATHOM_D][e % FATHOM_D] = q[(size_t)h0 * FATHOM_D + e];
-    if (MODE == 2 && tid < NH) s_thr[tid] = bin_lower_edge(fz.state[(h0 + tid) * 8]);   // fetched now, needed in the epilogue
+    if (MODE == 2 && tid < NH)                                // fetched now, needed in the epilogue
+      s_thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : bin_lower_edge(fz.state[(h0 + tid) * 8]);
     __syncthreads();
     int base = 0;
     for (int w = 0; w < warp; ++w) base += warp_tot[w];

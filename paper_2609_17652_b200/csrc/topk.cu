@@ -28,12 +28,23 @@ constexpr int FILT_THREADS = 256;
 constexpr int FILT_WARP_TOKENS = 1024;                       // 32 ballots -> 32 bitmap words per warp
 constexpr int FILT_TILE = (FILT_THREADS / 32) * FILT_WARP_TOKENS;   // 8192 tokens per CTA
 constexpr int FIN_THREADS = 1024;
-constexpr int FIN_CACHE = 8192;                              // candidate composites kept in shared memory (dynamic, 64 KB)
+constexpr int FIN_CACHE = 8192;                              // candidate composites kept in shared memory: two-pass select (64 KB)
+constexpr int FIN_CACHE_MAX = 16384;                         // ... direct select, when k leaves room (128 KB)
 
 __device__ __forceinline__ uint32_t ordered_key(float f) {
   uint32_t u = __float_as_uint(f);
   if ((u << 1) == 0u) u = 0u;                                // -0 -> +0
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// fp32 value whose ordered key is `key` (the inverse of ordered_key for non-NaN patterns)
+__device__ __forceinline__ float key_to_float(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+// Lower edge of a histogram bin as a score: the bins below -inf's (no finite score lies there) stand for "every score",
+// a bin past the last for "none" (a comparison with NaN is false).
+__device__ __forceinline__ float edge_of_bin(uint32_t bin) {
+  return bin >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bin <= 7u ? -INFINITY : key_to_float(bin << 20));
 }
 
 struct Forced { long long sink_end, local_begin; };          // eligible tokens: sink_end <= i < local_begin
@@ -117,7 +128,8 @@ topk_hist_kernel(const float* __restrict__ scores, long long n, long long score_
 }
 
 // state[head][0] = threshold bin, [1] = tokens in bins above it, [2] = tokens still needed from it, [3] = bound bin
-// of a sampled histogram, [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs.
+// of a sampled histogram, [4] = candidates appended by the filter, [5] = ticket counter of the histogram CTAs,
+// [6] = the score a candidate of the first attempt must reach (fp32 bits): the lower edge of bin [0].
 // Run by all THREADS threads of a CTA that sees the head's complete histogram h (in global memory: the CTA that
 // finished it last; or in shared memory): thread t owns bins 4095 - BPT t .. (descending), so a block prefix over
 // threads is a suffix count over bins.  s_warp: at least THREADS / 32 words of shared memory.
@@ -149,7 +161,7 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
     if (rank == 0) {                                          // nothing to select: no bin is above or equal
       if (tid == 0) {
         if (bound_slot) st[3] = FATHOM_TOPK_BINS;
-        else { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; }
+        else { st[0] = FATHOM_TOPK_BINS; st[1] = 0; st[2] = 0; st[6] = __float_as_uint(edge_of_bin(FATHOM_TOPK_BINS)); }
       }
       return;
     }
@@ -160,7 +172,7 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
         if (run < rank && run + c[x] >= rank) {
           const uint32_t bin = (uint32_t)(FATHOM_TOPK_BINS - 1 - (BPT * tid + x));
           if (bound_slot) st[3] = bin;
-          else { st[0] = bin; st[1] = run; st[2] = rank - run; }
+          else { st[0] = bin; st[1] = run; st[2] = rank - run; st[6] = __float_as_uint(edge_of_bin(bin)); }
         }
         run += c[x];
       }
@@ -168,7 +180,7 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
     if (tid == THREADS - 1 && above + local < rank) {         // fewer tokens than wanted: take them all
       if (!bound_slot && dev_status) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
       if (bound_slot) st[3] = 0;
-      else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; }
+      else { st[0] = 0; st[1] = above + local - c[BPT - 1]; st[2] = c[BPT - 1]; st[6] = __float_as_uint(edge_of_bin(0u)); }
     }
   };
   search(want, false);
@@ -209,10 +221,6 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
   find_threshold_bin<SAMPLE_THREADS, false>(sh, state + head * 8, want, nullptr, s_warp, want_bound);
 }
 
-// fp32 value whose ordered key is `key` (the inverse of ordered_key for non-NaN patterns)
-__device__ __forceinline__ float key_to_float(uint32_t key) {
-  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
-}
 
 // Bitmap layout: word (t / 128) * 4 + (t % 4), bit (t % 128) / 4.
 __device__ __forceinline__ long long bitmap_word(long long t) { return (t >> 7) * 4 + (t & 3); }
@@ -333,10 +341,8 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   // here on (a no-op unless this kernel was launched as a programmatic dependent of the sample kernel).
   asm volatile("griddepcontrol.wait;" ::: "memory");
   __syncthreads();
-  const uint32_t bstar = __ldcg(state + head * 8 + state_word);
-  // lower edge of the bin; the bins below -inf's (no finite score lies there) stand for "every score", a bin past the
-  // last for "none" (a comparison with NaN is false)
-  const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
+  // the score a candidate must reach: word 6 (first attempt: estimated, refined) or the lower edge of the bin in state_word
+  const float lo = state_word == 0 ? __uint_as_float(__ldcg(state + head * 8 + 6)) : edge_of_bin(__ldcg(state + head * 8 + state_word));
 #pragma unroll
   for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
     const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
@@ -414,7 +420,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
                    const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
                    Gate gate, const float* __restrict__ collect_scores, long long collect_stride, float* __restrict__ collect_score_out,
-                   int32_t* __restrict__ collect_idx_out) {
+                   int32_t* __restrict__ collect_idx_out, int cache_entries) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   if (!fathom_gate_open(gate, blockIdx.x)) return;
@@ -423,8 +429,8 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
   __shared__ uint32_t s_need, s_bucket, s_ntok;
   extern __shared__ __align__(16) unsigned char s_dyn[];      // composite cache; DIRECT: + range counters, chosen tokens, tokens by range
-  uint64_t* s_comp = reinterpret_cast<uint64_t*>(s_dyn);                        // [FIN_CACHE]
-  uint32_t* s_range = reinterpret_cast<uint32_t*>(s_comp + FIN_CACHE);          // [SORT_BUCKETS]
+  uint64_t* s_comp = reinterpret_cast<uint64_t*>(s_dyn);                        // [cache_entries]
+  uint32_t* s_range = reinterpret_cast<uint32_t*>(s_comp + cache_entries);      // [SORT_BUCKETS]
   int32_t* s_tok = reinterpret_cast<int32_t*>(s_range + SORT_BUCKETS);          // [k]
   int32_t* s_sorted = s_tok + k;                                                // [k]
   const int head = blockIdx.x, tid = threadIdx.x;
@@ -442,8 +448,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   if (own_list) {
     if (tid == 0) s_collected = 0u;
     __syncthreads();
-    const uint32_t bstar = state[head * 8 + 3];
-    const float lo = bstar >= FATHOM_TOPK_BINS ? __uint_as_float(0x7fc00000u) : (bstar <= 7u ? -INFINITY : key_to_float(bstar << 20));
+    const float lo = edge_of_bin(state[head * 8 + 3]);
     const float* srow = collect_scores + (size_t)head * (size_t)collect_stride;
     float* cs = collect_score_out + (size_t)head * (size_t)cand_capacity;
     int32_t* ci = collect_idx_out + (size_t)head * (size_t)cand_capacity;
@@ -487,7 +492,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   // The working set is either all m candidates in global memory or a subset kept in shared memory: everything when
   // m fits, otherwise the bucket of the first digit once it fits (what ranks above that bucket is taken at once).
   __shared__ uint32_t s_ncache;
-  bool cached = m <= FIN_CACHE;
+  bool cached = m <= (uint32_t)cache_entries;
   uint32_t mc = m;                                            // size of the working set
   // Called by all 32 lanes of a warp together; `take` says whether this lane's composite is chosen.
   auto mark = [&](bool take, uint64_t comp) {                 // the token sits in the low 32 bits of every composite
@@ -581,7 +586,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       __syncthreads();
       hi = lo;
       if (s_need == s_bucket) break;                          // the chosen bucket is taken entirely: done
-      if (!cached && s_bucket <= FIN_CACHE) {
+      if (!cached && s_bucket <= (uint32_t)cache_entries) {
         // the undecided bucket fits in shared memory: pull it in, take what ranks above it, go on from there
         const uint64_t pfx = s_prefix;
         for (uint32_t c0 = 0; c0 < mc; c0 += FIN_THREADS * 8) {
@@ -618,7 +623,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     if (DIRECT && cached) {
       // chosen tokens -> list: the warp counts its chosen candidates over all its rounds first and reserves their
       // places with ONE atomic (an atomic per round would serialise the rounds on its return value)
-      constexpr int ROUNDS = FIN_CACHE / FIN_THREADS;          // 8: a cached working set has at most that many rounds
+      constexpr int ROUNDS = FIN_CACHE_MAX / FIN_THREADS;      // 16: a cached working set has at most that many rounds
       uint32_t before = 0, mine = 0;                          // chosen by lower lanes / by this lane, over the rounds
       unsigned takes = 0;
 #pragma unroll
@@ -797,7 +802,13 @@ static int bucket_shift_for(long long n) {
 }
 
 static size_t select_cache_smem() { return (size_t)FIN_CACHE * 8; }
-static size_t direct_select_smem(int k) { return select_cache_smem() + (size_t)SORT_BUCKETS * 4 + (size_t)2 * k * 4; }
+// composite cache of the direct select: as many entries as k leaves room for in 216 KB, in steps of 1024, at most 16384
+static int direct_cache_entries(int k) {
+  long long room = (216LL * 1024 - (long long)SORT_BUCKETS * 4 - 2LL * k * 4) / 8;
+  room = room / 1024 * 1024;
+  return (int)(room > FIN_CACHE_MAX ? FIN_CACHE_MAX : (room < 1024 ? 1024 : room));
+}
+static size_t direct_select_smem(int k) { return (size_t)direct_cache_entries(k) * 8 + (size_t)SORT_BUCKETS * 4 + (size_t)2 * k * 4; }
 
 // The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
 // and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
@@ -808,15 +819,14 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
                                 int32_t* idx, int gate_mode, cudaStream_t st, const float* scores = nullptr, long long score_stride = 0) {
   static bool attr_set[64] = {};
   if (ctx->device >= 0 && ctx->device < 64 && !attr_set[ctx->device]) {
-    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)direct_select_smem(FATHOM_MAX_K)));
+    FATHOM_CUDA_TRY(ctx, cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
     attr_set[ctx->device] = true;
   }
   Gate g = {S.cand_count, want, Hq, gate_mode};
   topk_select_kernel<true><<<Hq, FIN_THREADS, direct_select_smem(k), st>>>(
       S.cand_score, n, 0, F, S.state, S.cand, nullptr, 0, k, idx, ctx->dev_status, nullptr, 0,
       gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g, gate_mode >= 4 ? scores : nullptr,
-      score_stride, S.cand_score, S.cand);
+      score_stride, S.cand_score, S.cand, direct_cache_entries(k));
   return FATHOM_OK;
 }
 
@@ -849,7 +859,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     }
     topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
                                                                             S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
-                                                                            ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr);
+                                                                            ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr, FIN_CACHE);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
@@ -991,7 +1001,8 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   // ---- full scan that keeps only the tokens reaching their head's threshold, then the exact selection among them
   fathom_scan_fuse fz = {};
   fz.tile_step = 1;
-  fz.state = S.state;
+  fz.state = S.state + 6;                                     // the (refined) score threshold of the first attempt
+  fz.state_is_score = 1;
   fz.sink_end = F.sink_end;
   fz.local_begin = F.local_begin;
   fz.cand_score = S.cand_score;
@@ -1005,6 +1016,7 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   if (rc != FATHOM_OK) return rc;
   if (two_attempts) {                                         // stands by: runs only if some head's estimate was too high
     fz.state = S.state + 3;
+    fz.state_is_score = 0;
     fz.cand_count = S.cand_count2;
     fz.gate = fathom_gate{S.cand_count, want, Hq, 2};
     rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
