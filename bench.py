@@ -64,6 +64,7 @@ def parse_args():
                     help="the budget sweep at n = 1M (water-filled budgets and fixed top-r channels) instead of the default step")
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--lanes", type=int, default=4, help="config 4: stream lanes over which the sessions are spread")
+    ap.add_argument("--no-batch", action="store_true", help="config 4: one fathom_scan per session instead of fathom_scan_batch")
     return ap.parse_args()
 
 
@@ -564,7 +565,7 @@ def run_config4(args):
                      "hs": torch.empty((Hkv, d, lay.scale_stride), dtype=torch.int16, pin_memory=True),
                      "Kr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, device=dev),
                      "Vr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, device=dev),
-                     "q": None, "var": None})
+                     "depth": torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev), "q": None, "var": None})
     planes = torch.empty((Hkv, d, 4, lay_max.plane_stride_words), dtype=torch.int64, device=dev)
     scales = torch.empty((Hkv, d, lay_max.scale_stride), dtype=torch.int16, device=dev)
     layer_ms, bytes_link = [], 0.0
@@ -588,13 +589,36 @@ def run_config4(args):
             fork.record(stream)
             for W in lanes[1:]:
                 W["stream"].wait_event(fork)
-            for s_i, S in enumerate(sess):
-                W = lanes[s_i % len(lanes)]
-                lay, st, c = S["lay"], W["stream"], W["ctx"]
-                c.fathom_alloc_depth(lay, S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, W["depth"], st)
-                c.fathom_scan(lay, S["hp"], S["hs"], S["q"], W["depth"], hpp, W["scores"], st)
-                c.fathom_topk(lay, W["scores"], k, 0, 0, W["idx"], st)
-                c.fathom_sparse_attend(lay, S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
+            if args.no_batch:
+                for s_i, S in enumerate(sess):
+                    W = lanes[s_i % len(lanes)]
+                    lay, st, c = S["lay"], W["stream"], W["ctx"]
+                    c.fathom_alloc_depth(lay, S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, W["depth"], st)
+                    c.fathom_scan(lay, S["hp"], S["hs"], S["q"], W["depth"], hpp, W["scores"], st)
+                    c.fathom_topk(lay, W["scores"], k, 0, 0, W["idx"], st)
+                    c.fathom_sparse_attend(lay, S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
+            else:
+                # the sessions in groups of len(lanes): one batched scan per group on the first lane keeps the host link
+                # busy, then each session's top-k and attention run on its own lane while the next group is scanned
+                nl = len(lanes)
+                for g0 in range(0, len(sess), nl):
+                    grp = sess[g0:g0 + nl]
+                    if g0:                                       # the group's score buffers are free again?
+                        for W in lanes[1:]:
+                            e = torch.cuda.Event(); e.record(W["stream"]); stream.wait_event(e)
+                    items = []
+                    for j, S in enumerate(grp):
+                        W = lanes[j]
+                        ctx.fathom_alloc_depth(S["lay"], S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, S["depth"], stream)
+                        items.append((S["lay"], S["hp"], S["hs"], S["q"], S["depth"], W["scores"]))
+                    ctx.fathom_scan_batch(items, hpp, stream)
+                    done = torch.cuda.Event(); done.record(stream)
+                    for j, S in enumerate(grp):
+                        W = lanes[j]
+                        st, c = W["stream"], W["ctx"]
+                        st.wait_event(done)
+                        c.fathom_topk(S["lay"], W["scores"], k, 0, 0, W["idx"], st)
+                        c.fathom_sparse_attend(S["lay"], S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
             for W in lanes[1:]:
                 join = torch.cuda.Event()
                 join.record(W["stream"])
@@ -621,7 +645,8 @@ def run_config4(args):
         "dtype": "u64 bit planes + f32 accumulate", "data": "synthetic",
         "config": {"workload": "agentic multi-session batch (config 4): 16 sessions, planes in pinned host memory",
                    "session_tokens": lengths, "total_tokens": total_tokens, "kv_heads": Hkv, "q_heads": Hq, "budget_bits": B,
-                   "k": k, "layers_measured": args.layers, "layers_of_the_model": 36, "stream_lanes": len(lanes)},
+                   "k": k, "layers_measured": args.layers, "layers_of_the_model": 36, "stream_lanes": len(lanes),
+                   "scan": "one fathom_scan per session" if args.no_batch else "fathom_scan_batch per group of sessions"},
         "bytes_over_link_per_layer": bytes_link, "host_link_gbs": round(bytes_link / (ms * 1e-3) / 1e9, 2),
         "device_status": status}))
     for W in lanes:

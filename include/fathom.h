@@ -130,6 +130,22 @@ int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* pl
                 const uint16_t* scales, const float* q, const uint8_t* depth, int heads_per_plan,
                 float* scores, void* stream);
 
+/* ---- (3b) the scans of several sessions in one launch — Sec. 4 "Offload harness" (many concurrent sessions) ------
+ * Equivalent to one fathom_scan per item (same arguments, bit-identical scores), but all items' tiles form one grid,
+ * so that short sessions do not each pay a launch, a ramp-up and a tail - which is what keeps a host link busy when
+ * the planes live in pinned host memory.  Every item has its own layout (its n and strides); all items must have
+ * the same n_kv_heads and n_q_heads.  items is a HOST array (read during the call); the pointers inside follow the
+ * rules of fathom_scan. */
+typedef struct fathom_scan_item {
+  fathom_layout layout;
+  const uint64_t* planes;
+  const uint16_t* scales;
+  const float* q;
+  const uint8_t* depth;
+  float* scores;
+} fathom_scan_item;
+int fathom_scan_batch(fathom_ctx* ctx, const fathom_scan_item* items, int n_items, int heads_per_plan, void* stream);
+
 /* ---- (4) top-k — Sec. 2 "Top-k decoding" ---------------------------------------------------
  * Per query head: the first n_sink and the last n_local tokens are always selected; the remaining
  * k - |forced| are the tokens with the highest scores among the others, ties to the lower token

@@ -23,7 +23,7 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
-           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated"]
+           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated", "fathom_scan_batch"]
 
 
 class Layout(C.Structure):
@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
     lib.fathom_channel_variance.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
     lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
+    lib.fathom_scan_batch.argtypes = [vp, vp, i32, i32, vp]
     lib.fathom_build_planes_rotated.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -77,6 +78,11 @@ def _load() -> C.CDLL:
 
 
 lib = _load()
+
+
+class ScanItem(C.Structure):
+    _fields_ = [("layout", Layout), ("planes", C.c_void_p), ("scales", C.c_void_p), ("q", C.c_void_p),
+                ("depth", C.c_void_p), ("scores", C.c_void_p)]
 
 
 class FathomError(RuntimeError):
@@ -149,6 +155,15 @@ class Context:
     def fathom_scan(self, layout, planes, scales, q, depth, heads_per_plan, scores, stream=None):
         self._check(lib.fathom_scan(self._h, C.byref(layout), _ptr(planes), _ptr(scales), _ptr(q), _ptr(depth),
                                     heads_per_plan, _ptr(scores), _stream(stream)))
+
+    def fathom_scan_batch(self, items, heads_per_plan, stream=None):
+        """items: sequence of (layout, planes, scales, q, depth, scores)."""
+        arr = (ScanItem * len(items))()
+        for i, (lay, planes, scales, q, depth, scores) in enumerate(items):
+            arr[i].layout = lay
+            arr[i].planes, arr[i].scales, arr[i].q = _ptr(planes), _ptr(scales), _ptr(q)
+            arr[i].depth, arr[i].scores = _ptr(depth), _ptr(scores)
+        self._check(lib.fathom_scan_batch(self._h, arr, len(items), heads_per_plan, _stream(stream)))
 
     def fathom_topk(self, layout, scores, k, n_sink, n_local, idx, stream=None):
         self._check(lib.fathom_topk(self._h, C.byref(layout), _ptr(scores), k, n_sink, n_local, _ptr(idx), _stream(stream)))

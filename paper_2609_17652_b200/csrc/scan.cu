@@ -79,12 +79,13 @@ struct alignas(16) WarpSmem {
 //         token positions 1024 i ..) - the sample from which fathom_scan_topk derives a safe threshold.
 // MODE 2: every tile is scanned, nothing is written but the tokens whose score reaches the head's threshold:
 //         (score, token) pairs appended to the head's candidate list.
+// bx: the CTA's tile (of the launch, or of its item in a batched launch); by: its group of NH query heads
 template <int NH, int MODE>
-__global__ void __launch_bounds__(SCAN_THREADS, 8)              // 64 registers: occupancy matters more than spills here
-scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
-            const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
-            long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
-            int G, int heads_per_plan, fathom_scan_fuse fz) {
+__device__ __forceinline__ void
+scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
+          const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
+          long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
+          int G, int heads_per_plan, const fathom_scan_fuse& fz, const long long bx, const int by) {
   using C = ScanCfg<NH>;
   constexpr int HP = C::HP, EB = C::EB, TSTRIDE = C::TSTRIDE;
   __shared__ uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];      // channel of active row r
@@ -100,7 +101,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
 
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
+  const int h0 = by * NH;                                      // first of the NH query heads of this CTA
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
   const int kv = h0 / G;
 
@@ -128,7 +129,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
   const int nrows = s_nrows;
 
   WarpSmem<NH>& S = s_warp[warp];
-  const long long blk0 = (long long)blockIdx.x * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;  // first block of this CTA
+  const long long blk0 = bx * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;  // first block of this CTA
   const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
   const int wb0 = warp * WB;                                   // first block of this warp within the tile
   const int nblk = max(0, min(WB, nblk_cta - wb0));
@@ -279,7 +280,7 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
     for (int b = 0; b < WB; ++b) {
       if (b < nblk) {
         const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;                       // token scanned
-        const long long dst = MODE == 1 ? tok - blk0 * FATHOM_BLOCK + (long long)blockIdx.x * (TILE_BLOCKS * FATHOM_BLOCK) : tok;
+        const long long dst = MODE == 1 ? tok - blk0 * FATHOM_BLOCK + bx * (TILE_BLOCKS * FATHOM_BLOCK) : tok;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
           float* row = scores + (size_t)(h0 + h) * (size_t)score_stride;
@@ -362,6 +363,41 @@ scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ sc
 }
 
 template <int NH, int MODE>
+__global__ void __launch_bounds__(SCAN_THREADS, 8)              // 64 registers: occupancy matters more than spills here
+scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
+            const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
+            long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
+            int G, int heads_per_plan, fathom_scan_fuse fz) {
+  scan_body<NH, MODE>(planes, scales, q, depth, scores, n, nb, plane_stride, scale_stride, score_stride, G, heads_per_plan, fz,
+                      (long long)blockIdx.x, (int)blockIdx.y);
+}
+
+// ---- several sessions in one launch (fathom_scan_batch): the items' tiles are laid end to end along grid.x
+struct ScanBatch {
+  static constexpr int MAX_ITEMS = 32;
+  const uint64_t* planes[MAX_ITEMS];
+  const uint16_t* scales[MAX_ITEMS];
+  const float* q[MAX_ITEMS];
+  const uint8_t* depth[MAX_ITEMS];
+  float* scores[MAX_ITEMS];
+  long long n[MAX_ITEMS], plane_stride[MAX_ITEMS], scale_stride[MAX_ITEMS], score_stride[MAX_ITEMS];
+  long long tile_end[MAX_ITEMS];                              // tiles of items 0 .. i, inclusive prefix
+  int items;
+};
+
+template <int NH>
+__global__ void __launch_bounds__(SCAN_THREADS, 8)
+scan_batch_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan) {
+  int it = 0;
+  while (it + 1 < B.items && (long long)blockIdx.x >= B.tile_end[it]) ++it;      // uniform over the CTA, at most 31 steps
+  const long long bx = (long long)blockIdx.x - (it ? B.tile_end[it - 1] : 0);
+  fathom_scan_fuse fz = {};
+  fz.tile_step = 1;
+  scan_body<NH, 0>(B.planes[it], B.scales[it], B.q[it], B.depth[it], B.scores[it], B.n[it], (B.n[it] + FATHOM_BLOCK - 1) / FATHOM_BLOCK, B.plane_stride[it],
+                   B.scale_stride[it], B.score_stride[it], G, heads_per_plan, fz, bx, (int)blockIdx.y);
+}
+
+template <int NH, int MODE>
 int launch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
                 const uint8_t* depth, int heads_per_plan, float* scores, long long score_stride,
                 const fathom_scan_fuse& fz, cudaStream_t st) {
@@ -417,6 +453,45 @@ extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64
   fz.tile_step = 1;
   rc = dispatch_scan<0>(L, planes, scales, q, depth, heads_per_plan, scores, L->score_stride, fz, static_cast<cudaStream_t>(stream));
   if (rc != FATHOM_OK) return rc;
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+extern "C" int fathom_scan_batch(fathom_ctx* ctx, const fathom_scan_item* items, int n_items, int heads_per_plan, void* stream) {
+  if (!ctx || !items || n_items < 1) return FATHOM_ERR_INVALID_ARG;
+  const int Hkv = items[0].layout.n_kv_heads, Hq = items[0].layout.n_q_heads;
+  for (int i = 0; i < n_items; ++i) {
+    const fathom_scan_item& it = items[i];
+    int rc = fathom_check_layout(&it.layout);
+    if (rc != FATHOM_OK) return rc;
+    if (it.layout.n_kv_heads != Hkv || it.layout.n_q_heads != Hq) return FATHOM_ERR_INVALID_ARG;   // one model, many sessions
+    if (!it.planes || !it.scales || !it.q || !it.depth || !it.scores) return FATHOM_ERR_INVALID_ARG;
+    if (!fathom_aligned16(it.planes) || !fathom_aligned16(it.scales) || !fathom_aligned16(it.scores)) return FATHOM_ERR_ALIGNMENT;
+  }
+  const int G = Hq / Hkv;
+  if (heads_per_plan < 1 || G % heads_per_plan != 0) return FATHOM_ERR_INVALID_ARG;
+  if (heads_per_plan != 1 && heads_per_plan != 2 && heads_per_plan != 4 && heads_per_plan != 8) return FATHOM_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int first = 0; first < n_items; first += ScanBatch::MAX_ITEMS) {       // at most 32 sessions per launch
+    ScanBatch B = {};
+    B.items = n_items - first < ScanBatch::MAX_ITEMS ? n_items - first : ScanBatch::MAX_ITEMS;
+    long long tiles = 0;
+    for (int i = 0; i < B.items; ++i) {
+      const fathom_scan_item& it = items[first + i];
+      B.planes[i] = it.planes; B.scales[i] = it.scales; B.q[i] = it.q; B.depth[i] = it.depth; B.scores[i] = it.scores;
+      B.n[i] = it.layout.n; B.plane_stride[i] = it.layout.plane_stride_words; B.scale_stride[i] = it.layout.scale_stride;
+      B.score_stride[i] = it.layout.score_stride;
+      tiles += (fathom_nblocks(it.layout.n) + TILE_BLOCKS - 1) / TILE_BLOCKS;
+      B.tile_end[i] = tiles;
+    }
+    const int nh = heads_per_plan == 8 ? 4 : heads_per_plan;  // plans of eight heads are served by two CTAs of four
+    dim3 grid((unsigned)tiles, (unsigned)(Hq / nh));
+    switch (nh) {
+      case 1: scan_batch_kernel<1><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
+      case 2: scan_batch_kernel<2><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
+      default: scan_batch_kernel<4><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
+    }
+  }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

@@ -540,3 +540,41 @@ def test_rotated_store_in_one_call_equals_rotate_then_build(n, dtype):
     assert torch.all(s_one[1, 5, :nb] == 0) and torch.all(p_one[1, 5, 1:, :nb] == 0)
     assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("hpp,host", [(4, False), (1, False), (4, True)])
+def test_batched_scan_equals_one_scan_per_session(hpp, host):
+    """fathom_scan_batch over ragged sessions (lengths that are not multiples of 64 or of the 1024-token tile, one of
+    a single token) gives bit for bit the scores of one fathom_scan per session, with the planes in HBM or in pinned
+    host memory, and more sessions than one launch takes (33 > 32)."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq = 2, 8
+    lengths = [1, 63, 1000, 1024, 1025, 5000, 70001] + [300 + 37 * i for i in range(26)]
+    assert len(lengths) == 33
+    ctx = fb.Context(0, 1 << 20)
+    items, singles = [], []
+    for s_i, n in enumerate(lengths):
+        L = make_layer(max(n, 64), Hkv, Hq, seed=60, session=s_i, device="cuda")
+        K = L.K[:, :n].contiguous()
+        lay = fb.make_layout(Hkv, Hq, n)
+        planes = torch.zeros((Hkv, 128, 4, lay.plane_stride_words), dtype=torch.int64, device="cuda")
+        scales = torch.zeros((Hkv, 128, lay.scale_stride), dtype=torch.int16, device="cuda")
+        ctx.fathom_build_planes(lay, K, planes, scales)
+        depth = torch.zeros((Hq // hpp, 128), dtype=torch.uint8, device="cuda")
+        ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, 48, hpp, depth)
+        if host:
+            hp = torch.empty(planes.shape, dtype=planes.dtype, pin_memory=True); hp.copy_(planes)
+            hs = torch.empty(scales.shape, dtype=scales.dtype, pin_memory=True); hs.copy_(scales)
+            planes, scales = hp, hs
+        one = torch.full((Hq, lay.score_stride), float("nan"), device="cuda")
+        ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, one)
+        many = torch.full((Hq, lay.score_stride), float("nan"), device="cuda")
+        items.append((lay, planes, scales, L.q, depth, many))
+        singles.append((one, n))
+    ctx.fathom_scan_batch(items, hpp)
+    torch.cuda.synchronize()
+    for (lay, _, _, _, _, many), (one, n) in zip(items, singles):
+        assert torch.equal(many[:, :n], one[:, :n])
+        assert torch.isnan(many[:, n:]).all()                                # padding untouched
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
