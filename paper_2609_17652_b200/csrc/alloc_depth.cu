@@ -19,6 +19,8 @@ __global__ void __launch_bounds__(AD_THREADS)
 alloc_depth_kernel(const float* __restrict__ q, const float* __restrict__ var, int mode, int budget,
                    int heads_per_plan, int G, uint8_t* __restrict__ depth) {
   __shared__ alignas(16) unsigned long long pri[NCAND];       // bit patterns of the (non-negative) priorities
+  FATHOM_PDL_WAIT();
+  FATHOM_PDL_RELEASE();                                       // the scan that follows may become resident now
   const int plan = blockIdx.x / CTAS_PER_PLAN, part = blockIdx.x % CTAS_PER_PLAN;
   const int tid = threadIdx.x;
   const int h0 = plan * heads_per_plan;

@@ -41,6 +41,28 @@ static inline int64_t fathom_nblocks(int64_t n) { return (n + FATHOM_BLOCK - 1) 
 static inline bool fathom_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t fathom_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// ---- programmatic dependent launch (sm_90+): a kernel launched with fathom_launch_dependent may become resident while
+// the previous kernel of the stream still runs (once every CTA of that kernel has passed FATHOM_PDL_RELEASE or exited) and
+// must execute FATHOM_PDL_WAIT before it touches anything the previous kernels wrote; the wait returns when they have
+// completed and their writes are visible.  Both are no-ops in a normally launched kernel, and a kernel that never
+// releases simply serialises.  Every kernel of the decode step waits at its top, so completion is transitive.
+#define FATHOM_PDL_WAIT() asm volatile("griddepcontrol.wait;" ::: "memory")
+#define FATHOM_PDL_RELEASE() asm volatile("griddepcontrol.launch_dependents;" ::: "memory")
+template <typename... P, typename... A>
+static inline cudaError_t fathom_launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
 // ---- pieces shared by scan.cu and topk.cu for the fused scan + selection (fathom_scan_topk) -------------------
 // A launch that belongs to one of two alternative continuations decides on the device whether it runs.  A first
 // attempt collects, per head, the tokens above an ESTIMATED threshold; it goes on only if every head collected at

@@ -99,6 +99,7 @@ scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scal
   __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
   __shared__ WarpSmem<NH> s_warp[SCAN_WARPS];
 
+  FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h0 = by * NH;                                      // first of the NH query heads of this CTA
@@ -405,6 +406,13 @@ int launch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* 
   const long long ntiles = (nb + TILE_BLOCKS - 1) / TILE_BLOCKS;
   const long long gx = MODE == 1 ? (ntiles + fz.tile_step - 1) / fz.tile_step : ntiles;
   dim3 grid((unsigned)gx, (unsigned)(L->n_q_heads / NH));
+  if (MODE == 0) {                                            // may become resident while fathom_alloc_depth's kernel runs
+    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(SCAN_THREADS), 0, st, planes, scales, q, depth, scores, (long long)L->n,
+                                (long long)nb, (long long)L->plane_stride_words, (long long)L->scale_stride, score_stride,
+                                L->n_q_heads / L->n_kv_heads, heads_per_plan, fz) != cudaSuccess)
+      return FATHOM_ERR_CUDA;
+    return 0;
+  }
   scan_kernel<NH, MODE><<<grid, SCAN_THREADS, 0, st>>>(planes, scales, q, depth, scores, L->n, nb, L->plane_stride_words,
                                                        L->scale_stride, score_stride, L->n_q_heads / L->n_kv_heads,
                                                        heads_per_plan, fz);

@@ -95,6 +95,7 @@ attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, 
   __shared__ float s_acc[AT_THREADS / 16][FATHOM_D];          // one partial sum per half-warp
   const int split = blockIdx.x, head = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kv = head / G;
+  FATHOM_PDL_WAIT();                                          // the indices come from the previous kernel
   const T* Kh = Krows + (size_t)kv * (size_t)n * FATHOM_D;
   const T* Vh = Vrows + (size_t)kv * (size_t)n * FATHOM_D;
   s_q[tid] = q[(size_t)head * FATHOM_D + tid];
@@ -216,14 +217,15 @@ extern "C" int fathom_sparse_attend(fathom_ctx* ctx, const fathom_layout* L, con
   unsigned int* tickets = ctx->dev_status + FATHOM_CTL_TICKETS;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid((unsigned)S.splits, (unsigned)Hq);
+  // launched so that its CTAs may become resident while the selection kernel (one CTA per head) still runs
   if (row_dtype == FATHOM_BF16)
-    attend_partial_kernel<__nv_bfloat16><<<grid, AT_THREADS, 0, st>>>(
-        q, static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k, L->n, G,
-        softmax_scale, S.partial, S.splits, tickets, out);
+    FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(attend_partial_kernel<__nv_bfloat16>, grid, dim3(AT_THREADS), 0, st, q,
+                                                 static_cast<const __nv_bfloat16*>(Krows), static_cast<const __nv_bfloat16*>(Vrows), idx, k,
+                                                 (long long)L->n, G, softmax_scale, S.partial, S.splits, tickets, out));
   else
-    attend_partial_kernel<float><<<grid, AT_THREADS, 0, st>>>(q, static_cast<const float*>(Krows),
-                                                              static_cast<const float*>(Vrows), idx, k, L->n, G,
-                                                              softmax_scale, S.partial, S.splits, tickets, out);
+    FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(attend_partial_kernel<float>, grid, dim3(AT_THREADS), 0, st, q,
+                                                 static_cast<const float*>(Krows), static_cast<const float*>(Vrows), idx, k,
+                                                 (long long)L->n, G, softmax_scale, S.partial, S.splits, tickets, out));
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

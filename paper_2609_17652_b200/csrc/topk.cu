@@ -339,7 +339,8 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   }
   // The scores were complete before the sample kernel started; its threshold and cleared counters are needed from
   // here on (a no-op unless this kernel was launched as a programmatic dependent of the sample kernel).
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  FATHOM_PDL_WAIT();
+  FATHOM_PDL_RELEASE();                                       // the selection that follows may become resident now
   __syncthreads();
   // the score a candidate must reach: word 6 (first attempt: estimated, refined) or the lower edge of the bin in state_word
   const float lo = state_word == 0 ? __uint_as_float(__ldcg(state + head * 8 + 6)) : edge_of_bin(__ldcg(state + head * 8 + state_word));
@@ -423,6 +424,8 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    int32_t* __restrict__ collect_idx_out, int cache_entries) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
+  FATHOM_PDL_WAIT();                                          // the candidates come from the previous kernel
+  FATHOM_PDL_RELEASE();                                       // the attention that follows may become resident now
   if (!fathom_gate_open(gate, blockIdx.x)) return;
   __shared__ uint32_t s_hist[DIGITS];
   __shared__ uint32_t s_warp[33];
@@ -823,10 +826,11 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
     attr_set[ctx->device] = true;
   }
   Gate g = {S.cand_count, want, Hq, gate_mode};
-  topk_select_kernel<true><<<Hq, FIN_THREADS, direct_select_smem(k), st>>>(
-      S.cand_score, n, 0, F, S.state, S.cand, nullptr, 0, k, idx, ctx->dev_status, nullptr, 0,
-      gate_mode == 2 ? S.cand_count2 : S.cand_count, n, want, bucket_shift_for(n), g, gate_mode >= 4 ? scores : nullptr,
-      score_stride, S.cand_score, S.cand, direct_cache_entries(k));
+  FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(
+      topk_select_kernel<true>, dim3(Hq), dim3(FIN_THREADS), direct_select_smem(k), st, (const float*)S.cand_score, n, 0LL, F,
+      (const uint32_t*)S.state, (const int32_t*)S.cand, (uint32_t*)nullptr, 0LL, k, idx, ctx->dev_status, (uint32_t*)nullptr, 0,
+      (const uint32_t*)(gate_mode == 2 ? S.cand_count2 : S.cand_count), n, want, bucket_shift_for(n), g,
+      (const float*)(gate_mode >= 4 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k)));
   return FATHOM_OK;
 }
 
