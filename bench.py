@@ -38,8 +38,12 @@ WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3
 # dram__bytes_read.sum + dram__bytes_write.sum per unit (one token of one KV head) from the ncu captures
 # summarised under profiles/: build at n = 131072 (596.1 MB / 1,048,576 units; traffic is proportional to
 # units), scan at n = 1,048,576 and B = 48 (136.9 MB / 8,388,608 units; part of the score writes is still in
-# L2 when the kernel ends).  Multiplied by the units of a launch in the JSON line.
-NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.3}
+# L2 when the kernel ends), the three top-k kernels at n = 1,048,576, k = 4096 (8.4 + 134.25 + 1.7 MB read, 0.5 MB
+# written / 8,388,608 units; valid for the single-pass path only), attention at k = 4096 (66.1 MB read + 1.05 MB
+# written; proportional to k, not to n: 67.1 MB / (32 heads x 4096 rows) = 512.3 B per selected row).
+# Multiplied by the units of a launch in the JSON line.
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.3, "topk_*": 17.3}
+NCU_TRAFFIC_BYTES_PER_SELECTED_ROW = 512.3
 
 
 def parse_args():
@@ -235,7 +239,9 @@ def run_ours(args):
         ach = alg_bytes[stage_key] / (t_us * 1e-6) / 1e9
         tr = NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD.get(kernel)
         return {"kernel": kernel, "bound": "hbm", "achieved": round(ach, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(ach / peak, 4), "traffic": (tr * unit_count if tr else None),
+                "frac": round(ach / peak, 4),
+                "traffic": (NCU_TRAFFIC_BYTES_PER_SELECTED_ROW * Hq * k if kernel == "attend_*" else
+                            (tr * unit_count if tr and not (kernel == "topk_*" and topk_passes != 1) else None)),
                 "algorithmic_bytes": alg_bytes[stage_key], "launch_us": round(t_us, 2), "peak_source": peak_src}
 
     # ---- isolated stage timings with an L2 flush before every launch (cold-cache view of each stage)
