@@ -93,3 +93,27 @@ def test_layer_budget_plan_host_function_matches_the_oracle(fb):
     assert fb.lib.fathom_plan_layer_budgets(None, 1, 1, None, C.c_double(1.0), None) == -1
     bad = (C.c_int * 2)(32, 32); e = (C.c_double * 2)(1.0, 0.5); out = (C.c_int * 1)()
     assert fb.lib.fathom_plan_layer_budgets(e, 1, 2, bad, C.c_double(40.0), out) == -1
+
+
+def test_topk_pass_plan_and_rejections_of_the_newer_entry_points(fb):
+    """Host logic only: which rows fathom_topk reads once, and NULL / inconsistent arguments of the entry points
+    beyond the five calls are refused before any launch."""
+    lay = fb.make_layout(8, 32, 1 << 20)
+    assert fb.fathom_topk_passes(lay, 4096) == 1 and fb.fathom_topk_passes(lay, 4096, 4, 32) == 1
+    assert fb.fathom_topk_passes(lay, 64) == 2                       # too few winners to estimate from a sample
+    assert fb.fathom_topk_passes(fb.make_layout(8, 32, 40000), 2048) == 2     # too short to sample
+    assert fb.fathom_topk_passes(fb.make_layout(8, 32, 131072), 2048) == 1
+    assert fb.lib.fathom_topk_passes(C.byref(lay), 0, 0, 0) < 0 and fb.lib.fathom_topk_passes(C.byref(lay), 10, 8, 8) < 0
+    for call, nargs in (("fathom_scan_topk", 12), ("fathom_gather_union", 12), ("fathom_calibrate", 7), ("fathom_rotate_keys", 8),
+                        ("fathom_rotate_query", 6), ("fathom_channel_variance", 7), ("fathom_build_planes_rotated", 9)):
+        fn = getattr(fb.lib, call)
+        args = [None, C.byref(lay)] + [16] * (nargs - 2)
+        if call in ("fathom_calibrate", "fathom_rotate_keys", "fathom_channel_variance", "fathom_build_planes_rotated"):
+            args[3] = 0                                              # k_dtype
+        if call == "fathom_scan_topk":
+            args[6:10] = [4, 10, 0, 0]
+        if call == "fathom_gather_union":
+            args[3] = 10; args[6] = 1
+        args[-1] = None                                              # stream
+        assert fn(*args) == -1, call                                 # FATHOM_ERR_INVALID_ARG: NULL context
+    assert fb.lib.fathom_scan_batch(None, None, 1, 4, None) == -1
