@@ -218,7 +218,7 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
  * the rest of the path is used as is: build planes from K_rot, pass q_rot to fathom_alloc_depth (with the
  * eigenvalues as `var`) and to fathom_scan, and run attention on the original rows.
  *   fathom_calibrate:    mean [Hkv][d] and unbiased covariance cov [Hkv][d][d] (fp32) of the session's own keys in ONE
- *                        read of the keys: the keys are centred on a shift (the mean of the head's first 64 keys),
+ *                        read of the keys: the keys are centred on a shift (the mean of 64 keys spread over the sequence),
  *                        sum (x - shift)(x - shift)^T is accumulated on the tensor cores (tf32 operands split in head
  *                        and tail, fp32 accumulation per CTA) together with the per-channel sums S, and a reduction
  *                        in fp64 gives mean = shift + S / n, cov = (sum - S S^T / n) / (n - 1); fixed order throughout.

@@ -530,19 +530,21 @@ __device__ __forceinline__ void umma_tf32_mn(uint32_t tmem_d, uint64_t a, uint64
       :: "r"(tmem_d), "l"(a), "l"(b), "r"(UMMA_IDESC_MN), "r"(accumulate), "r"(0u) : "memory");
 }
 
-// shift[kv][c] = mean of channel c over the head's first min(n, 64) keys (any value near the data would do; it only
-// has to keep S S^T / n small against the sum of squares)
+// shift[kv][c] = mean of channel c over 64 keys spread evenly over the head's sequence (any value near the data would
+// do; it only has to keep S S^T / n small against the sum of squares - keys from one place, e.g. the first tokens of a
+// prompt, may sit far from the rest)
 template <typename T>
 __global__ void __launch_bounds__(FATHOM_D)
 cov_shift_kernel(const T* __restrict__ K, long long n, float* __restrict__ shift) {
   const int kv = blockIdx.x, c = threadIdx.x;
   const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D;
   const int rows = (int)min((long long)64, n);
+  const long long step = n / rows;                            // >= 1
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   for (int r = 0; r < rows; r += 8)
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-      if (r + u < rows) acc[u] += (float)Kh[(size_t)(r + u) * FATHOM_D + c];
+      if (r + u < rows) acc[u] += (float)Kh[(size_t)((r + u) * step) * FATHOM_D + c];
   shift[(size_t)kv * FATHOM_D + c] = (((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]))) / (float)rows;
 }
 

@@ -578,3 +578,25 @@ def test_batched_scan_equals_one_scan_per_session(hpp, host):
         assert torch.isnan(many[:, n:]).all()                                # padding untouched
     assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+def test_single_pass_calibration_with_drifting_and_outlying_keys():
+    """The one-read covariance centres the keys on a shift taken from 64 keys spread over the sequence.  Keys whose mean
+    drifts along the sequence, with a few far-off keys at the start (as the first tokens of a prompt often are), must
+    still give the oracle's mean and covariance: nothing may cancel."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq, n = 2, 4, 30000
+    g = torch.Generator(device="cuda"); g.manual_seed(99)
+    K = torch.randn(Hkv, n, 128, device="cuda", generator=g)
+    K += torch.linspace(-4.0, 6.0, n, device="cuda")[None, :, None] * torch.rand(Hkv, 1, 128, device="cuda", generator=g)   # drift
+    K[:, :4] += 80.0                                                              # outlying first keys
+    K = K.contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, 1))
+    mean = torch.zeros((Hkv, 128), device="cuda"); cov = torch.zeros((Hkv, 128, 128), device="cuda")
+    ctx.fathom_calibrate(lay, K, mean, cov)
+    mu_ref, C_ref = O.calibrate(K.cpu().numpy())
+    assert np.allclose(mean.cpu().numpy(), mu_ref, rtol=1e-5, atol=1e-5)
+    scale = np.abs(C_ref).max(axis=(1, 2), keepdims=True)
+    assert np.all(np.abs(cov.cpu().numpy() - C_ref) <= 2e-5 * scale)
+    ctx.close()
