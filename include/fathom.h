@@ -249,7 +249,7 @@ int fathom_build_planes_rotated(fathom_ctx* ctx, const fathom_layout* layout, co
 /* ---- (8) per-channel key statistics — Sec. 3.3 (the Var(k_j) of g_j), Appendix B5 (from the session's own keys)
  * mean [Hkv][d] and var [Hkv][d] (device, fp32): mean and unbiased (n - 1) sample variance of every channel of
  * K [Hkv][n][d] (device, FATHOM_F32 or FATHOM_BF16, 16-byte aligned).  One pass over the keys; per 1024-token
- * tile fp32 sums of the keys shifted by the tile's first key, merged across tiles in fp64 in tile order
+ * tile fp32 sums of the keys shifted by the tile's middle key, merged across tiles in fp64 in tile order
  * (deterministic).  var feeds fathom_alloc_depth for the raw store.  n = 1 gives var = 0.  Uses the context scratch
  * (FATHOM_ERR_SCRATCH_TOO_SMALL if the context was created for a smaller layout). */
 int fathom_channel_variance(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype, float* mean,

@@ -160,7 +160,7 @@ cov_final_kernel(const float* __restrict__ partial, int tiles, long long n, floa
 
 // ---- per-channel mean and variance (the Var(k_j) of the importance g_j) -----------------------------------------
 // One pass over the keys.  A CTA takes MEAN_ROWS tokens of one KV head and, per channel, the sums of (x - s) and
-// (x - s)^2 with s the tile's first key (a shift inside the data keeps the squares free of cancellation); the
+// (x - s)^2 with s the tile's middle key (a shift inside the data keeps the squares free of cancellation); the
 // final kernel merges the tiles in fp64 in tile order: mean_t = s + S1/n_t, M2_t = S2 - S1^2/n_t,
 // M2 = sum M2_t + sum n_t (mean_t - mean)^2.
 __device__ __forceinline__ float4 load4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
@@ -178,7 +178,7 @@ var_partial_kernel(const T* __restrict__ K, long long n, float* __restrict__ par
   const long long r0 = (long long)blockIdx.x * MEAN_ROWS;
   const long long r1 = min(r0 + MEAN_ROWS, n);
   const T* Kh = K + (size_t)kv * (size_t)n * FATHOM_D + 4 * cq;
-  const float4 sh = load4(Kh + (size_t)r0 * FATHOM_D);
+  const float4 sh = load4(Kh + (size_t)(r0 + (r1 - r0) / 2) * FATHOM_D);   // the tile's middle key (a prompt's first keys may be far off)
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
 #pragma unroll 8
   for (long long r = r0 + rl; r < r1; r += 8) {

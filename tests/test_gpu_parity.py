@@ -594,6 +594,11 @@ def test_single_pass_calibration_with_drifting_and_outlying_keys():
     lay = fb.make_layout(Hkv, Hq, n)
     ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, 1))
     mean = torch.zeros((Hkv, 128), device="cuda"); cov = torch.zeros((Hkv, 128, 128), device="cuda")
+    var = torch.zeros((Hkv, 128), device="cuda")
+    ctx.fathom_channel_variance(lay, K, mean, var)
+    mu_v, var_ref = O.channel_variance(K.cpu().numpy())
+    assert np.all(np.abs(mean.cpu().numpy() - mu_v) <= 1e-6 * np.abs(mu_v) + 1e-5 * np.sqrt(var_ref))
+    assert np.all(np.abs(var.cpu().numpy() - var_ref) <= 1e-5 * var_ref)
     ctx.fathom_calibrate(lay, K, mean, cov)
     mu_ref, C_ref = O.calibrate(K.cpu().numpy())
     assert np.allclose(mean.cpu().numpy(), mu_ref, rtol=1e-5, atol=1e-5)
