@@ -73,16 +73,11 @@ struct fathom_gate {
   uint32_t want;
   int heads;
   int mode;                     // 0: always run; 1: only if every head collected enough; 2: only if some head did not;
-                                // 3 / 4: the CTA's own head (given by the kernel) collected enough / did not;
                                 // 5: always run - the kernel itself looks at its head's count and picks its input
 };
-// Called by every thread of the CTA at the top of a gated kernel; `head` is used by the per-head modes only.
-__device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g, int head = 0) {
+// Called by every thread of the CTA at the top of a gated kernel.
+__device__ __forceinline__ bool fathom_gate_open(const fathom_gate& g) {
   if (g.mode == 0 || g.mode == 5) return true;
-  if (g.mode >= 3) {
-    const bool ok = __ldcg(g.counts + head) >= g.want;
-    return g.mode == 3 ? ok : !ok;
-  }
   bool ok = true;
   for (int h = threadIdx.x; h < g.heads; h += blockDim.x) ok = ok && (__ldcg(g.counts + h) >= g.want);
   const bool all_ok = __syncthreads_and(ok) != 0;

@@ -313,16 +313,15 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
   for (uint32_t e = threadIdx.x; e < cnt; e += FILT_THREADS) cand_h[base + e] = (int32_t)(tile0 + s_list[e]);
 }
 
-// Collection pass of the sampled paths: every eligible token whose score reaches the lower edge of the head's
-// threshold bin is appended to the head's candidate list as a (score, token) pair.  state_word 0: the bin estimated
-// from a histogram of every 16th chunk (first attempt); 3: the bin that is a bound (second attempt, gated).
+// Collection pass of the single-pass top-k: every eligible token whose score reaches the head's estimated threshold
+// (state word 6, from the histogram of every 16th chunk) is appended to the head's candidate list as a (score, token)
+// pair.
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
-                    const uint32_t* state, int state_word, float* __restrict__ cand_score,
-                    int32_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_count, Gate gate) {
+                    const uint32_t* state, float* __restrict__ cand_score, int32_t* __restrict__ cand_idx,
+                    uint32_t* __restrict__ cand_count) {
   __shared__ uint16_t s_list[FILT_TILE];
   __shared__ uint32_t s_count, s_base;
-  if (!fathom_gate_open(gate)) return;
   // heads and tiles are walked from the last to the first: what the scan wrote last is the likeliest to be in L2 still
   const int head = gridDim.y - 1 - blockIdx.y, tile = gridDim.x - 1 - blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -342,8 +341,7 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   FATHOM_PDL_WAIT();
   FATHOM_PDL_RELEASE();                                       // the selection that follows may become resident now
   __syncthreads();
-  // the score a candidate must reach: word 6 (first attempt: estimated, refined) or the lower edge of the bin in state_word
-  const float lo = state_word == 0 ? __uint_as_float(__ldcg(state + head * 8 + 6)) : edge_of_bin(__ldcg(state + head * 8 + state_word));
+  const float lo = __uint_as_float(__ldcg(state + head * 8 + 6));   // the score a candidate must reach
 #pragma unroll
   for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
     const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
@@ -426,7 +424,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   FATHOM_PDL_WAIT();                                          // the candidates come from the previous kernel
   FATHOM_PDL_RELEASE();                                       // the attention that follows may become resident now
-  if (!fathom_gate_open(gate, blockIdx.x)) return;
+  if (!fathom_gate_open(gate)) return;
   __shared__ uint32_t s_hist[DIGITS];
   __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
@@ -440,7 +438,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   // dense: scores row of the head, candidate tokens [n];  direct: candidate scores and tokens [cand_capacity]
   // (when the CTA collects its own candidates they are read back through the pointers they were written through)
   const bool own_list = DIRECT && collect_scores != nullptr &&
-                        (gate.mode != 5 || __ldcg(gate.counts + head) < gate.want);   // the same for every thread of the CTA
+                        (gate.mode == 5 && __ldcg(gate.counts + head) < gate.want);   // the same for every thread of the CTA
   const float* row = (own_list ? collect_score_out : scores) + (size_t)head * (size_t)(DIRECT ? cand_capacity : score_stride);
   const int32_t* cand_h = (own_list ? collect_idx_out : cand) + (size_t)head * (size_t)(DIRECT ? cand_capacity : n);
   uint32_t* bm = DIRECT ? nullptr : bitmap + (size_t)head * (size_t)bitmap_words;
@@ -830,7 +828,7 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
       topk_select_kernel<true>, dim3(Hq), dim3(FIN_THREADS), direct_select_smem(k), st, (const float*)S.cand_score, n, 0LL, F,
       (const uint32_t*)S.state, (const int32_t*)S.cand, (uint32_t*)nullptr, 0LL, k, idx, ctx->dev_status, (uint32_t*)nullptr, 0,
       (const uint32_t*)(gate_mode == 2 ? S.cand_count2 : S.cand_count), n, want, bucket_shift_for(n), g,
-      (const float*)(gate_mode >= 4 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k)));
+      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k)));
   return FATHOM_OK;
 }
 
@@ -890,11 +888,10 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       attr[0].val.programmaticStreamSerializationAllowed = 1;
       cfg.attrs = attr;
       cfg.numAttrs = 1;
-      FATHOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, topk_collect_kernel, scores, n, score_stride, F, (const uint32_t*)S.state, 0,
-                                              S.cand_score, S.cand, S.cand_count, always));
+      FATHOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, topk_collect_kernel, scores, n, score_stride, F, (const uint32_t*)S.state,
+                                              S.cand_score, S.cand, S.cand_count));
     } else {
-      topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, 0, S.cand_score, S.cand, S.cand_count,
-                                                          always);
+      topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand_score, S.cand, S.cand_count);
     }
     // one launch serves both outcomes: a head whose estimate was low enough selects among its collected candidates; a
     // head that fell short collects above the bound bin itself (one CTA streaming its row) and selects among those
