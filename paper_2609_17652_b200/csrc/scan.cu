@@ -66,6 +66,9 @@ __device__ __forceinline__ float bin_lower_edge(uint32_t bin) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
+// first fp16 of staged row r in the padded scale array
+__device__ __forceinline__ int scale_offset(int r) { return r * TILE_BLOCKS + (r >> 2) * 8; }
+
 template <int NH>
 struct alignas(16) WarpSmem {
   using C = ScanCfg<NH>;
@@ -94,8 +97,11 @@ scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scal
   __shared__ int warp_tot[4];
   __shared__ float s_q[NH][FATHOM_D];
   __shared__ float s_thr[NH];                                 // MODE 2: score a token must reach, per head
-  __shared__ alignas(16) uint64_t s_words[STAGE_ROWS][TILE_BLOCKS];   // staged plane words
-  __shared__ alignas(16) uint16_t s_scale[STAGE_ROWS][TILE_BLOCKS];   // staged fp16 scales
+  // Both staged arrays are read by lanes that differ in the group g = (row / 4) mod 4, and rows four apart would fall on
+  // the same banks: the plane words of row r sit at block column c ^ 4 g, and the scales of each group of four rows
+  // start 16 bytes further on.
+  __shared__ alignas(16) uint64_t s_words[STAGE_ROWS][TILE_BLOCKS];   // staged plane words (block columns swizzled)
+  __shared__ alignas(16) uint16_t s_scale[STAGE_ROWS * TILE_BLOCKS + (STAGE_ROWS / 4) * 8];   // staged fp16 scales (padded)
   __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
   __shared__ WarpSmem<NH> s_warp[SCAN_WARPS];
 
@@ -184,9 +190,10 @@ scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scal
 #pragma unroll
       for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
         const int e = tid + k * SCAN_THREADS;
-        *reinterpret_cast<uint4*>(&s_words[e >> 3][2 * (e & 7)]) = wv[k];
+        const int r = e >> 3;
+        *reinterpret_cast<uint4*>(&s_words[r][(2 * (e & 7)) ^ (((r >> 2) & 3) << 2)]) = wv[k];
       }
-      if (tid < STAGE_ROWS * 2) *reinterpret_cast<uint4*>(&s_scale[tid >> 1][8 * (tid & 1)]) = sv;
+      if (tid < STAGE_ROWS * 2) *reinterpret_cast<uint4*>(&s_scale[scale_offset(tid >> 1) + 8 * (tid & 1)]) = sv;
     }
     __syncthreads();
 
@@ -204,7 +211,7 @@ scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scal
 #pragma unroll
           for (int x = 0; x < ROWS_PER_GROUP; ++x) {
             const int r = r0 + g * ROWS_PER_GROUP + x;            // staged rows beyond sc carry zero factors
-            const float s = __half2float(__ushort_as_half(s_scale[r][wb0 + beta]));
+            const float s = __half2float(__ushort_as_half(s_scale[scale_offset(r) + wb0 + beta]));
             if (NH == 1) {
               wa[x] = s_qs[r][0] * s; wb[x] = 0.0f;
             } else {
@@ -234,7 +241,7 @@ scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scal
       {
         const int half = lane & 1, beta = (lane >> 1) & 3, g = lane >> 3;
         if (g < gc) {
-          const uint32_t* w32 = reinterpret_cast<const uint32_t*>(&s_words[r0 + g * ROWS_PER_GROUP][wb0 + beta]) + half;
+          const uint32_t* w32 = reinterpret_cast<const uint32_t*>(&s_words[r0 + g * ROWS_PER_GROUP][(wb0 + beta) ^ (g << 2)]) + half;
           uint32_t a = w32[0 * TILE_BLOCKS * 2];
           uint32_t b = w32[1 * TILE_BLOCKS * 2];
           uint32_t c = w32[2 * TILE_BLOCKS * 2];

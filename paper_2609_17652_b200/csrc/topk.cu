@@ -1,6 +1,19 @@
 // fathom_topk: per-query-head top-k over n scores with deterministic ties (Sec. 2 "Top-k decoding").
 //
-// Bucket select on the order-preserving integer image of the fp32 score (-0 folded onto +0):
+// Both paths select on the order-preserving integer image of the fp32 score (-0 folded onto +0), and both give the
+// one set the definition fixes (ties to the lower token index), in ascending token order.
+//
+// Single pass (rows of 64K scores or more, at least 256 wanted): one read of the scores.
+//   a. one CTA per head histograms every 16th 1024-score chunk (12 leading key bits, shared memory) and finds two bins:
+//      the ESTIMATE, whose suffix count in the sample reaches the expected rank plus four standard deviations, and
+//      the BOUND, whose suffix count reaches k in the sample alone and therefore in the whole row;
+//   b. every CTA of the collection pass loads its 8192 scores before the sample kernel has finished (programmatic
+//      dependent launch), then appends the (score, token) pairs that reach the estimate's lower edge to the head's list;
+//   c. per head, a radix select over that list on the composite (key << 32 | ~index); the winners are placed in
+//      ascending order by a counting sort over 4096 token ranges. A head whose list came out shorter than wanted
+//      (the estimate was too high) collects again itself above the bound bin, which cannot fall short.
+//
+// Two passes (short rows, or FATHOM_TOPK_PATH=two_pass): bucket select.
 //   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores); the CTA that
 //      finishes a head's histogram last (ticket counter) finds
 //   2. the threshold bin b* whose suffix count first reaches the number wanted;
