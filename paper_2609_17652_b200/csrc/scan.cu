@@ -2,60 +2,39 @@
 //
 // A t-plane read of channel j dequantises to  a * sum_{p<t} (2 b_p - 1) 2^-(p+1)  with a = 8 s the
 // block range, so a score is a signed sum of per-(block, channel, plane) weights
-//     w[beta][j][p][h] = q_hj * a_{beta,j} * 2^-(p+1),      score_i = sum_rows (b_i ? +w : -w).
-// One add per (token, row, head) makes the scan arithmetic-bound (Sec. 6 "Arithmetic per byte"), so the
-// kernel trades adds for table lookups: the active (channel, plane) rows of a plan are taken four at a
-// time, and for every (64-token block, group of four rows) the 16 possible signed sums are tabulated once
-// (15 adds per head) and then looked up per token with the token's four plane bits as the index.
+//     w[beta][j][p][h] = q_hj * a_{beta,j} * 2^-(p+1),      score_i = sum_rows (b_i ? +w : -w)
+//                                                                   = -sum_rows w + sum_{rows with b_i = 1} 2 w.
+// The first term is a constant of the (block, head); every active (channel, plane) row then costs one predicated
+// add per (token, head).  One add per (token, row, head) is what bounds the scan (Sec. 6 "Arithmetic per byte"): at
+// 48 rows and 32 heads the plane bytes would take 9 us of HBM time and the adds take 43 us of the fp32 pipe, so the
+// kernel is built around instruction issue, not bandwidth.
 //
-// A CTA owns one plan (NH query heads that share the planes read) and 16 blocks (1024 tokens).  Up to 48
-// rows at a time it stages, with 16-byte loads, the rows' plane words (128 contiguous bytes per row: every
-// row is one contiguous run, Sec. 3.5) and fp16 scales (32 bytes per row) in shared memory; all these loads
-// are issued before anything waits, which is what a store in pinned host memory needs to run at link rate.
-// Then each of the four warps owns four consecutive blocks (256 tokens) and runs on its own (only
-// __syncwarp), walking the staged rows in chunks of four groups.  Per chunk a warp builds its
-//   tables     lane (group, head pair, block) takes the four staged scales, forms the weights and writes the
-//              16-entry table (8 bytes per entry = two heads); tables are 136 bytes apart so that the 32 lanes
-//              store to distinct banks;
-//   indices    lane (group, block, half) turns four 32-token row words into 32 four-bit indices with a
-//              4 x 4 bit-block transpose across the four registers (20 logic operations);
-// and then looks up: lane l owns tokens l and l + 32 of a block: one 8-byte load of the packed indices, then per
-//              head pair one 8-byte table load (all lanes hit one 128-byte table: conflict-free) and one
-//              packed add.
+// A tile is 16 blocks (1024 tokens) of one plan (NH query heads that share the planes read).  CTAs are persistent:
+// gridDim.x CTAs per plan walk the tiles round-robin, build the plan's list of active rows once, and fetch the next
+// tile's plane words and scales with asynchronous copies (cp.async, 16 bytes each: a row's 16 words are one
+// contiguous 128-byte run, Sec. 3.5) into the second half of a double buffer while they scan the current one.  (Short
+// CTAs that load, wait, compute and store in lockstep leave the issue slots idle for half of the time.)
+// Per tile and pass of up to 48 rows:
+//   weights    thread (block, rows r = k mod 8) multiplies the staged fp16 scale with the row's query factors
+//              q_hj 2^(3-p) and keeps 2 w of (row, block) for the NH heads; the negated half sums give the bases;
+//   adds       lane (block of the warp, octet of its tokens) reads ONE byte of the row's plane word - its eight
+//              tokens - and the NH weights, and adds them to the accumulators of the tokens whose bit is set
+//              (and + setp + NH predicated adds per token).
 // Only planes p < t_j and the scales of active channels are ever read.
 #include "fathom_common.cuh"
+
+#include <cstdlib>
+#include <cstring>
 
 namespace {
 
 constexpr int SCAN_WARPS = 4;
 constexpr int SCAN_THREADS = SCAN_WARPS * 32;
 constexpr int WB = 4;                                        // blocks per warp
-constexpr int TILE_BLOCKS = SCAN_WARPS * WB;                 // 1024 tokens per CTA
-constexpr int ROWS_PER_GROUP = 4;
-constexpr int GC = 4;                                        // groups per chunk
-constexpr int CHUNK_ROWS = GC * ROWS_PER_GROUP;              // 16
-constexpr int STAGE_ROWS = 3 * CHUNK_ROWS;                   // rows staged per CTA pass (a B = 48 plan in one pass)
-
-template <int NH> struct ScanCfg {
-  static constexpr int HP = NH == 1 ? 1 : NH / 2;            // head pairs (tables per block and group)
-  static constexpr int EB = NH == 1 ? 4 : 8;                 // bytes per table entry
-  static constexpr int TSTRIDE = 16 * EB + EB;               // bytes between tables (padded: 34 or 17 words)
-  static constexpr int NTAB = GC * HP * WB;                  // tables per warp and chunk
-};
-
-__device__ __forceinline__ void add2(unsigned long long& acc, unsigned long long v) {
-  asm("add.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(v));
-}
-
-// 4 x 4 bit-block transpose across four words: afterwards nibble k of word w holds, for token 4 k + w,
-// the bits of rows a, b, c, d at bit 0, 1, 2, 3.
-__device__ __forceinline__ void transpose_rows(uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
-  uint32_t t;
-  t = ((a >> 1) ^ b) & 0x55555555u; b ^= t; a ^= t << 1;
-  t = ((c >> 1) ^ d) & 0x55555555u; d ^= t; c ^= t << 1;
-  t = ((a >> 2) ^ c) & 0x33333333u; c ^= t; a ^= t << 2;
-  t = ((b >> 2) ^ d) & 0x33333333u; d ^= t; b ^= t << 2;
-}
+constexpr int TILE_BLOCKS = SCAN_WARPS * WB;                 // 1024 tokens per tile
+constexpr int STAGE_ROWS = 48;                               // rows staged per pass (a B = 48 plan in one pass)
+constexpr int TOK = 8;                                       // tokens per lane
+constexpr int CTAS_PER_SM = 7;
 
 // fp32 value whose order-preserving integer image (see topk.cu) has `bin` as its 12 leading bits and zeros below:
 // the lower edge of that histogram bin
@@ -66,321 +45,50 @@ __device__ __forceinline__ float bin_lower_edge(uint32_t bin) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
-// first fp16 of staged row r in the padded scale array
-__device__ __forceinline__ int scale_offset(int r) { return r * TILE_BLOCKS + (r >> 2) * 8; }
-
-template <int NH>
-struct alignas(16) WarpSmem {
-  using C = ScanCfg<NH>;
-  uint32_t idx[GC][WB * 4 * 2 + 2];                          // [group][(block, token mod 4, half)] + 2 pad words: 8 nibbles each;
-                                                             // the pad spreads the four groups over different banks
-  alignas(8) unsigned char tab[C::NTAB * C::TSTRIDE];
-};
-
-// MODE 0: scores of every token are written (fathom_scan).
-// MODE 1: only every tile_step-th tile is scanned and its scores are written compactly (tile i of the launch at
-//         token positions 1024 i ..) - the sample from which fathom_scan_topk derives a safe threshold.
-// MODE 2: every tile is scanned, nothing is written but the tokens whose score reaches the head's threshold:
-//         (score, token) pairs appended to the head's candidate list.
-// bx: the CTA's tile (of the launch, or of its item in a batched launch); by: its group of NH query heads
-template <int NH, int MODE>
-__device__ __forceinline__ void
-scan_body(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
-          const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
-          long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
-          int G, int heads_per_plan, const fathom_scan_fuse& fz, const long long bx, const int by) {
-  using C = ScanCfg<NH>;
-  constexpr int HP = C::HP, EB = C::EB, TSTRIDE = C::TSTRIDE;
-  __shared__ uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];      // channel of active row r
-  __shared__ uint8_t row_pl[FATHOM_D * FATHOM_NPLANES];       // plane of active row r
-  __shared__ int s_nrows;
-  __shared__ int warp_tot[4];
-  __shared__ float s_q[NH][FATHOM_D];
-  __shared__ float s_thr[NH];                                 // MODE 2: score a token must reach, per head
-  // Both staged arrays are read by lanes that differ in the group g = (row / 4) mod 4, and rows four apart would fall on
-  // the same banks: the plane words of row r sit at block column c ^ 4 g, and the scales of each group of four rows
-  // start 16 bytes further on.
-  __shared__ alignas(16) uint64_t s_words[STAGE_ROWS][TILE_BLOCKS];   // staged plane words (block columns swizzled)
-  __shared__ alignas(16) uint16_t s_scale[STAGE_ROWS * TILE_BLOCKS + (STAGE_ROWS / 4) * 8];   // staged fp16 scales (padded)
-  __shared__ float s_qs[STAGE_ROWS][NH];                               // q_hj * 2^(2 - p) per staged row
-  __shared__ WarpSmem<NH> s_warp[SCAN_WARPS];
-
-  FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
-  if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int h0 = by * NH;                                      // first of the NH query heads of this CTA
-  const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
-  const int kv = h0 / G;
-
-  // ---- active row list of this plan, ordered by channel then plane (thread = channel)
-  {
-    const int t = depth[(size_t)plan * FATHOM_D + tid];
-    int incl = t;                                             // inclusive prefix of depths over channels
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += y;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    for (int e = tid; e < NH * FATHOM_D; e += SCAN_THREADS) s_q[e / FATHOM_D][e % FATHOM_D] = q[(size_t)h0 * FATHOM_D + e];
-    if (MODE == 2 && tid < NH)                                // fetched now, needed in the epilogue
-      s_thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : bin_lower_edge(fz.state[(h0 + tid) * 8]);
-    __syncthreads();
-    int base = 0;
-    for (int w = 0; w < warp; ++w) base += warp_tot[w];
-    const int start = base + incl - t;
-    for (int p = 0; p < t; ++p) { row_ch[start + p] = (uint16_t)tid; row_pl[start + p] = (uint8_t)p; }
-    if (tid == FATHOM_D - 1) s_nrows = base + incl;
-    __syncthreads();
-  }
-  const int nrows = s_nrows;
-
-  WarpSmem<NH>& S = s_warp[warp];
-  const long long blk0 = bx * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;  // first block of this CTA
-  const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
-  const int wb0 = warp * WB;                                   // first block of this warp within the tile
-  const int nblk = max(0, min(WB, nblk_cta - wb0));
-
-  // lookup role: lane owns tokens lane (low word half) and lane + 32 (high half) of each of the warp's blocks
-  const int my_w = lane & 3;                                  // word of the transposed quadruple that holds my token
-  const int rot = (4 * (lane >> 2) - (EB == 8 ? 3 : 2)) & 31; // brings my nibble to the byte-offset position
-  constexpr uint32_t OFFMASK = 15u * EB;
-  unsigned long long acc2[WB][2][HP];                         // packed head pairs (NH >= 2)
-  float acc1[WB][2];                                          // NH == 1
-#pragma unroll
-  for (int b = 0; b < WB; ++b)
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-      acc1[b][x] = 0.0f;
-#pragma unroll
-      for (int hp = 0; hp < HP; ++hp) acc2[b][x][hp] = 0ull;
-    }
-
-  const uint64_t* planes_kv = planes + (size_t)kv * FATHOM_D * FATHOM_NPLANES * (size_t)plane_stride + blk0;
-  const uint16_t* scales_kv = scales + (size_t)kv * FATHOM_D * (size_t)scale_stride + blk0;
-
-  for (int s0 = 0; s0 < nrows; s0 += STAGE_ROWS) {
-    const int sc = min(STAGE_ROWS, nrows - s0);                // rows staged in this pass
-    if (s0 > 0) __syncthreads();                               // every warp is done with the previous pass
-    // ---- stage plane words (8 x 16 B per row), scales (2 x 16 B per row) and per-row query factors
-    {
-      uint4 wv[STAGE_ROWS * 8 / SCAN_THREADS];
-#pragma unroll
-      for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
-        const int e = tid + k * SCAN_THREADS, r = e >> 3, c = e & 7;
-        wv[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (r < sc && 2 * c < nblk_cta) {
-          const int j = row_ch[s0 + r], p = row_pl[s0 + r];
-          wv[k] = __ldg(reinterpret_cast<const uint4*>(planes_kv + ((size_t)j * FATHOM_NPLANES + p) * (size_t)plane_stride + 2 * c));
-        }
-      }
-      uint4 sv = make_uint4(0u, 0u, 0u, 0u);
-      if (tid < STAGE_ROWS * 2) {
-        const int r = tid >> 1, c = tid & 1;
-        if (r < sc && 8 * c < nblk_cta)
-          sv = __ldg(reinterpret_cast<const uint4*>(scales_kv + (size_t)row_ch[s0 + r] * (size_t)scale_stride + 8 * c));
-      }
-      if (tid < STAGE_ROWS) {
-        const bool valid = tid < sc;
-        const int j = valid ? row_ch[s0 + tid] : 0, p = valid ? row_pl[s0 + tid] : 0;
-        const float pw = valid ? __int_as_float((129 - p) << 23) : 0.0f;   // 8 * 2^-(p+1) = 2^(2-p), exact
-#pragma unroll
-        for (int h = 0; h < NH; ++h) s_qs[tid][h] = s_q[h][j] * pw;
-      }
-#pragma unroll
-      for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
-        const int e = tid + k * SCAN_THREADS;
-        const int r = e >> 3;
-        *reinterpret_cast<uint4*>(&s_words[r][(2 * (e & 7)) ^ (((r >> 2) & 3) << 2)]) = wv[k];
-      }
-      if (tid < STAGE_ROWS * 2) *reinterpret_cast<uint4*>(&s_scale[scale_offset(tid >> 1) + 8 * (tid & 1)]) = sv;
-    }
-    __syncthreads();
-
-    for (int r0 = 0; r0 < sc; r0 += CHUNK_ROWS) {
-      const int rc = min(CHUNK_ROWS, sc - r0);                   // rows in this chunk
-      const int gc = (rc + ROWS_PER_GROUP - 1) / ROWS_PER_GROUP; // groups in this chunk (the last may be padded)
-
-      // ---- tables: lane = (group, head pair, block)
-#pragma unroll
-      for (int t0 = 0; t0 < C::NTAB; t0 += 32) {
-        const int t = t0 + lane;
-        const int beta = t % WB, hp = (t / WB) % HP, g = t / (WB * HP);
-        if (t < C::NTAB && g < gc) {
-          float wa[ROWS_PER_GROUP], wb[ROWS_PER_GROUP];
-#pragma unroll
-          for (int x = 0; x < ROWS_PER_GROUP; ++x) {
-            const int r = r0 + g * ROWS_PER_GROUP + x;            // staged rows beyond sc carry zero factors
-            const float s = __half2float(__ushort_as_half(s_scale[scale_offset(r) + wb0 + beta]));
-            if (NH == 1) {
-              wa[x] = s_qs[r][0] * s; wb[x] = 0.0f;
-            } else {
-              const float2 qq = *reinterpret_cast<const float2*>(&s_qs[r][2 * hp]);
-              wa[x] = qq.x * s; wb[x] = qq.y * s;
-            }
-          }
-          float ta[16], tb[16];
-          ta[0] = -((wa[0] + wa[1]) + (wa[2] + wa[3]));
-          tb[0] = -((wb[0] + wb[1]) + (wb[2] + wb[3]));
-#pragma unroll
-          for (int x = 0; x < ROWS_PER_GROUP; ++x) {
-            const float da = 2.0f * wa[x], db = 2.0f * wb[x];
-#pragma unroll
-            for (int e = 0; e < (1 << x); ++e) { ta[e + (1 << x)] = ta[e] + da; tb[e + (1 << x)] = tb[e] + db; }
-          }
-          unsigned char* tab = S.tab + t * TSTRIDE;
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            if (NH == 1) reinterpret_cast<float*>(tab)[e] = ta[e];
-            else reinterpret_cast<float2*>(tab)[e] = make_float2(ta[e], tb[e]);
-          }
-        }
-      }
-
-      // ---- indices: lane = (group, block, half)
-      {
-        const int half = lane & 1, beta = (lane >> 1) & 3, g = lane >> 3;
-        if (g < gc) {
-          const uint32_t* w32 = reinterpret_cast<const uint32_t*>(&s_words[r0 + g * ROWS_PER_GROUP][(wb0 + beta) ^ (g << 2)]) + half;
-          uint32_t a = w32[0 * TILE_BLOCKS * 2];
-          uint32_t b = w32[1 * TILE_BLOCKS * 2];
-          uint32_t c = w32[2 * TILE_BLOCKS * 2];
-          uint32_t d = w32[3 * TILE_BLOCKS * 2];
-          transpose_rows(a, b, c, d);
-          S.idx[g][(beta * 4 + 0) * 2 + half] = a;
-          S.idx[g][(beta * 4 + 1) * 2 + half] = b;
-          S.idx[g][(beta * 4 + 2) * 2 + half] = c;
-          S.idx[g][(beta * 4 + 3) * 2 + half] = d;
-        }
-      }
-      __syncwarp();
-
-      // ---- lookup
-#pragma unroll
-      for (int b = 0; b < WB; ++b) {
-#pragma unroll
-        for (int g = 0; g < GC; ++g) {
-          if (g < gc) {
-            const uint2 nib = *reinterpret_cast<const uint2*>(&S.idx[g][(b * 4 + my_w) * 2]);
-            const uint32_t off_lo = __funnelshift_r(nib.x, nib.x, rot) & OFFMASK;
-            const uint32_t off_hi = __funnelshift_r(nib.y, nib.y, rot) & OFFMASK;
-            const unsigned char* tab = S.tab + ((g * HP) * WB + b) * TSTRIDE;
-            if (NH == 1) {
-              acc1[b][0] += *reinterpret_cast<const float*>(tab + off_lo);
-              acc1[b][1] += *reinterpret_cast<const float*>(tab + off_hi);
-            } else {
-#pragma unroll
-              for (int hp = 0; hp < HP; ++hp) {
-                add2(acc2[b][0][hp], *reinterpret_cast<const unsigned long long*>(tab + hp * (WB * TSTRIDE) + off_lo));
-                add2(acc2[b][1][hp], *reinterpret_cast<const unsigned long long*>(tab + hp * (WB * TSTRIDE) + off_hi));
-              }
-            }
-          }
-        }
-      }
-      __syncwarp();
-    }
-  }
-
-  // ---- epilogue
-  if (MODE != 2) {
-#pragma unroll
-    for (int b = 0; b < WB; ++b) {
-      if (b < nblk) {
-        const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;                       // token scanned
-        const long long dst = MODE == 1 ? tok - blk0 * FATHOM_BLOCK + bx * (TILE_BLOCKS * FATHOM_BLOCK) : tok;
-#pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          float* row = scores + (size_t)(h0 + h) * (size_t)score_stride;
-#pragma unroll
-          for (int x = 0; x < 2; ++x) {
-            float v;
-            if (NH == 1) v = acc1[b][x];
-            else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
-            if (tok + 32 * x < n) row[dst + 32 * x] = v;
-          }
-        }
-      }
-    }
-  } else {
-    // candidates of this warp's 256 tokens, per head, collected in the (now idle) table memory and appended to
-    // the head's global list; entry = (score bits, token)
-    constexpr int LIST = (int)(sizeof(S.tab) / sizeof(uint2)) / NH;    // entries per head
-    uint2* list = reinterpret_cast<uint2*>(S.tab);
-    uint32_t* cnt = S.idx[0];                                          // NH counters (index memory is idle too)
-    __syncwarp();
-    if (lane < NH) cnt[lane] = 0u;
-    __syncwarp();
-    float thr[NH];
-#pragma unroll
-    for (int h = 0; h < NH; ++h) thr[h] = s_thr[h];
-#pragma unroll
-    for (int b = 0; b < WB; ++b) {
-      if (b < nblk) {
-        const long long tok = (blk0 + wb0 + b) * FATHOM_BLOCK + lane;
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const long long t = tok + 32 * x;
-          const bool elig = t < n && t >= fz.sink_end && t < fz.local_begin;
-#pragma unroll
-          for (int h = 0; h < NH; ++h) {
-            float v;
-            if (NH == 1) v = acc1[b][x];
-            else v = __uint_as_float((uint32_t)(acc2[b][x][h >> 1] >> ((h & 1) * 32)));
-            if (elig && v >= thr[h]) {
-              const uint32_t p = atomicAdd(&cnt[h], 1u);
-              if (p < (uint32_t)LIST) list[h * LIST + p] = make_uint2(__float_as_uint(v), (uint32_t)t);
-              else {                                                   // list full: straight to the global list
-                const uint32_t gp = atomicAdd(&fz.cand_count[h0 + h], 1u);
-                if ((long long)gp < fz.capacity) {
-                  fz.cand_score[(size_t)(h0 + h) * fz.capacity + gp] = v;
-                  fz.cand_idx[(size_t)(h0 + h) * fz.capacity + gp] = (int32_t)t;
-                }
-              }
-            }
-          }
-        }
-      }
-    }
-    // one global atomic per (CTA, head): the four warps' counts are summed, the slice is reserved once
-    __shared__ uint32_t s_wcnt[SCAN_WARPS][NH], s_cbase[NH];
-    __syncwarp();
-    if (lane < NH) s_wcnt[warp][lane] = min(cnt[lane], (uint32_t)LIST);
-    __syncthreads();
-    if (tid < NH) {
-      uint32_t tot = 0;
-#pragma unroll
-      for (int w = 0; w < SCAN_WARPS; ++w) tot += s_wcnt[w][tid];
-      s_cbase[tid] = tot ? atomicAdd(&fz.cand_count[h0 + tid], tot) : 0u;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int h = 0; h < NH; ++h) {
-      const uint32_t c = s_wcnt[warp][h];
-      uint32_t base = s_cbase[h];
-      for (int w = 0; w < warp; ++w) base += s_wcnt[w][h];
-      for (uint32_t e = lane; e < c; e += 32) {
-        const uint2 it = list[h * LIST + e];
-        if ((long long)(base + e) < fz.capacity) {
-          fz.cand_score[(size_t)(h0 + h) * fz.capacity + base + e] = __uint_as_float(it.x);
-          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + base + e] = (int32_t)it.y;
-        }
-      }
-    }
-  }
+// a[h] += w[h] for the NH heads if bit MASK of `bits` is set.  (A predicated add.f32x2 is not issued as one
+// instruction, so the adds are scalar.)
+template <int MASK>
+__device__ __forceinline__ void add_if(float (&a)[4], uint32_t bits, const float (&w)[4]) {
+  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %4, %5;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %6;\n\t@p add.f32 %1, %1, %7;\n\t"
+      "@p add.f32 %2, %2, %8;\n\t@p add.f32 %3, %3, %9;\n\t}"
+      : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]) : "r"(bits), "n"(MASK), "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
+}
+template <int MASK>
+__device__ __forceinline__ void add_if(float (&a)[2], uint32_t bits, const float (&w)[2]) {
+  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %2, %3;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %4;\n\t@p add.f32 %1, %1, %5;\n\t}"
+      : "+f"(a[0]), "+f"(a[1]) : "r"(bits), "n"(MASK), "f"(w[0]), "f"(w[1]));
+}
+template <int MASK>
+__device__ __forceinline__ void add_if(float (&a)[1], uint32_t bits, const float (&w)[1]) {
+  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %1, %2;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %3;\n\t}"
+      : "+f"(a[0]) : "r"(bits), "n"(MASK), "f"(w[0]));
 }
 
-template <int NH, int MODE>
-__global__ void __launch_bounds__(SCAN_THREADS, 8)              // 64 registers: occupancy matters more than spills here
-scan_kernel(const uint64_t* __restrict__ planes, const uint16_t* __restrict__ scales,
-            const float* __restrict__ q, const uint8_t* __restrict__ depth, float* __restrict__ scores,
-            long long n, long long nb, long long plane_stride, long long scale_stride, long long score_stride,
-            int G, int heads_per_plan, fathom_scan_fuse fz) {
-  scan_body<NH, MODE>(planes, scales, q, depth, scores, n, nb, plane_stride, scale_stride, score_stride, G, heads_per_plan, fz,
-                      (long long)blockIdx.x, (int)blockIdx.y);
+// NH consecutive floats as one shared-memory access
+__device__ __forceinline__ void load_heads(const float* p, float (&v)[4]) {
+  const float4 x = *reinterpret_cast<const float4*>(p); v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
 }
+__device__ __forceinline__ void load_heads(const float* p, float (&v)[2]) {
+  const float2 x = *reinterpret_cast<const float2*>(p); v[0] = x.x; v[1] = x.y;
+}
+__device__ __forceinline__ void load_heads(const float* p, float (&v)[1]) { v[0] = *p; }
+__device__ __forceinline__ void store_heads(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store_heads(float* p, const float (&v)[2]) { *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]); }
+__device__ __forceinline__ void store_heads(float* p, const float (&v)[1]) { *p = v[0]; }
 
-// ---- several sessions in one launch (fathom_scan_batch): the items' tiles are laid end to end along grid.x
+// 16-byte asynchronous copy global -> shared; `valid` false writes zeros and reads nothing
+__device__ __forceinline__ void copy16_async(void* dst, const void* src, bool valid) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+  const int bytes = valid ? 16 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void copies_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void copies_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// ---- the sessions of one launch: their tiles are laid end to end (fathom_scan has one item)
 struct ScanBatch {
   static constexpr int MAX_ITEMS = 32;
   const uint64_t* planes[MAX_ITEMS];
@@ -394,49 +102,355 @@ struct ScanBatch {
 };
 
 template <int NH>
-__global__ void __launch_bounds__(SCAN_THREADS, 8)
-scan_batch_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan) {
-  int it = 0;
-  while (it + 1 < B.items && (long long)blockIdx.x >= B.tile_end[it]) ++it;      // uniform over the CTA, at most 31 steps
-  const long long bx = (long long)blockIdx.x - (it ? B.tile_end[it - 1] : 0);
-  fathom_scan_fuse fz = {};
-  fz.tile_step = 1;
-  scan_body<NH, 0>(B.planes[it], B.scales[it], B.q[it], B.depth[it], B.scores[it], B.n[it], (B.n[it] + FATHOM_BLOCK - 1) / FATHOM_BLOCK, B.plane_stride[it],
-                   B.scale_stride[it], B.score_stride[it], G, heads_per_plan, fz, bx, (int)blockIdx.y);
+struct alignas(16) ScanSmem {
+  uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];                 // channel of active row r
+  uint8_t row_pl[FATHOM_D * FATHOM_NPLANES];                  // plane of active row r
+  int nrows;
+  int warp_tot[4];
+  float thr[NH];                                              // MODE 2: score a token must reach, per head
+  alignas(16) uint64_t words[2][STAGE_ROWS][TILE_BLOCKS];     // staged plane words, double buffered
+  alignas(16) uint16_t scale[2][STAGE_ROWS][TILE_BLOCKS];     // staged fp16 scales, double buffered
+  alignas(16) float qs[2 * STAGE_ROWS][NH];                   // q_hj * 2^(3 - p) of every row (plans of up to 96 rows) or of a pass
+  alignas(16) float w2[STAGE_ROWS][TILE_BLOCKS][NH];          // 2 w of (row, block, head)
+  alignas(16) float pb[SCAN_WARPS][TILE_BLOCKS][NH];          // -sum of w over the rows a warp weighted, per block
+  uint32_t cnt[SCAN_WARPS][NH], wcnt[SCAN_WARPS][NH], cbase[NH];   // MODE 2: candidate counters
+};
+
+// MODE 0: scores of every token are written (fathom_scan, fathom_scan_batch).
+// MODE 1: only every tile_step-th tile is scanned and its scores are written compactly (tile i of the launch at
+//         token positions 1024 i ..) - the sample from which fathom_scan_topk derives a safe threshold.
+// MODE 2: every tile is scanned, nothing is written but the tokens whose score reaches the head's threshold:
+//         (score, token) pairs appended to the head's candidate list.
+// grid = (CTAs per plan, groups of NH query heads); MODE 1 and 2 are launched with one item.
+template <int NH, int MODE>
+__global__ void __launch_bounds__(SCAN_THREADS, CTAS_PER_SM)
+scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fathom_scan_fuse fz) {
+  __shared__ ScanSmem<NH> M;
+  constexpr int QS_ROWS = (int)(sizeof(M.qs) / sizeof(M.qs[0]));
+
+  FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
+  if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
+  const long long total = B.tile_end[B.items - 1];             // tiles of this launch
+  long long g = blockIdx.x;                                    // my current tile of the launch
+  if (g >= total) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
+  const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
+  const int kv = h0 / G;
+  const int beta = lane >> 3, oct = lane & 7;                  // lane = (block of the warp, octet of its tokens)
+  const int myb = warp * WB + beta;                            // my block within the tile
+  if (MODE == 2 && tid < NH)                                   // read after the barriers of the first item's row list
+    M.thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : bin_lower_edge(fz.state[(h0 + tid) * 8]);
+
+  int item = -1, nrows = 0, npass = 1;
+
+  // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), and
+  //      the rows' query factors if they all fit
+  auto enter_item = [&](long long tile) {
+    int it = item < 0 ? 0 : item;
+    while (tile >= B.tile_end[it]) ++it;                       // uniform over the CTA; items only move forward
+    if (it == item) return;
+    item = it;
+    const int t = B.depth[it][(size_t)plan * FATHOM_D + tid];
+    int incl = t;                                              // inclusive prefix of depths over channels
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) M.warp_tot[warp] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < warp; ++w) before += M.warp_tot[w];
+    const int start = before + incl - t;
+    for (int p = 0; p < t; ++p) { M.row_ch[start + p] = (uint16_t)tid; M.row_pl[start + p] = (uint8_t)p; }
+    if (tid == FATHOM_D - 1) M.nrows = before + incl;
+    __syncthreads();
+    nrows = M.nrows;
+    npass = nrows > 0 ? (nrows + STAGE_ROWS - 1) / STAGE_ROWS : 1;
+    if (nrows <= QS_ROWS && tid < nrows) {                     // made visible by the barrier that precedes the first weights
+      const int j = M.row_ch[tid], p = M.row_pl[tid];
+      const float pw = __int_as_float((130 - p) << 23);        // 2 * 8 * 2^-(p+1) = 2^(3-p), exact
+#pragma unroll
+      for (int h = 0; h < NH; ++h) M.qs[tid][h] = __ldg(B.q[it] + (size_t)(h0 + h) * FATHOM_D + j) * pw;
+    }
+  };
+
+  // first block of launch tile `tile` within its session
+  auto first_block = [&](long long tile) -> long long {
+    const long long tl = tile - (item ? B.tile_end[item - 1] : 0);
+    return tl * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;
+  };
+
+  // ---- asynchronous copies of the plane words (8 x 16 B per row) and scales (2 x 16 B per row) of one pass of a tile
+  auto prefetch = [&](long long tile, int pass, int buf) {
+    const long long blk0 = first_block(tile);
+    const long long nb = (B.n[item] + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
+    const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
+    const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
+    const long long plane_stride = B.plane_stride[item], scale_stride = B.scale_stride[item];
+    const uint64_t* planes_kv = B.planes[item] + (size_t)kv * FATHOM_D * FATHOM_NPLANES * (size_t)plane_stride + blk0;
+    const uint16_t* scales_kv = B.scales[item] + (size_t)kv * FATHOM_D * (size_t)scale_stride + blk0;
+#pragma unroll
+    for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
+      const int e = tid + k * SCAN_THREADS, r = e >> 3, c = e & 7;
+      if (r < sc) {
+        const int j = M.row_ch[s0 + r], p = M.row_pl[s0 + r];
+        const bool valid = 2 * c < nblk_cta;
+        copy16_async(&M.words[buf][r][2 * c],
+                     valid ? (const void*)(planes_kv + ((size_t)j * FATHOM_NPLANES + p) * (size_t)plane_stride + 2 * c) : (const void*)B.planes[item],
+                     valid);
+      }
+    }
+    if (tid < STAGE_ROWS * 2) {
+      const int r = tid >> 1, c = tid & 1;
+      if (r < sc) {
+        const bool valid = 8 * c < nblk_cta;
+        copy16_async(&M.scale[buf][r][8 * c],
+                     valid ? (const void*)(scales_kv + (size_t)M.row_ch[s0 + r] * (size_t)scale_stride + 8 * c) : (const void*)B.scales[item], valid);
+      }
+    }
+    copies_commit();
+  };
+
+  enter_item(g);
+  int pass = 0, buf = 0;
+  prefetch(g, 0, 0);
+  float acc[TOK][NH], base[NH];
+
+  while (true) {
+    // ---- the stage after this one: the next pass of the tile, or the first pass of my next tile
+    long long g_next = g;
+    int pass_next = pass + 1;
+    if (pass_next == npass) { g_next = g + gridDim.x; pass_next = 0; }
+    const bool more = g_next < total;
+    const bool same_item = more && g_next < B.tile_end[item];
+    if (same_item) {
+      prefetch(g_next, pass_next, buf ^ 1);                    // lands while this stage is scanned
+      copies_wait<1>();
+    } else {
+      copies_wait<0>();
+    }
+    __syncthreads();                                           // this stage's words and scales are in place
+
+    const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
+    const int q0 = nrows <= QS_ROWS ? s0 : 0;                  // where this pass's query factors start in M.qs
+    if (nrows > QS_ROWS) {                                     // too many rows to keep all factors: those of this pass
+      if (tid < sc) {
+        const int j = M.row_ch[s0 + tid], p = M.row_pl[s0 + tid];
+        const float pw = __int_as_float((130 - p) << 23);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) M.qs[tid][h] = __ldg(B.q[item] + (size_t)(h0 + h) * FATHOM_D + j) * pw;
+      }
+      __syncthreads();
+    }
+
+    // ---- doubled weights of every (row, block) and the blocks' bases: thread = (block, rows r = k mod 8)
+    {
+      const int b = tid & 15, k = tid >> 4;
+      float pb[NH];
+#pragma unroll
+      for (int h = 0; h < NH; ++h) pb[h] = 0.0f;
+      for (int r = k; r < sc; r += SCAN_THREADS / 16) {
+        const float s = __half2float(__ushort_as_half(M.scale[buf][r][b]));
+        float w2[NH];
+        load_heads(&M.qs[q0 + r][0], w2);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) { w2[h] *= s; pb[h] += w2[h]; }
+        store_heads(&M.w2[r][b][0], w2);
+      }
+#pragma unroll
+      for (int h = 0; h < NH; ++h) pb[h] = -0.5f * (pb[h] + __shfl_xor_sync(0xffffffffu, pb[h], 16));
+      if (lane < 16) store_heads(&M.pb[warp][b][0], pb);
+    }
+    __syncthreads();
+
+    if (pass == 0) {
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        base[h] = 0.0f;
+#pragma unroll
+        for (int t = 0; t < TOK; ++t) acc[t][h] = 0.0f;
+      }
+    }
+#pragma unroll
+    for (int w = 0; w < SCAN_WARPS; ++w) {
+      float pb[NH];
+      load_heads(&M.pb[w][myb][0], pb);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) base[h] += pb[h];
+    }
+
+    // ---- one predicated add per (token, row, head)
+    {
+      const unsigned char* my_bytes = reinterpret_cast<const unsigned char*>(&M.words[buf][0][myb]) + oct;
+      const float* my_w = &M.w2[0][myb][0];
+#pragma unroll 4
+      for (int r = 0; r < sc; ++r) {
+        const uint32_t bits = my_bytes[r * (TILE_BLOCKS * 8)];
+        float w[NH];
+        load_heads(my_w + r * (TILE_BLOCKS * NH), w);
+        add_if<1>(acc[0], bits, w);
+        add_if<2>(acc[1], bits, w);
+        add_if<4>(acc[2], bits, w);
+        add_if<8>(acc[3], bits, w);
+        add_if<16>(acc[4], bits, w);
+        add_if<32>(acc[5], bits, w);
+        add_if<64>(acc[6], bits, w);
+        add_if<128>(acc[7], bits, w);
+      }
+    }
+
+    if (pass == npass - 1) {
+      // ---- scores of my eight tokens: base + what the set bits added
+      float v[NH][TOK];
+#pragma unroll
+      for (int t = 0; t < TOK; ++t)
+#pragma unroll
+        for (int h = 0; h < NH; ++h) v[h][t] = acc[t][h] + base[h];
+      const long long n = B.n[item];
+      const long long blk0 = first_block(g);
+      const bool have_block = blk0 + myb < (n + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
+      const long long tok = (blk0 + myb) * FATHOM_BLOCK + oct * TOK;                        // my first token
+
+      if (MODE != 2) {
+        if (have_block) {
+          const long long dst = MODE == 1 ? g * (TILE_BLOCKS * FATHOM_BLOCK) + myb * FATHOM_BLOCK + oct * TOK : tok;
+#pragma unroll
+          for (int h = 0; h < NH; ++h) {
+            float* row = B.scores[item] + (size_t)(h0 + h) * (size_t)B.score_stride[item] + dst;
+            if (tok + TOK <= n) {
+              *reinterpret_cast<float4*>(row) = make_float4(v[h][0], v[h][1], v[h][2], v[h][3]);
+              *reinterpret_cast<float4*>(row + 4) = make_float4(v[h][4], v[h][5], v[h][6], v[h][7]);
+            } else {
+#pragma unroll
+              for (int t = 0; t < TOK; ++t)
+                if (tok + t < n) row[t] = v[h][t];
+            }
+          }
+        }
+      } else {
+        // candidates of this warp's 256 tokens, per head, collected in the (now idle) weight memory and appended to
+        // the head's global list; entry = (score bits, token)
+        constexpr int LIST = (int)(sizeof(M.w2) / sizeof(uint2)) / SCAN_WARPS / NH;    // entries per warp and head
+        __syncthreads();                                                   // every warp is done with the weights
+        uint2* list = reinterpret_cast<uint2*>(&M.w2[0][0][0]) + warp * (LIST * NH);
+        uint32_t* cnt = M.cnt[warp];
+        if (lane < NH) cnt[lane] = 0u;
+        __syncwarp();
+        if (have_block) {
+#pragma unroll
+          for (int t = 0; t < TOK; ++t) {
+            const long long ti = tok + t;
+            const bool elig = ti < n && ti >= fz.sink_end && ti < fz.local_begin;
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+              if (elig && v[h][t] >= M.thr[h]) {
+                const uint32_t p = atomicAdd(&cnt[h], 1u);
+                if (p < (uint32_t)LIST) list[h * LIST + p] = make_uint2(__float_as_uint(v[h][t]), (uint32_t)ti);
+                else {                                                   // list full: straight to the global list
+                  const uint32_t gp = atomicAdd(&fz.cand_count[h0 + h], 1u);
+                  if ((long long)gp < fz.capacity) {
+                    fz.cand_score[(size_t)(h0 + h) * fz.capacity + gp] = v[h][t];
+                    fz.cand_idx[(size_t)(h0 + h) * fz.capacity + gp] = (int32_t)ti;
+                  }
+                }
+              }
+            }
+          }
+        }
+        // one global atomic per (tile, head): the four warps' counts are summed, the slice is reserved once
+        __syncwarp();
+        if (lane < NH) M.wcnt[warp][lane] = min(cnt[lane], (uint32_t)LIST);
+        __syncthreads();
+        if (tid < NH) {
+          uint32_t tot = 0;
+#pragma unroll
+          for (int w = 0; w < SCAN_WARPS; ++w) tot += M.wcnt[w][tid];
+          M.cbase[tid] = tot ? atomicAdd(&fz.cand_count[h0 + tid], tot) : 0u;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          const uint32_t c = M.wcnt[warp][h];
+          uint32_t at = M.cbase[h];
+          for (int w = 0; w < warp; ++w) at += M.wcnt[w][h];
+          for (uint32_t e = lane; e < c; e += 32) {
+            const uint2 it = list[h * LIST + e];
+            if ((long long)(at + e) < fz.capacity) {
+              fz.cand_score[(size_t)(h0 + h) * fz.capacity + at + e] = __uint_as_float(it.x);
+              fz.cand_idx[(size_t)(h0 + h) * fz.capacity + at + e] = (int32_t)it.y;
+            }
+          }
+        }
+      }
+    }
+
+    if (!more) break;
+    __syncthreads();                                           // every warp is done with this stage's buffers
+    g = g_next;
+    pass = pass_next;
+    buf ^= 1;
+    if (!same_item) {                                          // first tile of another session: nothing was fetched ahead
+      enter_item(g);
+      prefetch(g, 0, buf);
+    }
+  }
+}
+
+// CTAs per plan: as many as are resident at once, and no more than there are tiles
+static int scan_ctas_per_plan(long long tiles, int plans) {
+  static int sms[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  if (!sms[dev]) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    sms[dev] = v;
+  }
+  long long x = (long long)sms[dev] * CTAS_PER_SM / plans;
+  if (x < 1) x = 1;
+  return (int)(x < tiles ? x : tiles);
 }
 
 template <int NH, int MODE>
-int launch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
-                const uint8_t* depth, int heads_per_plan, float* scores, long long score_stride,
-                const fathom_scan_fuse& fz, cudaStream_t st) {
-  const long long nb = fathom_nblocks(L->n);
-  const long long ntiles = (nb + TILE_BLOCKS - 1) / TILE_BLOCKS;
-  const long long gx = MODE == 1 ? (ntiles + fz.tile_step - 1) / fz.tile_step : ntiles;
-  dim3 grid((unsigned)gx, (unsigned)(L->n_q_heads / NH));
-  if (MODE == 0) {                                            // may become resident while fathom_alloc_depth's kernel runs
-    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(SCAN_THREADS), 0, st, planes, scales, q, depth, scores, (long long)L->n,
-                                (long long)nb, (long long)L->plane_stride_words, (long long)L->scale_stride, score_stride,
-                                L->n_q_heads / L->n_kv_heads, heads_per_plan, fz) != cudaSuccess)
+int launch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const fathom_scan_fuse& fz, bool dependent,
+                cudaStream_t st) {
+  const long long tiles = B.tile_end[B.items - 1];
+  if (tiles <= 0) return FATHOM_OK;
+  const int plans = Hq / NH;
+  dim3 grid((unsigned)scan_ctas_per_plan(tiles, plans), (unsigned)plans);
+  if (dependent) {                                            // may become resident while the previous kernel of the stream runs
+    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(SCAN_THREADS), 0, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
       return FATHOM_ERR_CUDA;
-    return 0;
+    return FATHOM_OK;
   }
-  scan_kernel<NH, MODE><<<grid, SCAN_THREADS, 0, st>>>(planes, scales, q, depth, scores, L->n, nb, L->plane_stride_words,
-                                                       L->scale_stride, score_stride, L->n_q_heads / L->n_kv_heads,
-                                                       heads_per_plan, fz);
-  return 0;
+  scan_kernel<NH, MODE><<<grid, SCAN_THREADS, 0, st>>>(B, Hq / Hkv, heads_per_plan, fz);
+  return FATHOM_OK;
 }
 
 template <int MODE>
-int dispatch_scan(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
-                  const uint8_t* depth, int heads_per_plan, float* scores, long long score_stride,
-                  const fathom_scan_fuse& fz, cudaStream_t st) {
+int dispatch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const fathom_scan_fuse& fz, bool dependent,
+                  cudaStream_t st) {
   switch (heads_per_plan) {
-    case 1: return launch_scan<1, MODE>(L, planes, scales, q, depth, 1, scores, score_stride, fz, st);
-    case 2: return launch_scan<2, MODE>(L, planes, scales, q, depth, 2, scores, score_stride, fz, st);
-    case 4: return launch_scan<4, MODE>(L, planes, scales, q, depth, 4, scores, score_stride, fz, st);
-    case 8: return launch_scan<4, MODE>(L, planes, scales, q, depth, 8, scores, score_stride, fz, st);   // two CTAs of four heads share a plan
+    case 1: return launch_scan<1, MODE>(B, Hkv, Hq, 1, fz, dependent, st);
+    case 2: return launch_scan<2, MODE>(B, Hkv, Hq, 2, fz, dependent, st);
+    case 4: return launch_scan<4, MODE>(B, Hkv, Hq, 4, fz, dependent, st);
+    case 8: return launch_scan<4, MODE>(B, Hkv, Hq, 8, fz, dependent, st);   // two CTAs of four heads share a plan
     default: return FATHOM_ERR_UNSUPPORTED;
   }
+}
+
+// one session as a batch of one; `tile_step` > 1 lists only the sampled tiles
+ScanBatch single_item(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q, const uint8_t* depth,
+                      float* scores, long long score_stride, int tile_step) {
+  ScanBatch B = {};
+  B.items = 1;
+  B.planes[0] = planes; B.scales[0] = scales; B.q[0] = q; B.depth[0] = depth; B.scores[0] = scores;
+  B.n[0] = L->n; B.plane_stride[0] = L->plane_stride_words; B.scale_stride[0] = L->scale_stride; B.score_stride[0] = score_stride;
+  const long long tiles = (fathom_nblocks(L->n) + TILE_BLOCKS - 1) / TILE_BLOCKS;
+  B.tile_end[0] = (tiles + tile_step - 1) / tile_step;
+  return B;
 }
 
 }  // namespace
@@ -448,12 +462,14 @@ int fathom_launch_scan_sample(const fathom_layout* L, const uint64_t* planes, co
                               int tile_step, cudaStream_t st) {
   fathom_scan_fuse fz = {};
   fz.tile_step = tile_step;
-  return dispatch_scan<1>(L, planes, scales, q, depth, heads_per_plan, sample, sample_stride, fz, st);
+  return dispatch_scan<1>(single_item(L, planes, scales, q, depth, sample, sample_stride, tile_step), L->n_kv_heads, L->n_q_heads,
+                          heads_per_plan, fz, false, st);
 }
 
 int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
                               const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st) {
-  return dispatch_scan<2>(L, planes, scales, q, depth, heads_per_plan, nullptr, 0, fz, st);
+  return dispatch_scan<2>(single_item(L, planes, scales, q, depth, nullptr, 0, 1), L->n_kv_heads, L->n_q_heads, heads_per_plan, fz,
+                          false, st);
 }
 
 extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64_t* planes, const uint16_t* scales,
@@ -466,7 +482,8 @@ extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64
   if (!fathom_aligned16(planes) || !fathom_aligned16(scales) || !fathom_aligned16(scores)) return FATHOM_ERR_ALIGNMENT;
   fathom_scan_fuse fz = {};
   fz.tile_step = 1;
-  rc = dispatch_scan<0>(L, planes, scales, q, depth, heads_per_plan, scores, L->score_stride, fz, static_cast<cudaStream_t>(stream));
+  rc = dispatch_scan<0>(single_item(L, planes, scales, q, depth, scores, L->score_stride, 1), L->n_kv_heads, L->n_q_heads, heads_per_plan,
+                        fz, true, static_cast<cudaStream_t>(stream));
   if (rc != FATHOM_OK) return rc;
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
@@ -487,6 +504,8 @@ extern "C" int fathom_scan_batch(fathom_ctx* ctx, const fathom_scan_item* items,
   if (heads_per_plan < 1 || G % heads_per_plan != 0) return FATHOM_ERR_INVALID_ARG;
   if (heads_per_plan != 1 && heads_per_plan != 2 && heads_per_plan != 4 && heads_per_plan != 8) return FATHOM_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  fathom_scan_fuse fz = {};
+  fz.tile_step = 1;
   for (int first = 0; first < n_items; first += ScanBatch::MAX_ITEMS) {       // at most 32 sessions per launch
     ScanBatch B = {};
     B.items = n_items - first < ScanBatch::MAX_ITEMS ? n_items - first : ScanBatch::MAX_ITEMS;
@@ -499,13 +518,8 @@ extern "C" int fathom_scan_batch(fathom_ctx* ctx, const fathom_scan_item* items,
       tiles += (fathom_nblocks(it.layout.n) + TILE_BLOCKS - 1) / TILE_BLOCKS;
       B.tile_end[i] = tiles;
     }
-    const int nh = heads_per_plan == 8 ? 4 : heads_per_plan;  // plans of eight heads are served by two CTAs of four
-    dim3 grid((unsigned)tiles, (unsigned)(Hq / nh));
-    switch (nh) {
-      case 1: scan_batch_kernel<1><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
-      case 2: scan_batch_kernel<2><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
-      default: scan_batch_kernel<4><<<grid, SCAN_THREADS, 0, st>>>(B, G, heads_per_plan); break;
-    }
+    const int rc = dispatch_scan<0>(B, Hkv, Hq, heads_per_plan, fz, false, st);
+    if (rc != FATHOM_OK) return rc;
   }
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
