@@ -42,7 +42,7 @@ WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3
 # written / 8,388,608 units; valid for the single-pass path only), attention at k = 4096 (66.1 MB read + 1.05 MB
 # written; proportional to k, not to n: 67.1 MB / (32 heads x 4096 rows) = 512.3 B per selected row).
 # Multiplied by the units of a launch in the JSON line.
-NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.3, "topk_*": 17.3}
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 15.9, "topk_*": 17.3}
 NCU_TRAFFIC_BYTES_PER_SELECTED_ROW = 512.3
 
 
@@ -307,14 +307,17 @@ def run_ours(args):
         f"topk ({topk_passes} pass{'es' if topk_passes > 1 else ''} over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
         "sparse_attend": roof("sparse_attend", stage_us["sparse_attend"], "attend_*", n * Hkv),
     }
-    # the scan is bound by shared-memory table lookups and issue slots, not by HBM: also report it that way
-    groups_per_plan = [(int(r.sum()) + 3) // 4 for r in depth_h]            # groups of four active rows
-    lookups = n * sum(groups_per_plan) * max(1, hpp // 2)                    # per token, group and head pair
-    lookup_peak = 148 * 15.8 * 1.965e9                          # measured: 15.8 eight-byte lookups per clock per SM
+    # the scan is bound by arithmetic, not by HBM (one fp32 add per token, active row and head): also report it that way
+    adds = float(n) * sum(int(r.sum()) for r in depth_h) * hpp               # per token, active (channel, plane) row and head
+    add_peak = 148 * 128 * 1.965e9                              # fp32 lanes x SMs x clocks.max.sm: one add per lane and clock
+    issue_peak = 148 * 4 * 1.965e9                              # warp instructions per second (four schedulers per SM)
+    scan_s = stage_us["scan"] * 1e-6
     result["roofline_other_kernels"]["scan"]["alt_bound"] = {
-        "bound": "shared-memory lookups", "achieved": round(lookups / (stage_us["scan"] * 1e-6) / 1e12, 3), "peak": round(lookup_peak / 1e12, 3),
-        "unit": "T lookups/s", "frac": round(lookups / (stage_us["scan"] * 1e-6) / lookup_peak, 4),
-        "note": "one 8-byte table load per token, group of four rows and head pair; peak = 148 SMs x 15.8 lookups per clock (micro-benchmark of 8-byte shared-memory loads) x 1.965 GHz"}
+        "bound": "alu", "achieved": round(adds / scan_s / 1e12, 3), "peak": round(add_peak / 1e12, 3), "unit": "T fp32 adds/s",
+        "frac": round(adds / scan_s / add_peak, 4),
+        "issue_frac": round(adds / 32 * 1.25 / scan_s / issue_peak, 4),
+        "note": "peak = 148 SMs x 128 fp32 lanes x 1.965 GHz; the adds are predicated on the token's plane bit, which costs a fifth "
+                "instruction per four adds: issue_frac = (adds / 32 lanes x 5/4) / (148 SMs x 4 schedulers x 1.965 GHz)"}
 
     # ---- attention gathers 256-byte rows scattered over 2 + 2 GiB: every row opens a DRAM page, so the copy peak is not
     #      the bound that matters.  A micro-benchmark of a pure gather (half a warp per row, 8 loads in flight, rows

@@ -398,8 +398,19 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   }
 }
 
-// CTAs per plan: as many as are resident at once, and no more than there are tiles
-static int scan_ctas_per_plan(long long tiles, int plans) {
+// Whether the planes are read over the host link (pinned host memory mapped into the device's address space)
+static bool planes_in_host_memory(const void* planes) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, planes) != cudaSuccess) { cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost;
+}
+
+// CTAs per plan.  Planes in HBM: as many as are resident at once (and no more than there are tiles), each walking
+// several tiles.  Planes read over the host link: one CTA per tile, so that CTAs become resident in block order - all
+// tiles of one plan before the next plan's - and the link sees a few long sequential streams (48 rows of one KV head)
+// instead of eight times as many short ones; the link, not instruction issue, bounds that scan.
+static int scan_ctas_per_plan(long long tiles, int plans, bool host_planes) {
+  if (host_planes) return (int)tiles;
   static int sms[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
@@ -419,7 +430,7 @@ int launch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const f
   const long long tiles = B.tile_end[B.items - 1];
   if (tiles <= 0) return FATHOM_OK;
   const int plans = Hq / NH;
-  dim3 grid((unsigned)scan_ctas_per_plan(tiles, plans), (unsigned)plans);
+  dim3 grid((unsigned)scan_ctas_per_plan(tiles, plans, planes_in_host_memory(B.planes[0])), (unsigned)plans);
   if (dependent) {                                            // may become resident while the previous kernel of the stream runs
     if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(SCAN_THREADS), 0, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
       return FATHOM_ERR_CUDA;
