@@ -123,7 +123,9 @@ int fathom_alloc_depth(fathom_ctx* ctx, const fathom_layout* layout, const float
  * For every plan, every query head h of it and every token i < n:
  *   scores[h][i] = sum_{j : depth_j > 0} q_hj * (c_ij >> (4 - t_j) + 1/2 - 2^(t_j - 1)) * (8 s_{beta(i), j}) / 2^(t_j - 1)
  * reading only planes p < t_j and the scales of the active channels; fp32 accumulation; no 1/sqrt(d)
- * factor.  `planes` / `scales` may be device memory or device-addressable pinned host memory.
+ * factor.  `planes` / `scales` may be device memory or device-addressable pinned host memory (the call asks the
+ * runtime which it is: planes in device memory are scanned by persistent CTAs that fetch their next tile ahead, planes
+ * in host memory by one CTA per tile in block order, which keeps the requests on the host link sequential).
  *   scores  out  [Hq][score_stride] fp32; elements i >= n of a row are not written
  * heads_per_plan must be 1, 2, 4 or 8 and divide G. */
 int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes,
