@@ -126,6 +126,8 @@ int fathom_alloc_depth(fathom_ctx* ctx, const fathom_layout* layout, const float
  * factor.  `planes` / `scales` may be device memory or device-addressable pinned host memory (the call asks the
  * runtime which it is: planes in device memory are scanned by persistent CTAs that fetch their next tile ahead, planes
  * in host memory by one CTA per tile in block order, which keeps the requests on the host link sequential).
+ * Environment: FATHOM_SCAN_CTAS_PER_PLAN=<count> (read at every call) fixes the number of CTAs that share a plan's
+ * tiles instead; the scores do not depend on it.
  *   scores  out  [Hq][score_stride] fp32; elements i >= n of a row are not written
  * heads_per_plan must be 1, 2, 4 or 8 and divide G. */
 int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes,

@@ -410,6 +410,10 @@ static bool planes_in_host_memory(const void* planes) {
 // tiles of one plan before the next plan's - and the link sees a few long sequential streams (48 rows of one KV head)
 // instead of eight times as many short ones; the link, not instruction issue, bounds that scan.
 static int scan_ctas_per_plan(long long tiles, int plans, bool host_planes) {
+  if (const char* e = getenv("FATHOM_SCAN_CTAS_PER_PLAN")) {   // tests and tuning: a fixed number (read at every call)
+    const long long v = atoll(e);
+    if (v >= 1) return (int)(v < tiles ? v : tiles);
+  }
   if (host_planes) return (int)tiles;
   static int sms[64] = {};
   int dev = 0;
