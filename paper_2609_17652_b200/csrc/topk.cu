@@ -332,11 +332,13 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                     const uint32_t* state, float* __restrict__ cand_score, int32_t* __restrict__ cand_idx,
-                    uint32_t* __restrict__ cand_count) {
+                    uint32_t* __restrict__ cand_count, int heads) {
   __shared__ uint16_t s_list[FILT_TILE];
   __shared__ uint32_t s_count, s_base;
-  // heads and tiles are walked from the last to the first: what the scan wrote last is the likeliest to be in L2 still
-  const int head = gridDim.y - 1 - blockIdx.y, tile = gridDim.x - 1 - blockIdx.x;
+  // one CTA per (tile, head), tiles from the last to the first and all heads of a tile together: the scan writes the
+  // heads' rows side by side from the first token to the last, so what it wrote last is the likeliest to be in L2 still
+  const int head = heads - 1 - (int)(blockIdx.x % (unsigned)heads);
+  const int tile = (int)(gridDim.x / (unsigned)heads) - 1 - (int)(blockIdx.x / (unsigned)heads);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) s_count = 0u;
   const float* row = scores + (size_t)head * (size_t)score_stride;
@@ -892,7 +894,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       // programmatic dependent launch: the collection's CTAs become resident and load their scores while the 32 CTAs of
       // the sample kernel work; they wait for its completion (griddepcontrol.wait) before they read the threshold
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = fgrid;
+      cfg.gridDim = dim3((unsigned)ntiles * (unsigned)Hq);
       cfg.blockDim = dim3(FILT_THREADS);
       cfg.dynamicSmemBytes = 0;
       cfg.stream = st;
@@ -902,9 +904,10 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       cfg.attrs = attr;
       cfg.numAttrs = 1;
       FATHOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, topk_collect_kernel, scores, n, score_stride, F, (const uint32_t*)S.state,
-                                              S.cand_score, S.cand, S.cand_count));
+                                              S.cand_score, S.cand, S.cand_count, Hq));
     } else {
-      topk_collect_kernel<<<fgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand_score, S.cand, S.cand_count);
+      topk_collect_kernel<<<(unsigned)ntiles * (unsigned)Hq, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand_score, S.cand,
+                                                                                 S.cand_count, Hq);
     }
     // one launch serves both outcomes: a head whose estimate was low enough selects among its collected candidates; a
     // head that fell short collects above the bound bin itself (one CTA streaming its row) and selects among those
