@@ -9,11 +9,12 @@
 // 48 rows and 32 heads the plane bytes would take 9 us of HBM time and the adds take 43 us of the fp32 pipe, so the
 // kernel is built around instruction issue, not bandwidth.
 //
-// A tile is 16 blocks (1024 tokens) of one plan (NH query heads that share the planes read).  CTAs are persistent:
-// gridDim.x CTAs per plan walk the tiles round-robin, build the plan's list of active rows once, and fetch the next
-// tile's plane words and scales with asynchronous copies (cp.async, 16 bytes each: a row's 16 words are one
-// contiguous 128-byte run, Sec. 3.5) into the second half of a double buffer while they scan the current one.  (Short
-// CTAs that load, wait, compute and store in lockstep leave the issue slots idle for half of the time.)
+// A tile is 16 blocks (1024 tokens) of one plan (NH query heads that share the planes read).  With the planes in device
+// memory the CTAs are persistent: gridDim.x CTAs per plan walk the tiles round-robin, build the plan's list of active rows
+// once, and fetch the next tile's plane words and scales with asynchronous copies (cp.async, 16 bytes each: a row's 16
+// words are one contiguous 128-byte run, Sec. 3.5) into the second half of a double buffer while they scan the current
+// one; that pays at small budgets (40 against 48 us at B = 4) and is neutral at B = 48, where the adds dominate.  With the
+// planes in pinned host memory the grid is one CTA per tile, which keeps the requests on the host link sequential.
 // Per tile and pass of up to 48 rows:
 //   weights    thread (block, rows r = k mod 8) multiplies the staged fp16 scale with the row's query factors
 //              q_hj 2^(3-p) and keeps 2 w of (row, block) for the NH heads; the negated half sums give the bases;
