@@ -4,7 +4,8 @@
 // one set the definition fixes (ties to the lower token index), in ascending token order.
 //
 // Single pass (rows of 64K scores or more, at least 256 wanted): one read of the scores.
-//   a. one CTA per head histograms every 16th 1024-score chunk (12 leading key bits, shared memory) and finds two bins:
+//   a. a cluster of four CTAs per head histograms every 16th 1024-score chunk (12 leading key bits, shared memory,
+//      merged through distributed shared memory) and finds two bins:
 //      the ESTIMATE, whose suffix count in the sample reaches the expected rank plus four standard deviations, and
 //      the BOUND, whose suffix count reaches k in the sample alone and therefore in the whole row;
 //   b. every CTA of the collection pass loads its 8192 scores before the sample kernel has finished (programmatic
@@ -29,9 +30,13 @@
 // The selected set is unique, so neither the append order nor atomics can show in the output.
 #include "fathom_common.cuh"
 
+#include <cooperative_groups.h>
+
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -200,20 +205,24 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
   if (want_bound) search(want_bound, true);
 }
 
-// Histogram of a head's sample (every 16th whole chunk of 1024 scores) by ONE CTA, which then finds the estimated and
-// the bound bin itself: no global histogram, no flush, no ticket.  For rows of up to a few million scores.
+// Histogram of a head's sample (every 16th whole chunk of 1024 scores) by a cluster of SAMPLE_CLUSTER CTAs: each
+// histograms its share of the chunks in its own shared memory, the first CTA of the cluster adds the others' histograms
+// to its own through distributed shared memory and finds the estimated and the bound bin: no global histogram, no
+// flush, no ticket.  For rows of up to a few million scores.
 constexpr int SAMPLE_THREADS = 1024;
-__global__ void __launch_bounds__(SAMPLE_THREADS)
+constexpr int SAMPLE_CLUSTER = 4;
+__global__ void __cluster_dims__(SAMPLE_CLUSTER, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 topk_sample_kernel(const float* __restrict__ scores, long long sampled, long long chunk_stride, long long score_stride,
                    uint32_t* __restrict__ state, uint32_t want, uint32_t want_bound, uint32_t* __restrict__ cand_count,
                    uint32_t* __restrict__ cand_count2) {
   __shared__ uint32_t sh[FATHOM_TOPK_BINS];
   __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
-  const int head = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int head = blockIdx.x / SAMPLE_CLUSTER, part = (int)cluster.block_rank();
   // the collection kernel may be launched as a programmatic dependent: let it start at once, it loads its scores while
   // this kernel runs and waits for this kernel's results only before it compares
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (threadIdx.x == 0) {                                     // the collection that follows counts from zero
+  if (part == 0 && threadIdx.x == 0) {                        // the collection that follows counts from zero
     cand_count[head] = 0u;
     if (cand_count2) cand_count2[head] = 0u;
   }
@@ -221,16 +230,26 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
   __syncthreads();
   const float* row = scores + (size_t)head * (size_t)score_stride;
   // `sampled` whole chunks of 1024 scores, chunk_stride scores apart (16384: every 16th chunk of a score row; 1024: a
-  // compact array of sampled scores)
-#pragma unroll 8
-  for (long long v = threadIdx.x; v < sampled * 256; v += SAMPLE_THREADS) {
+  // compact array of sampled scores); CTA `part` of the cluster takes every SAMPLE_CLUSTER-th group of 1024 float4
+#pragma unroll 4
+  for (long long v = (long long)part * SAMPLE_THREADS + threadIdx.x; v < sampled * 256; v += SAMPLE_CLUSTER * SAMPLE_THREADS) {
     const float4 x = __ldg(reinterpret_cast<const float4*>(row + (v >> 8) * chunk_stride) + (v & 255));
     atomicAdd(&sh[ordered_key(x.x) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.y) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
   }
-  __syncthreads();
+  cluster.sync();                                             // every CTA's histogram is complete
+  if (part == 0) {
+    for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) {
+      uint32_t c = sh[b];
+#pragma unroll
+      for (int r = 1; r < SAMPLE_CLUSTER; ++r) c += cluster.map_shared_rank(sh, r)[b];
+      sh[b] = c;
+    }
+  }
+  cluster.sync();                                             // the others' shared memory has been read: they may exit
+  if (part != 0) return;
   find_threshold_bin<SAMPLE_THREADS, false>(sh, state + head * 8, want, nullptr, s_warp, want_bound);
 }
 
@@ -856,7 +875,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
   const long long chunks = n / 1024, sampled = (chunks + 15) / 16;           // whole chunks; chunks 0, 16, 32, .. are sampled
   uint32_t rank = 0;
   const bool single = single_pass_plan(n, k, want, &rank);
-  // histograms, per-head states and candidate counters are contiguous at the start of the arena; the one-CTA sample
+  // histograms, per-head states and candidate counters are contiguous at the start of the arena; the sample
   // kernel keeps its histogram in shared memory
   // (the sample kernel writes every state word that path reads and clears the candidate counter: nothing to clear then)
   if (!(single && sampled <= 256)) FATHOM_CUDA_TRY(ctx, cudaMemsetAsync(S.hist, 0, (char*)S.bitmap - (char*)S.hist, st));
@@ -882,7 +901,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
     // reach the bound bin, hence at least k - forced = want eligible ones
     if (sampled <= 256) {                                              // up to 4M scores per row: one CTA per head
-      topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k,
+      topk_sample_kernel<<<Hq * SAMPLE_CLUSTER, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k,
                                                         S.cand_count, nullptr);
     } else {
       const int reps = 8;                                              // sampled chunks per CTA
@@ -1005,7 +1024,7 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)n_forced;
   const bool two_attempts = !force_two_pass() && want >= 256 && (long long)rank * 2 <= k;
   if (one_cta_sample) {                                       // one CTA per head, histogram in shared memory only
-    topk_sample_kernel<<<Hq, SAMPLE_THREADS, 0, st>>>(S.sample, n_sample / 1024, 1024LL, S.sample_stride, S.state,
+    topk_sample_kernel<<<Hq * SAMPLE_CLUSTER, SAMPLE_THREADS, 0, st>>>(S.sample, n_sample / 1024, 1024LL, S.sample_stride, S.state,
                                                       two_attempts ? rank : (uint32_t)k, two_attempts ? (uint32_t)k : 0u, S.cand_count,
                                                       S.cand_count2);
   } else {
