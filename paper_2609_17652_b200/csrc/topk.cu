@@ -376,16 +376,22 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   FATHOM_PDL_RELEASE();                                       // the selection that follows may become resident now
   __syncthreads();
   const float lo = __uint_as_float(__ldcg(state + head * 8 + 6));   // the score a candidate must reach
+  const uint32_t woff = (uint32_t)warp * FILT_WARP_TOKENS + (uint32_t)lane * 4u;   // my first token's offset in the tile
 #pragma unroll
   for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
     const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
     if (fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])) >= lo) {  // divergent on purpose: candidates are rare
-      const long long t0 = wbase + it * 128 + lane * 4;
+      const uint32_t off = woff + it * 128u;
+      if (all_elig) {                                         // (uniform over the warp) nothing else to check
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const long long t = t0 + c;
-        if (e[c] >= lo && (all_elig || (t < n && t >= F.sink_end && t < F.local_begin)))
-          s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(t - tile0);
+        for (int c = 0; c < 4; ++c)
+          if (e[c] >= lo) s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(off + c);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const long long t = tile0 + off + c;
+          if (e[c] >= lo && t < n && t >= F.sink_end && t < F.local_begin) s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(off + c);
+        }
       }
     }
   }
