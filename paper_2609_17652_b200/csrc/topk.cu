@@ -351,13 +351,15 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
 __global__ void __launch_bounds__(FILT_THREADS)
 topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                     const uint32_t* state, float* __restrict__ cand_score, int32_t* __restrict__ cand_idx,
-                    uint32_t* __restrict__ cand_count, int heads) {
+                    uint32_t* __restrict__ cand_count, int ntiles) {
   __shared__ uint16_t s_list[FILT_TILE];
   __shared__ uint32_t s_count, s_base;
-  // one CTA per (tile, head), tiles from the last to the first and all heads of a tile together: the scan writes the
-  // heads' rows side by side from the first token to the last, so what it wrote last is the likeliest to be in L2 still
-  const int head = heads - 1 - (int)(blockIdx.x % (unsigned)heads);
-  const int tile = (int)(gridDim.x / (unsigned)heads) - 1 - (int)(blockIdx.x / (unsigned)heads);
+  // one CTA per (head, tile): grid = (heads, tiles in y and z), tiles from the last to the first and all heads of a tile
+  // together: the scan writes the heads' rows side by side from the first token to the last, so what it wrote last is
+  // the likeliest to be in L2 still
+  const int head = gridDim.x - 1 - blockIdx.x;
+  const int tile = ntiles - 1 - (int)(blockIdx.z * gridDim.y + blockIdx.y);
+  if (tile < 0) return;                                        // padding of the last z slice
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) s_count = 0u;
   const float* row = scores + (size_t)head * (size_t)score_stride;
@@ -365,10 +367,16 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
   const bool all_elig = wbase >= F.sink_end && wbase + FILT_WARP_TOKENS <= F.local_begin && wbase + FILT_WARP_TOKENS <= n;
   float4 x[FILT_WARP_TOKENS / 128];
+  if (wbase + FILT_WARP_TOKENS <= n) {                        // (uniform over the warp) no load needs a guard
+    const float4* src = reinterpret_cast<const float4*>(row + wbase) + lane;
 #pragma unroll
-  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
-    const long long t0 = wbase + it * 128 + lane * 4;
-    x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) x[it] = __ldg(src + it * 32);
+  } else {
+#pragma unroll
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+      const long long t0 = wbase + it * 128 + lane * 4;
+      x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
   // The scores were complete before the sample kernel started; its threshold and cleared counters are needed from
   // here on (a no-op unless this kernel was launched as a programmatic dependent of the sample kernel).
@@ -915,11 +923,13 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       topk_hist_kernel<<<sgrid, HIST_THREADS, 0, st>>>(scores, n, score_stride, F, S.hist, S.state, rank, nullptr, 1024, 16 * 1024LL,
                                                        reps, (uint32_t)k);
     }
+    const unsigned ty = (unsigned)(ntiles < 65535 ? ntiles : 65535);
+    const dim3 cgrid((unsigned)Hq, ty, (unsigned)((ntiles + ty - 1) / ty));
     if (sampled <= 256) {
       // programmatic dependent launch: the collection's CTAs become resident and load their scores while the 32 CTAs of
       // the sample kernel work; they wait for its completion (griddepcontrol.wait) before they read the threshold
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)ntiles * (unsigned)Hq);
+      cfg.gridDim = cgrid;
       cfg.blockDim = dim3(FILT_THREADS);
       cfg.dynamicSmemBytes = 0;
       cfg.stream = st;
@@ -929,10 +939,9 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
       cfg.attrs = attr;
       cfg.numAttrs = 1;
       FATHOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, topk_collect_kernel, scores, n, score_stride, F, (const uint32_t*)S.state,
-                                              S.cand_score, S.cand, S.cand_count, Hq));
+                                              S.cand_score, S.cand, S.cand_count, ntiles));
     } else {
-      topk_collect_kernel<<<(unsigned)ntiles * (unsigned)Hq, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand_score, S.cand,
-                                                                                 S.cand_count, Hq);
+      topk_collect_kernel<<<cgrid, FILT_THREADS, 0, st>>>(scores, n, score_stride, F, S.state, S.cand_score, S.cand, S.cand_count, ntiles);
     }
     // one launch serves both outcomes: a head whose estimate was low enough selects among its collected candidates; a
     // head that fell short collects above the bound bin itself (one CTA streaming its row) and selects among those
