@@ -189,17 +189,17 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     const long long nb = (B.n[item] + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
     const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
     const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
-    const long long plane_stride = B.plane_stride[item], scale_stride = B.scale_stride[item];
-    const uint64_t* planes_kv = B.planes[item] + (size_t)kv * FATHOM_D * FATHOM_NPLANES * (size_t)plane_stride + blk0;
-    const uint16_t* scales_kv = B.scales[item] + (size_t)kv * FATHOM_D * (size_t)scale_stride + blk0;
+    // (strides are below 2^32 elements: one 32 x 32 -> 64-bit multiply per address)
+    const uint32_t plane_stride = (uint32_t)B.plane_stride[item], scale_stride = (uint32_t)B.scale_stride[item];
+    const uint64_t* planes_kv = B.planes[item] + (uint64_t)(kv * FATHOM_D * FATHOM_NPLANES) * plane_stride + blk0;
+    const uint16_t* scales_kv = B.scales[item] + (uint64_t)(kv * FATHOM_D) * scale_stride + blk0;
 #pragma unroll
     for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
       const int e = tid + k * SCAN_THREADS, r = e >> 3, c = e & 7;
       if (r < sc) {
-        const int j = M.row_ch[s0 + r], p = M.row_pl[s0 + r];
+        const uint32_t row = (uint32_t)M.row_ch[s0 + r] * FATHOM_NPLANES + M.row_pl[s0 + r];
         const bool valid = 2 * c < nblk_cta;
-        copy16_async(&M.words[buf][r][2 * c],
-                     valid ? (const void*)(planes_kv + ((size_t)j * FATHOM_NPLANES + p) * (size_t)plane_stride + 2 * c) : (const void*)B.planes[item],
+        copy16_async(&M.words[buf][r][2 * c], valid ? (const void*)(planes_kv + (uint64_t)row * plane_stride + 2 * c) : (const void*)B.planes[item],
                      valid);
       }
     }
@@ -208,7 +208,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       if (r < sc) {
         const bool valid = 8 * c < nblk_cta;
         copy16_async(&M.scale[buf][r][8 * c],
-                     valid ? (const void*)(scales_kv + (size_t)M.row_ch[s0 + r] * (size_t)scale_stride + 8 * c) : (const void*)B.scales[item], valid);
+                     valid ? (const void*)(scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride + 8 * c) : (const void*)B.scales[item], valid);
       }
     }
     copies_commit();
