@@ -131,8 +131,8 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
 
   FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
-  const long long total = B.tile_end[B.items - 1];             // tiles of this launch
-  long long g = blockIdx.x;                                    // my current tile of the launch
+  const int total = (int)B.tile_end[B.items - 1];              // tiles of this launch (tile and block indices fit 32 bits)
+  int g = blockIdx.x;                                          // my current tile of the launch
   if (g >= total) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
@@ -147,7 +147,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
 
   // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), and
   //      the rows' query factors if they all fit
-  auto enter_item = [&](long long tile) {
+  auto enter_item = [&](int tile) {
     int it = item < 0 ? 0 : item;
     while (tile >= B.tile_end[it]) ++it;                       // uniform over the CTA; items only move forward
     if (it == item) return;
@@ -178,16 +178,16 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   };
 
   // first block of launch tile `tile` within its session
-  auto first_block = [&](long long tile) -> long long {
-    const long long tl = tile - (item ? B.tile_end[item - 1] : 0);
+  auto first_block = [&](int tile) -> int {
+    const int tl = tile - (item ? (int)B.tile_end[item - 1] : 0);
     return tl * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;
   };
 
   // ---- asynchronous copies of the plane words (8 x 16 B per row) and scales (2 x 16 B per row) of one pass of a tile
-  auto prefetch = [&](long long tile, int pass, int buf) {
-    const long long blk0 = first_block(tile);
-    const long long nb = (B.n[item] + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
-    const int nblk_cta = (int)min((long long)TILE_BLOCKS, nb - blk0);
+  auto prefetch = [&](int tile, int pass, int buf) {
+    const int blk0 = first_block(tile);
+    const int nb = (int)((B.n[item] + FATHOM_BLOCK - 1) / FATHOM_BLOCK);
+    const int nblk_cta = min(TILE_BLOCKS, nb - blk0);
     const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
     // (strides are below 2^32 elements: one 32 x 32 -> 64-bit multiply per address)
     const uint32_t plane_stride = (uint32_t)B.plane_stride[item], scale_stride = (uint32_t)B.scale_stride[item];
@@ -221,7 +221,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
 
   while (true) {
     // ---- the stage after this one: the next pass of the tile, or the first pass of my next tile
-    long long g_next = g;
+    int g_next = g;
     int pass_next = pass + 1;
     if (pass_next == npass) { g_next = g + gridDim.x; pass_next = 0; }
     const bool more = g_next < total;
@@ -309,14 +309,14 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       for (int t = 0; t < TOK; ++t)
 #pragma unroll
         for (int h = 0; h < NH; ++h) v[h][t] = acc[t][h] + base[h];
-      const long long n = B.n[item];
-      const long long blk0 = first_block(g);
+      const uint32_t n = (uint32_t)B.n[item];                  // n < 2^31
+      const int blk0 = first_block(g);
       const bool have_block = blk0 + myb < (n + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
-      const long long tok = (blk0 + myb) * FATHOM_BLOCK + oct * TOK;                        // my first token
+      const uint32_t tok = (uint32_t)(blk0 + myb) * FATHOM_BLOCK + oct * TOK;                // my first token
 
       if (MODE != 2) {
         if (have_block) {
-          const long long dst = MODE == 1 ? g * (TILE_BLOCKS * FATHOM_BLOCK) + myb * FATHOM_BLOCK + oct * TOK : tok;
+          const uint32_t dst = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + myb * FATHOM_BLOCK + oct * TOK : tok;
 #pragma unroll
           for (int h = 0; h < NH; ++h) {
             float* row = B.scores[item] + (size_t)(h0 + h) * (size_t)B.score_stride[item] + dst;
@@ -342,7 +342,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         if (have_block) {
 #pragma unroll
           for (int t = 0; t < TOK; ++t) {
-            const long long ti = tok + t;
+            const long long ti = (long long)tok + t;
             const bool elig = ti < n && ti >= fz.sink_end && ti < fz.local_begin;
 #pragma unroll
             for (int h = 0; h < NH; ++h) {
