@@ -123,11 +123,15 @@ int fathom_alloc_depth(fathom_ctx* ctx, const fathom_layout* layout, const float
  * For every plan, every query head h of it and every token i < n:
  *   scores[h][i] = sum_{j : depth_j > 0} q_hj * (c_ij >> (4 - t_j) + 1/2 - 2^(t_j - 1)) * (8 s_{beta(i), j}) / 2^(t_j - 1)
  * reading only planes p < t_j and the scales of the active channels; fp32 accumulation; no 1/sqrt(d)
- * factor.  `planes` / `scales` may be device memory or device-addressable pinned host memory (the call asks the
+ * factor.  The accumulate runs on the tensor cores: the plane bit becomes the sign of the stored fp16 scale (exact), the
+ * query factors are split into two fp16 parts (the precision of an fp32 weight), products are exact in fp32 accumulators
+ * and summed in an order that the plan alone fixes, so scores do not depend on the launch geometry.
+ * `planes` / `scales` may be device memory or device-addressable pinned host memory (the call asks the
  * runtime which it is: planes in device memory are scanned by persistent CTAs that fetch their next tile ahead, planes
  * in host memory by one CTA per tile in block order, which keeps the requests on the host link sequential).
- * Environment: FATHOM_SCAN_CTAS_PER_PLAN=<count> (read at every call) fixes the number of CTAs that share a plan's
- * tiles instead; the scores do not depend on it.
+ * Depth values above 4 are read as 4.
+ * Environment: FATHOM_SCAN_PATH=simt (read once per process) selects the earlier CUDA-core kernel (one predicated fp32
+ * add per plane bit and head) for every scan; both meet the same tolerance.
  *   scores  out  [Hq][score_stride] fp32; elements i >= n of a row are not written
  * heads_per_plan must be 1, 2, 4 or 8 and divide G. */
 int fathom_scan(fathom_ctx* ctx, const fathom_layout* layout, const uint64_t* planes,
@@ -149,6 +153,10 @@ typedef struct fathom_scan_item {
   float* scores;
 } fathom_scan_item;
 int fathom_scan_batch(fathom_ctx* ctx, const fathom_scan_item* items, int n_items, int heads_per_plan, void* stream);
+/* Tuning and test knob, process-wide, no GPU work (the paper has no counterpart): a positive `ctas` fixes the number of
+ * CTAs that share a plan's tiles in every later scan launch (each then walks several tiles, also across the sessions of
+ * a batch); 0 restores the automatic choice.  Scores never depend on it.  Always returns FATHOM_OK. */
+int fathom_scan_set_ctas_per_plan(int ctas);
 
 /* ---- (4) top-k — Sec. 2 "Top-k decoding" ---------------------------------------------------
  * Per query head: the first n_sink and the last n_local tokens are always selected; the remaining

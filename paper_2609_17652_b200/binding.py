@@ -23,7 +23,8 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_device_status", "fathom_version", "fathom_build_planes", "fathom_alloc_depth", "fathom_scan",
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
-           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated", "fathom_scan_batch"]
+           "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated", "fathom_scan_batch",
+           "fathom_scan_set_ctas_per_plan"]
 
 
 class Layout(C.Structure):
@@ -67,6 +68,7 @@ def _load() -> C.CDLL:
     lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
     lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
     lib.fathom_scan_batch.argtypes = [vp, vp, i32, i32, vp]
+    lib.fathom_scan_set_ctas_per_plan.argtypes = [i32]
     lib.fathom_build_planes_rotated.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -240,6 +242,11 @@ def fathom_topk_passes(layout: Layout, k: int, n_sink: int = 0, n_local: int = 0
     if rc < 0:
         raise FathomError(rc)
     return rc
+
+
+def fathom_scan_set_ctas_per_plan(ctas: int) -> None:
+    """Process-wide tuning knob: CTAs per plan of every later scan launch; 0 = automatic."""
+    lib.fathom_scan_set_ctas_per_plan(int(ctas))
 
 
 def fathom_scratch_bytes(layout: Layout, k: int) -> int:

@@ -1,121 +1,84 @@
-// fathom_scan: variable-depth bit-plane key scan (Sec. 3.2 prefix dequantiser, Sec. 3.3).
+// fathom_scan: variable-depth bit-plane key scan (Sec. 3.2 prefix dequantiser, Sec. 3.3), accumulate on the tensor cores.
 //
-// A t-plane read of channel j dequantises to  a * sum_{p<t} (2 b_p - 1) 2^-(p+1)  with a = 8 s the
-// block range, so a score is a signed sum of per-(block, channel, plane) weights
-//     w[beta][j][p][h] = q_hj * a_{beta,j} * 2^-(p+1),      score_i = sum_rows (b_i ? +w : -w)
-//                                                                   = -sum_rows w + sum_{rows with b_i = 1} 2 w.
-// The first term is a constant of the (block, head); every active (channel, plane) row then costs one predicated
-// add per (token, head).  One add per (token, row, head) is what bounds the scan (Sec. 6 "Arithmetic per byte"): at
-// 48 rows and 32 heads the plane bytes would take 9 us of HBM time and the adds take 43 us of the fp32 pipe, so the
-// kernel is built around instruction issue, not bandwidth.
+// A t-plane read of channel j dequantises to  a * sum_{p<t} (2 b_p - 1) 2^-(p+1)  with a = 8 s the block range, so with
+// the active (channel, plane) pairs of a plan as "rows" r = (j, p) a score is
+//     score[i][h] = sum_r  sigma[i][r] * s[beta(i)][j(r)]  *  q_h,j(r) 2^(2 - p(r)),        sigma = +1 if the bit is set, else -1:
+// a [tokens x rows] . [rows x heads] product whose left operand is the stored fp16 scale with the plane bit as its sign
+// - exact in fp16 - and whose right operand depends on neither token nor block.  One add per (token, row, head) on the
+// CUDA cores is what bounds the scan (Sec. 7 "Arithmetic per byte": 1.6 G adds at n = 1M, B = 48, 43 us of fp32 pipe
+// against 9 us of HBM time for the planes); here the adds go to the tensor cores and the CUDA cores only expand the
+// plane bits into the left operand, two integer instructions per pair of elements:
+//   * left operand (registers): a lane holds, for 8 consecutive tokens of a block (one byte of each plane word) and 4 of
+//     every 16 rows, the half2 (s_r, s_r') of a row pair; the element of token i is that pair with the sign bits flipped
+//     where the tokens' bits are clear:  pair ^ (~(bytes << shift_i) & 0x80008000);
+//   * right operand: q_hj 2^(2-p) / E_h (E_h a power of two near max_j |q_hj|) split into an fp16 head and an fp16 tail
+//     scaled by 2^11 (together 22 significant bits + rounding = the precision of an fp32 weight), columns
+//     (head, part) = 4 x 2 = the 8 columns of mma.sync.m16n8k16; built once per session and plan in shared memory;
+//   * fp16 x fp16 products are exact in the fp32 accumulators; score = E_h (acc_head + 2^-11 acc_tail).  The order of
+//     the accumulation is fixed by the row list alone, so scores do not depend on the launch geometry.
+// The tcgen05 path was not taken for this contraction: its left operand must sit in shared or tensor memory, i.e. every
+// expanded element would be written and read once more (2 bytes per (token, row) against 1/8 byte of plane bits), and
+// the expansion, not the multiply-add, is what costs here (12 mma per 64 tokens x 48 rows against ~100 integer ops).
 //
 // A tile is 16 blocks (1024 tokens) of one plan (NH query heads that share the planes read).  With the planes in device
-// memory the CTAs are persistent: gridDim.x CTAs per plan walk the tiles round-robin, build the plan's list of active rows
-// once, and fetch the next tile's plane words and scales with asynchronous copies (cp.async, 16 bytes each: a row's 16
-// words are one contiguous 128-byte run, Sec. 3.5) into the second half of a double buffer while they scan the current
-// one; that pays at small budgets (40 against 48 us at B = 4) and is neutral at B = 48, where the adds dominate.  With the
-// planes in pinned host memory the grid is one CTA per tile, which keeps the requests on the host link sequential.
-// Per tile and pass of up to 48 rows:
-//   weights    thread (block, rows r = k mod 8) multiplies the staged fp16 scale with the row's query factors
-//              q_hj 2^(3-p) and keeps 2 w of (row, block) for the NH heads; the negated half sums give the bases;
-//   adds       lane (block of the warp, octet of its tokens) reads ONE byte of the row's plane word - its eight
-//              tokens - and the NH weights, and adds them to the accumulators of the tokens whose bit is set
-//              (and + setp + NH predicated adds per token).
+// memory the CTAs are persistent: gridDim.x CTAs per plan walk the tiles round-robin, build the plan's row list and right
+// operand once, and fetch the next stage's plane words and scales with asynchronous copies (cp.async; a row's words are
+// one contiguous run, Sec. 3.6) into the other half of a double buffer.  A stage is a sub-tile of TB blocks and up to
+// ROWS rows: plans of up to 48 rows take whole tiles (TB = 16: 128-byte runs, a warp owns 4 blocks), up to 96 rows half
+// tiles (TB = 8), deeper plans quarter tiles (TB = 4, a warp owns one block and carries its accumulators over passes of
+// 160 rows), so that the staging buffers do not grow with the budget.  With the planes in pinned host memory the grid is
+// one CTA per tile, which keeps the requests on the host link sequential.
 // Only planes p < t_j and the scales of active channels are ever read.
-#include "fathom_common.cuh"
+#include "scan_shared.cuh"
 
 #include <cstdlib>
 #include <cstring>
+#include <type_traits>
 
 namespace {
 
-constexpr int SCAN_WARPS = 4;
-constexpr int SCAN_THREADS = SCAN_WARPS * 32;
-constexpr int WB = 4;                                        // blocks per warp
-constexpr int TILE_BLOCKS = SCAN_WARPS * WB;                 // 1024 tokens per tile
-constexpr int STAGE_ROWS = 48;                               // rows staged per pass (a B = 48 plan in one pass)
-constexpr int TOK = 8;                                       // tokens per lane
-constexpr int CTAS_PER_SM = 7;
+constexpr int THREADS = 128, WARPS = 4;
+constexpr int TILE_BLOCKS = FATHOM_SCAN_TILE_BLOCKS;
+constexpr int MAX_ROWS = FATHOM_D * FATHOM_NPLANES;          // 512 (channel, plane) pairs
+constexpr int MAX_KSTEPS = MAX_ROWS / 16;                    // 16 rows per mma
+constexpr int WORD_STAGE_BYTES = 7680;                       // staged plane words of one stage (padded rows)
+constexpr int SCALE_STAGE_BYTES = 4608;                      // staged fp16 scales of one stage (padded rows)
+constexpr int CTAS_PER_SM = 6;
 
-// fp32 value whose order-preserving integer image (see topk.cu) has `bin` as its 12 leading bits and zeros below:
-// the lower edge of that histogram bin
-__device__ __forceinline__ float bin_lower_edge(uint32_t bin) {
-  if (bin >= FATHOM_TOPK_BINS) return __uint_as_float(0x7fc00000u);   // past the last bin: nothing reaches it (NaN compares false)
-  if (bin <= 7u) return -INFINITY;                                    // bins below -inf's hold no finite score: everything reaches them
-  const uint32_t key = bin << 20;
-  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
-}
-
-// a[h] += w[h] for the NH heads if bit MASK of `bits` is set.  (A predicated add.f32x2 is not issued as one
-// instruction, so the adds are scalar.)
-template <int MASK>
-__device__ __forceinline__ void add_if(float (&a)[4], uint32_t bits, const float (&w)[4]) {
-  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %4, %5;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %6;\n\t@p add.f32 %1, %1, %7;\n\t"
-      "@p add.f32 %2, %2, %8;\n\t@p add.f32 %3, %3, %9;\n\t}"
-      : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]) : "r"(bits), "n"(MASK), "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
-}
-template <int MASK>
-__device__ __forceinline__ void add_if(float (&a)[2], uint32_t bits, const float (&w)[2]) {
-  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %2, %3;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %4;\n\t@p add.f32 %1, %1, %5;\n\t}"
-      : "+f"(a[0]), "+f"(a[1]) : "r"(bits), "n"(MASK), "f"(w[0]), "f"(w[1]));
-}
-template <int MASK>
-__device__ __forceinline__ void add_if(float (&a)[1], uint32_t bits, const float (&w)[1]) {
-  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %1, %2;\n\tsetp.ne.u32 p, t, 0;\n\t@p add.f32 %0, %0, %3;\n\t}"
-      : "+f"(a[0]) : "r"(bits), "n"(MASK), "f"(w[0]));
-}
-
-// NH consecutive floats as one shared-memory access
-__device__ __forceinline__ void load_heads(const float* p, float (&v)[4]) {
-  const float4 x = *reinterpret_cast<const float4*>(p); v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-}
-__device__ __forceinline__ void load_heads(const float* p, float (&v)[2]) {
-  const float2 x = *reinterpret_cast<const float2*>(p); v[0] = x.x; v[1] = x.y;
-}
-__device__ __forceinline__ void load_heads(const float* p, float (&v)[1]) { v[0] = *p; }
-__device__ __forceinline__ void store_heads(float* p, const float (&v)[4]) {
-  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-__device__ __forceinline__ void store_heads(float* p, const float (&v)[2]) { *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]); }
-__device__ __forceinline__ void store_heads(float* p, const float (&v)[1]) { *p = v[0]; }
-
-// 16-byte asynchronous copy global -> shared; `valid` false writes zeros and reads nothing
-__device__ __forceinline__ void copy16_async(void* dst, const void* src, bool valid) {
-  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
-  const int bytes = valid ? 16 : 0;
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void copies_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int PENDING>
-__device__ __forceinline__ void copies_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
-
-// ---- the sessions of one launch: their tiles are laid end to end (fathom_scan has one item)
-struct ScanBatch {
-  static constexpr int MAX_ITEMS = 32;
-  const uint64_t* planes[MAX_ITEMS];
-  const uint16_t* scales[MAX_ITEMS];
-  const float* q[MAX_ITEMS];
-  const uint8_t* depth[MAX_ITEMS];
-  float* scores[MAX_ITEMS];
-  long long n[MAX_ITEMS], plane_stride[MAX_ITEMS], scale_stride[MAX_ITEMS], score_stride[MAX_ITEMS];
-  long long tile_end[MAX_ITEMS];                              // tiles of items 0 .. i, inclusive prefix
-  int items;
+// Stage geometry for sub-tiles of TB blocks.  The row pitches are padded so that the four lanes of a quad, which read
+// rows two apart, hit different banks (plane bytes: pitch / 4 = 4 mod 32 for TB = 16, ...).
+template <int TB>
+struct Geo {
+  static constexpr int ROW_BYTES = 8 * TB + 16;               // pitch of a staged plane-word row
+  static constexpr int SCALE_ELEMS = TB == 4 ? 12 : 24;       // pitch of a staged scale row, fp16 elements
+  static constexpr int ROWS = TB == 16 ? 48 : TB == 8 ? 96 : 160;   // rows per stage (multiples of 16)
+  static_assert(ROWS * ROW_BYTES <= WORD_STAGE_BYTES && ROWS * SCALE_ELEMS * 2 <= SCALE_STAGE_BYTES, "stage buffers too small");
 };
 
-template <int NH>
-struct alignas(16) ScanSmem {
-  uint16_t row_ch[FATHOM_D * FATHOM_NPLANES];                 // channel of active row r
-  uint8_t row_pl[FATHOM_D * FATHOM_NPLANES];                  // plane of active row r
+struct alignas(16) Smem {
+  uint16_t row_ch[MAX_ROWS];                                  // channel of active row r
+  uint8_t row_pl[MAX_ROWS];                                   // plane of active row r
   int nrows;
-  int warp_tot[4];
-  float thr[NH];                                              // MODE 2: score a token must reach, per head
-  alignas(16) uint64_t words[2][STAGE_ROWS][TILE_BLOCKS];     // staged plane words, double buffered
-  alignas(16) uint16_t scale[2][STAGE_ROWS][TILE_BLOCKS];     // staged fp16 scales, double buffered
-  alignas(16) float qs[2 * STAGE_ROWS][NH];                   // q_hj * 2^(3 - p) of every row (plans of up to 96 rows) or of a pass
-  alignas(16) float w2[STAGE_ROWS][TILE_BLOCKS][NH];          // 2 w of (row, block, head)
-  alignas(16) float pb[SCAN_WARPS][TILE_BLOCKS][NH];          // -sum of w over the rows a warp weighted, per block
-  uint32_t cnt[SCAN_WARPS][NH], wcnt[SCAN_WARPS][NH], cbase[NH];   // MODE 2: candidate counters
+  int warp_tot[WARPS];
+  float wmax[WARPS][4];                                       // per warp: max_j |q_hj| of its channels
+  float hscale[4], hinv[4];                                   // E_h and 1 / E_h
+  float thr[4];                                               // MODE 2: score a token must reach, per head
+  alignas(16) uint2 bfr[MAX_KSTEPS][32];                      // right operand: per 16 rows, the two B registers of every lane
+  alignas(16) unsigned char words[2][WORD_STAGE_BYTES];       // staged plane words, double buffered
+  alignas(16) unsigned char scale[2][SCALE_STAGE_BYTES];      // staged fp16 scales, double buffered
 };
+
+// D += A B, A 16 x 16 (row), B 16 x 8 (col), fp16 operands, fp32 accumulators
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// the scale pair with each half's sign flipped where bit (15 - SH) resp. (31 - SH) of `bytes` is clear
+template <int SH>
+__device__ __forceinline__ uint32_t signed_pair(uint32_t pair, uint32_t bytes) {
+  return pair ^ (~(bytes << SH) & 0x80008000u);
+}
 
 // MODE 0: scores of every token are written (fathom_scan, fathom_scan_batch).
 // MODE 1: only every tile_step-th tile is scanned and its scores are written compactly (tile i of the launch at
@@ -124,10 +87,9 @@ struct alignas(16) ScanSmem {
 //         (score, token) pairs appended to the head's candidate list.
 // grid = (CTAs per plan, groups of NH query heads); MODE 1 and 2 are launched with one item.
 template <int NH, int MODE>
-__global__ void __launch_bounds__(SCAN_THREADS, CTAS_PER_SM)
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
 scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fathom_scan_fuse fz) {
-  __shared__ ScanSmem<NH> M;
-  constexpr int QS_ROWS = (int)(sizeof(M.qs) / sizeof(M.qs[0]));
+  __shared__ Smem M;
 
   FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
@@ -135,45 +97,85 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   int g = blockIdx.x;                                          // my current tile of the launch
   if (g >= total) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gq = lane >> 2, t4 = lane & 3;                     // mma fragment coordinates: lane = (row group, column pair)
   const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
   const int kv = h0 / G;
-  const int beta = lane >> 3, oct = lane & 7;                  // lane = (block of the warp, octet of its tokens)
-  const int myb = warp * WB + beta;                            // my block within the tile
+  const int myh = t4 < NH ? t4 : 0;                            // the head whose scores this lane receives (lanes t4 >= NH: none)
   if (MODE == 2 && tid < NH)                                   // read after the barriers of the first item's row list
-    M.thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : bin_lower_edge(fz.state[(h0 + tid) * 8]);
+    M.thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : fathom_bin_lower_edge(fz.state[(h0 + tid) * 8]);
 
-  int item = -1, nrows = 0, npass = 1;
+  int item = -1, nrows = 0, tb = TILE_BLOCKS, rows_stage = Geo<16>::ROWS, npass = 1, nb_item = 0;
+  float hs = 1.0f, hs_tail = 0.0f;                             // E of my head and E 2^-11
 
-  // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), and
-  //      the rows' query factors if they all fit
+  // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), the
+  //      heads' power-of-two scales and the right operand of every 16 rows
   auto enter_item = [&](int tile) {
     int it = item < 0 ? 0 : item;
     while (tile >= B.tile_end[it]) ++it;                       // uniform over the CTA; items only move forward
     if (it == item) return;
     item = it;
-    const int t = B.depth[it][(size_t)plan * FATHOM_D + tid];
+    nb_item = (int)((B.n[it] + FATHOM_BLOCK - 1) / FATHOM_BLOCK);
+    const int t = min((int)B.depth[it][(size_t)plan * FATHOM_D + tid], FATHOM_NPLANES);   // a depth above 4 (an unwritten buffer) must not index past the row list
     int incl = t;                                              // inclusive prefix of depths over channels
+    float qa[NH];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) qa[h] = fabsf(__ldg(B.q[it] + (size_t)(h0 + h) * FATHOM_D + tid));
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += y;
+#pragma unroll
+      for (int h = 0; h < NH; ++h) qa[h] = fmaxf(qa[h], __shfl_xor_sync(0xffffffffu, qa[h], o));
     }
     if (lane == 31) M.warp_tot[warp] = incl;
+#pragma unroll
+    for (int h = 0; h < NH; ++h)
+      if (lane == h) M.wmax[warp][h] = qa[h];
     __syncthreads();
     int before = 0;
     for (int w = 0; w < warp; ++w) before += M.warp_tot[w];
     const int start = before + incl - t;
     for (int p = 0; p < t; ++p) { M.row_ch[start + p] = (uint16_t)tid; M.row_pl[start + p] = (uint8_t)p; }
     if (tid == FATHOM_D - 1) M.nrows = before + incl;
+    if (tid < NH) {                                            // E = 2^floor(log2 max|q|), kept inside the normal range
+      float m = 0.0f;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) m = fmaxf(m, M.wmax[w][tid]);
+      int eb = (int)(__float_as_uint(m) >> 23);
+      eb = eb < 1 ? 1 : (eb > 253 ? 253 : eb);
+      M.hscale[tid] = __int_as_float(eb << 23);
+      M.hinv[tid] = __int_as_float((254 - eb) << 23);
+    }
     __syncthreads();
     nrows = M.nrows;
-    npass = nrows > 0 ? (nrows + STAGE_ROWS - 1) / STAGE_ROWS : 1;
-    if (nrows <= QS_ROWS && tid < nrows) {                     // made visible by the barrier that precedes the first weights
-      const int j = M.row_ch[tid], p = M.row_pl[tid];
-      const float pw = __int_as_float((130 - p) << 23);        // 2 * 8 * 2^-(p+1) = 2^(3-p), exact
+    if (nrows <= Geo<16>::ROWS) { tb = 16; rows_stage = Geo<16>::ROWS; }
+    else if (nrows <= Geo<8>::ROWS) { tb = 8; rows_stage = Geo<8>::ROWS; }
+    else { tb = 4; rows_stage = Geo<4>::ROWS; }
+    npass = nrows > rows_stage ? (nrows + rows_stage - 1) / rows_stage : 1;
+    hs = M.hscale[myh];
+    hs_tail = hs * 4.8828125e-4f;                              // 2^-11
+    // right operand (made visible by the barrier that precedes the first stage's arithmetic): entry (kstep, lane, i)
+    // holds rows 16 kstep + 2 (lane & 3) + 8 i and the next one, column lane >> 2 = (head, part)
+    const int entries = ((nrows + 15) >> 4) * 64;
+    for (int e = tid; e < entries; e += THREADS) {
+      const int ks = e >> 6, ln = (e >> 1) & 31, i = e & 1;
+      const int col = ln >> 2, head = col >> 1, part = col & 1;
+      const int r0 = ks * 16 + 2 * (ln & 3) + 8 * i;
+      uint32_t packed = 0u;
+      if (head < NH) {
+        const float inv = M.hinv[head];
 #pragma unroll
-      for (int h = 0; h < NH; ++h) M.qs[tid][h] = __ldg(B.q[it] + (size_t)(h0 + h) * FATHOM_D + j) * pw;
+        for (int z = 0; z < 2; ++z) {
+          const int r = r0 + z;
+          float v = 0.0f;
+          if (r < nrows) v = __ldg(B.q[it] + (size_t)(h0 + head) * FATHOM_D + M.row_ch[r]) * inv * __int_as_float((129 - (int)M.row_pl[r]) << 23);
+          const __half hi = __float2half_rn(v);
+          const __half out = part ? __float2half_rn((v - __half2float(hi)) * 2048.0f) : hi;
+          packed |= (uint32_t)__half_as_ushort(out) << (16 * z);
+        }
+      }
+      reinterpret_cast<uint32_t*>(&M.bfr[ks][ln])[i] = packed;
     }
   };
 
@@ -183,250 +185,171 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     return tl * (MODE == 1 ? fz.tile_step : 1) * TILE_BLOCKS;
   };
 
-  // ---- asynchronous copies of the plane words (8 x 16 B per row) and scales (2 x 16 B per row) of one pass of a tile
-  auto prefetch = [&](int tile, int pass, int buf) {
-    const int blk0 = first_block(tile);
-    const int nb = (int)((B.n[item] + FATHOM_BLOCK - 1) / FATHOM_BLOCK);
-    const int nblk_cta = min(TILE_BLOCKS, nb - blk0);
-    const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
+  // ---- asynchronous copies of the plane words and scales of one stage: sub-tile u of `tile`, rows of `pass`
+  auto prefetch = [&](int tile, int u, int pass, int buf) {
+    const int blk0 = first_block(tile) + u * tb;
+    const int nblk = min(tb, nb_item - blk0);                  // >= 1: stages past the last block are never entered
+    const int s0 = pass * rows_stage, sc = min(rows_stage, nrows - s0);
     // (strides are below 2^32 elements: one 32 x 32 -> 64-bit multiply per address)
     const uint32_t plane_stride = (uint32_t)B.plane_stride[item], scale_stride = (uint32_t)B.scale_stride[item];
     const uint64_t* planes_kv = B.planes[item] + (uint64_t)(kv * FATHOM_D * FATHOM_NPLANES) * plane_stride + blk0;
     const uint16_t* scales_kv = B.scales[item] + (uint64_t)(kv * FATHOM_D) * scale_stride + blk0;
-#pragma unroll
-    for (int k = 0; k < STAGE_ROWS * 8 / SCAN_THREADS; ++k) {
-      const int e = tid + k * SCAN_THREADS, r = e >> 3, c = e & 7;
-      if (r < sc) {
-        const uint32_t row = (uint32_t)M.row_ch[s0 + r] * FATHOM_NPLANES + M.row_pl[s0 + r];
-        const bool valid = 2 * c < nblk_cta;
-        copy16_async(&M.words[buf][r][2 * c], valid ? (const void*)(planes_kv + (uint64_t)row * plane_stride + 2 * c) : (const void*)B.planes[item],
-                     valid);
-      }
+    const int sh = tb == 16 ? 3 : (tb == 8 ? 2 : 1);           // 16-byte copies per row of plane words: tb / 2
+    const int row_bytes = 8 * tb + 16;
+    unsigned char* wdst = M.words[buf];
+    for (int e = tid; e < (sc << sh); e += THREADS) {
+      const int r = e >> sh, c = e & ((1 << sh) - 1);
+      const uint32_t row = (uint32_t)M.row_ch[s0 + r] * FATHOM_NPLANES + M.row_pl[s0 + r];
+      const bool valid = 2 * c < nblk;
+      fathom_copy_async<16>(wdst + r * row_bytes + c * 16,
+                            valid ? (const void*)(planes_kv + (uint64_t)row * plane_stride + 2 * c) : (const void*)B.planes[item], valid);
     }
-    if (tid < STAGE_ROWS * 2) {
-      const int r = tid >> 1, c = tid & 1;
-      if (r < sc) {
-        const bool valid = 8 * c < nblk_cta;
-        copy16_async(&M.scale[buf][r][8 * c],
-                     valid ? (const void*)(scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride + 8 * c) : (const void*)B.scales[item], valid);
+    unsigned char* sdst = M.scale[buf];
+    if (tb == 16) {
+      for (int e = tid; e < sc * 2; e += THREADS) {
+        const int r = e >> 1, c = e & 1;
+        const bool valid = 8 * c < nblk;
+        fathom_copy_async<16>(sdst + r * (Geo<16>::SCALE_ELEMS * 2) + c * 16,
+                              valid ? (const void*)(scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride + 8 * c) : (const void*)B.scales[item], valid);
       }
+    } else if (tb == 8) {
+      for (int r = tid; r < sc; r += THREADS)
+        fathom_copy_async<16>(sdst + r * (Geo<8>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride, true);
+    } else {
+      for (int r = tid; r < sc; r += THREADS)
+        fathom_copy_async<8>(sdst + r * (Geo<4>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride, true);
     }
-    copies_commit();
+    // rows that pad the last 16: scale 0, so that whatever the stale plane bytes say they contribute +-0
+    const int pad = ((sc + 15) & ~15) - sc;
+    const int wpr = (tb == 4 ? Geo<4>::SCALE_ELEMS : Geo<16>::SCALE_ELEMS) / 2;   // 32-bit words per scale row
+    for (int e = tid; e < pad * wpr; e += THREADS)
+      reinterpret_cast<uint32_t*>(sdst)[(sc + e / wpr) * wpr + e % wpr] = 0u;
+    fathom_copies_commit();
   };
 
+  float acc[4][4];                                             // [16-token slice of the block][c0..c3]
+
   enter_item(g);
-  int pass = 0, buf = 0;
-  prefetch(g, 0, 0);
-  float acc[TOK][NH], base[NH];
+  const float my_thr = MODE == 2 ? M.thr[myh] : 0.0f;
+  int u = 0, pass = 0, buf = 0;
+  prefetch(g, 0, 0, 0);
 
   while (true) {
-    // ---- the stage after this one: the next pass of the tile, or the first pass of my next tile
-    int g_next = g;
-    int pass_next = pass + 1;
-    if (pass_next == npass) { g_next = g + gridDim.x; pass_next = 0; }
+    // ---- the stage after this one: the next pass of the sub-tile, the next sub-tile of the tile, or my next tile
+    int g_next = g, u_next = u, pass_next = pass + 1;
+    if (pass_next == npass) {
+      pass_next = 0;
+      u_next = u + 1;
+      if (u_next * tb >= TILE_BLOCKS || first_block(g) + u_next * tb >= nb_item) { u_next = 0; g_next = g + gridDim.x; }
+    }
     const bool more = g_next < total;
     const bool same_item = more && g_next < B.tile_end[item];
     if (same_item) {
-      prefetch(g_next, pass_next, buf ^ 1);                    // lands while this stage is scanned
-      copies_wait<1>();
+      prefetch(g_next, u_next, pass_next, buf ^ 1);            // lands while this stage is scanned
+      fathom_copies_wait<1>();
     } else {
-      copies_wait<0>();
+      fathom_copies_wait<0>();
     }
     __syncthreads();                                           // this stage's words and scales are in place
 
-    const int s0 = pass * STAGE_ROWS, sc = min(STAGE_ROWS, nrows - s0);
-    const int q0 = nrows <= QS_ROWS ? s0 : 0;                  // where this pass's query factors start in M.qs
-    if (nrows > QS_ROWS) {                                     // too many rows to keep all factors: those of this pass
-      if (tid < sc) {
-        const int j = M.row_ch[s0 + tid], p = M.row_pl[s0 + tid];
-        const float pw = __int_as_float((130 - p) << 23);
-#pragma unroll
-        for (int h = 0; h < NH; ++h) M.qs[tid][h] = __ldg(B.q[item] + (size_t)(h0 + h) * FATHOM_D + j) * pw;
-      }
-      __syncthreads();
-    }
-
-    // ---- doubled weights of every (row, block) and the blocks' bases: thread = (block, rows r = k mod 8)
-    {
-      const int b = tid & 15, k = tid >> 4;
-      float pb[NH];
-#pragma unroll
-      for (int h = 0; h < NH; ++h) pb[h] = 0.0f;
-      for (int r = k; r < sc; r += SCAN_THREADS / 16) {
-        const float s = __half2float(__ushort_as_half(M.scale[buf][r][b]));
-        float w2[NH];
-        load_heads(&M.qs[q0 + r][0], w2);
-#pragma unroll
-        for (int h = 0; h < NH; ++h) { w2[h] *= s; pb[h] += w2[h]; }
-        store_heads(&M.w2[r][b][0], w2);
-      }
-#pragma unroll
-      for (int h = 0; h < NH; ++h) pb[h] = -0.5f * (pb[h] + __shfl_xor_sync(0xffffffffu, pb[h], 16));
-      if (lane < 16) store_heads(&M.pb[warp][b][0], pb);
-    }
-    __syncthreads();
-
-    if (pass == 0) {
-#pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        base[h] = 0.0f;
-#pragma unroll
-        for (int t = 0; t < TOK; ++t) acc[t][h] = 0.0f;
-      }
-    }
-#pragma unroll
-    for (int w = 0; w < SCAN_WARPS; ++w) {
-      float pb[NH];
-      load_heads(&M.pb[w][myb][0], pb);
-#pragma unroll
-      for (int h = 0; h < NH; ++h) base[h] += pb[h];
-    }
-
-    // ---- one predicated add per (token, row, head)
-    {
-      const unsigned char* my_bytes = reinterpret_cast<const unsigned char*>(&M.words[buf][0][myb]) + oct;
-      const float* my_w = &M.w2[0][myb][0];
-#pragma unroll 4
-      for (int r = 0; r < sc; ++r) {
-        const uint32_t bits = my_bytes[r * (TILE_BLOCKS * 8)];
-        float w[NH];
-        load_heads(my_w + r * (TILE_BLOCKS * NH), w);
-        add_if<1>(acc[0], bits, w);
-        add_if<2>(acc[1], bits, w);
-        add_if<4>(acc[2], bits, w);
-        add_if<8>(acc[3], bits, w);
-        add_if<16>(acc[4], bits, w);
-        add_if<32>(acc[5], bits, w);
-        add_if<64>(acc[6], bits, w);
-        add_if<128>(acc[7], bits, w);
-      }
-    }
-
-    if (pass == npass - 1) {
-      // ---- scores of my eight tokens: base + what the set bits added
-      float v[NH][TOK];
-#pragma unroll
-      for (int t = 0; t < TOK; ++t)
-#pragma unroll
-        for (int h = 0; h < NH; ++h) v[h][t] = acc[t][h] + base[h];
+    auto compute = [&](auto tbc) {
+      constexpr int TB = decltype(tbc)::value;
+      using GE = Geo<TB>;
+      constexpr int BW = TB / WARPS;                           // blocks per warp and stage
+      const int s0 = pass * GE::ROWS, sc = min(GE::ROWS, nrows - s0), nks = (sc + 15) >> 4, ks0 = s0 >> 4;
+      const int blk0 = first_block(g) + u * TB;
       const uint32_t n = (uint32_t)B.n[item];                  // n < 2^31
-      const int blk0 = first_block(g);
-      const bool have_block = blk0 + myb < (n + FATHOM_BLOCK - 1) / FATHOM_BLOCK;
-      const uint32_t tok = (uint32_t)(blk0 + myb) * FATHOM_BLOCK + oct * TOK;                // my first token
-
-      if (MODE != 2) {
-        if (have_block) {
-          const uint32_t dst = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + myb * FATHOM_BLOCK + oct * TOK : tok;
+#pragma unroll 1
+      for (int i = 0; i < BW; ++i) {
+        const int b = warp * BW + i;                           // my block within the sub-tile
+        if (pass == 0) {
 #pragma unroll
-          for (int h = 0; h < NH; ++h) {
-            float* row = B.scores[item] + (size_t)(h0 + h) * (size_t)B.score_stride[item] + dst;
-            if (tok + TOK <= n) {
-              *reinterpret_cast<float4*>(row) = make_float4(v[h][0], v[h][1], v[h][2], v[h][3]);
-              *reinterpret_cast<float4*>(row + 4) = make_float4(v[h][4], v[h][5], v[h][6], v[h][7]);
-            } else {
-#pragma unroll
-              for (int t = 0; t < TOK; ++t)
-                if (tok + t < n) row[t] = v[h][t];
-            }
-          }
+          for (int j = 0; j < 4; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f;
         }
-      } else {
-        // candidates of this warp's 256 tokens, per head, collected in the (now idle) weight memory and appended to
-        // the head's global list; entry = (score bits, token)
-        constexpr int LIST = (int)(sizeof(M.w2) / sizeof(uint2)) / SCAN_WARPS / NH;    // entries per warp and head
-        __syncthreads();                                                   // every warp is done with the weights
-        uint2* list = reinterpret_cast<uint2*>(&M.w2[0][0][0]) + warp * (LIST * NH);
-        uint32_t* cnt = M.cnt[warp];
-        if (lane < NH) cnt[lane] = 0u;
-        __syncwarp();
-        if (have_block) {
+        // my byte (tokens 8 gq .. 8 gq + 7) of the plane words and the scales of rows 2 t4, 2 t4 + 1 (+ 8, + 9) of every 16
+        const unsigned char* wp = M.words[buf] + (2 * t4) * GE::ROW_BYTES + b * 8 + gq;
+        const uint16_t* sp = reinterpret_cast<const uint16_t*>(M.scale[buf]) + (2 * t4) * GE::SCALE_ELEMS + b;
+#pragma unroll 1
+        for (int ks = 0; ks < nks; ++ks) {
+          const uint2 bf = M.bfr[ks0 + ks][lane];
+          const uint32_t x0 = __byte_perm(wp[0], wp[GE::ROW_BYTES], 0x5410);
+          const uint32_t x1 = __byte_perm(wp[8 * GE::ROW_BYTES], wp[9 * GE::ROW_BYTES], 0x5410);
+          const uint32_t S0 = __byte_perm(sp[0], sp[GE::SCALE_ELEMS], 0x5410);
+          const uint32_t S1 = __byte_perm(sp[8 * GE::SCALE_ELEMS], sp[9 * GE::SCALE_ELEMS], 0x5410);
+          // slice j: mma row gq = token 8 gq + 2 j, row gq + 8 = token 8 gq + 2 j + 1
+          mma_16816(acc[0], signed_pair<15>(S0, x0), signed_pair<14>(S0, x0), signed_pair<15>(S1, x1), signed_pair<14>(S1, x1), bf.x, bf.y);
+          mma_16816(acc[1], signed_pair<13>(S0, x0), signed_pair<12>(S0, x0), signed_pair<13>(S1, x1), signed_pair<12>(S1, x1), bf.x, bf.y);
+          mma_16816(acc[2], signed_pair<11>(S0, x0), signed_pair<10>(S0, x0), signed_pair<11>(S1, x1), signed_pair<10>(S1, x1), bf.x, bf.y);
+          mma_16816(acc[3], signed_pair<9>(S0, x0), signed_pair<8>(S0, x0), signed_pair<9>(S1, x1), signed_pair<8>(S1, x1), bf.x, bf.y);
+          wp += 16 * GE::ROW_BYTES;
+          sp += 16 * GE::SCALE_ELEMS;
+        }
+        if (pass != npass - 1) continue;
+
+        // ---- scores of head t4 for my eight tokens: columns 2 t4 (head part) and 2 t4 + 1 (tail part)
+        float v[8];
 #pragma unroll
-          for (int t = 0; t < TOK; ++t) {
-            const long long ti = (long long)tok + t;
-            const bool elig = ti < n && ti >= fz.sink_end && ti < fz.local_begin;
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] = fmaf(acc[j][1], hs_tail, acc[j][0] * hs);
+          v[2 * j + 1] = fmaf(acc[j][3], hs_tail, acc[j][2] * hs);
+        }
+        const bool have_block = blk0 + b < nb_item;
+        const uint32_t tok = (uint32_t)(blk0 + b) * FATHOM_BLOCK + gq * 8;                     // my first token
+        if (t4 >= NH || !have_block) continue;
+        if (MODE != 2) {
+          const uint32_t dst = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok;
+          float* row = B.scores[item] + (size_t)(h0 + t4) * (size_t)B.score_stride[item] + dst;
+          if (tok + 8 <= n) {
+            *reinterpret_cast<float4*>(row) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(row + 4) = make_float4(v[4], v[5], v[6], v[7]);
+          } else {
 #pragma unroll
-            for (int h = 0; h < NH; ++h) {
-              if (elig && v[h][t] >= M.thr[h]) {
-                const uint32_t p = atomicAdd(&cnt[h], 1u);
-                if (p < (uint32_t)LIST) list[h * LIST + p] = make_uint2(__float_as_uint(v[h][t]), (uint32_t)ti);
-                else {                                                   // list full: straight to the global list
-                  const uint32_t gp = atomicAdd(&fz.cand_count[h0 + h], 1u);
-                  if ((long long)gp < fz.capacity) {
-                    fz.cand_score[(size_t)(h0 + h) * fz.capacity + gp] = v[h][t];
-                    fz.cand_idx[(size_t)(h0 + h) * fz.capacity + gp] = (int32_t)ti;
+            for (int x = 0; x < 8; ++x)
+              if (tok + x < n) row[x] = v[x];
+          }
+        } else {
+          // candidates: (score, token) pairs appended to the head's list; their order in the list is irrelevant
+          uint32_t m = 0u;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) m |= (v[x] >= my_thr ? 1u : 0u) << x;
+          if (m) {
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+              const long long ti = (long long)tok + x;
+              if (!(ti < (long long)n && ti >= fz.sink_end && ti < fz.local_begin)) m &= ~(1u << x);
+            }
+            if (m) {
+              uint32_t at = atomicAdd(&fz.cand_count[h0 + t4], (uint32_t)__popc(m));
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                if ((m >> x) & 1u) {
+                  if ((long long)at < fz.capacity) {
+                    fz.cand_score[(size_t)(h0 + t4) * fz.capacity + at] = v[x];
+                    fz.cand_idx[(size_t)(h0 + t4) * fz.capacity + at] = (int32_t)(tok + x);
                   }
+                  ++at;
                 }
               }
             }
           }
         }
-        // one global atomic per (tile, head): the four warps' counts are summed, the slice is reserved once
-        __syncwarp();
-        if (lane < NH) M.wcnt[warp][lane] = min(cnt[lane], (uint32_t)LIST);
-        __syncthreads();
-        if (tid < NH) {
-          uint32_t tot = 0;
-#pragma unroll
-          for (int w = 0; w < SCAN_WARPS; ++w) tot += M.wcnt[w][tid];
-          M.cbase[tid] = tot ? atomicAdd(&fz.cand_count[h0 + tid], tot) : 0u;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          const uint32_t c = M.wcnt[warp][h];
-          uint32_t at = M.cbase[h];
-          for (int w = 0; w < warp; ++w) at += M.wcnt[w][h];
-          for (uint32_t e = lane; e < c; e += 32) {
-            const uint2 it = list[h * LIST + e];
-            if ((long long)(at + e) < fz.capacity) {
-              fz.cand_score[(size_t)(h0 + h) * fz.capacity + at + e] = __uint_as_float(it.x);
-              fz.cand_idx[(size_t)(h0 + h) * fz.capacity + at + e] = (int32_t)it.y;
-            }
-          }
-        }
       }
-    }
+    };
+    if (tb == 16) compute(std::integral_constant<int, 16>());
+    else if (tb == 8) compute(std::integral_constant<int, 8>());
+    else compute(std::integral_constant<int, 4>());
 
     if (!more) break;
     __syncthreads();                                           // every warp is done with this stage's buffers
     g = g_next;
+    u = u_next;
     pass = pass_next;
     buf ^= 1;
     if (!same_item) {                                          // first tile of another session: nothing was fetched ahead
       enter_item(g);
-      prefetch(g, 0, buf);
+      prefetch(g, 0, 0, buf);
     }
   }
-}
-
-// Whether the planes are read over the host link (pinned host memory mapped into the device's address space)
-static bool planes_in_host_memory(const void* planes) {
-  cudaPointerAttributes a;
-  if (cudaPointerGetAttributes(&a, planes) != cudaSuccess) { cudaGetLastError(); return false; }
-  return a.type == cudaMemoryTypeHost;
-}
-
-// CTAs per plan.  Planes in HBM: as many as are resident at once (and no more than there are tiles), each walking
-// several tiles.  Planes read over the host link: one CTA per tile, so that CTAs become resident in block order - all
-// tiles of one plan before the next plan's - and the link sees a few long sequential streams (48 rows of one KV head)
-// instead of eight times as many short ones; the link, not instruction issue, bounds that scan.
-static int scan_ctas_per_plan(long long tiles, int plans, bool host_planes) {
-  if (const char* e = getenv("FATHOM_SCAN_CTAS_PER_PLAN")) {   // tests and tuning: a fixed number (read at every call)
-    const long long v = atoll(e);
-    if (v >= 1) return (int)(v < tiles ? v : tiles);
-  }
-  if (host_planes) return (int)tiles;
-  static int sms[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-  if (!sms[dev]) {
-    int v = 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-    sms[dev] = v;
-  }
-  long long x = (long long)sms[dev] * CTAS_PER_SM / plans;
-  if (x < 1) x = 1;
-  return (int)(x < tiles ? x : tiles);
 }
 
 template <int NH, int MODE>
@@ -435,19 +358,26 @@ int launch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const f
   const long long tiles = B.tile_end[B.items - 1];
   if (tiles <= 0) return FATHOM_OK;
   const int plans = Hq / NH;
-  dim3 grid((unsigned)scan_ctas_per_plan(tiles, plans, planes_in_host_memory(B.planes[0])), (unsigned)plans);
+  dim3 grid((unsigned)fathom_scan_grid_ctas(tiles, plans, fathom_planes_in_host_memory(B.planes[0]), CTAS_PER_SM), (unsigned)plans);
   if (dependent) {                                            // may become resident while the previous kernel of the stream runs
-    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(SCAN_THREADS), 0, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
+    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(THREADS), 0, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
       return FATHOM_ERR_CUDA;
     return FATHOM_OK;
   }
-  scan_kernel<NH, MODE><<<grid, SCAN_THREADS, 0, st>>>(B, Hq / Hkv, heads_per_plan, fz);
+  scan_kernel<NH, MODE><<<grid, THREADS, 0, st>>>(B, Hq / Hkv, heads_per_plan, fz);
   return FATHOM_OK;
+}
+
+// FATHOM_SCAN_PATH=simt (read once) selects the CUDA-core kernel of scan_simt.cu for every scan of the process
+bool simt_path() {
+  static const bool v = [] { const char* e = getenv("FATHOM_SCAN_PATH"); return e && strcmp(e, "simt") == 0; }();
+  return v;
 }
 
 template <int MODE>
 int dispatch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const fathom_scan_fuse& fz, bool dependent,
                   cudaStream_t st) {
+  if (simt_path()) return fathom_scan_simt_dispatch(MODE, B, Hkv, Hq, heads_per_plan, fz, dependent, st);
   switch (heads_per_plan) {
     case 1: return launch_scan<1, MODE>(B, Hkv, Hq, 1, fz, dependent, st);
     case 2: return launch_scan<2, MODE>(B, Hkv, Hq, 2, fz, dependent, st);
@@ -469,7 +399,34 @@ ScanBatch single_item(const fathom_layout* L, const uint64_t* planes, const uint
   return B;
 }
 
+int g_ctas_override = 0;                                       // fathom_scan_set_ctas_per_plan
+
 }  // namespace
+
+// Whether the planes are read over the host link (pinned host memory mapped into the device's address space)
+bool fathom_planes_in_host_memory(const void* planes) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, planes) != cudaSuccess) { cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost;
+}
+
+int fathom_scan_ctas_override() { return g_ctas_override; }
+
+int fathom_scan_grid_ctas(long long tiles, int plans, bool host_planes, int ctas_per_sm) {
+  if (g_ctas_override >= 1) return (int)(g_ctas_override < tiles ? g_ctas_override : tiles);
+  if (host_planes) return (int)tiles;
+  static int sms[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  if (!sms[dev]) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    sms[dev] = v;
+  }
+  long long x = (long long)sms[dev] * ctas_per_sm / plans;
+  if (x < 1) x = 1;
+  return (int)(x < tiles ? x : tiles);
+}
 
 int fathom_scan_tile_tokens() { return TILE_BLOCKS * FATHOM_BLOCK; }
 
@@ -486,6 +443,11 @@ int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, co
                               const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st) {
   return dispatch_scan<2>(single_item(L, planes, scales, q, depth, nullptr, 0, 1), L->n_kv_heads, L->n_q_heads, heads_per_plan, fz,
                           false, st);
+}
+
+extern "C" int fathom_scan_set_ctas_per_plan(int ctas) {
+  g_ctas_override = ctas > 0 ? ctas : 0;
+  return FATHOM_OK;
 }
 
 extern "C" int fathom_scan(fathom_ctx* ctx, const fathom_layout* L, const uint64_t* planes, const uint16_t* scales,

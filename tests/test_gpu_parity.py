@@ -141,14 +141,18 @@ def test_planes_in_pinned_host_memory_give_identical_scores():
 
 @pytest.mark.parametrize("n,Hkv,Hq,B,hpp,ctas", [(70001, 2, 8, 136, 4, 5), (33000, 2, 8, 48, 1, 3), (40000, 1, 8, 200, 8, 1),
                                                  (5000, 2, 8, 80, 2, 2)])
-def test_scan_with_few_persistent_ctas_walking_many_tiles(n, Hkv, Hq, B, hpp, ctas, monkeypatch):
+def test_scan_with_few_persistent_ctas_walking_many_tiles(n, Hkv, Hq, B, hpp, ctas):
     """A CTA of the scan walks several tiles and several passes per tile (its next tile's planes fetched ahead into the
     other half of its double buffer): with only `ctas` CTAs per plan the scores are those of the oracle, and bit for
     bit those of the default launch."""
+    from paper_2609_17652_b200 import binding as fb
     L = make_layer(n, Hkv=Hkv, Hq=Hq, seed=21, device="cuda")
     a = run_gpu(L, B, 64, hpp, stages=("scan",))
-    monkeypatch.setenv("FATHOM_SCAN_CTAS_PER_PLAN", str(ctas))
-    b = run_gpu(L, B, 64, hpp, stages=("scan",))
+    fb.fathom_scan_set_ctas_per_plan(ctas)
+    try:
+        b = run_gpu(L, B, 64, hpp, stages=("scan",))
+    finally:
+        fb.fathom_scan_set_ctas_per_plan(0)
     assert np.array_equal(a["scores"], b["scores"])
     H = host(L)
     planes, scales = O.build_planes(H["K"])
@@ -562,7 +566,7 @@ def test_rotated_store_in_one_call_equals_rotate_then_build(n, dtype):
 
 
 @pytest.mark.parametrize("hpp,host,ctas", [(4, False, None), (1, False, None), (4, True, None), (4, False, 7), (2, True, 3)])
-def test_batched_scan_equals_one_scan_per_session(hpp, host, ctas, monkeypatch):
+def test_batched_scan_equals_one_scan_per_session(hpp, host, ctas):
     """fathom_scan_batch over ragged sessions (lengths that are not multiples of 64 or of the 1024-token tile, one of
     a single token) gives bit for bit the scores of one fathom_scan per session, with the planes in HBM or in pinned
     host memory, more sessions than one launch takes (33 > 32), and with so few CTAs that each crosses from one session
@@ -591,10 +595,12 @@ def test_batched_scan_equals_one_scan_per_session(hpp, host, ctas, monkeypatch):
         many = torch.full((Hq, lay.score_stride), float("nan"), device="cuda")
         items.append((lay, planes, scales, L.q, depth, many))
         singles.append((one, n))
-    if ctas:                                          # few CTAs per plan: each walks tiles of several sessions in turn
-        monkeypatch.setenv("FATHOM_SCAN_CTAS_PER_PLAN", str(ctas))
-    ctx.fathom_scan_batch(items, hpp)
-    torch.cuda.synchronize()
+    fb.fathom_scan_set_ctas_per_plan(ctas or 0)         # few CTAs per plan: each walks tiles of several sessions in turn
+    try:
+        ctx.fathom_scan_batch(items, hpp)
+        torch.cuda.synchronize()
+    finally:
+        fb.fathom_scan_set_ctas_per_plan(0)
     for (lay, _, _, _, _, many), (one, n) in zip(items, singles):
         assert torch.equal(many[:, :n], one[:, :n])
         assert torch.isnan(many[:, n:]).all()                                # padding untouched
