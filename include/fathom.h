@@ -66,7 +66,7 @@ typedef struct {
   int32_t d;                   /* channels per head; must be 128 */
   int32_t reserved;            /* set to 0 */
   int64_t n;                   /* tokens, n >= 1 */
-  int64_t plane_stride_words;  /* uint64 words per (KV head, channel, plane) row; >= nb, multiple of 2 (16 B), < 2^32 */
+  int64_t plane_stride_words;  /* uint64 words per (KV head, channel, plane) row; >= nb, multiple of 2 (16 B), < 2^24 */
   int64_t scale_stride;        /* fp16 elements per (KV head, channel) row; >= nb, multiple of 8 (16 B), < 2^32 */
   int64_t score_stride;        /* floats per query-head score row; >= n, multiple of 4 (16 B) */
 } fathom_layout;

@@ -12,7 +12,7 @@ int fathom_check_layout(const fathom_layout* L) {
   const int64_t nb = fathom_nblocks(L->n);
   if (L->plane_stride_words < nb || L->scale_stride < nb || L->score_stride < L->n) return FATHOM_ERR_INVALID_ARG;
   if (L->plane_stride_words % 2 != 0 || L->scale_stride % 8 != 0 || L->score_stride % 4 != 0) return FATHOM_ERR_ALIGNMENT;
-  if (L->plane_stride_words > (int64_t)0xffffffff || L->scale_stride > (int64_t)0xffffffff) return FATHOM_ERR_UNSUPPORTED;   // 32-bit strides
+  if (L->plane_stride_words >= ((int64_t)1 << 24) || L->scale_stride > (int64_t)0xffffffff) return FATHOM_ERR_UNSUPPORTED;   // row offsets in 16-byte units fit 32 bits
   return FATHOM_OK;
 }
 

@@ -40,10 +40,13 @@ namespace {
 constexpr int THREADS = 128, WARPS = 4;
 constexpr int TILE_BLOCKS = FATHOM_SCAN_TILE_BLOCKS;
 constexpr int MAX_ROWS = FATHOM_D * FATHOM_NPLANES;          // 512 (channel, plane) pairs
-constexpr int MAX_KSTEPS = MAX_ROWS / 16;                    // 16 rows per mma
+constexpr int STAGE_KSTEPS = 10;                             // 16 rows per mma; a stage holds at most 160 rows
 constexpr int WORD_STAGE_BYTES = 7680;                       // staged plane words of one stage (padded rows)
 constexpr int SCALE_STAGE_BYTES = 4608;                      // staged fp16 scales of one stage (padded rows)
-constexpr int CTAS_PER_SM = 6;
+#ifndef FATHOM_SCAN_CTAS_PER_SM
+#define FATHOM_SCAN_CTAS_PER_SM 6
+#endif
+constexpr int CTAS_PER_SM = FATHOM_SCAN_CTAS_PER_SM;
 
 // Stage geometry for sub-tiles of TB blocks.  The row pitches are padded so that the four lanes of a quad, which read
 // rows two apart, hit different banks (plane bytes: pitch / 4 = 4 mod 32 for TB = 16, ...).
@@ -55,15 +58,21 @@ struct Geo {
   static_assert(ROWS * ROW_BYTES <= WORD_STAGE_BYTES && ROWS * SCALE_ELEMS * 2 <= SCALE_STAGE_BYTES, "stage buffers too small");
 };
 
+constexpr int CAND_CAP = 32;                                 // MODE 2: candidates a warp keeps per head before it appends them to the global lists
+
+template <int MODE>
 struct alignas(16) Smem {
-  uint16_t row_ch[MAX_ROWS];                                  // channel of active row r
-  uint8_t row_pl[MAX_ROWS];                                   // plane of active row r
+  uint16_t row_id[MAX_ROWS];                                  // active row r: channel * 4 + plane
+  uint32_t woff[MAX_ROWS];                                    // where its plane words start within the KV head, in 16-byte units
+  uint32_t soff[MAX_ROWS];                                    // where its channel's scales start within the KV head, in 16-byte units
   int nrows;
   int warp_tot[WARPS];
   float wmax[WARPS][4];                                       // per warp: max_j |q_hj| of its channels
   float hscale[4], hinv[4];                                   // E_h and 1 / E_h
   float thr[4];                                               // MODE 2: score a token must reach, per head
-  alignas(16) uint2 bfr[MAX_KSTEPS][32];                      // right operand: per 16 rows, the two B registers of every lane
+  uint32_t ccnt[WARPS][4];                                    // MODE 2: candidates in the warp's lists
+  uint2 cand[MODE == 2 ? WARPS * 4 * CAND_CAP : 1];           // MODE 2: (score bits, token) per warp and head
+  alignas(16) uint2 bfr[STAGE_KSTEPS][32];                    // right operand of the rows of a pass: per 16 rows, the two B registers of every lane
   alignas(16) unsigned char words[2][WORD_STAGE_BYTES];       // staged plane words, double buffered
   alignas(16) unsigned char scale[2][SCALE_STAGE_BYTES];      // staged fp16 scales, double buffered
 };
@@ -80,6 +89,45 @@ __device__ __forceinline__ uint32_t signed_pair(uint32_t pair, uint32_t bytes) {
   return pair ^ (~(bytes << SH) & 0x80008000u);
 }
 
+// eight consecutive scores: one 32-byte store where the address allows it (a whole sector per lane), else two of 16 bytes
+__device__ __forceinline__ void store_scores8(float* row, const float (&v)[8]) {
+  if ((reinterpret_cast<uintptr_t>(row) & 31u) == 0) {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(row), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]),
+                 "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+  } else {
+    *reinterpret_cast<float4*>(row) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(row + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// One block (64 tokens: this lane's eight are byte `wp[0]` of every staged plane word) times the rows of a stage, 16 rows per
+// step: the lane's two row pairs of a step are rows 2 t4, 2 t4 + 1 and 2 t4 + 8, 2 t4 + 9 of the sixteen.  NKS > 0: that
+// many steps, unrolled (the loads of all steps are in flight at once); NKS = 0: `nks` steps in a loop.
+// Slice j of the accumulators: mma row gq = token 8 gq + 2 j, row gq + 8 = token 8 gq + 2 j + 1.
+template <int ROW_BYTES, int SCALE_ELEMS, int NKS>
+__device__ __forceinline__ void mma_rows(float (&acc)[4][4], const unsigned char* wp, const uint16_t* sp, const uint2* bfr_lane, int nks) {
+  auto step = [&](int ks) {
+    const uint2 bf = bfr_lane[ks * 32];
+    const unsigned char* w = wp + ks * (16 * ROW_BYTES);
+    const uint16_t* sc = sp + ks * (16 * SCALE_ELEMS);
+    const uint32_t x0 = __byte_perm(w[0], w[ROW_BYTES], 0x5410);
+    const uint32_t x1 = __byte_perm(w[8 * ROW_BYTES], w[9 * ROW_BYTES], 0x5410);
+    const uint32_t S0 = __byte_perm(sc[0], sc[SCALE_ELEMS], 0x5410);
+    const uint32_t S1 = __byte_perm(sc[8 * SCALE_ELEMS], sc[9 * SCALE_ELEMS], 0x5410);
+    mma_16816(acc[0], signed_pair<15>(S0, x0), signed_pair<14>(S0, x0), signed_pair<15>(S1, x1), signed_pair<14>(S1, x1), bf.x, bf.y);
+    mma_16816(acc[1], signed_pair<13>(S0, x0), signed_pair<12>(S0, x0), signed_pair<13>(S1, x1), signed_pair<12>(S1, x1), bf.x, bf.y);
+    mma_16816(acc[2], signed_pair<11>(S0, x0), signed_pair<10>(S0, x0), signed_pair<11>(S1, x1), signed_pair<10>(S1, x1), bf.x, bf.y);
+    mma_16816(acc[3], signed_pair<9>(S0, x0), signed_pair<8>(S0, x0), signed_pair<9>(S1, x1), signed_pair<8>(S1, x1), bf.x, bf.y);
+  };
+  if (NKS > 0) {
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) step(ks);
+  } else {
+#pragma unroll 1
+    for (int ks = 0; ks < nks; ++ks) step(ks);
+  }
+}
+
 // MODE 0: scores of every token are written (fathom_scan, fathom_scan_batch).
 // MODE 1: only every tile_step-th tile is scanned and its scores are written compactly (tile i of the launch at
 //         token positions 1024 i ..) - the sample from which fathom_scan_topk derives a safe threshold.
@@ -89,7 +137,7 @@ __device__ __forceinline__ uint32_t signed_pair(uint32_t pair, uint32_t bytes) {
 template <int NH, int MODE>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
 scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fathom_scan_fuse fz) {
-  __shared__ Smem M;
+  __shared__ Smem<MODE> M;
 
   FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
@@ -102,11 +150,41 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
   const int kv = h0 / G;
   const int myh = t4 < NH ? t4 : 0;                            // the head whose scores this lane receives (lanes t4 >= NH: none)
+  if (MODE == 2 && tid < WARPS * 4) (&M.ccnt[0][0])[tid] = 0u;
   if (MODE == 2 && tid < NH)                                   // read after the barriers of the first item's row list
     M.thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : fathom_bin_lower_edge(fz.state[(h0 + tid) * 8]);
 
   int item = -1, nrows = 0, tb = TILE_BLOCKS, rows_stage = Geo<16>::ROWS, npass = 1, nb_item = 0;
   float hs = 1.0f, hs_tail = 0.0f;                             // E of my head and E 2^-11
+
+  // ---- right operand of the rows of pass `pass` (made visible by the barrier that precedes the pass's arithmetic): entry
+  //      (kstep, lane, i) holds rows 16 kstep + 2 (lane & 3) + 8 i and the next one of the pass, column lane >> 2 = (head, part)
+  auto fill_bfr = [&](int pass) {
+    const int s0 = pass * rows_stage, sc = min(rows_stage, nrows - s0);
+    const int entries = ((sc + 15) >> 4) * 64;
+    for (int e = tid; e < entries; e += THREADS) {
+      const int ks = e >> 6, ln = (e >> 1) & 31, i = e & 1;
+      const int col = ln >> 2, head = col >> 1, part = col & 1;
+      const int r0 = s0 + ks * 16 + 2 * (ln & 3) + 8 * i;
+      uint32_t packed = 0u;
+      if (head < NH) {
+        const float inv = M.hinv[head];
+#pragma unroll
+        for (int z = 0; z < 2; ++z) {
+          const int r = r0 + z;
+          float v = 0.0f;
+          if (r < nrows) {
+            const int id = M.row_id[r];
+            v = __ldg(B.q[item] + (size_t)(h0 + head) * FATHOM_D + (id >> 2)) * inv * __int_as_float((129 - (id & 3)) << 23);
+          }
+          const __half hi = __float2half_rn(v);
+          const __half out = part ? __float2half_rn((v - __half2float(hi)) * 2048.0f) : hi;
+          packed |= (uint32_t)__half_as_ushort(out) << (16 * z);
+        }
+      }
+      reinterpret_cast<uint32_t*>(&M.bfr[ks][ln])[i] = packed;
+    }
+  };
 
   // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), the
   //      heads' power-of-two scales and the right operand of every 16 rows
@@ -136,7 +214,12 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     int before = 0;
     for (int w = 0; w < warp; ++w) before += M.warp_tot[w];
     const int start = before + incl - t;
-    for (int p = 0; p < t; ++p) { M.row_ch[start + p] = (uint16_t)tid; M.row_pl[start + p] = (uint8_t)p; }
+    const uint32_t half_stride = (uint32_t)(B.plane_stride[it] >> 1), eighth_stride = (uint32_t)(B.scale_stride[it] >> 3);
+    for (int p = 0; p < t; ++p) {                              // (511 * half_stride < 2^32: fathom_check_layout)
+      M.row_id[start + p] = (uint16_t)(tid * FATHOM_NPLANES + p);
+      M.woff[start + p] = (uint32_t)(tid * FATHOM_NPLANES + p) * half_stride;
+      M.soff[start + p] = (uint32_t)tid * eighth_stride;
+    }
     if (tid == FATHOM_D - 1) M.nrows = before + incl;
     if (tid < NH) {                                            // E = 2^floor(log2 max|q|), kept inside the normal range
       float m = 0.0f;
@@ -155,28 +238,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     npass = nrows > rows_stage ? (nrows + rows_stage - 1) / rows_stage : 1;
     hs = M.hscale[myh];
     hs_tail = hs * 4.8828125e-4f;                              // 2^-11
-    // right operand (made visible by the barrier that precedes the first stage's arithmetic): entry (kstep, lane, i)
-    // holds rows 16 kstep + 2 (lane & 3) + 8 i and the next one, column lane >> 2 = (head, part)
-    const int entries = ((nrows + 15) >> 4) * 64;
-    for (int e = tid; e < entries; e += THREADS) {
-      const int ks = e >> 6, ln = (e >> 1) & 31, i = e & 1;
-      const int col = ln >> 2, head = col >> 1, part = col & 1;
-      const int r0 = ks * 16 + 2 * (ln & 3) + 8 * i;
-      uint32_t packed = 0u;
-      if (head < NH) {
-        const float inv = M.hinv[head];
-#pragma unroll
-        for (int z = 0; z < 2; ++z) {
-          const int r = r0 + z;
-          float v = 0.0f;
-          if (r < nrows) v = __ldg(B.q[it] + (size_t)(h0 + head) * FATHOM_D + M.row_ch[r]) * inv * __int_as_float((129 - (int)M.row_pl[r]) << 23);
-          const __half hi = __float2half_rn(v);
-          const __half out = part ? __float2half_rn((v - __half2float(hi)) * 2048.0f) : hi;
-          packed |= (uint32_t)__half_as_ushort(out) << (16 * z);
-        }
-      }
-      reinterpret_cast<uint32_t*>(&M.bfr[ks][ln])[i] = packed;
-    }
+    fill_bfr(0);
   };
 
   // first block of launch tile `tile` within its session
@@ -190,34 +252,30 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     const int blk0 = first_block(tile) + u * tb;
     const int nblk = min(tb, nb_item - blk0);                  // >= 1: stages past the last block are never entered
     const int s0 = pass * rows_stage, sc = min(rows_stage, nrows - s0);
-    // (strides are below 2^32 elements: one 32 x 32 -> 64-bit multiply per address)
-    const uint32_t plane_stride = (uint32_t)B.plane_stride[item], scale_stride = (uint32_t)B.scale_stride[item];
-    const uint64_t* planes_kv = B.planes[item] + (uint64_t)(kv * FATHOM_D * FATHOM_NPLANES) * plane_stride + blk0;
-    const uint16_t* scales_kv = B.scales[item] + (uint64_t)(kv * FATHOM_D) * scale_stride + blk0;
+    // 16-byte units throughout: plane_stride is even, scale_stride a multiple of 8, blk0 a multiple of tb
+    const uint4* planes_kv = reinterpret_cast<const uint4*>(B.planes[item]) +
+                             (uint64_t)(kv * FATHOM_D * FATHOM_NPLANES) * (uint64_t)(B.plane_stride[item] >> 1) + (blk0 >> 1);
+    const unsigned char* scales_kv = reinterpret_cast<const unsigned char*>(B.scales[item]) +
+                                     (uint64_t)(kv * FATHOM_D) * (uint64_t)B.scale_stride[item] * 2 + (uint64_t)blk0 * 2;
     const int sh = tb == 16 ? 3 : (tb == 8 ? 2 : 1);           // 16-byte copies per row of plane words: tb / 2
     const int row_bytes = 8 * tb + 16;
     unsigned char* wdst = M.words[buf];
-    for (int e = tid; e < (sc << sh); e += THREADS) {
-      const int r = e >> sh, c = e & ((1 << sh) - 1);
-      const uint32_t row = (uint32_t)M.row_ch[s0 + r] * FATHOM_NPLANES + M.row_pl[s0 + r];
-      const bool valid = 2 * c < nblk;
-      fathom_copy_async<16>(wdst + r * row_bytes + c * 16,
-                            valid ? (const void*)(planes_kv + (uint64_t)row * plane_stride + 2 * c) : (const void*)B.planes[item], valid);
-    }
+    const int c = tid & ((1 << sh) - 1);                       // my 16-byte column of every row I copy
+    const bool valid = 2 * c < nblk;
+    for (int r = tid >> sh; r < sc; r += THREADS >> sh)
+      fathom_copy_async<16>(wdst + r * row_bytes + c * 16, valid ? planes_kv + M.woff[s0 + r] + c : planes_kv, valid);
     unsigned char* sdst = M.scale[buf];
     if (tb == 16) {
-      for (int e = tid; e < sc * 2; e += THREADS) {
-        const int r = e >> 1, c = e & 1;
-        const bool valid = 8 * c < nblk;
-        fathom_copy_async<16>(sdst + r * (Geo<16>::SCALE_ELEMS * 2) + c * 16,
-                              valid ? (const void*)(scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride + 8 * c) : (const void*)B.scales[item], valid);
-      }
+      const int cs = tid & 1;
+      const bool vs = 8 * cs < nblk;
+      for (int r = tid >> 1; r < sc; r += THREADS >> 1)
+        fathom_copy_async<16>(sdst + r * (Geo<16>::SCALE_ELEMS * 2) + cs * 16, vs ? scales_kv + (uint64_t)M.soff[s0 + r] * 16 + cs * 16 : scales_kv, vs);
     } else if (tb == 8) {
       for (int r = tid; r < sc; r += THREADS)
-        fathom_copy_async<16>(sdst + r * (Geo<8>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride, true);
+        fathom_copy_async<16>(sdst + r * (Geo<8>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.soff[s0 + r] * 16, true);
     } else {
       for (int r = tid; r < sc; r += THREADS)
-        fathom_copy_async<8>(sdst + r * (Geo<4>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.row_ch[s0 + r] * scale_stride, true);
+        fathom_copy_async<8>(sdst + r * (Geo<4>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.soff[s0 + r] * 16, true);
     }
     // rows that pad the last 16: scale 0, so that whatever the stale plane bytes say they contribute +-0
     const int pad = ((sc + 15) & ~15) - sc;
@@ -252,13 +310,144 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     }
     __syncthreads();                                           // this stage's words and scales are in place
 
+    // ---- eight consecutive scores of head t4 (lanes with t4 < NH, tokens of an existing block): tokens tok .. tok + 7 of
+    //      the session, written at position dst of the head's row (MODE 0, 1) or tested against the head's threshold (MODE 2)
+    auto emit = [&](const float (&v)[8], uint32_t tok, uint32_t dst, uint32_t n) {
+      if (MODE != 2) {
+        float* row = B.scores[item] + (size_t)(h0 + t4) * (size_t)B.score_stride[item] + dst;
+        if (tok + 8 <= n) {
+          store_scores8(row, v);
+        } else {
+#pragma unroll
+          for (int x = 0; x < 8; ++x)
+            if (tok + x < n) row[x] = v[x];
+        }
+      } else {
+        // candidates: (score, token) pairs appended to the head's list; their order in the list is irrelevant.  They are
+        // rare (a fraction of a percent of the tokens), so the common path is a maximum and one comparison
+        const float vmax = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
+        if (vmax >= my_thr) {
+          uint32_t m = 0u;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) m |= (v[x] >= my_thr ? 1u : 0u) << x;
+          const uint32_t hi = (uint32_t)(fz.local_begin < (long long)n ? fz.local_begin : (long long)n);   // eligible: lo <= token < hi
+          const uint32_t lo = (uint32_t)(fz.sink_end < (long long)hi ? fz.sink_end : (long long)hi);
+#pragma unroll 1
+          while (m) {
+            const int x = __ffs(m) - 1;
+            m &= m - 1;
+            const uint32_t ti = tok + x;
+            if (ti - lo < hi - lo) {
+              const float a01 = (x & 1) ? v[1] : v[0], a23 = (x & 1) ? v[3] : v[2], a45 = (x & 1) ? v[5] : v[4], a67 = (x & 1) ? v[7] : v[6];
+              const float a03 = (x & 2) ? a23 : a01, a47 = (x & 2) ? a67 : a45;
+              const float val = (x & 4) ? a47 : a03;
+              const uint32_t p = atomicAdd(&M.ccnt[warp][t4], 1u);
+              if (p < (uint32_t)CAND_CAP) {
+                M.cand[(warp * 4 + t4) * CAND_CAP + p] = make_uint2(__float_as_uint(val), ti);
+              } else {                                         // list full (only with a threshold far too low): straight to the global list
+                const uint32_t at = atomicAdd(&fz.cand_count[h0 + t4], 1u);
+                if ((long long)at < fz.capacity) {
+                  fz.cand_score[(size_t)(h0 + t4) * fz.capacity + at] = val;
+                  fz.cand_idx[(size_t)(h0 + t4) * fz.capacity + at] = (int32_t)ti;
+                }
+              }
+            }
+          }
+        }
+      }
+    };
+
+    // ---- MODE 2, whole warp, after the last emit of a stage: the warp's lists go to the heads' global lists, one atomic
+    //      per head (same-address atomics are what the global lists can take least of)
+    auto flush_candidates = [&]() {
+      if (MODE != 2) return;
+      __syncwarp();
+      uint32_t c = 0u, base = 0u;
+      if (lane < NH) {
+        c = min(M.ccnt[warp][lane], (uint32_t)CAND_CAP);
+        if (c) base = atomicAdd(&fz.cand_count[h0 + lane], c);
+      }
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const uint32_t ch = __shfl_sync(0xffffffffu, c, h), bh = __shfl_sync(0xffffffffu, base, h);
+        if (lane < ch && (long long)(bh + lane) < fz.capacity) {
+          const uint2 it = M.cand[(warp * 4 + h) * CAND_CAP + lane];
+          fz.cand_score[(size_t)(h0 + h) * fz.capacity + bh + lane] = __uint_as_float(it.x);
+          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + bh + lane] = (int32_t)it.y;
+        }
+      }
+      __syncwarp();
+      if (lane < 4) M.ccnt[warp][lane] = 0u;
+      __syncwarp();
+    };
+
+    // ---- a whole 16-block stage of NKS x 16 rows, single pass: the warp's four blocks are 256 tokens, and a lane takes 32
+    //      consecutive ones (half a block: ONE 32-bit load per row gives all their bits, and one scale pair per row pair
+    //      serves them all), eight at a time (byte k of the loaded words): slice j of the accumulators then holds
+    //      tokens 8 k + 2 j (mma row gq) and 8 k + 2 j + 1 (row gq + 8) of the lane's 32
+    auto half_blocks = [&](auto nksc, int blk0) {
+      constexpr int NKS = decltype(nksc)::value;
+      using GE = Geo<16>;
+      const int mine = warp * 4 + (gq >> 1);                   // my block of the stage, and my half of it
+      const unsigned char* wp = M.words[buf] + (2 * t4) * GE::ROW_BYTES + mine * 8 + (gq & 1) * 4;
+      const uint16_t* sp = reinterpret_cast<const uint16_t*>(M.scale[buf]) + (2 * t4) * GE::SCALE_ELEMS + mine;
+      uint32_t w[NKS][4], S[NKS][2];
+      uint2 bf[NKS];
+#pragma unroll
+      for (int ks = 0; ks < NKS; ++ks) {
+        bf[ks] = M.bfr[ks][lane];
+        const unsigned char* wk = wp + ks * (16 * GE::ROW_BYTES);
+        w[ks][0] = *reinterpret_cast<const uint32_t*>(wk);
+        w[ks][1] = *reinterpret_cast<const uint32_t*>(wk + GE::ROW_BYTES);
+        w[ks][2] = *reinterpret_cast<const uint32_t*>(wk + 8 * GE::ROW_BYTES);
+        w[ks][3] = *reinterpret_cast<const uint32_t*>(wk + 9 * GE::ROW_BYTES);
+        const uint16_t* sk = sp + ks * (16 * GE::SCALE_ELEMS);
+        S[ks][0] = __byte_perm(sk[0], sk[GE::SCALE_ELEMS], 0x5410);
+        S[ks][1] = __byte_perm(sk[8 * GE::SCALE_ELEMS], sk[9 * GE::SCALE_ELEMS], 0x5410);
+      }
+      const uint32_t n = (uint32_t)B.n[item];
+      const uint32_t tok0 = (uint32_t)(blk0 + mine) * FATHOM_BLOCK + (gq & 1) * 32;      // my first token
+      const uint32_t dst0 = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)mine * FATHOM_BLOCK + (gq & 1) * 32 : tok0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f;
+#pragma unroll
+        for (int ks = 0; ks < NKS; ++ks) {
+          // byte k of the two rows of a pair side by side: bits 0..7 and 16..23 (the other bytes are masked away later)
+          const uint32_t x0 = __byte_perm(w[ks][0], w[ks][1], 0x0400 + 0x0101 * k);
+          const uint32_t x1 = __byte_perm(w[ks][2], w[ks][3], 0x0400 + 0x0101 * k);
+          const uint32_t S0 = S[ks][0], S1 = S[ks][1];
+          mma_16816(acc[0], signed_pair<15>(S0, x0), signed_pair<14>(S0, x0), signed_pair<15>(S1, x1), signed_pair<14>(S1, x1), bf[ks].x, bf[ks].y);
+          mma_16816(acc[1], signed_pair<13>(S0, x0), signed_pair<12>(S0, x0), signed_pair<13>(S1, x1), signed_pair<12>(S1, x1), bf[ks].x, bf[ks].y);
+          mma_16816(acc[2], signed_pair<11>(S0, x0), signed_pair<10>(S0, x0), signed_pair<11>(S1, x1), signed_pair<10>(S1, x1), bf[ks].x, bf[ks].y);
+          mma_16816(acc[3], signed_pair<9>(S0, x0), signed_pair<8>(S0, x0), signed_pair<9>(S1, x1), signed_pair<8>(S1, x1), bf[ks].x, bf[ks].y);
+        }
+        float v[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] = fmaf(acc[j][1], hs_tail, acc[j][0] * hs);
+          v[2 * j + 1] = fmaf(acc[j][3], hs_tail, acc[j][2] * hs);
+        }
+        if (t4 < NH) emit(v, tok0 + 8 * k, dst0 + 8 * k, n);
+      }
+      flush_candidates();
+    };
+
     auto compute = [&](auto tbc) {
       constexpr int TB = decltype(tbc)::value;
       using GE = Geo<TB>;
       constexpr int BW = TB / WARPS;                           // blocks per warp and stage
-      const int s0 = pass * GE::ROWS, sc = min(GE::ROWS, nrows - s0), nks = (sc + 15) >> 4, ks0 = s0 >> 4;
+      const int s0 = pass * GE::ROWS, sc = min(GE::ROWS, nrows - s0), nks = (sc + 15) >> 4;
       const int blk0 = first_block(g) + u * TB;
       const uint32_t n = (uint32_t)B.n[item];                  // n < 2^31
+      if (TB == 16 && npass == 1 && nks >= 1 && nks <= 3 && (uint32_t)(blk0 + TB) * FATHOM_BLOCK <= n) {
+        // ---- the common stage (a plan of up to 48 rows, a whole tile of a long sequence)
+        if (nks == 3) half_blocks(std::integral_constant<int, 3>(), blk0);
+        else if (nks == 2) half_blocks(std::integral_constant<int, 2>(), blk0);
+        else half_blocks(std::integral_constant<int, 1>(), blk0);
+        return;
+      }
 #pragma unroll 1
       for (int i = 0; i < BW; ++i) {
         const int b = warp * BW + i;                           // my block within the sub-tile
@@ -269,21 +458,9 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         // my byte (tokens 8 gq .. 8 gq + 7) of the plane words and the scales of rows 2 t4, 2 t4 + 1 (+ 8, + 9) of every 16
         const unsigned char* wp = M.words[buf] + (2 * t4) * GE::ROW_BYTES + b * 8 + gq;
         const uint16_t* sp = reinterpret_cast<const uint16_t*>(M.scale[buf]) + (2 * t4) * GE::SCALE_ELEMS + b;
-#pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks) {
-          const uint2 bf = M.bfr[ks0 + ks][lane];
-          const uint32_t x0 = __byte_perm(wp[0], wp[GE::ROW_BYTES], 0x5410);
-          const uint32_t x1 = __byte_perm(wp[8 * GE::ROW_BYTES], wp[9 * GE::ROW_BYTES], 0x5410);
-          const uint32_t S0 = __byte_perm(sp[0], sp[GE::SCALE_ELEMS], 0x5410);
-          const uint32_t S1 = __byte_perm(sp[8 * GE::SCALE_ELEMS], sp[9 * GE::SCALE_ELEMS], 0x5410);
-          // slice j: mma row gq = token 8 gq + 2 j, row gq + 8 = token 8 gq + 2 j + 1
-          mma_16816(acc[0], signed_pair<15>(S0, x0), signed_pair<14>(S0, x0), signed_pair<15>(S1, x1), signed_pair<14>(S1, x1), bf.x, bf.y);
-          mma_16816(acc[1], signed_pair<13>(S0, x0), signed_pair<12>(S0, x0), signed_pair<13>(S1, x1), signed_pair<12>(S1, x1), bf.x, bf.y);
-          mma_16816(acc[2], signed_pair<11>(S0, x0), signed_pair<10>(S0, x0), signed_pair<11>(S1, x1), signed_pair<10>(S1, x1), bf.x, bf.y);
-          mma_16816(acc[3], signed_pair<9>(S0, x0), signed_pair<8>(S0, x0), signed_pair<9>(S1, x1), signed_pair<8>(S1, x1), bf.x, bf.y);
-          wp += 16 * GE::ROW_BYTES;
-          sp += 16 * GE::SCALE_ELEMS;
-        }
+        const uint2* bfr_lane = &M.bfr[0][lane];
+        if (nks == 3) mma_rows<GE::ROW_BYTES, GE::SCALE_ELEMS, 3>(acc, wp, sp, bfr_lane, 3);   // 33 .. 48 rows: a B = 48 plan
+        else mma_rows<GE::ROW_BYTES, GE::SCALE_ELEMS, 0>(acc, wp, sp, bfr_lane, nks);
         if (pass != npass - 1) continue;
 
         // ---- scores of head t4 for my eight tokens: columns 2 t4 (head part) and 2 t4 + 1 (tail part)
@@ -296,44 +473,9 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         const bool have_block = blk0 + b < nb_item;
         const uint32_t tok = (uint32_t)(blk0 + b) * FATHOM_BLOCK + gq * 8;                     // my first token
         if (t4 >= NH || !have_block) continue;
-        if (MODE != 2) {
-          const uint32_t dst = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok;
-          float* row = B.scores[item] + (size_t)(h0 + t4) * (size_t)B.score_stride[item] + dst;
-          if (tok + 8 <= n) {
-            *reinterpret_cast<float4*>(row) = make_float4(v[0], v[1], v[2], v[3]);
-            *reinterpret_cast<float4*>(row + 4) = make_float4(v[4], v[5], v[6], v[7]);
-          } else {
-#pragma unroll
-            for (int x = 0; x < 8; ++x)
-              if (tok + x < n) row[x] = v[x];
-          }
-        } else {
-          // candidates: (score, token) pairs appended to the head's list; their order in the list is irrelevant
-          uint32_t m = 0u;
-#pragma unroll
-          for (int x = 0; x < 8; ++x) m |= (v[x] >= my_thr ? 1u : 0u) << x;
-          if (m) {
-#pragma unroll
-            for (int x = 0; x < 8; ++x) {
-              const long long ti = (long long)tok + x;
-              if (!(ti < (long long)n && ti >= fz.sink_end && ti < fz.local_begin)) m &= ~(1u << x);
-            }
-            if (m) {
-              uint32_t at = atomicAdd(&fz.cand_count[h0 + t4], (uint32_t)__popc(m));
-#pragma unroll
-              for (int x = 0; x < 8; ++x) {
-                if ((m >> x) & 1u) {
-                  if ((long long)at < fz.capacity) {
-                    fz.cand_score[(size_t)(h0 + t4) * fz.capacity + at] = v[x];
-                    fz.cand_idx[(size_t)(h0 + t4) * fz.capacity + at] = (int32_t)(tok + x);
-                  }
-                  ++at;
-                }
-              }
-            }
-          }
-        }
+        emit(v, tok, MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok, n);
       }
+      if (pass == npass - 1) flush_candidates();
     };
     if (tb == 16) compute(std::integral_constant<int, 16>());
     else if (tb == 8) compute(std::integral_constant<int, 8>());
@@ -348,6 +490,8 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     if (!same_item) {                                          // first tile of another session: nothing was fetched ahead
       enter_item(g);
       prefetch(g, 0, 0, buf);
+    } else if (npass > 1) {
+      fill_bfr(pass);                                          // plans of more than 160 rows: the right operand of the next pass
     }
   }
 }

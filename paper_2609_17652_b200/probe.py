@@ -28,9 +28,11 @@ def main():
     ap.add_argument("--q-heads", type=int, default=32)
     ap.add_argument("--heads-per-plan", type=int, default=4)
     ap.add_argument("--host-planes", action="store_true", help="planes and scales in pinned host memory")
+    ap.add_argument("--ctas", type=int, default=0, help="CTAs per plan of the scan (0 = automatic)")
     ap.add_argument("--no-flush", action="store_true", help="do not write a 256 MB buffer between iterations")
     a = ap.parse_args()
     dev = torch.device("cuda", 0)
+    fb.fathom_scan_set_ctas_per_plan(a.ctas)
     torch.manual_seed(0)
     n, Hkv, Hq, d, hpp = a.n, a.kv_heads, a.q_heads, 128, a.heads_per_plan
     lay = fb.make_layout(Hkv, Hq, n, d)
