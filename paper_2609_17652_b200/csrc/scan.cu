@@ -357,16 +357,16 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       }
     };
 
-    // ---- MODE 2, whole warp, after the last emit of a stage: the warp's lists go to the heads' global lists, one atomic
-    //      per head (same-address atomics are what the global lists can take least of)
-    auto flush_candidates = [&]() {
+    // ---- MODE 2, whole warp, after the last emit of a stage: once a list is half full (or at the end of the warp's work:
+    //      `final`) the warp's lists go to the heads' global lists, one atomic per head (same-address atomics are what the
+    //      global lists can take least of, and waiting for their result is what a warp can afford least often)
+    auto flush_candidates = [&](bool final) {
       if (MODE != 2) return;
       __syncwarp();
       uint32_t c = 0u, base = 0u;
-      if (lane < NH) {
-        c = min(M.ccnt[warp][lane], (uint32_t)CAND_CAP);
-        if (c) base = atomicAdd(&fz.cand_count[h0 + lane], c);
-      }
+      if (lane < NH) c = min(M.ccnt[warp][lane], (uint32_t)CAND_CAP);
+      if (!final && !__any_sync(0xffffffffu, c >= (uint32_t)(CAND_CAP / 2))) return;
+      if (c) base = atomicAdd(&fz.cand_count[h0 + lane], c);
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
         const uint32_t ch = __shfl_sync(0xffffffffu, c, h), bh = __shfl_sync(0xffffffffu, base, h);
@@ -431,7 +431,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         }
         if (t4 < NH) emit(v, tok0 + 8 * k, dst0 + 8 * k, n);
       }
-      flush_candidates();
+      flush_candidates(!more);
     };
 
     auto compute = [&](auto tbc) {
@@ -475,7 +475,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         if (t4 >= NH || !have_block) continue;
         emit(v, tok, MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok, n);
       }
-      if (pass == npass - 1) flush_candidates();
+      if (pass == npass - 1) flush_candidates(!more);
     };
     if (tb == 16) compute(std::integral_constant<int, 16>());
     else if (tb == 8) compute(std::integral_constant<int, 8>());
