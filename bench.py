@@ -1,10 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the Fathom decode-step hot path on B200.
 
-One "step" is one pass of the whole hot path over one synthetic Qwen3-8B-shaped layer:
-    fathom_build_planes -> fathom_alloc_depth -> fathom_scan -> fathom_topk -> fathom_sparse_attend
+One "step" is one decode step of one synthetic Qwen3-8B-shaped layer:
+    fathom_alloc_depth -> fathom_scan -> fathom_topk -> fathom_sparse_attend
 at n = 1,048,576 tokens, 8 KV heads / 32 query heads, d = 128, budget B = 48, k = 4096, planes in HBM
-(the million-token configuration the metric is quoted on).  Prints ONE JSON line (rank 0).
+(the million-token configuration the metric is quoted on).  fathom_build_planes runs once per sequence,
+before the steps, and is timed on its own (once_per_sequence).  Prints ONE JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -33,17 +34,19 @@ from paper_2609_17652_b200 import dist as fdist
 
 METRIC = "keys_scanned_per_s"
 UNIT = "keys/s"
+N_LAYERS = 4                                                    # layer stores a session's steps rotate over
 WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3, planes in HBM)",
                 n=1 << 20, Hkv=8, Hq=32, d=128, B=48, k=4096, heads_per_plan=4)
 # dram__bytes_read.sum + dram__bytes_write.sum per unit (one token of one KV head) from the ncu captures
 # summarised under profiles/: build at n = 131072 (596.1 MB / 1,048,576 units; traffic is proportional to
-# units), scan at n = 1,048,576 and B = 48 (136.9 MB / 8,388,608 units; part of the score writes is still in
+# units), scan at n = 1,048,576 and B = 48 (139.7 MB / 8,388,608 units; part of the score writes is still in
 # L2 when the kernel ends), the three top-k kernels at n = 1,048,576, k = 4096 (8.4 + 134.25 + 1.7 MB read, 0.5 MB
 # written / 8,388,608 units; valid for the single-pass path only), attention at k = 4096 (66.1 MB read + 1.05 MB
 # written; proportional to k, not to n: 67.1 MB / (32 heads x 4096 rows) = 512.3 B per selected row).
 # Multiplied by the units of a launch in the JSON line.
-NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 15.9, "topk_*": 17.3}
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.65, "topk_*": 17.3}
 NCU_TRAFFIC_BYTES_PER_SELECTED_ROW = 512.3
+NCU_SCAN_WARP_INSTRUCTIONS_PER_BLOCK_OF_48_ROWS = 232.0         # smsp__inst_executed.sum / (n * Hkv / 64) at B = 48 (profiles/scan_kernel_n1M_B48.md)
 
 
 def parse_args():
@@ -124,6 +127,10 @@ class ClockSampler:
                 pass
             time.sleep(self._period)
 
+    def mark(self):
+        """The timed region starts here (samples before it belong to the warm-up steps, which run the same kernels)."""
+        self.marked = len(self.samples)
+
     def stop(self):
         if self._nv is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable: " + self.err]}
@@ -132,6 +139,7 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
                 "sm_mhz_min": min(self.samples) if self.samples else None,
                 "power_w_max": max(self.power) if self.power else None, "samples": len(self.samples),
+                "samples_in_timed_region": len(self.samples) - getattr(self, "marked", 0),
                 "reasons": sorted(self.reasons)}
 
 
@@ -152,83 +160,107 @@ def run_ours(args):
     B, k, hpp = args.budget, args.k, WORKLOAD["heads_per_plan"]
     G = Hq // Hkv
 
-    # weak scaling: every rank owns one independent session (its own seed); no data-path collective
+    # weak scaling: every rank owns one independent session (its own seed); no data-path collective.
+    # The session has N_LAYERS independently seeded layers' stores; consecutive steps take consecutive layers, as the
+    # decode step of a model does, so no plane byte of a step is still in L2 from the step before (4 x 58 MB > 126 MB).
     session = fdist.sessions_of_rank(rank, world, n_sessions=world)[0]
-    L = make_layer(n, Hkv, Hq, d, seed=2, session=session, device=str(dev))
     lay = fb.make_layout(Hkv, Hq, n, d)
     ctx = fb.Context(local_rank, fb.fathom_scratch_bytes(lay, k))
-    planes = torch.zeros((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
-    scales = torch.zeros((Hkv, d, lay.scale_stride), dtype=torch.int16, device=dev)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    layers = []
+    build_ts = []
+    for li in range(N_LAYERS):
+        Ll = make_layer(n, Hkv, Hq, d, seed=2, session=session, layer=li, device=str(dev), want_rows=(li == 0))
+        pl = torch.zeros((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
+        sc = torch.zeros((Hkv, d, lay.scale_stride), dtype=torch.int16, device=dev)
+        for it in range(4 if li == 0 else 3):                    # once per sequence: timed here, L2 flushed, not part of the step
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); ctx.fathom_build_planes(lay, Ll.K, pl, sc, stream); b.record(stream)
+            torch.cuda.synchronize()
+            if it or li:
+                build_ts.append(a.elapsed_time(b) * 1e3)
+        if li == 0:
+            L = Ll
+        layers.append({"planes": pl, "scales": sc, "q": Ll.q, "var": Ll.var})
+        if li:
+            del Ll
+    build_us = statistics.median(build_ts)
+    planes, scales = layers[0]["planes"], layers[0]["scales"]
     depth = torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev)
     scores = torch.zeros((Hq, lay.score_stride), dtype=torch.float32, device=dev)
     idx = torch.zeros((Hq, k), dtype=torch.int32, device=dev)
     out = torch.zeros((Hq, d), dtype=torch.float32, device=dev)
     sm_scale = 1.0 / math.sqrt(d)
-    stream = torch.cuda.current_stream()
 
-    stage_names = ["build_planes", "alloc_depth", "scan", "topk", "sparse_attend"]
+    stage_names = ["alloc_depth", "scan", "topk", "sparse_attend"]
     topk_passes = fb.fathom_topk_passes(lay, k)                 # 1: sampled estimate + one collection pass; 2: histogram + filter
     # single pass: sample histogram, collection, selection (3 kernels); two passes: histogram, filter, select, emit (4)
-    launches_per_step = {"build_planes": 1, "alloc_depth": 1, "scan": 1, "topk": 3 if topk_passes == 1 else 4, "sparse_attend": 1}
+    launches_per_step = {"alloc_depth": 1, "scan": 1, "topk": 3 if topk_passes == 1 else 4, "sparse_attend": 1}
 
-    def stage(i, K=L.K, Kr=L.Krows, Vr=L.Vrows, q=L.q, var=L.var, pl=planes, sc=scales):
+    def stage(i, W, st, q=None, var=None):
+        """Stage i of the decode step on layer store W: alloc_depth, scan, topk, sparse_attend."""
+        q = W["q"] if q is None else q
+        var = W["var"] if var is None else var
         if i == 0:
-            ctx.fathom_build_planes(lay, K, pl, sc, stream)
+            ctx.fathom_alloc_depth(lay, q, var, fb.DEPTH_WATERFILL, B, hpp, depth, st)
         elif i == 1:
-            ctx.fathom_alloc_depth(lay, q, var, fb.DEPTH_WATERFILL, B, hpp, depth, stream)
+            ctx.fathom_scan(lay, W["planes"], W["scales"], q, depth, hpp, scores, st)
         elif i == 2:
-            ctx.fathom_scan(lay, pl, sc, q, depth, hpp, scores, stream)
-        elif i == 3:
-            ctx.fathom_topk(lay, scores, k, 0, 0, idx, stream)
-        else:
-            ctx.fathom_sparse_attend(lay, q, Kr, Vr, idx, k, sm_scale, out, stream)
-
-    def stage_on(i, st):
-        if i == 1:
-            ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, B, hpp, depth, st)
-        elif i == 2:
-            ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, scores, st)
-        elif i == 3:
             ctx.fathom_topk(lay, scores, k, 0, 0, idx, st)
         else:
-            ctx.fathom_sparse_attend(lay, L.q, L.Krows, L.Vrows, idx, k, sm_scale, out, st)
+            ctx.fathom_sparse_attend(lay, q, L.Krows, L.Vrows, idx, k, sm_scale, out, st)
 
-    def step(events=None):
-        for i in range(5):
+    def step(s, events=None):
+        W = layers[s % N_LAYERS]
+        for i in range(4):
             if events is not None:
                 events[i].record(stream)
-            stage(i)
+            stage(i, W, stream)
         if events is not None:
-            events[5].record(stream)
+            events[4].record(stream)
 
-    for _ in range(max(args.warmup, 3)):
-        step()
+    sampler = ClockSampler(local_rank, period_s=0.0005) if rank == 0 else None   # samples from the warm-up steps on: same load
+    for s in range(max(args.warmup, 3)):
+        step(s)
     torch.cuda.synchronize()
 
-    # ---- timed region: exactly `steps` steps, CUDA events on the launching stream, clocks sampled meanwhile
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    # ---- timed region: exactly `steps` decode steps, CUDA events on the launching stream, clocks sampled meanwhile
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     fdist.barrier()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.mark()
     t_wall = time.perf_counter()
     for s in range(args.steps):
-        step(ev[s])
+        step(s, ev[s])
     torch.cuda.synchronize()
     t_wall = time.perf_counter() - t_wall
     fdist.barrier()
     clocks = sampler.stop() if sampler else None
-    total_ms = ev[0][0].elapsed_time(ev[-1][5])
+    total_ms = ev[0][0].elapsed_time(ev[-1][4])
     total_ms = fdist.max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
     stage_us = {nm: 1e3 * statistics.mean(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps))
                 for i, nm in enumerate(stage_names)}
+    stage_us["build_planes"] = build_us
     status = ctx.fathom_device_status()
+    step(0)                                                     # depth, scores, idx of layer 0 for the legs below
+    torch.cuda.synchronize()
 
-    depth_h = depth.cpu().numpy()
-    bits = float(np.mean([bits_per_token(r) for r in depth_h]))
     # per launch, all plans: a plan's rows are read once by the CTAs that serve it (twice for plans of eight heads, which two
-    # groups of four heads share)
-    plane_bytes_read = sum(bits_per_token(r) for r in depth_h) / 8.0 * n * max(1, hpp // 4)
+    # groups of four heads share); mean over the layers the steps rotate over (their plans differ slightly)
+    per_layer_bytes, per_layer_bits = [], []
+    for W in reversed(layers):                                  # layer 0 last: its depths stay in `depth`
+        stage(0, W, stream)
+        torch.cuda.synchronize()
+        dh = depth.cpu().numpy()
+        per_layer_bytes.append(sum(bits_per_token(r) for r in dh) / 8.0 * n * max(1, hpp // 4))
+        per_layer_bits.append(float(np.mean([bits_per_token(r) for r in dh])))
+    depth_h = depth.cpu().numpy()
+    bits = float(np.mean(per_layer_bits))
+    plane_bytes_read = float(np.mean(per_layer_bytes))
     alg_bytes = {
         "build_planes": n * Hkv * (d * 4 + 68.0),
         "scan": plane_bytes_read + 4.0 * Hq * n,
@@ -247,14 +279,13 @@ def run_ours(args):
                 "algorithmic_bytes": alg_bytes[stage_key], "launch_us": round(t_us, 2), "peak_source": peak_src}
 
     # ---- isolated stage timings with an L2 flush before every launch (cold-cache view of each stage)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    iso_us = {}
+    iso_us = {"build_planes": build_us}
     for i, nm in enumerate(stage_names):
         ts = []
         for _ in range(10):
             flush.zero_()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); stage(i); b.record(stream)
+            a.record(stream); stage(i, layers[0], stream); b.record(stream)
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(b) * 1e3)
         iso_us[nm] = statistics.median(ts)
@@ -265,7 +296,11 @@ def run_ours(args):
         "dtype": "u64 bit planes + f32 accumulate", "data": "synthetic",
         "config": {"workload": WORKLOAD["name"], "n": n, "kv_heads": Hkv, "q_heads": Hq, "d": d, "budget_bits": B,
                    "k": k, "heads_per_plan": hpp, "sessions_per_gpu": 1, "parallelism": f"{world} independent session(s), one per GPU",
-                   "l2": "step inputs (4 GiB of fp32 keys, 4 GiB of bf16 rows) exceed the 126 MB L2; no explicit flush in the timed region"},
+                   "step": "one decode step of one layer: fathom_alloc_depth -> fathom_scan -> fathom_topk -> fathom_sparse_attend; "
+                           "fathom_build_planes runs once per sequence and is timed separately (once_per_sequence)",
+                   "l2": f"consecutive steps take the stores of {N_LAYERS} independently seeded layers in turn ({N_LAYERS} x 58 MB of plane "
+                         "rows read, 134 MB of scores written and re-read, 67 MB of rows gathered from 4 GiB per step): nothing a step "
+                         "reads is left in the 126 MB L2 by the step before; no explicit flush in the timed region"},
     }
     keys_per_step = n * Hkv * world
     result["value"] = keys_per_step / (ms_per_step * 1e-3)
@@ -273,7 +308,10 @@ def run_ours(args):
     result["clocks"] = clocks
     result["stage_us"] = {k_: round(v, 2) for k_, v in stage_us.items()}
     result["stage_us_isolated_l2_flushed"] = {k_: round(v, 2) for k_, v in iso_us.items()}
-    result["decode_step_us_per_layer"] = round(sum(v for k_, v in stage_us.items() if k_ != "build_planes"), 2)
+    result["decode_step_us_per_layer"] = round(1e3 * ms_per_step, 2)
+    result["once_per_sequence"] = {"build_planes_us": round(build_us, 2), "keys_per_s": n * Hkv / (build_us * 1e-6),
+                                   "step_with_build_ms": round(ms_per_step + build_us * 1e-3, 4),
+                                   "keys_per_s_step_with_build": keys_per_step / (ms_per_step * 1e-3 + build_us * 1e-6)}
     result["bits_per_token"] = round(bits, 2)
     result["scan"] = {
         "keys_per_s": n * Hkv / (stage_us["scan"] * 1e-6),
@@ -318,26 +356,35 @@ def run_ours(args):
         result["scan_per_query_head_plans"] = {"heads_per_plan": 1, "scan_us_l2_flushed": round(t1, 2), "plane_and_scale_bytes_read": rd,
                                                "gbs_index_bytes_only": round(rd / (t1 * 1e-6) / 1e9, 1),
                                                "gbs_with_score_writes": round((rd + 4.0 * Hq * n) / (t1 * 1e-6) / 1e9, 1)}
-    ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, scores, stream)      # scores of the default budget again
-    ctx.fathom_topk(lay, scores, k, 0, 0, idx, stream)
+    stage(1, layers[0], stream); stage(2, layers[0], stream)      # scores and picks of the default budget again
     result["scan_other_budgets"] = other
-    result["roofline"] = roof("build_planes", stage_us["build_planes"], "build_planes_kernel", n * Hkv)
+    # the headline roofline is the scan kernel's: the kernel the metric and the targets are written for
+    scan_s = stage_us["scan"] * 1e-6
+    result["roofline"] = roof("scan", stage_us["scan"], "scan_kernel", n * Hkv)
+    result["roofline"]["frac_index_bytes_only"] = round(plane_bytes_read / scan_s / 1e9 / peak, 4)
+    result["roofline"]["note"] = ("algorithmic bytes = plane words and scales read + fp32 scores written; frac_index_bytes_only counts the "
+                                  "plane words and scales alone (the paper's GB/s convention); with the scores materialised that figure "
+                                  "cannot exceed bytes_read / (bytes_read + bytes_written) = %.2f" % (plane_bytes_read / alg_bytes["scan"]))
     result["roofline_other_kernels"] = {
-        "scan": roof("scan", stage_us["scan"], "scan_kernel", n * Hkv),
+        "build_planes (once per sequence)": roof("build_planes", build_us, "build_planes_kernel", n * Hkv),
         f"topk ({topk_passes} pass{'es' if topk_passes > 1 else ''} over the scores)": roof("topk", stage_us["topk"], "topk_*", n * Hkv),
         "sparse_attend": roof("sparse_attend", stage_us["sparse_attend"], "attend_*", n * Hkv),
     }
-    # the scan is bound by arithmetic, not by HBM (one fp32 add per token, active row and head): also report it that way
-    adds = float(n) * sum(int(r.sum()) for r in depth_h) * hpp               # per token, active (channel, plane) row and head
-    add_peak = 148 * 128 * 1.965e9                              # fp32 lanes x SMs x clocks.max.sm: one add per lane and clock
+    # the scan's arithmetic: one tensor-core multiply-add per (token, active row, head part) and, on the CUDA cores, the
+    # expansion of every plane bit into a signed fp16 operand (one shift + one logic op per pair of elements)
+    elements = float(n) * sum(int(r.sum()) for r in depth_h)                 # (token, active row) pairs of one launch, all plans
     issue_peak = 148 * 4 * 1.965e9                              # warp instructions per second (four schedulers per SM)
-    scan_s = stage_us["scan"] * 1e-6
-    result["roofline_other_kernels"]["scan"]["alt_bound"] = {
-        "bound": "alu", "achieved": round(adds / scan_s / 1e12, 3), "peak": round(add_peak / 1e12, 3), "unit": "T fp32 adds/s",
-        "frac": round(adds / scan_s / add_peak, 4),
-        "issue_frac": round(adds / 32 * 1.25 / scan_s / issue_peak, 4),
-        "note": "peak = 148 SMs x 128 fp32 lanes x 1.965 GHz; the adds are predicated on the token's plane bit, which costs a fifth "
-                "instruction per four adds: issue_frac = (adds / 32 lanes x 5/4) / (148 SMs x 4 schedulers x 1.965 GHz)"}
+    result["roofline"]["alt_bound"] = {
+        "bound": "alu", "unit": "G warp instructions/s", "peak": round(issue_peak / 1e9, 1),
+        "achieved": round(elements / 3072.0 * NCU_SCAN_WARP_INSTRUCTIONS_PER_BLOCK_OF_48_ROWS / scan_s / 1e9, 1),
+        "frac": round(elements / 3072.0 * NCU_SCAN_WARP_INSTRUCTIONS_PER_BLOCK_OF_48_ROWS / scan_s / issue_peak, 4),
+        "note": "issue-slot view: warp instructions per 64 tokens x 48 rows from the committed ncu summary (profiles/), scaled by the "
+                "launch's (token, row) pairs; peak = 148 SMs x 4 schedulers x 1.965 GHz"}
+    result["targets"] = {
+        "hbm_resident_scan_frac_of_hbm_peak": {"target": 0.70, "achieved_with_score_writes": result["roofline"]["frac"],
+                                               "achieved_index_bytes_only": result["roofline"]["frac_index_bytes_only"],
+                                               "met": bool(result["roofline"]["frac"] >= 0.70)},
+    }
 
     # ---- attention gathers 256-byte rows scattered over 2 + 2 GiB: every row opens a DRAM page, so the copy peak is not
     #      the bound that matters.  A micro-benchmark of a pure gather (half a warp per row, 8 loads in flight, rows
@@ -356,23 +403,25 @@ def run_ours(args):
         gs = torch.cuda.Stream()
         gs.wait_stream(stream)
         with torch.cuda.stream(gs):
-            for i in range(1, 5):
-                stage_on(i, gs)
+            for W in layers:
+                for i in range(4):
+                    stage(i, W, gs)
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=gs):
-                for i in range(1, 5):
-                    stage_on(i, gs)
+                for W in layers:                                    # one graph = the decode steps of N_LAYERS layers
+                    for i in range(4):
+                        stage(i, W, gs)
         torch.cuda.synchronize()
         ts = []
-        for it in range(13):                                        # ten replays back to back per sample, as the layers
+        for it in range(13):                                        # three replays back to back per sample, as the layers
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)   # of a model would follow each other
             a.record(stream)
-            for _ in range(10):
+            for _ in range(3):
                 g.replay()
             b.record(stream)
             torch.cuda.synchronize()
             if it >= 3:
-                ts.append(a.elapsed_time(b) * 1e3 / 10.0)
+                ts.append(a.elapsed_time(b) * 1e3 / (3.0 * N_LAYERS))
         graph_us = round(statistics.median(ts), 2)
         del g
     except Exception as e:                                      # report, never hide
@@ -380,26 +429,31 @@ def run_ours(args):
     result["decode_step_us_per_layer_cuda_graph"] = graph_us
 
     # ---- the same decode step with scan and selection fused (scores never written): alloc, scan_topk, attend
-    def fused_on(st):
-        ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, B, hpp, depth, st)
-        ctx.fathom_scan_topk(lay, planes, scales, L.q, depth, hpp, k, 0, 0, idx, st)
-        ctx.fathom_sparse_attend(lay, L.q, L.Krows, L.Vrows, idx, k, sm_scale, out, st)
-    ts = []
-    for it in range(33):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream); fused_on(stream); b.record(stream)
-        torch.cuda.synchronize()
-        if it >= 3:
-            ts.append(a.elapsed_time(b) * 1e3)
-    result["decode_step_fused_us_per_layer"] = round(statistics.median(ts), 2)
+    def fused_on(W, st):
+        ctx.fathom_alloc_depth(lay, W["q"], W["var"], fb.DEPTH_WATERFILL, B, hpp, depth, st)
+        ctx.fathom_scan_topk(lay, W["planes"], W["scales"], W["q"], depth, hpp, k, 0, 0, idx, st)
+        ctx.fathom_sparse_attend(lay, W["q"], L.Krows, L.Vrows, idx, k, sm_scale, out, st)
+    for s_ in range(3):
+        fused_on(layers[s_ % N_LAYERS], stream)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for s_ in range(args.steps):
+        fused_on(layers[s_ % N_LAYERS], stream)
+    b.record(stream)
+    torch.cuda.synchronize()
+    result["decode_step_fused_us_per_layer"] = round(a.elapsed_time(b) * 1e3 / args.steps, 2)
+    stage(0, layers[0], stream); stage(1, layers[0], stream); stage(2, layers[0], stream)   # layer 0's depths, scores, picks again
     result["device_status"] = status
     result["wall_ms_per_step"] = round(1e3 * t_wall / args.steps, 4)
 
     # ---- planes in pinned host memory, read zero-copy by the scan kernel over the host link
     if rank == 0 and not args.no_host_resident:
-        result["host_resident_scan"] = host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, plane_bytes_read)
+        result["host_resident_scan"] = host_resident_leg(ctx, lay, planes, scales, L, depth, hpp, scores, stream, per_layer_bytes[-1])
         result["host_resident_row_fetch"] = row_fetch_leg(ctx, lay, L, idx, k, G, stream,
                                                           result["host_resident_scan"]["link_peak_gbs"])
+        result["targets"]["host_resident_scan_frac_of_measured_link"] = {
+            "target": 0.80, "achieved": result["host_resident_scan"]["frac_of_measured_link"],
+            "met": bool(result["host_resident_scan"]["frac_of_measured_link"] >= 0.80)}
 
     # ---- once-per-session kernels of the raw and the KLT-rotated store (not part of the step): statistics, rotation
     if rank == 0 and not args.no_session_kernels:
@@ -407,7 +461,7 @@ def run_ours(args):
 
     # ---- end to end through the C ABI from HOST buffers: H2D of the step's inputs and D2H of its result are timed
     if not args.no_e2e:
-        result["e2e"] = e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step)
+        result["e2e"] = e2e_leg(args, layers, stage, out, stream, keys_per_step)
     else:
         result["e2e"] = None
 
@@ -524,38 +578,42 @@ def row_fetch_leg(ctx, lay, L, idx, k, G, stream, link_gbs):
             "gbs": round(gbs, 2), "frac_of_measured_link": round(gbs / link_gbs, 4)}
 
 
-def e2e_leg(args, fb, ctx, lay, L, stage, out, stream, keys_per_step):
-    hK = torch.empty(L.K.shape, dtype=L.K.dtype, pin_memory=True); hK.copy_(L.K)
-    hKr = torch.empty(L.Krows.shape, dtype=L.Krows.dtype, pin_memory=True); hKr.copy_(L.Krows)
-    hVr = torch.empty(L.Vrows.shape, dtype=L.Vrows.dtype, pin_memory=True); hVr.copy_(L.Vrows)
-    hq = torch.empty(L.q.shape, dtype=L.q.dtype, pin_memory=True); hq.copy_(L.q)
-    hvar = torch.empty(L.var.shape, dtype=L.var.dtype, pin_memory=True); hvar.copy_(L.var)
+def e2e_leg(args, layers, stage, out, stream, keys_per_step):
+    """The decode step end to end from HOST buffers: what a decode step ships is the layer's query and channel statistics
+    in (pinned host memory -> device, inside the timed region, every step) and the attention output back (device ->
+    pinned host); the store and the K/V rows are resident, as they are between the steps of a session."""
+    hq = [torch.empty(W["q"].shape, dtype=W["q"].dtype, pin_memory=True) for W in layers]
+    hvar = [torch.empty(W["var"].shape, dtype=W["var"].dtype, pin_memory=True) for W in layers]
+    for W, a, b in zip(layers, hq, hvar):
+        a.copy_(W["q"]); b.copy_(W["var"])
     hout = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
-    dK, dKr, dVr, dq, dvar = (torch.empty_like(L.K), torch.empty_like(L.Krows), torch.empty_like(L.Vrows),
-                              torch.empty_like(L.q), torch.empty_like(L.var))
-    h2d = sum(t.numel() * t.element_size() for t in (hK, hKr, hVr, hq, hvar))
+    dq, dvar = torch.empty_like(layers[0]["q"]), torch.empty_like(layers[0]["var"])
+    h2d = sum(t.numel() * t.element_size() for t in (hq[0], hvar[0]))
     d2h = hout.numel() * hout.element_size()
 
-    def e2e_step():
-        dK.copy_(hK, non_blocking=True); dKr.copy_(hKr, non_blocking=True); dVr.copy_(hVr, non_blocking=True)
-        dq.copy_(hq, non_blocking=True); dvar.copy_(hvar, non_blocking=True)
-        for i in range(5):
-            stage(i, K=dK, Kr=dKr, Vr=dVr, q=dq, var=dvar)
+    def e2e_step(s):
+        li = s % len(layers)
+        dq.copy_(hq[li], non_blocking=True); dvar.copy_(hvar[li], non_blocking=True)
+        for i in range(4):
+            stage(i, layers[li], stream, q=dq, var=dvar)
         hout.copy_(out, non_blocking=True)
 
-    steps = max(3, min(args.steps, 5))
-    e2e_step(); torch.cuda.synchronize()
+    steps = args.steps
+    for s in range(3):
+        e2e_step(s)
+    torch.cuda.synchronize()
     fdist.barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(stream)
-    for _ in range(steps):
-        e2e_step()
+    for s in range(steps):
+        e2e_step(s)
     b.record(stream)
     torch.cuda.synchronize()
     ms = fdist.max_over_ranks(a.elapsed_time(b)) / steps
-    return {"value": keys_per_step / (ms * 1e-3), "unit": UNIT, "ms_per_step": round(ms, 3), "steps": steps,
+    return {"value": keys_per_step / (ms * 1e-3), "unit": UNIT, "ms_per_step": round(ms, 4), "steps": steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "what": "pinned host K (fp32), K/V rows (bf16), q, var copied to the device, five C-ABI calls, result copied back"}
+            "what": "per step: q [32][128] and var [8][128] (fp32) copied from pinned host memory to the device, the four C-ABI calls "
+                    "of the decode step on the resident store and rows, out [32][128] copied back to pinned host memory"}
 
 
 # ------------------------------------------------------------------------------------------------ config 4
@@ -748,29 +806,88 @@ def run_config5(args):
 
 
 # ------------------------------------------------------------------------------------------------ oracle legs
-def oracle_step(n_s, B, k, hpp, seed):
+def oracle_step(n_s, B, k, hpp, seed, Hkv=None, barrier=None):
+    """One decode step of the oracle (alloc_depth, scan, topk, sparse_attend) on a synthetic layer of n_s tokens; the
+    store is built first, untimed, as in the GPU arm.  Returns (seconds of the decode step, seconds of the build)."""
     from oracle import fathom_oracle as O
     from workloads.synth import make_layer
-    L = make_layer(n_s, WORKLOAD["Hkv"], WORKLOAD["Hq"], WORKLOAD["d"], seed=seed, device="cpu")
+    Hkv = WORKLOAD["Hkv"] if Hkv is None else Hkv
+    G = WORKLOAD["Hq"] // WORKLOAD["Hkv"]
+    L = make_layer(n_s, Hkv, Hkv * G, WORKLOAD["d"], seed=seed, device="cpu")
     K, q, var = L.K.numpy(), L.q.numpy(), L.var.numpy()
     Kr, Vr = L.Krows.float().numpy(), L.Vrows.float().numpy()
     t0 = time.perf_counter()
     planes, scales = O.build_planes(K)
+    t_build = time.perf_counter() - t0
+    if barrier is not None:
+        barrier.wait(timeout=300)
+    t0 = time.perf_counter()
     depth = O.alloc_depth(q, var, "waterfill", B, hpp)
     s = O.scan(planes, scales, q, depth, n_s, hpp)
     idx = O.topk(s, k)
     O.sparse_attend(q, Kr, Vr, idx, 1.0 / math.sqrt(WORKLOAD["d"]))
-    return time.perf_counter() - t0
+    return time.perf_counter() - t0, t_build
+
+
+def _oracle_worker(n_s, B, k, hpp, seed, heads, barrier, queue):
+    from threadpoolctl import threadpool_limits
+    torch.set_num_threads(1)
+    with threadpool_limits(limits=1):
+        dt, _ = oracle_step(n_s, B, k, hpp, seed, Hkv=heads, barrier=barrier)
+    queue.put(dt)
+
+
+def oracle_all_cores(n_s, B, k, hpp, seed):
+    """The same oracle step with the KV heads (independent problems) spread over worker processes, one thread each; the
+    oracle itself is unchanged.  Returns (seconds = the slowest worker's decode step after a common barrier, workers)."""
+    import multiprocessing as mp
+    Hkv = WORKLOAD["Hkv"]
+    workers = max(1, min(os.cpu_count() or 1, Hkv))
+    while Hkv % workers:
+        workers -= 1
+    ctx = mp.get_context("spawn")                                # the parent may hold a CUDA context: no fork
+    barrier, queue = ctx.Barrier(workers), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_worker, args=(n_s, B, k, hpp, seed + 1000 * w, Hkv // workers, barrier, queue))
+             for w in range(workers)]
+    for p_ in procs:
+        p_.start()
+    import queue as pyqueue
+    dts, deadline = [], time.time() + 600
+    try:
+        while len(dts) < workers:
+            try:
+                dts.append(queue.get(timeout=2))
+            except pyqueue.Empty:
+                if any(p_.exitcode not in (None, 0) for p_ in procs):
+                    raise RuntimeError("an oracle worker exited with an error")
+                if time.time() > deadline:
+                    raise RuntimeError("oracle workers timed out")
+    finally:
+        for p_ in procs:
+            if p_.is_alive() and len(dts) < workers:
+                p_.terminate()
+            p_.join(timeout=10)
+    return max(dts), workers
 
 
 def cpu_baseline(n_s, B, k, hpp):
     from threadpoolctl import threadpool_limits
     torch.set_num_threads(1)
     with threadpool_limits(limits=1):
-        dt = oracle_step(n_s, B, k, hpp, seed=2)
-    return {"value": n_s * WORKLOAD["Hkv"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
-            "host_cores_available": os.cpu_count(),
-            "sample": f"one step of the same layer shape at n = {n_s} tokens (8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread"}
+        dt, t_build = oracle_step(n_s, B, k, hpp, seed=2)
+    keys = n_s * WORKLOAD["Hkv"]
+    out = {"value": keys / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
+           "config": {"n": n_s, "kv_heads": 8, "q_heads": 32, "d": 128, "budget_bits": B, "k": k, "heads_per_plan": hpp},
+           "build_planes_seconds_untimed": round(t_build, 2), "host_cores_available": os.cpu_count(),
+           "sample": f"one decode step (alloc_depth, scan, topk, sparse_attend) of the same layer shape at n = {n_s} tokens "
+                     f"(8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread"}
+    try:
+        dt_all, workers = oracle_all_cores(n_s, B, k, hpp, seed=2)
+        out["all_cores"] = {"value": keys / dt_all, "unit": UNIT, "cores": workers, "seconds": round(dt_all, 2),
+                            "how": "KV heads spread over worker processes (one thread each), the slowest worker's time after a common barrier"}
+    except Exception as e:                                      # report, never hide
+        out["all_cores"] = {"error": repr(e)}
+    return out
 
 
 def run_reference(args):
@@ -784,16 +901,17 @@ def run_reference(args):
     with threadpool_limits(limits=1):
         for w in range(args.warmup):
             oracle_step(n_s, B, k, hpp, seed=100 + w)
-        ts = [oracle_step(n_s, B, k, hpp, seed=200 + s) for s in range(args.steps)]
+        ts = [oracle_step(n_s, B, k, hpp, seed=200 + s)[0] for s in range(args.steps)]
     dt = sum(ts) / len(ts)
     val = n_s * WORKLOAD["Hkv"] / dt
-    sample = f"each step = one layer of the same shape at n = {n_s} tokens (8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread"
+    sample = (f"each step = one decode step (alloc_depth, scan, topk, sparse_attend) on one layer of the same shape at n = {n_s} tokens "
+              f"(8 KV / 32 Q heads, B = {B}, k = {k}), numpy fp64, 1 thread; a bounded sample of the n = {args.n}, k = {args.k} workload")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD["name"], "n": args.n, "kv_heads": 8, "q_heads": 32, "d": 128,
-                   "budget_bits": B, "k": args.k, "heads_per_plan": hpp},
+        "config": {"workload": WORKLOAD["name"] + " - bounded sample", "n": n_s, "kv_heads": 8, "q_heads": 32, "d": 128,
+                   "budget_bits": B, "k": k, "heads_per_plan": hpp, "sample_of": {"n": args.n, "k": args.k}},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
