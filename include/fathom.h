@@ -9,13 +9,13 @@
  *    reads KV head h / G), d = 128 channels, n tokens, nb = ceil(n / 64) blocks of 64 tokens.
  *  - Every data pointer is a DEVICE pointer unless the argument says otherwise.  `planes` and
  *    `scales` may instead point to pinned host memory that the device can address (the paper's
- *    host-resident store, Sec. 3.5): the scan then reads it directly over the host link.
+ *    host-resident store, Sec. 3.6): the scan then reads it directly over the host link.
  *  - All buffers are allocated and owned by the caller.  The library allocates only the scratch
  *    arena and one status word when a context is created, and frees them when it is destroyed.
  *  - The five data-path calls only ENQUEUE work on `stream` (a cudaStream_t passed as void*;
  *    NULL = the legacy default stream).  None of them synchronises; results (`depth`, `scores`,
  *    `idx`) stay on the device and feed the next call, so a decode step needs no host round trip
- *    (Sec. 3.5, Appendix A6: fixed-size plan, no host synchronisation).
+ *    (Sec. 3.6 and Sec. 6, ablation A6: fixed-size plan, no host synchronisation).
  *  - Return value: FATHOM_OK (0) or a negative fathom_status.  Arguments that can be checked on
  *    the host (null pointers, d != 128, strides too small or misaligned, k out of range, scratch
  *    too small) are rejected before anything is launched and leave all outputs untouched.
@@ -89,6 +89,11 @@ const char* fathom_strerror(int status);
 const char* fathom_last_cuda_error(const fathom_ctx* ctx);
 /* Copies the device status word to *status (host pointer) and clears it.  Synchronises `stream`. */
 int fathom_device_status(fathom_ctx* ctx, void* stream, uint32_t* status);
+/* Self-test of the bounded device-side waits (the paper has no counterpart): enqueues a one-warp kernel in which one
+ * thread polls, at most `tries` (1 .. 4096) times, a barrier that nothing will ever complete - no copy or tensor-core
+ * operation is outstanding - then sets FATHOM_DEV_WAIT_EXPIRED in the status word and returns.  The kernels that wait
+ * on copies or tensor-core work take the same path when a wait runs out; the context stays usable afterwards. */
+int fathom_selftest_wait_expiry(fathom_ctx* ctx, int tries, void* stream);
 /* Library version, major * 100 + minor. */
 int fathom_version(void);
 
@@ -179,7 +184,7 @@ int fathom_topk(fathom_ctx* ctx, const fathom_layout* layout, const float* score
  * status for arguments fathom_topk would reject. */
 int fathom_topk_passes(const fathom_layout* layout, int k, int n_sink, int n_local);
 
-/* ---- (3+4) fused scan and top-k, scores never materialised — Sec. 6 ("a fused kernel would narrow the gap") ------
+/* ---- (3+4) fused scan and top-k, scores never materialised — Sec. 9 Conclusion (fusing the scan with what follows it) ------
  * Gives exactly the idx that fathom_topk would give on the scores of fathom_scan (same arguments), without writing
  * or re-reading the n * Hq scores: (a) every 16th 1024-token tile is scanned and histogrammed per head (12 leading
  * score-key bits); (b) the full scan keeps only the (score, token) pairs that reach a threshold bin's lower edge;

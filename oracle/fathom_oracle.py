@@ -147,8 +147,8 @@ def waterfill_depths(g: np.ndarray, B: int) -> np.ndarray:
 
     round(log4(g_j / theta)) >= m  <=>  theta <= 2 * g_j * 4^-m, so at water line
     theta channel j holds every plane m in 1..4 whose priority pi = g_j 4^-m satisfies
-    2 pi >= theta.  "The smallest theta that fits" therefore admits the longest
-    prefix (at most B items) of the planes sorted by priority.  Ties: lower channel,
+    2 pi >= theta.  The water line of Sec. 3.3 (the least theta whose depths still fit B)
+    therefore admits the longest prefix (at most B items) of the planes sorted by priority.  Ties: lower channel,
     then lower plane.  Zero priorities sort last, so B >= 4d gives depth 4 everywhere.
     """
     g = np.asarray(g, dtype=np.float64)
@@ -378,7 +378,7 @@ def exact_scores(q, Krows) -> np.ndarray:
 
 # --------------------------------------------------------------------------
 # O6  union of a group's winners  (Sec. 1: the union of the G heads' winners is fetched once per KV head;
-#     Sec. 4 "Offload harness": "the gather of the union of the selected rows")
+#     Sec. 4 "Offload harness": the row fetch of a step is that union)
 # --------------------------------------------------------------------------
 def gather_union(idx: np.ndarray, G: int, Krows, Vrows):
     """O6: per KV head kv, the ascending list u of distinct tokens picked by its G query heads, the rows
@@ -435,7 +435,7 @@ def klt_basis(C: np.ndarray):
 
 
 def rotate_keys(K: np.ndarray, mu: np.ndarray, V: np.ndarray) -> np.ndarray:
-    """(k - mu) V per KV head (Sec. 3.5: "stores planes of (k - mu) V"), fp64."""
+    """(k - mu) V per KV head (Sec. 3.5: the rotated keys whose planes the store keeps), fp64."""
     K = np.asarray(K, dtype=np.float32).astype(np.float64)
     return np.stack([(K[h] - np.asarray(mu, dtype=np.float64)[h]) @ np.asarray(V, dtype=np.float64)[h] for h in range(K.shape[0])])
 

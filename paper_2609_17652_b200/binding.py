@@ -24,7 +24,7 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
            "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated", "fathom_scan_batch",
-           "fathom_scan_set_ctas_per_plan"]
+           "fathom_scan_set_ctas_per_plan", "fathom_selftest_wait_expiry"]
 
 
 class Layout(C.Structure):
@@ -69,6 +69,7 @@ def _load() -> C.CDLL:
     lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
     lib.fathom_scan_batch.argtypes = [vp, vp, i32, i32, vp]
     lib.fathom_scan_set_ctas_per_plan.argtypes = [i32]
+    lib.fathom_selftest_wait_expiry.argtypes = [vp, i32, vp]
     lib.fathom_build_planes_rotated.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp, vp]
     lib.fathom_scan_topk.argtypes = [vp, LP, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
     lib.fathom_gather_union.argtypes = [vp, LP, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -201,6 +202,9 @@ class Context:
         self._check(lib.fathom_gather_union(self._h, C.byref(layout), _ptr(idx), k, _ptr(Krows), _ptr(Vrows),
                                             _dtype_code(Krows) if row_dtype is None else row_dtype, _ptr(K_stage),
                                             _ptr(V_stage), _ptr(idx_local), _ptr(union_count), _stream(stream)))
+
+    def fathom_selftest_wait_expiry(self, tries: int = 200, stream=None):
+        self._check(lib.fathom_selftest_wait_expiry(self._h, tries, _stream(stream)))
 
     def fathom_device_status(self, stream=None) -> int:
         st = C.c_uint32(0)

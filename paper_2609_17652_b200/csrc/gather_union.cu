@@ -1,6 +1,6 @@
 // fathom_gather_union: union of the winners of the query heads that share a KV head, fetched once
-// (Sec. 1: "fetches the union of the four heads' winners, at most 2048 rows per KV head"; Sec. 4 "Offload harness":
-// "the gather of the union of the selected rows over PCIe").
+// (Sec. 1: the heads of a group mostly pick the same tokens, so a KV head's distinct rows - at most G k - cross the link
+// once; Sec. 4 "Offload harness": the row fetch of a decode step is that union).
 //
 // Three kernels on the caller's stream, no host round trip:
 //   mark    every selected token sets its bit in a per-KV-head bitmap (atomic OR: idempotent, so order-free);

@@ -5,13 +5,13 @@
 //   fathom_rotate_keys    K' = (K - mu) V, the keys whose planes the rotated variant stores;
 //   fathom_rotate_query   q' = q V, from which g_j = sum_h (q'_hj)^2 lambda_j is formed by fathom_alloc_depth
 //                         (eigenvalues passed as `var`).
-// The eigen-decomposition of the 128 x 128 covariances is left to the caller (once per session and KV head).
 //
-// Rotation and covariance are the same register-tiled product  C[i][j] += P[t][i] * Q[t][j]  over a shared-memory
-// panel: 256 threads, each an 8 x 8 block of the 128 x 128 result (columns split 4 + 4 so that the 16-byte panel
-// loads of neighbouring lanes are contiguous).  They run in plain fp32 FMAs in a fixed order: the rotated keys feed
-// a quantiser whose codes must not depend on the machine, which rules out tf32; a tensor-core version would need a
-// three-way split of the operands.
+// This file holds the statistics kernels, the entry points and the plain-fp32 variants of rotation and covariance
+// (FATHOM_ROTATE_PATH=simt, FATHOM_CALIBRATE_PATH=simt); the default paths are the tcgen05 kernels of klt_tc.cu, which
+// split both operands into tf32 head and tail so that the rotated keys, which feed a quantiser, keep fp32 accuracy.
+// The fp32 variants are the same register-tiled product  C[i][j] += P[t][i] * Q[t][j]  over a shared-memory panel:
+// 256 threads, each an 8 x 8 block of the 128 x 128 result (columns split 4 + 4 so that the 16-byte panel loads of
+// neighbouring lanes are contiguous), plain FMAs in a fixed order.
 #include "fathom_common.cuh"
 
 #include <cstdlib>

@@ -67,8 +67,8 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
 }
 // Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < WAIT_TRIES; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t tries = WAIT_TRIES) {
+  for (uint32_t i = 0; i < tries; ++i) {
     uint32_t done;
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                  : "=r"(done) : "r"(bar), "r"(parity) : "memory");
@@ -76,6 +76,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (i > 64) __nanosleep(32);
   }
   return false;
+}
+
+// The give-up path of the bounded wait, exercised on its own: one thread waits `tries` times on a barrier that nothing will
+// ever arrive on (no copy, no MMA, nothing asynchronous is outstanding), reports FATHOM_DEV_WAIT_EXPIRED and returns.
+__global__ void wait_expiry_selftest_kernel(uint32_t* dev_status, uint32_t tries) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(b, 0, tries)) atomicOr(dev_status, FATHOM_DEV_WAIT_EXPIRED);
+  }
 }
 
 // ---- basis prepared for the MMA: transposed (K-major for the B operand) and split into tf32 head and tail
@@ -776,6 +788,13 @@ int fathom_launch_rotate_build_tc(fathom_ctx* ctx, const fathom_layout* L, const
                                                                               scales, n, L->plane_stride_words, L->scale_stride,
                                                                               ctx->dev_status);
   }
+  FATHOM_CUDA_TRY(ctx, cudaGetLastError());
+  return FATHOM_OK;
+}
+
+extern "C" int fathom_selftest_wait_expiry(fathom_ctx* ctx, int tries, void* stream) {
+  if (!ctx || tries < 1 || tries > 4096) return FATHOM_ERR_INVALID_ARG;
+  wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->dev_status, (uint32_t)tries);
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

@@ -15,34 +15,6 @@ namespace {
 constexpr int AT_THREADS = FATHOM_ATTN_CHUNK;   // 128 threads: one per row, then one per channel
 constexpr int AT_WARPS = AT_THREADS / 32;
 
-__device__ __forceinline__ float dot_row(const __nv_bfloat16* row, const float* sq) {
-  const uint4* r = reinterpret_cast<const uint4*>(row);
-  float acc = 0.0f;
-#pragma unroll
-  for (int v = 0; v < FATHOM_D / 8; ++v) {
-    const uint4 x = __ldg(r + v);
-    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      acc = fmaf(__uint_as_float(w[c] << 16), sq[v * 8 + 2 * c], acc);
-      acc = fmaf(__uint_as_float(w[c] & 0xffff0000u), sq[v * 8 + 2 * c + 1], acc);
-    }
-  }
-  return acc;
-}
-__device__ __forceinline__ float dot_row(const float* row, const float* sq) {
-  const float4* r = reinterpret_cast<const float4*>(row);
-  float acc = 0.0f;
-#pragma unroll
-  for (int v = 0; v < FATHOM_D / 4; ++v) {
-    const float4 x = __ldg(r + v);
-    acc = fmaf(x.x, sq[v * 4 + 0], acc);
-    acc = fmaf(x.y, sq[v * 4 + 1], acc);
-    acc = fmaf(x.z, sq[v * 4 + 2], acc);
-    acc = fmaf(x.w, sq[v * 4 + 3], acc);
-  }
-  return acc;
-}
 // eight consecutive channels of a row, as loaded (converted to fp32 only when used, to keep many rows in flight)
 struct Raw8h { uint4 x; };
 struct Raw8f { float4 a, b; };
@@ -61,27 +33,6 @@ __device__ __forceinline__ void unpack(const Raw8f& r, float v[8]) {
 template <typename T> struct RawOf;
 template <> struct RawOf<__nv_bfloat16> { using type = Raw8h; };
 template <> struct RawOf<float> { using type = Raw8f; };
-// eight consecutive channels of a row (one 16-byte load in bf16, two in fp32)
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float v[8]) {
-  const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
-  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-  for (int c = 0; c < 4; ++c) { v[2 * c] = __uint_as_float(w[c] << 16); v[2 * c + 1] = __uint_as_float(w[c] & 0xffff0000u); }
-}
-__device__ __forceinline__ void load8(const float* p, float v[8]) {
-  const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-}
-__device__ __forceinline__ void load4(const __nv_bfloat16* p, float v[4]) {
-  const uint2 x = __ldg(reinterpret_cast<const uint2*>(p));
-  v[0] = __uint_as_float(x.x << 16); v[1] = __uint_as_float(x.x & 0xffff0000u);
-  v[2] = __uint_as_float(x.y << 16); v[3] = __uint_as_float(x.y & 0xffff0000u);
-}
-__device__ __forceinline__ void load4(const float* p, float v[4]) {
-  const float4 x = __ldg(reinterpret_cast<const float4*>(p));
-  v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(AT_THREADS)
 attend_partial_kernel(const float* __restrict__ q, const T* __restrict__ Krows, const T* __restrict__ Vrows,

@@ -40,6 +40,28 @@ def test_static_entry_matches_context_entry_on_two_calls_in_a_row():
         assert np.array_equal(g, w), call                     # same kernels, same order: in fact identical
 
 
+def test_static_entry_at_its_limit_then_a_small_call_with_fp32_rows():
+    """Exactly FATHOM_ATTEND_STATIC_MAX_CHUNKS chunks (32 heads x ceil(8192 / 128) = 2048: the last element of the built-in
+    array is used), then a much smaller call with fp32 rows: both bit for bit what the context-based entry point gives."""
+    from paper_2609_17652_b200 import binding as fb
+    scale = 1.0 / math.sqrt(128)
+    for call, (seed, n, Hkv, Hq, k, f32) in enumerate([(5, 9000, 8, 32, 8192, False), (6, 3000, 2, 8, 200, True)]):
+        assert Hq * ((k + 127) // 128) <= fb.ATTEND_STATIC_MAX_CHUNKS
+        lay = fb.make_layout(Hkv, Hq, n)
+        q, Kr, Vr, idx = _case(seed, n, Hkv, Hq, k)
+        if f32:
+            Kr, Vr = Kr.float(), Vr.float()
+        ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+        want = torch.full((Hq, 128), float("nan"), device="cuda")
+        ctx.fathom_sparse_attend(lay, q, Kr, Vr, idx, k, scale, want)
+        got = torch.full((Hq, 128), float("nan"), device="cuda")
+        fb.fathom_sparse_attend_static(lay, q, Kr, Vr, idx, k, scale, got)
+        torch.cuda.synchronize()
+        ctx.close()
+        assert torch.isfinite(got).all(), call
+        assert torch.equal(got, want), call
+
+
 def test_static_entry_rejects_sizes_beyond_its_built_in_scratch():
     from paper_2609_17652_b200 import binding as fb
     lay = fb.make_layout(8, 32, 20000)
