@@ -239,7 +239,7 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
  *                        sum (x - shift)(x - shift)^T is accumulated on the tensor cores (tf32 operands split in head
  *                        and tail, fp32 accumulation per CTA) together with the per-channel sums S, and a reduction
  *                        in fp64 gives mean = shift + S / n, cov = (sum - S S^T / n) / (n - 1); fixed order throughout.
- *                        The eigen-decomposition of the 128 x 128 covariances is the caller's (once per session).
+ *                        fathom_klt_basis turns the covariances into bases and eigenvalues.
  *                        Uses the context scratch.  FATHOM_CALIBRATE_PATH=simt: two passes in plain fp32 FMAs.
  *   fathom_rotate_keys:  K_rot [Hkv][n][d] fp32 = (K - mean) basis, basis [Hkv][d][d] row-major with the
  *                        directions in its columns; tensor cores, tf32 operands split in head and tail (three
@@ -248,6 +248,13 @@ int fathom_gather_union(fathom_ctx* ctx, const fathom_layout* layout, const int3
  * K is [Hkv][n][d], FATHOM_F32 or FATHOM_BF16, 16-byte aligned, like basis, cov and K_rot. */
 int fathom_calibrate(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype, float* mean,
                      float* cov, void* stream);
+/*   fathom_klt_basis:    basis [Hkv][d][d] (fp32, row-major, directions in its columns) and eigenvalues [Hkv][d] (fp32,
+ *                        descending) of cov [Hkv][d][d] (its symmetric part is used): two-sided cyclic Jacobi in fp64, one
+ *                        CTA per KV head, rotations accumulated in fp32, fixed order (bit-reproducible); every direction is
+ *                        signed so that its largest component is positive.  About 6 ms for 8 KV heads, once per session.  The eigenvalues
+ *                        are the `var` of fathom_alloc_depth for the rotated store. */
+int fathom_klt_basis(fathom_ctx* ctx, const fathom_layout* layout, const float* cov, float* basis, float* eigenvalues,
+                     void* stream);
 int fathom_rotate_keys(fathom_ctx* ctx, const fathom_layout* layout, const void* K, int k_dtype,
                        const float* mean, const float* basis, float* K_rot, void* stream);
 int fathom_rotate_query(fathom_ctx* ctx, const fathom_layout* layout, const float* q, const float* basis,

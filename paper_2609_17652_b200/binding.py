@@ -24,7 +24,7 @@ EXPORTS = ["fathom_create", "fathom_destroy", "fathom_scratch_bytes", "fathom_st
            "fathom_topk", "fathom_sparse_attend", "fathom_sparse_attend_static", "fathom_gather_union",
            "fathom_scan_topk", "fathom_calibrate", "fathom_rotate_keys", "fathom_rotate_query",
            "fathom_channel_variance", "fathom_plan_layer_budgets", "fathom_topk_passes", "fathom_build_planes_rotated", "fathom_scan_batch",
-           "fathom_scan_set_ctas_per_plan", "fathom_selftest_wait_expiry"]
+           "fathom_scan_set_ctas_per_plan", "fathom_selftest_wait_expiry", "fathom_klt_basis"]
 
 
 class Layout(C.Structure):
@@ -64,6 +64,7 @@ def _load() -> C.CDLL:
     lib.fathom_calibrate.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_rotate_keys.argtypes = [vp, LP, vp, i32, vp, vp, vp, vp]
     lib.fathom_rotate_query.argtypes = [vp, LP, vp, vp, vp, vp]
+    lib.fathom_klt_basis.argtypes = [vp, LP, vp, vp, vp, vp]
     lib.fathom_channel_variance.argtypes = [vp, LP, vp, i32, vp, vp, vp]
     lib.fathom_plan_layer_budgets.argtypes = [vp, i32, i32, vp, C.c_double, vp]
     lib.fathom_topk_passes.argtypes = [LP, i32, i32, i32]
@@ -181,6 +182,9 @@ class Context:
 
     def fathom_channel_variance(self, layout, K, mean, var, stream=None):
         self._check(lib.fathom_channel_variance(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(var), _stream(stream)))
+
+    def fathom_klt_basis(self, layout, cov, basis, eigenvalues, stream=None):
+        self._check(lib.fathom_klt_basis(self._h, C.byref(layout), _ptr(cov), _ptr(basis), _ptr(eigenvalues), _stream(stream)))
 
     def fathom_rotate_keys(self, layout, K, mean, basis, K_rot, stream=None):
         self._check(lib.fathom_rotate_keys(self._h, C.byref(layout), _ptr(K), _dtype_code(K), _ptr(mean), _ptr(basis),

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfathom.so")
-SOURCES = ["fathom_api.cu", "build_planes.cu", "alloc_depth.cu", "scan.cu", "scan_simt.cu", "topk.cu", "sparse_attend.cu", "gather_union.cu", "klt.cu", "klt_tc.cu", "layer_plan.cu"]
+SOURCES = ["fathom_api.cu", "build_planes.cu", "alloc_depth.cu", "scan.cu", "scan_simt.cu", "topk.cu", "sparse_attend.cu", "gather_union.cu", "klt.cu", "klt_tc.cu", "klt_eig.cu", "layer_plan.cu"]
 
 
 def nvcc_path() -> str:

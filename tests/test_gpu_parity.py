@@ -405,6 +405,94 @@ def test_klt_rotated_store(n):
     assert np.all(g["depth"].sum(1) == 48)
 
 
+@pytest.mark.parametrize("case", ["keys", "few_keys", "identity", "blocks"])
+def test_klt_basis_on_the_device(case):
+    """fathom_klt_basis against the oracle's eigen-decomposition on what does not depend on signs or on the order inside
+    (nearly) equal eigenvalues: the eigenvalues themselves, V^T V = I, V diag(lambda) V^T = C, the directions of
+    well-separated eigenvalues; covariances of correlated keys, of fewer keys than channels (rank-deficient), the
+    identity (fully degenerate) and a block matrix with repeated eigenvalues."""
+    from paper_2609_17652_b200 import binding as fb
+    Hkv, Hq = 2, 8
+    g = torch.Generator(device="cuda").manual_seed(5)
+    if case in ("keys", "few_keys"):
+        n = 5000 if case == "keys" else 60
+        L = make_layer(max(n, 256), Hkv, Hq, seed=43, device="cuda")
+        mix = torch.linalg.qr(torch.randn(Hkv, 128, 128, generator=g, device="cuda"))[0]
+        K = (torch.bmm(L.K[:, :n], mix) + 0.25).contiguous()
+        C = torch.stack([torch.cov(K[h].double().T) for h in range(Hkv)]).float().contiguous()
+    elif case == "identity":
+        C = torch.eye(128, device="cuda").repeat(Hkv, 1, 1).contiguous()
+    else:
+        B4 = torch.tensor([[2.0, 1.0, 0, 0], [1.0, 2.0, 0, 0], [0, 0, 5.0, 0], [0, 0, 0, 5.0]], device="cuda")
+        C = torch.block_diag(*[B4] * 32).repeat(Hkv, 1, 1).contiguous()
+    lay = fb.make_layout(Hkv, Hq, 1000)
+    ctx = fb.Context(0, 0)
+    V = torch.full((Hkv, 128, 128), float("nan"), device="cuda"); lam = torch.full((Hkv, 128), float("nan"), device="cuda")
+    ctx.fathom_klt_basis(lay, C, V, lam)
+    V2 = torch.empty_like(V); lam2 = torch.empty_like(lam)
+    ctx.fathom_klt_basis(lay, C, V2, lam2)
+    torch.cuda.synchronize()
+    assert torch.equal(V, V2) and torch.equal(lam, lam2)                       # bit-reproducible
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+    Ch = C.cpu().numpy().astype(np.float64)
+    Ch = 0.5 * (Ch + Ch.transpose(0, 2, 1))
+    V_ref, lam_ref = O.klt_basis(Ch)
+    Vh, lh = V.cpu().numpy().astype(np.float64), lam.cpu().numpy().astype(np.float64)
+    for h in range(Hkv):
+        top = max(lam_ref[h].max(), 1e-30)
+        assert np.all(np.diff(lh[h]) <= 0) and np.all(lh[h] >= 0)
+        assert np.all(np.abs(lh[h] - lam_ref[h]) <= 1e-5 * top)
+        assert np.abs(Vh[h].T @ Vh[h] - np.eye(128)).max() <= 2e-5
+        assert np.abs(Vh[h] @ np.diag(lh[h]) @ Vh[h].T - Ch[h]).max() <= 2e-5 * np.abs(Ch[h]).max()
+        assert np.all(Vh[h][np.abs(Vh[h]).argmax(axis=0), np.arange(128)] > 0)  # every direction's largest component is positive
+        gap = np.minimum(np.abs(np.diff(lam_ref[h], prepend=np.inf)), np.abs(np.diff(lam_ref[h], append=-np.inf)))
+        for j in np.nonzero(gap > 1e-3 * top)[0]:                             # a well-separated eigenvalue fixes its direction
+            assert abs(Vh[h][:, j] @ V_ref[h][:, j]) >= 1 - 1e-4, (h, j)
+
+
+def test_rotated_store_built_with_library_calls_only():
+    """Session calibration end to end on the device: fathom_calibrate -> fathom_klt_basis -> fathom_rotate_keys /
+    fathom_rotate_query, then the five calls on the rotated store, every stage against the oracle on the stage's own input."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hkv, Hq, G, k = 9000, 2, 8, 4, 128
+    L = make_layer(n, Hkv, Hq, seed=47, device="cuda")
+    mix = torch.linalg.qr(torch.randn(Hkv, 128, 128, device="cuda"))[0]
+    K = (torch.bmm(L.K, mix) + 0.5).contiguous()
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    mean = torch.zeros((Hkv, 128), device="cuda"); cov = torch.zeros((Hkv, 128, 128), device="cuda")
+    V = torch.zeros((Hkv, 128, 128), device="cuda"); lam = torch.zeros((Hkv, 128), device="cuda")
+    K_rot = torch.full((Hkv, n, 128), float("nan"), device="cuda"); q_rot = torch.zeros((Hq, 128), device="cuda")
+    ctx.fathom_calibrate(lay, K, mean, cov)
+    ctx.fathom_klt_basis(lay, cov, V, lam)
+    ctx.fathom_rotate_keys(lay, K, mean, V, K_rot)
+    ctx.fathom_rotate_query(lay, L.q, V, q_rot)
+    torch.cuda.synchronize()
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+    Kh = K.cpu().numpy()
+    Kr_ref = O.rotate_keys(Kh, mean.cpu().numpy(), V.cpu().numpy())
+    rown = np.linalg.norm(Kr_ref, axis=2, keepdims=True)
+    assert np.all(np.abs(K_rot.cpu().numpy() - Kr_ref) <= 1e-5 * rown + 1e-6)
+    # the rotated keys are decorrelated: their covariance is diag(lambda) up to the accuracy of the statistics
+    Cr = np.stack([np.cov(Kr_ref[h].T) for h in range(Hkv)])
+    lh = lam.cpu().numpy().astype(np.float64)
+    for h in range(Hkv):
+        assert np.abs(Cr[h] - np.diag(lh[h])).max() <= 1e-4 * lh[h].max()
+    # scores are preserved up to the constant q . mu (Sec. 3.5): q'.k' + q.mu = q.k
+    qh, muh = L.q.cpu().numpy().astype(np.float64), mean.cpu().numpy().astype(np.float64)
+    i = np.arange(0, n, 997)
+    for hq in range(Hq):
+        kv = hq // G
+        lhs = Kr_ref[kv][i] @ q_rot.cpu().numpy().astype(np.float64)[hq] + qh[hq] @ muh[kv]
+        rhs = Kh[kv][i].astype(np.float64) @ qh[hq]
+        assert np.all(np.abs(lhs - rhs) <= 1e-4 * np.linalg.norm(Kh[kv][i], axis=1) * np.linalg.norm(qh[hq]))
+    L.K, L.q, L.var = K_rot, q_rot, lam
+    g_, ref = check_all(L, B=48, k=k, hpp=G)
+    assert np.all(g_["depth"].sum(1) == 48)
+
+
 @pytest.mark.parametrize("n,dtype", [(1, torch.float32), (777, torch.float32), (1024, torch.float32), (40000 + 13, torch.float32),
                                      (9000, torch.bfloat16)])
 def test_channel_variance_kernel(n, dtype):
