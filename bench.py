@@ -69,6 +69,9 @@ def parse_args():
                          "one decode step over --layers independently seeded layers")
     ap.add_argument("--config5", action="store_true",
                     help="the budget sweep at n = 1M (water-filled budgets and fixed top-r channels) instead of the default step")
+    ap.add_argument("--plan-layers", action="store_true",
+                    help="per-layer budgets: measure every layer's error at every level, plan at mean --budget, re-run; use with "
+                         "--layers L --n N")
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--lanes", type=int, default=4, help="config 4: stream lanes over which the sessions are spread")
     ap.add_argument("--no-batch", action="store_true", help="config 4: one fathom_scan per session instead of fathom_scan_batch")
@@ -814,6 +817,91 @@ def run_config5(args):
                               "a needle is off by about 1; every stage is in parity with the oracle at every budget"}))
 
 
+# ------------------------------------------------------------------------------------------------ per-layer budgets
+PLAN_LEVELS = [24, 32, 40, 48, 64, 80, 96, 128]
+
+
+def layer_recipe(layer: int):
+    """How the synthetic layers of the per-layer budget experiment differ: the spread of the channel scales and the number
+    of outlier channels change from layer to layer (a concentrated layer needs fewer bits than a flat one)."""
+    his = [4.0, 2.0, 8.0, 1.0, 3.0, 6.0]
+    return dict(sigma_lo=0.1, sigma_hi=his[layer % len(his)], n_outliers=[4, 2, 0, 4, 1, 3][layer % 6])
+
+
+def measure_layer_errors(fb, ctx, lay, layers_inputs, levels, k, hpp, stream):
+    """err[l][i]: mean over the query heads of the relative L2 error of the attention output of layer l at budget levels[i]
+    (decode step through the library: alloc_depth, scan, topk, sparse_attend) against dense attention over all rows (a
+    measurement aid in plain torch fp64 on the stored bf16 rows, not part of the library).  Also returns, per layer and
+    level, the bits per token read and the depth sums (the budgets as fathom_alloc_depth granted them)."""
+    dev = layers_inputs[0].K.device
+    Hkv, Hq, d, n = lay.n_kv_heads, lay.n_q_heads, lay.d, lay.n
+    G = Hq // Hkv
+    planes = torch.zeros((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
+    scales = torch.zeros((Hkv, d, lay.scale_stride), dtype=torch.int16, device=dev)
+    depth = torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev)
+    scores = torch.zeros((Hq, lay.score_stride), dtype=torch.float32, device=dev)
+    idx = torch.zeros((Hq, k), dtype=torch.int32, device=dev)
+    out = torch.zeros((Hq, d), dtype=torch.float32, device=dev)
+    err, bits, sums = [], [], []
+    for L in layers_inputs:
+        ctx.fathom_build_planes(lay, L.K, planes, scales, stream)
+        dense = torch.zeros((Hq, d), dtype=torch.float64, device=dev)
+        for kv in range(Hkv):
+            e = (L.q[kv * G:(kv + 1) * G].double() @ L.Krows[kv].double().T) / math.sqrt(d)
+            dense[kv * G:(kv + 1) * G] = torch.softmax(e, dim=1) @ L.Vrows[kv].double()
+        row_e, row_b, row_s = [], [], []
+        for B in levels:
+            ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, B, hpp, depth, stream)
+            ctx.fathom_scan(lay, planes, scales, L.q, depth, hpp, scores, stream)
+            ctx.fathom_topk(lay, scores, k, 0, 0, idx, stream)
+            ctx.fathom_sparse_attend(lay, L.q, L.Krows, L.Vrows, idx, k, 1.0 / math.sqrt(d), out, stream)
+            torch.cuda.synchronize()
+            rel = torch.linalg.norm(out.double() - dense, dim=1) / torch.linalg.norm(dense, dim=1)
+            dh = depth.cpu().numpy()
+            row_e.append(float(rel.mean())); row_b.append(float(np.mean([bits_per_token(r) for r in dh])))
+            row_s.append([int(r.sum()) for r in dh])
+        err.append(row_e); bits.append(row_b); sums.append(row_s)
+    return err, bits, sums
+
+
+def run_plan_layers(args):
+    """Per-layer budgets (Sec. 3.4) closed on synthetic data: the error of every layer at every budget level is measured
+    through the library, fathom_plan_layer_budgets turns the table into one budget per layer at the target mean, and the
+    decode step is run again with those budgets; reported against the flat budget at the same mean."""
+    from paper_2609_17652_b200 import binding as fb
+    from workloads.synth import make_layer
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n, Hkv, Hq, d, k, hpp = args.n, WORKLOAD["Hkv"], WORKLOAD["Hq"], WORKLOAD["d"], args.k, WORKLOAD["heads_per_plan"]
+    nl, target = args.layers, float(args.budget)
+    lay = fb.make_layout(Hkv, Hq, n, d)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    st = torch.cuda.current_stream()
+    Ls = [make_layer(n, Hkv, Hq, d, seed=6, layer=l, device=str(dev), **layer_recipe(l)) for l in range(nl)]
+    err, bits, sums = measure_layer_errors(fb, ctx, lay, Ls, PLAN_LEVELS, k, hpp, st)
+    choice = fb.fathom_plan_layer_budgets(err, PLAN_LEVELS, target)
+    planned = [PLAN_LEVELS[c] for c in choice]
+    flat_i = PLAN_LEVELS.index(int(target)) if int(target) in PLAN_LEVELS else None
+    res = {"metric": "attention_rel_l2_error_at_equal_mean_bits", "unit": "relative L2 error (mean over layers and heads)",
+           "data": "synthetic", "n_gpus": 1,
+           "config": {"workload": "per-layer budgets (Sec. 3.4) on synthetic layers of varying channel spread", "n": n, "layers": nl,
+                      "kv_heads": Hkv, "q_heads": Hq, "k": k, "levels": PLAN_LEVELS, "target_mean_budget": target,
+                      "layer_recipes": [layer_recipe(l) for l in range(nl)]},
+           "error_table": [[round(e, 5) for e in row] for row in err],
+           "planned_budgets": planned, "planned_mean_budget": sum(planned) / nl,
+           "planned_mean_error": float(np.mean([err[l][choice[l]] for l in range(nl)])),
+           "planned_mean_bits_per_token": float(np.mean([bits[l][choice[l]] for l in range(nl)])),
+           "granted_depth_sums_at_planned_budgets": [sums[l][choice[l]] for l in range(nl)]}
+    if flat_i is not None:
+        res["flat_mean_error"] = float(np.mean([err[l][flat_i] for l in range(nl)]))
+        res["flat_mean_bits_per_token"] = float(np.mean([bits[l][flat_i] for l in range(nl)]))
+    res["value"] = res["planned_mean_error"]
+    res["higher_is_better"] = False
+    res["device_status"] = ctx.fathom_device_status()
+    ctx.close()
+    print(json.dumps(res))
+
+
 # ------------------------------------------------------------------------------------------------ one stage
 STAGES = ["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "rotate_build", "calibrate", "variance", "union"]
 
@@ -1031,6 +1119,8 @@ if __name__ == "__main__":
     a = parse_args()
     if a.stage:
         run_stage(a)
+    elif a.plan_layers:
+        run_plan_layers(a)
     elif a.config4:
         run_config4(a)
     elif a.config5:

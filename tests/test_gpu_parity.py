@@ -764,3 +764,33 @@ def test_single_pass_calibration_with_drifting_and_outlying_keys():
     scale = np.abs(C_ref).max(axis=(1, 2), keepdims=True)
     assert np.all(np.abs(cov.cpu().numpy() - C_ref) <= 2e-5 * scale)
     ctx.close()
+
+
+def test_per_layer_budgets_closed_on_synthetic_layers():
+    """Sec. 3.4 end to end: the error of every synthetic layer at every level measured through the library, the greedy plan
+    of fathom_plan_layer_budgets (equal to the oracle's on the same table), and the planned budgets passed through
+    fathom_alloc_depth: the granted depths of layer l sum to its planned budget, and the budgets stay within the target."""
+    import bench
+    from paper_2609_17652_b200 import binding as fb
+    n, Hkv, Hq, k, hpp, nl, target = 20000, 2, 8, 256, 4, 5, 48.0
+    levels = [24, 32, 48, 64, 96]
+    lay = fb.make_layout(Hkv, Hq, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    Ls = [make_layer(n, Hkv, Hq, seed=6, layer=l, device="cuda", **bench.layer_recipe(l)) for l in range(nl)]
+    err, bits, sums = bench.measure_layer_errors(fb, ctx, lay, Ls, levels, k, hpp, torch.cuda.current_stream())
+    assert ctx.fathom_device_status() == 0
+    choice = fb.fathom_plan_layer_budgets(err, levels, target)
+    assert choice == list(O.plan_layer_budgets(np.array(err), levels, target))
+    planned = [levels[c] for c in choice]
+    assert sum(planned) <= target * nl
+    # no single raise still fits that would lower the error: the plan is not trivially stuck at the lowest level
+    assert sum(planned) > levels[0] * nl
+    depth = torch.zeros((Hq // hpp, 128), dtype=torch.uint8, device="cuda")
+    for l, L in enumerate(Ls):
+        ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, planned[l], hpp, depth)
+        torch.cuda.synchronize()
+        assert np.all(depth.cpu().numpy().sum(1) == planned[l])
+        assert sums[l][choice[l]] == [planned[l]] * (Hq // hpp)
+    for l in range(nl):                                                        # more bits are read at higher levels
+        assert all(b1 > b0 for b0, b1 in zip(bits[l], bits[l][1:]))
+    ctx.close()

@@ -56,17 +56,19 @@ def mix_seed(seed0: int, session: int = 0, layer: int = 0) -> int:
 
 def make_layer(n: int, Hkv: int = 8, Hq: int = 32, d: int = 128, seed: int = 0,
                session: int = 0, layer: int = 0, device: str = "cpu",
-               want_rows: bool = True) -> LayerInputs:
+               want_rows: bool = True, sigma_lo: float = 0.1, sigma_hi: float = 4.0, n_outliers: int = 4) -> LayerInputs:
+    """sigma_lo, sigma_hi, n_outliers: the channel spread of the recipe (defaults: the recipe of the module docstring);
+    the per-layer budget experiments vary them from layer to layer, as real layers differ in how concentrated they are."""
     dev = torch.device(device)
     gen = torch.Generator(device=dev)
     gen.manual_seed(mix_seed(seed, session, layer))
     G = Hq // Hkv
 
     u = torch.rand(Hkv, d, generator=gen, device=dev, dtype=torch.float64)
-    sigma = torch.exp(math.log(0.1) + u * (math.log(4.0) - math.log(0.1)))
+    sigma = torch.exp(math.log(sigma_lo) + u * (math.log(sigma_hi) - math.log(sigma_lo)))
     for h in range(Hkv):
         out_ch = torch.randperm(d, generator=gen, device=dev)[:4]
-        sigma[h, out_ch] = 16.0
+        sigma[h, out_ch[:n_outliers]] = 16.0
     sigma = sigma.to(torch.float32)
 
     q = torch.randn(Hq, d, generator=gen, device=dev, dtype=torch.float32)
