@@ -903,7 +903,7 @@ def run_plan_layers(args):
 
 
 # ------------------------------------------------------------------------------------------------ one stage
-STAGES = ["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "rotate_build", "calibrate", "variance", "union"]
+STAGES = ["build", "alloc", "scan", "topk", "attend", "scan_topk", "rotate", "rotate_build", "calibrate", "variance", "union", "klt_basis"]
 
 
 def run_stage(a):
@@ -933,6 +933,11 @@ def run_stage(a):
         cov = torch.zeros(Hkv, d, d, device=dev)
         basis = torch.linalg.qr(torch.randn(Hkv, d, d, device=dev))[0].contiguous()
         K_rot = torch.empty(Hkv, n, d, device=dev) if a.stage == "rotate" else None
+    if a.stage == "klt_basis":
+        X = torch.randn(Hkv, 4096, d, device=dev) * torch.exp(torch.randn(Hkv, 1, d, device=dev))
+        cov = torch.stack([torch.cov((X[h] @ torch.linalg.qr(torch.randn(d, d, device=dev))[0]).T) for h in range(Hkv)]).contiguous()
+        basis = torch.empty(Hkv, d, d, device=dev)
+        lam = torch.empty(Hkv, d, device=dev)
     if a.stage in ("build", "rotate_build", "scan", "scan_topk"):
         planes = torch.randint(-(1 << 62), 1 << 62, (Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, device=dev)
         scales = torch.rand(Hkv, d, lay.scale_stride, device=dev).mul_(0.5).add_(0.01).to(torch.float16).view(torch.int16)
@@ -966,6 +971,8 @@ def run_stage(a):
     def run():
         if a.stage == "union":
             ctx.fathom_gather_union(lay, idx, a.k, Kr, Vr, Kst, Vst, loc, cnt, st)
+        elif a.stage == "klt_basis":
+            ctx.fathom_klt_basis(lay, cov, basis, lam, st)
         elif a.stage == "build":
             ctx.fathom_build_planes(lay, K, planes, scales, st)
         elif a.stage == "alloc":

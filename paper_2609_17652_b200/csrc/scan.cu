@@ -44,7 +44,7 @@ constexpr int STAGE_KSTEPS = 10;                             // 16 rows per mma;
 constexpr int WORD_STAGE_BYTES = 7680;                       // staged plane words of one stage (padded rows)
 constexpr int SCALE_STAGE_BYTES = 4608;                      // staged fp16 scales of one stage (padded rows)
 #ifndef FATHOM_SCAN_CTAS_PER_SM
-#define FATHOM_SCAN_CTAS_PER_SM 6
+#define FATHOM_SCAN_CTAS_PER_SM 4                               // 16 warps per SM with ~115 registers each beat 24 warps with 80
 #endif
 constexpr int CTAS_PER_SM = FATHOM_SCAN_CTAS_PER_SM;
 
