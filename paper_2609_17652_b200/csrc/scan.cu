@@ -381,35 +381,41 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       __syncwarp();
     };
 
-    // ---- a whole 16-block stage of NKS x 16 rows, single pass: the warp's four blocks are 256 tokens, and a lane takes 32
-    //      consecutive ones (half a block: ONE 32-bit load per row gives all their bits, and one scale pair per row pair
-    //      serves them all), eight at a time (byte k of the loaded words): slice j of the accumulators then holds
-    //      tokens 8 k + 2 j (mma row gq) and 8 k + 2 j + 1 (row gq + 8) of the lane's 32
-    auto half_blocks = [&](auto nksc, int blk0) {
-      constexpr int NKS = decltype(nksc)::value;
-      using GE = Geo<16>;
-      const int mine = warp * 4 + (gq >> 1);                   // my block of the stage, and my half of it
-      const unsigned char* wp = M.words[buf] + (2 * t4) * GE::ROW_BYTES + mine * 8 + (gq & 1) * 4;
+    // ---- a whole stage of TB blocks and NKS x 16 rows, single pass: the warp's TB / 4 blocks are 16 TB tokens, and a lane
+    //      takes 2 TB consecutive ones (TB = 16: half a block, TB = 8: a quarter): ONE load of TB / 4 bytes per row gives all
+    //      their bits, and one scale pair per row pair serves them all.  They are worked eight at a time (byte k of the
+    //      loaded words): slice j of the accumulators then holds tokens 8 k + 2 j (mma row gq) and 8 k + 2 j + 1 (row gq + 8)
+    //      of the lane's tokens
+    auto owned_tokens = [&](auto tbc, auto nksc, int blk0) {
+      constexpr int TB = decltype(tbc)::value, NKS = decltype(nksc)::value;
+      constexpr int BYTES = TB / 4;                            // plane bytes per row and lane
+      using GE = Geo<TB>;
+      const int mine = warp * (TB / 4) + (gq * BYTES) / 8;     // my block of the stage
+      const int off = (gq * BYTES) % 8;                        // where my bytes start in its words
+      const unsigned char* wp = M.words[buf] + (2 * t4) * GE::ROW_BYTES + mine * 8 + off;
       const uint16_t* sp = reinterpret_cast<const uint16_t*>(M.scale[buf]) + (2 * t4) * GE::SCALE_ELEMS + mine;
       uint32_t w[NKS][4], S[NKS][2];
       uint2 bf[NKS];
+      auto plane_bytes = [](const unsigned char* p) -> uint32_t {
+        return BYTES == 4 ? *reinterpret_cast<const uint32_t*>(p) : (uint32_t)*reinterpret_cast<const uint16_t*>(p);
+      };
 #pragma unroll
       for (int ks = 0; ks < NKS; ++ks) {
         bf[ks] = M.bfr[ks][lane];
         const unsigned char* wk = wp + ks * (16 * GE::ROW_BYTES);
-        w[ks][0] = *reinterpret_cast<const uint32_t*>(wk);
-        w[ks][1] = *reinterpret_cast<const uint32_t*>(wk + GE::ROW_BYTES);
-        w[ks][2] = *reinterpret_cast<const uint32_t*>(wk + 8 * GE::ROW_BYTES);
-        w[ks][3] = *reinterpret_cast<const uint32_t*>(wk + 9 * GE::ROW_BYTES);
+        w[ks][0] = plane_bytes(wk);
+        w[ks][1] = plane_bytes(wk + GE::ROW_BYTES);
+        w[ks][2] = plane_bytes(wk + 8 * GE::ROW_BYTES);
+        w[ks][3] = plane_bytes(wk + 9 * GE::ROW_BYTES);
         const uint16_t* sk = sp + ks * (16 * GE::SCALE_ELEMS);
         S[ks][0] = __byte_perm(sk[0], sk[GE::SCALE_ELEMS], 0x5410);
         S[ks][1] = __byte_perm(sk[8 * GE::SCALE_ELEMS], sk[9 * GE::SCALE_ELEMS], 0x5410);
       }
       const uint32_t n = (uint32_t)B.n[item];
-      const uint32_t tok0 = (uint32_t)(blk0 + mine) * FATHOM_BLOCK + (gq & 1) * 32;      // my first token
-      const uint32_t dst0 = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)mine * FATHOM_BLOCK + (gq & 1) * 32 : tok0;
+      const uint32_t tok0 = (uint32_t)(blk0 + mine) * FATHOM_BLOCK + off * 8;            // my first token
+      const uint32_t dst0 = MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + mine) * FATHOM_BLOCK + off * 8 : tok0;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < BYTES; ++k) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f;
 #pragma unroll
@@ -441,11 +447,12 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       const int s0 = pass * GE::ROWS, sc = min(GE::ROWS, nrows - s0), nks = (sc + 15) >> 4;
       const int blk0 = first_block(g) + u * TB;
       const uint32_t n = (uint32_t)B.n[item];                  // n < 2^31
-      if (TB == 16 && npass == 1 && nks >= 1 && nks <= 3 && (uint32_t)(blk0 + TB) * FATHOM_BLOCK <= n) {
-        // ---- the common stage (a plan of up to 48 rows, a whole tile of a long sequence)
-        if (nks == 3) half_blocks(std::integral_constant<int, 3>(), blk0);
-        else if (nks == 2) half_blocks(std::integral_constant<int, 2>(), blk0);
-        else half_blocks(std::integral_constant<int, 1>(), blk0);
+      if constexpr (TB >= 8) if (npass == 1 && nks >= 1 && (uint32_t)(blk0 + TB) * FATHOM_BLOCK <= n) {
+        // ---- the common stages (plans of up to 96 rows, whole sub-tiles of a long sequence)
+        constexpr int K0 = TB == 16 ? 0 : 3;                   // TB = 8 serves 49 .. 96 rows: 4 .. 6 steps of 16
+        if (nks == K0 + 3) owned_tokens(tbc, std::integral_constant<int, K0 + 3>(), blk0);
+        else if (nks == K0 + 2) owned_tokens(tbc, std::integral_constant<int, K0 + 2>(), blk0);
+        else owned_tokens(tbc, std::integral_constant<int, K0 + 1>(), blk0);
         return;
       }
 #pragma unroll 1
