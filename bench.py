@@ -72,9 +72,8 @@ def parse_args():
     ap.add_argument("--plan-layers", action="store_true",
                     help="per-layer budgets: measure every layer's error at every level, plan at mean --budget, re-run; use with "
                          "--layers L --n N")
-    ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--layers", type=int, default=None, help="config 4: layers timed (default 36); --plan-layers: synthetic layers (default 12)")
     ap.add_argument("--lanes", type=int, default=4, help="config 4: stream lanes over which the sessions are spread")
-    ap.add_argument("--no-batch", action="store_true", help="config 4: one fathom_scan per session instead of fathom_scan_batch")
     ap.add_argument("--stage", choices=STAGES, help="time ONE stage on small synthetic buffers instead of the bench (for profilers)")
     ap.add_argument("--iters", type=int, default=10, help="--stage: timed launches")
     ap.add_argument("--kv-heads", type=int, default=WORKLOAD["Hkv"], help="--stage only")
@@ -629,127 +628,185 @@ def e2e_leg(args, layers, stage, out, stream, keys_per_step):
 
 
 # ------------------------------------------------------------------------------------------------ config 4
-def run_config4(args):
-    """Agentic multi-session batch: 16 concurrent sessions, n log-uniform in [65536, 1048576] (ragged, not multiples
-    of 64), Qwen3-8B layer shape, planes of all sessions in pinned host memory, B = 48, k = 2048.  One decode step =
-    for every layer and every session: alloc_depth -> scan (planes read over the host link) -> top-k -> attention.
-    Layers are independently seeded and processed one at a time with reused buffers (36 layers of planes would be
-    111 GB of pinned memory); the time per layer is what is reported."""
-    from paper_2609_17652_b200 import binding as fb
-    from workloads.synth import make_layer, session_lengths
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    Hkv, Hq, d, B, k, hpp = 8, 32, 128, 48, 2048, 4
-    lengths = session_lengths(16, 65536, 1048576, seed=0)
-    nmax = max(lengths)
-    lay_max = fb.make_layout(Hkv, Hq, nmax, d)
-    # stream lanes (context + stream + work buffers each): while one session's top-k and attention run, the next
-    # sessions' scans already pull their planes over the host link
-    stream = torch.cuda.current_stream()
-    lanes = []
-    for li in range(max(1, args.lanes)):
-        lanes.append({"ctx": fb.Context(0, fb.fathom_scratch_bytes(lay_max, k)),
-                      "stream": stream if li == 0 else torch.cuda.Stream(),
-                      "depth": torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev),
-                      "scores": torch.zeros((Hq, lay_max.score_stride), dtype=torch.float32, device=dev),
-                      "idx": torch.zeros((Hq, k), dtype=torch.int32, device=dev),
-                      "out": torch.zeros((Hq, d), dtype=torch.float32, device=dev)})
-    ctx = lanes[0]["ctx"]
-    # per-session device state (rows stay in HBM) and pinned host stores, allocated once and reused by every layer
-    sess = []
-    for s_i, n in enumerate(lengths):
-        lay = fb.make_layout(Hkv, Hq, n, d)
-        sess.append({"n": n, "lay": lay,
-                     "hp": torch.empty((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, pin_memory=True),
-                     "hs": torch.empty((Hkv, d, lay.scale_stride), dtype=torch.int16, pin_memory=True),
-                     "Kr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, device=dev),
-                     "Vr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, device=dev),
-                     "depth": torch.zeros((Hq // hpp, d), dtype=torch.uint8, device=dev), "q": None, "var": None})
-    planes = torch.empty((Hkv, d, 4, lay_max.plane_stride_words), dtype=torch.int64, device=dev)
-    scales = torch.empty((Hkv, d, lay_max.scale_stride), dtype=torch.int16, device=dev)
-    layer_ms, bytes_link = [], 0.0
-    for layer in range(args.layers):
-        for s_i, S in enumerate(sess):                           # build this layer's stores (not timed: once per sequence)
-            L = make_layer(S["n"], Hkv, Hq, d, seed=4, session=s_i, layer=layer, device=str(dev))
+class Config4:
+    """Agentic multi-session batch (config 4): 16 concurrent sessions, n log-uniform in [65536, 1048576] (ragged, not
+    multiples of 64), Qwen3-8B layer shape, B = 48, k = 2048.  As in the paper's offload harness (Sec. 4) the planes, the
+    scales AND the K/V rows of every session live in pinned host memory.  One decode step of a layer = for every session:
+    alloc_depth -> scan (planes read over the host link; the sessions of a group in one fathom_scan_batch launch) ->
+    top-k -> union of each group's winners fetched once from the host rows (fathom_gather_union) -> attention over the
+    staged rows.  The scans run on the main stream; top-k, row fetch and attention of a session run on one of `lanes` side
+    streams, so the link carries the next group's planes while the previous group's rows and selection are worked on.
+    Layers are independently seeded and processed one at a time with reused buffers (36 layers of planes and rows would be
+    1.1 TB of pinned memory): build_layer() refills the host stores (untimed), decode_layer() enqueues the step."""
+
+    def __init__(self, fb, dev, lanes=4, n_sessions=16, lo=65536, hi=1048576, k=2048, budget=48, host_rows=True):
+        from workloads.synth import session_lengths
+        self.fb, self.dev = fb, dev
+        self.Hkv, self.Hq, self.d, self.B, self.k, self.hpp = 8, 32, 128, budget, k, 4
+        self.G = self.Hq // self.Hkv
+        Hkv, Hq, d = self.Hkv, self.Hq, self.d
+        self.lengths = session_lengths(n_sessions, lo, hi, seed=0)
+        nmax = max(self.lengths)
+        self.lay_max = fb.make_layout(Hkv, Hq, nmax, d)
+        self.lay_stage = fb.make_layout(Hkv, Hq, self.G * k, d)
+        self.main = torch.cuda.current_stream()
+        self.ctx = fb.Context(dev.index or 0, fb.fathom_scratch_bytes(self.lay_max, k))
+        self.lanes = []
+        for _ in range(max(1, lanes)):
+            self.lanes.append({"ctx": fb.Context(dev.index or 0, fb.fathom_scratch_bytes(self.lay_max, k)), "stream": torch.cuda.Stream(),
+                               "Kst": torch.empty((Hkv, self.G * k, d), dtype=torch.bfloat16, device=dev),
+                               "Vst": torch.empty((Hkv, self.G * k, d), dtype=torch.bfloat16, device=dev)})
+        self.sess = []
+        for n in self.lengths:
+            lay = fb.make_layout(Hkv, Hq, n, d)
+            rows = dict(pin_memory=True) if host_rows else dict(device=dev)
+            self.sess.append({
+                "n": n, "lay": lay,
+                "hp": torch.empty((Hkv, d, 4, lay.plane_stride_words), dtype=torch.int64, pin_memory=True),
+                "hs": torch.empty((Hkv, d, lay.scale_stride), dtype=torch.int16, pin_memory=True),
+                "Kr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, **rows), "Vr": torch.empty((Hkv, n, d), dtype=torch.bfloat16, **rows),
+                "q": None, "var": None,
+                "depth": torch.zeros((Hq // self.hpp, d), dtype=torch.uint8, device=dev),
+                "scores": torch.zeros((Hq, lay.score_stride), dtype=torch.float32, device=dev),
+                "idx": torch.zeros((Hq, k), dtype=torch.int32, device=dev), "idx_local": torch.zeros((Hq, k), dtype=torch.int32, device=dev),
+                "ucount": torch.zeros((Hkv,), dtype=torch.int32, device=dev), "out": torch.zeros((Hq, d), dtype=torch.float32, device=dev)})
+        self.planes = torch.empty((Hkv, d, 4, self.lay_max.plane_stride_words), dtype=torch.int64, device=dev)
+        self.scales = torch.empty((Hkv, d, self.lay_max.scale_stride), dtype=torch.int16, device=dev)
+
+    def build_layer(self, layer, seed=4, on_session=None):
+        """The stores of one layer for every session (not timed: once per sequence).  on_session(i, L, planes, scales) is
+        called while the session's generated layer L and its device-side planes are alive."""
+        from workloads.synth import make_layer
+        Hkv, d = self.Hkv, self.d
+        for i, S in enumerate(self.sess):
+            L = make_layer(S["n"], Hkv, self.Hq, d, seed=seed, session=i, layer=layer, device=str(self.dev))
             lay = S["lay"]
-            pv = planes.view(-1)[:Hkv * d * 4 * lay.plane_stride_words].view(Hkv, d, 4, lay.plane_stride_words)
-            sv = scales.view(-1)[:Hkv * d * lay.scale_stride].view(Hkv, d, lay.scale_stride)
-            ctx.fathom_build_planes(lay, L.K, pv, sv, stream)
+            pv = self.planes.view(-1)[:Hkv * d * 4 * lay.plane_stride_words].view(Hkv, d, 4, lay.plane_stride_words)
+            sv = self.scales.view(-1)[:Hkv * d * lay.scale_stride].view(Hkv, d, lay.scale_stride)
+            self.ctx.fathom_build_planes(lay, L.K, pv, sv, self.main)
             S["hp"].copy_(pv); S["hs"].copy_(sv)
             S["Kr"].copy_(L.Krows); S["Vr"].copy_(L.Vrows)
             S["q"], S["var"] = L.q, L.var
+            if on_session is not None:
+                torch.cuda.synchronize()
+                on_session(i, L, pv, sv)
             del L
         torch.cuda.synchronize()
+
+    def decode_layer(self):
+        """Enqueues the decode step of the current layer over all sessions; everything is joined back on the main stream."""
+        fb, k, hpp, main = self.fb, self.k, self.hpp, self.main
+        nl = len(self.lanes)
+        sm = 1.0 / math.sqrt(self.d)
+        fork = torch.cuda.Event(); fork.record(main)
+        for W in self.lanes:
+            W["stream"].wait_event(fork)
+        for g0 in range(0, len(self.sess), nl):
+            grp = self.sess[g0:g0 + nl]
+            items = []
+            for S in grp:
+                self.ctx.fathom_alloc_depth(S["lay"], S["q"], S["var"], fb.DEPTH_WATERFILL, self.B, hpp, S["depth"], main)
+                items.append((S["lay"], S["hp"], S["hs"], S["q"], S["depth"], S["scores"]))
+            self.ctx.fathom_scan_batch(items, hpp, main)
+            done = torch.cuda.Event(); done.record(main)
+            for j, S in enumerate(grp):
+                W = self.lanes[j]
+                st, c = W["stream"], W["ctx"]
+                st.wait_event(done)
+                c.fathom_topk(S["lay"], S["scores"], k, 0, 0, S["idx"], st)
+                c.fathom_gather_union(S["lay"], S["idx"], k, S["Kr"], S["Vr"], W["Kst"], W["Vst"], S["idx_local"], S["ucount"], st)
+                c.fathom_sparse_attend(self.lay_stage, S["q"], W["Kst"], W["Vst"], S["idx_local"], k, sm, S["out"], st)
+        for W in self.lanes:
+            join = torch.cuda.Event(); join.record(W["stream"])
+            main.wait_event(join)
+
+    def link_bytes(self):
+        """Bytes one decode step of the current layer moves over the host link: plane words and scales of the active
+        rows (from the depths the step left behind) and the distinct rows fetched (from the union counts)."""
+        pl = 0.0
+        for S in self.sess:
+            pl += sum(bits_per_token(r) for r in S["depth"].cpu().numpy()) / 8.0 * S["n"] * max(1, self.hpp // 4)
+        rows = sum(int(S["ucount"].sum().item()) for S in self.sess) * self.d * 2 * 2
+        return pl, float(rows)
+
+    def status(self):
+        st = self.ctx.fathom_device_status(self.main)
+        for W in self.lanes:
+            st |= W["ctx"].fathom_device_status(W["stream"])
+        return st
+
+    def close(self):
+        self.ctx.close()
+        for W in self.lanes:
+            W["ctx"].close()
+
+
+def probe_host_link(dev, stream):
+    """One pinned -> device copy of 1 GiB, best of 10: the denominator of every host-link fraction."""
+    src = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    best = 1e9
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); dst.copy_(src, non_blocking=True); b.record(stream)
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b))
+    return (1 << 30) / (best * 1e-3) / 1e9
+
+
+def run_config4(args):
+    """Times one decode step per layer over --layers independently seeded layers (default here: all 36) of the 16-session
+    batch; reports the per-layer median, the total over the layers measured, and the host-link rate (planes + rows)."""
+    from paper_2609_17652_b200 import binding as fb
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    C = Config4(fb, dev, lanes=args.lanes)
+    link = probe_host_link(dev, C.main)
+    layer_ms, plane_b, row_b = [], [], []
+    for layer in range(args.layers):
+        C.build_layer(layer)
         ts = []
-        for it in range(4):                                      # the decode step of this layer over the 16 sessions
+        for it in range(3):                                      # one untimed pass, then two timed ones of the same layer
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            fork = torch.cuda.Event()
-            a.record(stream)
-            fork.record(stream)
-            for W in lanes[1:]:
-                W["stream"].wait_event(fork)
-            if args.no_batch:
-                for s_i, S in enumerate(sess):
-                    W = lanes[s_i % len(lanes)]
-                    lay, st, c = S["lay"], W["stream"], W["ctx"]
-                    c.fathom_alloc_depth(lay, S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, W["depth"], st)
-                    c.fathom_scan(lay, S["hp"], S["hs"], S["q"], W["depth"], hpp, W["scores"], st)
-                    c.fathom_topk(lay, W["scores"], k, 0, 0, W["idx"], st)
-                    c.fathom_sparse_attend(lay, S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
-            else:
-                # the sessions in groups of len(lanes): one batched scan per group on the first lane keeps the host link
-                # busy, then each session's top-k and attention run on its own lane while the next group is scanned
-                nl = len(lanes)
-                for g0 in range(0, len(sess), nl):
-                    grp = sess[g0:g0 + nl]
-                    if g0:                                       # the group's score buffers are free again?
-                        for W in lanes[1:]:
-                            e = torch.cuda.Event(); e.record(W["stream"]); stream.wait_event(e)
-                    items = []
-                    for j, S in enumerate(grp):
-                        W = lanes[j]
-                        ctx.fathom_alloc_depth(S["lay"], S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, S["depth"], stream)
-                        items.append((S["lay"], S["hp"], S["hs"], S["q"], S["depth"], W["scores"]))
-                    ctx.fathom_scan_batch(items, hpp, stream)
-                    done = torch.cuda.Event(); done.record(stream)
-                    for j, S in enumerate(grp):
-                        W = lanes[j]
-                        st, c = W["stream"], W["ctx"]
-                        st.wait_event(done)
-                        c.fathom_topk(S["lay"], W["scores"], k, 0, 0, W["idx"], st)
-                        c.fathom_sparse_attend(S["lay"], S["q"], S["Kr"], S["Vr"], W["idx"], k, 1.0 / math.sqrt(d), W["out"], st)
-            for W in lanes[1:]:
-                join = torch.cuda.Event()
-                join.record(W["stream"])
-                stream.wait_event(join)
-            b.record(stream)
+            a.record(C.main); C.decode_layer(); b.record(C.main)
             torch.cuda.synchronize()
             if it:
                 ts.append(a.elapsed_time(b))
-        layer_ms.append(statistics.median(ts))
-        if layer == 0:
-            depth = lanes[0]["depth"]
-            for S in sess:
-                ctx.fathom_alloc_depth(S["lay"], S["q"], S["var"], fb.DEPTH_WATERFILL, B, hpp, depth, stream)
-                torch.cuda.synchronize()
-                bytes_link += sum(bits_per_token(r) for r in depth.cpu().numpy()) / 8.0 * S["n"] * max(1, hpp // 4)
-    status = 0
-    for W in lanes:
-        status |= W["ctx"].fathom_device_status(W["stream"])
-    total_tokens = sum(lengths)
-    ms = statistics.mean(layer_ms)
+        layer_ms.append(min(ts))
+        pb, rb = C.link_bytes()
+        plane_b.append(pb); row_b.append(rb)
+    # the zero-copy scan alone, session by session (layer: the last one built): link rate against session length
+    per_session = []
+    for S in C.sess:
+        ts = []
+        for it in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(C.main); C.ctx.fathom_scan(S["lay"], S["hp"], S["hs"], S["q"], S["depth"], C.hpp, S["scores"], C.main); b.record(C.main)
+            torch.cuda.synchronize()
+            if it:
+                ts.append(a.elapsed_time(b))
+        nbytes = sum(bits_per_token(r) for r in S["depth"].cpu().numpy()) / 8.0 * S["n"]
+        g = nbytes / (statistics.median(ts) * 1e-3) / 1e9
+        per_session.append({"n": S["n"], "scan_ms": round(statistics.median(ts), 3), "gbs": round(g, 2), "frac_of_measured_link": round(g / link, 3)})
+    status = C.status()
+    total_tokens = sum(C.lengths)
+    med = statistics.median(layer_ms)
+    total_b = float(np.mean(plane_b) + np.mean(row_b))
     print(json.dumps({
-        "metric": METRIC, "value": total_tokens * Hkv / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.layers,
-        "ms_per_layer": round(ms, 3), "ms_per_decode_step_36_layers": round(ms * 36, 1), "higher_is_better": True,
+        "metric": METRIC, "value": total_tokens * C.Hkv / (med * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.layers,
+        "ms_per_layer_median": round(med, 3), "ms_per_layer_min": round(min(layer_ms), 3), "ms_per_layer_max": round(max(layer_ms), 3),
+        "ms_decode_step_all_layers_measured": round(sum(layer_ms), 2), "layers_measured": args.layers, "higher_is_better": True,
         "dtype": "u64 bit planes + f32 accumulate", "data": "synthetic",
-        "config": {"workload": "agentic multi-session batch (config 4): 16 sessions, planes in pinned host memory",
-                   "session_tokens": lengths, "total_tokens": total_tokens, "kv_heads": Hkv, "q_heads": Hq, "budget_bits": B,
-                   "k": k, "layers_measured": args.layers, "layers_of_the_model": 36, "stream_lanes": len(lanes),
-                   "scan": "one fathom_scan per session" if args.no_batch else "fathom_scan_batch per group of sessions"},
-        "bytes_over_link_per_layer": bytes_link, "host_link_gbs": round(bytes_link / (ms * 1e-3) / 1e9, 2),
-        "device_status": status}))
-    for W in lanes:
-        W["ctx"].close()
+        "config": {"workload": "agentic multi-session batch (config 4): 16 sessions, planes, scales and K/V rows in pinned host memory",
+                   "session_tokens": C.lengths, "total_tokens": total_tokens, "kv_heads": C.Hkv, "q_heads": C.Hq, "budget_bits": C.B,
+                   "k": C.k, "layers_of_the_model": 36, "stream_lanes": len(C.lanes),
+                   "step": "per session: alloc_depth, scan (fathom_scan_batch per group of sessions), topk, gather_union from host rows, "
+                           "sparse_attend over the staged rows"},
+        "bytes_over_link_per_layer": {"planes_and_scales": float(np.mean(plane_b)), "rows": float(np.mean(row_b)), "total": total_b},
+        "host_link_gbs": round(total_b / (med * 1e-3) / 1e9, 2), "link_peak_gbs": round(link, 2),
+        "frac_of_measured_link": round(total_b / (med * 1e-3) / 1e9 / link, 4),
+        "zero_copy_scan_alone_by_session": per_session, "device_status": status}))
+    C.close()
 
 
 # ------------------------------------------------------------------------------------------------ config 5
@@ -1124,6 +1181,8 @@ def run_reference(args):
 
 if __name__ == "__main__":
     a = parse_args()
+    if a.layers is None:
+        a.layers = 36 if a.config4 else 12
     if a.stage:
         run_stage(a)
     elif a.plan_layers:

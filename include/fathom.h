@@ -71,6 +71,10 @@ typedef struct {
   int64_t score_stride;        /* floats per query-head score row; >= n, multiple of 4 (16 B) */
 } fathom_layout;
 
+/* Strides that are multiples of 128 bytes (16 words, 64 scales, 32 scores) make every row start on a memory-line boundary;
+ * the scan of a host-resident store reaches its best link rate only then (a 128-byte run that straddles two lines costs two
+ * requests on the link). */
+
 typedef struct fathom_ctx fathom_ctx;   /* opaque: device id, scratch arena, status word */
 
 /* ---- context ------------------------------------------------------------------------------

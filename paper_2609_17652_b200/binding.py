@@ -33,10 +33,15 @@ class Layout(C.Structure):
                 ("score_stride", C.c_int64)]
 
 
-def make_layout(Hkv: int, Hq: int, n: int, d: int = 128) -> Layout:
-    """Tight strides rounded up to the 16-byte multiples the layout requires."""
+def make_layout(Hkv: int, Hq: int, n: int, d: int = 128, row_align_bytes: int = 128) -> Layout:
+    """Strides rounded up so that every (head, channel, plane) row of words, every row of scales and every score row
+    starts on a `row_align_bytes` boundary (default 128: a row's 128-byte runs then never straddle a memory line, which
+    matters most when the store is read over the host link).  row_align_bytes = 16 gives the tightest strides the
+    layout allows."""
     nb = (n + 63) // 64
-    return Layout(Hkv, Hq, d, 0, n, (nb + 1) // 2 * 2, (nb + 7) // 8 * 8, (n + 3) // 4 * 4)
+    a = max(16, row_align_bytes)
+    rnd = lambda x, m: (x + m - 1) // m * m
+    return Layout(Hkv, Hq, d, 0, n, rnd(nb, a // 8), rnd(nb, a // 2), rnd(n, a // 4))
 
 
 def _load() -> C.CDLL:

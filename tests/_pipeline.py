@@ -8,11 +8,11 @@ import torch
 
 
 def run_gpu(L, B, k, hpp, mode=0, n_sink=0, n_local=0, ctx=None, rows_dtype=torch.bfloat16, host_planes=False,
-            depth_override=None, stages=("build", "alloc", "scan", "topk", "attend")):
+            depth_override=None, stages=("build", "alloc", "scan", "topk", "attend"), row_align_bytes=128):
     """L: workloads.synth.LayerInputs with tensors on cuda.  Returns a dict of numpy arrays (tight strides)."""
     from paper_2609_17652_b200 import binding as fb
     dev = L.K.device
-    lay = fb.make_layout(L.Hkv, L.Hq, L.n, L.d)
+    lay = fb.make_layout(L.Hkv, L.Hq, L.n, L.d, row_align_bytes=row_align_bytes)
     nb = (L.n + 63) // 64
     own = ctx is None
     if own:

@@ -43,8 +43,10 @@ def test_layout_struct_matches_header(fb):
     assert C.sizeof(fb.Layout) == 4 * 4 + 4 * 8
     lay = fb.make_layout(8, 32, 1 << 20)
     assert lay.plane_stride_words == 16384 and lay.scale_stride == 16384 and lay.score_stride == 1 << 20
-    odd = fb.make_layout(1, 1, 65)
+    odd = fb.make_layout(1, 1, 65, row_align_bytes=16)              # the tightest strides the layout allows
     assert odd.plane_stride_words == 2 and odd.scale_stride == 8 and odd.score_stride == 68
+    odd = fb.make_layout(1, 1, 65)                                  # default: every row starts on a 128-byte boundary
+    assert odd.plane_stride_words == 16 and odd.scale_stride == 64 and odd.score_stride == 96
 
 
 def test_scratch_bytes_and_host_side_rejection(fb):

@@ -179,3 +179,66 @@ def test_fused_scan_topk_on_a_sequence_longer_than_the_one_cta_sample_covers():
     assert np.array_equal(idx.cpu().numpy(), g["idx"])
     assert ctx.fathom_device_status() == 0
     ctx.close()
+
+
+def test_config4_sixteen_sessions_three_layers_in_the_bench_configuration():
+    """Config 4 at its stated size, in the launch configuration bench.py --config4 times: 16 sessions of 96 k .. 1.04 M
+    tokens (ragged), planes, scales and K/V rows in pinned host memory, B = 48, k = 2048, three independently seeded
+    layers.  Per layer and session: depths bit-exact against the oracle; plane words and scales of sampled blocks against
+    the oracle's build on those blocks; sampled scores one by one from the plane words; the full top-k of the GPU's own
+    scores; the union of each group's winners; attention over the staged rows against the oracle on the picked rows."""
+    import bench
+    from paper_2609_17652_b200 import binding as fb
+    dev = torch.device("cuda", 0)
+    C = bench.Config4(fb, dev, lanes=4)
+    assert len(C.lengths) == 16 and min(C.lengths) >= 65536 and max(C.lengths) > 1_000_000
+    rng = np.random.default_rng(4)
+    G, k, hpp = C.G, C.k, C.hpp
+    for layer in range(3):
+        sampled = {}
+
+        def keep_blocks(i, L, pv, sv, sampled=sampled):
+            nb = (L.n + 63) // 64
+            blocks = np.unique(np.concatenate([[0, nb - 1], rng.integers(0, nb, 6)]))
+            sampled[i] = [(int(b), L.K[:, b * 64:min((b + 1) * 64, L.n)].cpu().numpy()) for b in blocks]
+
+        C.build_layer(layer, on_session=keep_blocks)
+        C.decode_layer()
+        torch.cuda.synchronize()
+        assert C.status() == 0
+        for i, S in enumerate(C.sess):
+            n, nb = S["n"], (S["n"] + 63) // 64
+            q, var = S["q"].cpu().numpy(), S["var"].cpu().numpy()
+            depth = S["depth"].cpu().numpy()
+            assert np.array_equal(depth, O.alloc_depth(q, var, "waterfill", C.B, hpp)), (layer, i)
+            planes = S["hp"].numpy().view(np.uint64)[..., :nb]
+            scales = S["hs"].numpy().view(np.float16)[..., :nb]
+            for b, Kb in sampled[i]:                                            # the store: sampled blocks, all heads and channels
+                p_ref, s_ref = O.build_planes(Kb)
+                assert np.array_equal(planes[..., b:b + 1], p_ref) and np.array_equal(scales[..., b:b + 1].view(np.uint16), s_ref.view(np.uint16)), (layer, i, b)
+            scores = S["scores"][:, :n].cpu().numpy()
+            tok = np.concatenate([[0, 63, 64, n - 1], rng.integers(0, n, 12)])
+            for h in range(0, C.Hq, 5):                                         # scores: sampled tokens of sampled heads, one by one
+                ref = O.scan_tokens(planes, scales, q, depth, hpp, h, tok)
+                rms = np.sqrt(np.mean(scores[h].astype(np.float64) ** 2))
+                assert np.all(np.abs(scores[h, tok] - ref) <= 1e-5 * np.maximum(np.abs(ref), rms)), (layer, i, h)
+            idx = S["idx"].cpu().numpy()
+            assert np.array_equal(idx, O.topk(scores.astype(np.float64), k)), (layer, i)      # full stable sort of the GPU's own scores
+            # union of the winners and attention over the staged rows; the oracle sees only the picked rows (compacted)
+            Kh, Vh = S["Kr"].view(torch.int16).numpy(), S["Vr"].view(torch.int16).numpy()
+            u_all = [np.unique(idx[kv * G:(kv + 1) * G]) for kv in range(C.Hkv)]
+            assert np.array_equal(S["ucount"].cpu().numpy(), [len(u) for u in u_all]), (layer, i)
+            loc = S["idx_local"].cpu().numpy()
+            bf = lambda a: (a.astype(np.uint16).astype(np.uint32) << 16).view(np.float32)   # bf16 bit patterns -> fp32
+            umax = max(len(u) for u in u_all)
+            Kc, Vc = np.zeros((C.Hkv, umax, 128), np.float32), np.zeros((C.Hkv, umax, 128), np.float32)
+            for kv in range(C.Hkv):
+                Kc[kv, :len(u_all[kv])] = bf(Kh[kv][u_all[kv]])
+                Vc[kv, :len(u_all[kv])] = bf(Vh[kv][u_all[kv]])
+            for h in range(C.Hq):
+                assert np.array_equal(u_all[h // G][loc[h]], idx[h]), (layer, i, h)          # every pick found at its staged position
+            o_ref = O.sparse_attend(q, Kc, Vc, loc, 1 / math.sqrt(128))
+            o = S["out"].cpu().numpy()
+            rel = np.linalg.norm(o - o_ref, axis=1) / np.linalg.norm(o_ref, axis=1)
+            assert rel.max() <= 2e-3, (layer, i, rel.max())
+    C.close()

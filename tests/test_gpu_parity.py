@@ -538,6 +538,18 @@ def test_channel_variance_kernel(n, dtype):
     ctx.close()
 
 
+@pytest.mark.parametrize("n,B", [(70001, 48), (5000, 80), (3001, 200)])
+def test_tight_strides_give_what_line_aligned_strides_give(n, B):
+    """The layout only asks for 16-byte strides; rows that start in the middle of a memory line (and stages whose copies
+    straddle lines) must give the same planes, scores, picks and outputs as the 128-byte-aligned default."""
+    L = make_layer(n, Hkv=2, Hq=8, seed=13, device="cuda")
+    a = run_gpu(L, B, 64, 4)
+    b = run_gpu(L, B, 64, 4, row_align_bytes=16)
+    for key in ("planes", "scales", "depth", "scores", "idx", "out"):
+        assert np.array_equal(a[key], b[key]), key
+    assert a["status"] == 0 and b["status"] == 0
+
+
 def test_depths_above_four_are_read_as_four():
     """A depth buffer that was never written (255s) must not send the scan past its row list: it scans like all-4."""
     from paper_2609_17652_b200 import binding as fb
