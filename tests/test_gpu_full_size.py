@@ -71,6 +71,35 @@ def test_config3_million_tokens_sampled():
     rel = np.linalg.norm(g["out"] - o_ref, axis=1) / np.linalg.norm(o_ref, axis=1)
     assert rel.max() <= 2e-3
     assert g["status"] == 0
+    # the same store in pinned host memory, read zero-copy: B = 48 bit for bit the scores of the HBM-resident scan, and
+    # B = 80 (the configuration's second budget) against the oracle on sampled tokens, from HBM and from host memory
+    from paper_2609_17652_b200 import binding as fb
+    lay = fb.make_layout(8, 32, n)
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    hp = torch.empty(g["planes_t"].shape, dtype=torch.int64, pin_memory=True); hp.copy_(g["planes_t"])
+    hs = torch.empty(g["scales_t"].shape, dtype=torch.int16, pin_memory=True); hs.copy_(g["scales_t"])
+    dd = torch.from_numpy(depth).cuda()
+    sc = torch.full((32, lay.score_stride), float("nan"), device="cuda")
+    ctx.fathom_scan(lay, hp, hs, L.q, dd, 4, sc)
+    torch.cuda.synchronize()
+    assert np.array_equal(sc[:, :n].cpu().numpy(), g["scores"])
+    d80 = torch.zeros_like(dd)
+    ctx.fathom_alloc_depth(lay, L.q, L.var, fb.DEPTH_WATERFILL, 80, 4, d80)
+    d80h = d80.cpu().numpy()
+    assert np.array_equal(d80h, O.alloc_depth(q, L.var.cpu().numpy(), "waterfill", 80, 4))
+    got = []
+    for pl_, sl_ in ((g["planes_t"], g["scales_t"]), (hp, hs)):
+        sc.fill_(float("nan"))
+        ctx.fathom_scan(lay, pl_, sl_, L.q, d80, 4, sc)
+        torch.cuda.synchronize()
+        got.append(sc[:, :n].cpu().numpy())
+    assert np.array_equal(got[0], got[1])
+    for h in range(0, 32, 3):
+        ref = O.scan_tokens(planes, scales, q, d80h, 4, h, tok)
+        rms = np.sqrt(np.mean(got[0][h].astype(np.float64) ** 2))
+        assert np.all(np.abs(got[0][h, tok] - ref) <= 1e-5 * np.maximum(np.abs(ref), rms))
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
 
 
 def test_config5_budget_sweep_at_1M():
