@@ -75,7 +75,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="config 4: layers timed (default 36); --plan-layers: synthetic layers (default 12)")
     ap.add_argument("--lanes", type=int, default=4, help="config 4: stream lanes over which the sessions are spread")
     ap.add_argument("--stage", choices=STAGES, help="time ONE stage on small synthetic buffers instead of the bench (for profilers)")
-    ap.add_argument("--iters", type=int, default=10, help="--stage: timed launches")
+    ap.add_argument("--iters", type=int, default=10, help="--stage: timed samples")
+    ap.add_argument("--repeat", type=int, default=1, help="--stage: launches per timed sample (back to back; the event timer resolves ~2 us)")
     ap.add_argument("--kv-heads", type=int, default=WORKLOAD["Hkv"], help="--stage only")
     ap.add_argument("--q-heads", type=int, default=WORKLOAD["Hq"], help="--stage only")
     ap.add_argument("--heads-per-plan", dest="heads_per_plan_arg", type=int, default=WORKLOAD["heads_per_plan"], help="--stage only")
@@ -1056,10 +1057,13 @@ def run_stage(a):
         if not a.no_flush:
             flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(st); run(); e1.record(st)
+        e0.record(st)
+        for _ in range(a.repeat):
+            run()
+        e1.record(st)
         torch.cuda.synchronize()
         if it >= 3:
-            ts.append(e0.elapsed_time(e1) * 1e3)
+            ts.append(e0.elapsed_time(e1) * 1e3 / a.repeat)
     print(f"stage={a.stage} n={n} budget={a.budget} k={a.k} median_us={statistics.median(ts):.2f} min_us={min(ts):.2f} "
           f"status={ctx.fathom_device_status()}")
     ctx.close()

@@ -302,13 +302,10 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     }
     const bool more = g_next < total;
     const bool same_item = more && g_next < B.tile_end[item];
-    if (same_item) {
-      prefetch(g_next, u_next, pass_next, buf ^ 1);            // lands while this stage is scanned
-      fathom_copies_wait<1>();
-    } else {
-      fathom_copies_wait<0>();
-    }
-    __syncthreads();                                           // this stage's words and scales are in place
+    fathom_copies_wait<0>();
+    __syncthreads();                                           // this stage's words and scales are in place, and every warp has
+                                                               // left the previous stage: its buffer may be refilled
+    if (same_item) prefetch(g_next, u_next, pass_next, buf ^ 1);   // lands while this stage is scanned
 
     // ---- eight consecutive scores of head t4 (lanes with t4 < NH, tokens of an existing block): tokens tok .. tok + 7 of
     //      the session, written at position dst of the head's row (MODE 0, 1) or tested against the head's threshold (MODE 2)
@@ -489,15 +486,16 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     else compute(std::integral_constant<int, 4>());
 
     if (!more) break;
-    __syncthreads();                                           // every warp is done with this stage's buffers
     g = g_next;
     u = u_next;
     pass = pass_next;
     buf ^= 1;
     if (!same_item) {                                          // first tile of another session: nothing was fetched ahead
+      __syncthreads();                                         // every warp is done with the previous session's row list
       enter_item(g);
       prefetch(g, 0, 0, buf);
     } else if (npass > 1) {
+      __syncthreads();                                         // every warp is done with the previous pass's right operand
       fill_bfr(pass);                                          // plans of more than 160 rows: the right operand of the next pass
     }
   }
