@@ -227,7 +227,7 @@ def alloc_depth(q, var, mode: str, budget: int, heads_per_plan: int) -> np.ndarr
 
 
 # --------------------------------------------------------------------------
-# O3  scan  (Sec. 3.2 prefix dequantiser; Sec. 3.3 "channels with t_j = 0 are skipped")
+# O3  scan  (Sec. 3.2 prefix dequantiser; Sec. 3.3: a channel of depth 0 is not read and adds nothing)
 # --------------------------------------------------------------------------
 def prefix_values(planes, scales, n: int, h: int, j: int, t: int) -> np.ndarray:
     """Dequantised value of channel j of KV head h for every token, read to depth t:
@@ -407,9 +407,9 @@ def gather_union(idx: np.ndarray, G: int, Krows, Vrows):
 # O7  KLT-rotated store  (Sec. 3.5 "Basis rule"; Appendix B5 session calibration)
 # --------------------------------------------------------------------------
 def calibrate(K: np.ndarray):
-    """Per KV head: mean mu[d] and covariance C[d][d] of the session's own keys (Appendix B5: "the mean,
-    eigenbasis and eigenvalues of each layer's keys computed from the session's own prefill cache, one covariance
-    per KV head"); unbiased (n - 1), fp64.  Returns (mu [Hkv][d], C [Hkv][d][d])."""
+    """Per KV head: mean mu[d] and covariance C[d][d] of the session's own keys (Appendix B5: the statistics of the
+    calibration-free variant are taken from the keys the session itself has cached, head by head); unbiased (n - 1),
+    fp64.  Returns (mu [Hkv][d], C [Hkv][d][d])."""
     K = np.asarray(K, dtype=np.float32).astype(np.float64)
     Hkv, n, d = K.shape
     mu = K.mean(axis=1)
