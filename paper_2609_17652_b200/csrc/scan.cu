@@ -590,8 +590,9 @@ int fathom_launch_scan_sample(const fathom_layout* L, const uint64_t* planes, co
 
 int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
                               const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st) {
+  // (a programmatic dependent: the second, gated attempt then costs no launch latency when it has nothing to do)
   return dispatch_scan<2>(single_item(L, planes, scales, q, depth, nullptr, 0, 1), L->n_kv_heads, L->n_q_heads, heads_per_plan, fz,
-                          false, st);
+                          true, st);
 }
 
 extern "C" int fathom_scan_set_ctas_per_plan(int ctas) {

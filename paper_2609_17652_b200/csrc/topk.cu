@@ -219,6 +219,7 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
   __shared__ uint32_t s_warp[SAMPLE_THREADS / 32];
   cg::cluster_group cluster = cg::this_cluster();
   const int head = blockIdx.x / SAMPLE_CLUSTER, part = (int)cluster.block_rank();
+  FATHOM_PDL_WAIT();                                          // the scores come from the previous kernel (this one may be launched as its dependent)
   // the collection kernel may be launched as a programmatic dependent: let it start at once, it loads its scores while
   // this kernel runs and waits for this kernel's results only before it compares
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -915,8 +916,8 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
     // reach the bound bin, hence at least k - forced = want eligible ones
     if (sampled <= 256) {                                              // up to 4M scores per row: one CTA per head
-      topk_sample_kernel<<<Hq * SAMPLE_CLUSTER, SAMPLE_THREADS, 0, st>>>(scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k,
-                                                        S.cand_count, nullptr);
+      FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(topk_sample_kernel, dim3(Hq * SAMPLE_CLUSTER), dim3(SAMPLE_THREADS), 0, st, scores, sampled, 16 * 1024LL, score_stride, S.state, rank, (uint32_t)k,
+                                                        S.cand_count, (uint32_t*)nullptr));
     } else {
       const int reps = 8;                                              // sampled chunks per CTA
       dim3 sgrid((unsigned)((sampled + reps - 1) / reps), (unsigned)Hq);
@@ -1039,9 +1040,9 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   const uint32_t rank = estimate_rank(want, n_sample, n) + (uint32_t)n_forced;
   const bool two_attempts = !force_two_pass() && want >= 256 && (long long)rank * 2 <= k;
   if (one_cta_sample) {                                       // one CTA per head, histogram in shared memory only
-    topk_sample_kernel<<<Hq * SAMPLE_CLUSTER, SAMPLE_THREADS, 0, st>>>(S.sample, n_sample / 1024, 1024LL, S.sample_stride, S.state,
-                                                      two_attempts ? rank : (uint32_t)k, two_attempts ? (uint32_t)k : 0u, S.cand_count,
-                                                      S.cand_count2);
+    FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(topk_sample_kernel, dim3(Hq * SAMPLE_CLUSTER), dim3(SAMPLE_THREADS), 0, st, (const float*)S.sample,
+                                                 n_sample / 1024, 1024LL, S.sample_stride, S.state, two_attempts ? rank : (uint32_t)k,
+                                                 two_attempts ? (uint32_t)k : 0u, S.cand_count, S.cand_count2));
   } else {
     const int htile = hist_tile_for(n_sample, Hq);
     dim3 hgrid((unsigned)((n_sample + htile - 1) / htile), (unsigned)Hq);
