@@ -9,10 +9,16 @@
 //      the ESTIMATE, whose suffix count in the sample reaches the expected rank plus four standard deviations, and
 //      the BOUND, whose suffix count reaches k in the sample alone and therefore in the whole row;
 //   b. every CTA of the collection pass loads its 8192 scores before the sample kernel has finished (programmatic
-//      dependent launch), then appends the (score, token) pairs that reach the estimate's lower edge to the head's list;
-//   c. per head, a radix select over that list on the composite (key << 32 | ~index); the winners are placed in
-//      ascending order by a counting sort over 4096 token ranges. A head whose list came out shorter than wanted
-//      (the estimate was too high) collects again itself above the bound bin, which cannot fall short.
+//      dependent launch), marks its candidates (scores that reach the estimate's lower edge), gives each a place by a
+//      prefix count over the CTA and ONE atomic on the head's counter, and appends the (score, token) pairs;
+//   c. per head, one CTA selects among the list on the composite (key << 32 | ~index).  The short way (lists of up to
+//      16384, sequences whose bitmap fits in shared memory): a fine histogram of the candidates' distance from the
+//      threshold finds the bin of the wanted-th largest, the few members of that bin are ranked against one another,
+//      the chosen tokens are set in a bitmap and read off it in ascending order with popcounts.  The general way: a
+//      radix select over the list (11-bit digits; a chosen digit with few members is finished by ranking them), the
+//      winners placed in ascending order by a counting sort over 4096 token ranges.  A head whose list came out
+//      shorter than wanted (the estimate was too high) collects again itself above the bound bin, which cannot fall
+//      short.
 //
 // Two passes (short rows, or FATHOM_TOPK_PATH=two_pass): bucket select.
 //   1. histogram of the 12 leading key bits over all eligible tokens (one read of the scores); the CTA that
@@ -349,12 +355,12 @@ topk_filter_kernel(const float* __restrict__ scores, long long n, long long scor
 // Collection pass of the single-pass top-k: every eligible token whose score reaches the head's estimated threshold
 // (state word 6, from the histogram of every 16th chunk) is appended to the head's candidate list as a (score, token)
 // pair.
-__global__ void __launch_bounds__(FILT_THREADS)
+__global__ void __launch_bounds__(FILT_THREADS, 5)
 topk_collect_kernel(const float* __restrict__ scores, long long n, long long score_stride, Forced F,
                     const uint32_t* state, float* __restrict__ cand_score, int32_t* __restrict__ cand_idx,
                     uint32_t* __restrict__ cand_count, int ntiles) {
-  __shared__ uint16_t s_list[FILT_TILE];
-  __shared__ uint32_t s_count, s_base;
+  __shared__ uint32_t s_warp_total[FILT_THREADS / 32];
+  __shared__ uint32_t s_base;
   // one CTA per (head, tile): grid = (heads, tiles in y and z), tiles from the last to the first and all heads of a tile
   // together: the scan writes the heads' rows side by side from the first token to the last, so what it wrote last is
   // the likeliest to be in L2 still
@@ -362,7 +368,6 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   const int tile = ntiles - 1 - (int)(blockIdx.z * gridDim.y + blockIdx.y);
   if (tile < 0) return;                                        // padding of the last z slice
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) s_count = 0u;
   const float* row = scores + (size_t)head * (size_t)score_stride;
   const long long tile0 = (long long)tile * FILT_TILE;
   const long long wbase = tile0 + (long long)warp * FILT_WARP_TOKENS;
@@ -371,51 +376,76 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   if (wbase + FILT_WARP_TOKENS <= n) {                        // (uniform over the warp) no load needs a guard
     const float4* src = reinterpret_cast<const float4*>(row + wbase) + lane;
 #pragma unroll
-    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) x[it] = __ldg(src + it * 32);
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) x[it] = __ldcs(src + it * 32);     // read once: first to be evicted
   } else {
 #pragma unroll
     for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
       const long long t0 = wbase + it * 128 + lane * 4;
-      x[it] = (t0 < n) ? __ldg(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      x[it] = (t0 < n) ? __ldcs(reinterpret_cast<const float4*>(row + t0)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
   // The scores were complete before the sample kernel started; its threshold and cleared counters are needed from
   // here on (a no-op unless this kernel was launched as a programmatic dependent of the sample kernel).
   FATHOM_PDL_WAIT();
   FATHOM_PDL_RELEASE();                                       // the selection that follows may become resident now
-  __syncthreads();
   const float lo = __uint_as_float(__ldcg(state + head * 8 + 6));   // the score a candidate must reach
-  const uint32_t woff = (uint32_t)warp * FILT_WARP_TOKENS + (uint32_t)lane * 4u;   // my first token's offset in the tile
+  // ---- which of my 32 scores are candidates (bit 4 it + c), then a place for each: my candidates follow those of the
+  //      lanes before me, the warp's those of the warps before it, the CTA's block comes from ONE atomic on the head's count
+  uint32_t mine = 0;
+  if (all_elig) {                                             // (uniform over the warp) nothing else to check
 #pragma unroll
-  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
-    const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
-    if (fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])) >= lo) {  // divergent on purpose: candidates are rare
-      const uint32_t off = woff + it * 128u;
-      if (all_elig) {                                         // (uniform over the warp) nothing else to check
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+      mine |= (x[it].x >= lo ? 1u : 0u) << (4 * it);
+      mine |= (x[it].y >= lo ? 1u : 0u) << (4 * it + 1);
+      mine |= (x[it].z >= lo ? 1u : 0u) << (4 * it + 2);
+      mine |= (x[it].w >= lo ? 1u : 0u) << (4 * it + 3);
+    }
+  } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          if (e[c] >= lo) s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(off + c);
-      } else {
+    for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+      const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const long long t = tile0 + off + c;
-          if (e[c] >= lo && t < n && t >= F.sink_end && t < F.local_begin) s_list[atomicAdd(&s_count, 1u)] = (uint16_t)(off + c);
-        }
+      for (int c = 0; c < 4; ++c) {
+        const long long t = wbase + it * 128 + lane * 4 + c;
+        mine |= (e[c] >= lo && t < n && t >= F.sink_end && t < F.local_begin ? 1u : 0u) << (4 * it + c);
       }
     }
   }
+  const uint32_t cnt = __popc(mine);
+  uint32_t incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_warp_total[warp] = incl;
   __syncthreads();
-  const uint32_t cnt = s_count;
-  if (cnt == 0u) return;
-  if (threadIdx.x == 0) s_base = atomicAdd(&cand_count[head], cnt);
+  uint32_t before = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < FILT_THREADS / 32; ++w) {
+    const uint32_t c = s_warp_total[w];
+    before += w < warp ? c : 0u;
+    total += c;
+  }
+  if (total == 0u) return;                                    // (the same for every thread)
+  if (threadIdx.x == 0) s_base = atomicAdd(&cand_count[head], total);
   __syncthreads();
-  const uint32_t base = s_base;
+  if (mine == 0u) return;
+  uint32_t pos = s_base + before + incl - cnt;
   float* cs = cand_score + (size_t)head * (size_t)n;
   int32_t* ci = cand_idx + (size_t)head * (size_t)n;
-  for (uint32_t e = threadIdx.x; e < cnt; e += FILT_THREADS) {
-    const long long t = tile0 + s_list[e];
-    cs[base + e] = row[t];
-    ci[base + e] = (int32_t)t;
+#pragma unroll
+  for (int it = 0; it < FILT_WARP_TOKENS / 128; ++it) {
+    const float e[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+    if ((mine >> (4 * it)) & 15u) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if ((mine >> (4 * it + c)) & 1u) {
+          cs[pos] = e[c];
+          ci[pos] = (int32_t)(wbase + it * 128 + lane * 4 + c);
+          ++pos;
+        }
+    }
   }
 }
 
@@ -452,6 +482,206 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return s_warp[warp] + incl - v;
 }
 
+
+// The short way of the direct select, for a head whose candidates had to reach a known score `lo` and whose selection
+// bitmap fits in shared memory.  The candidates (at most 16 per thread, loaded once, kept in registers as bin and token) are counted in a
+// fine histogram of the key's distance from lo's key (2048 bins of 2^13 keys: 16 bins of the 12-bit histogram lo came
+// from; the last bin takes everything beyond).  Its suffix counts give the bin b that holds the wanted-th largest
+// candidate; candidates in bins above b are chosen at once, the few dozen members of b are listed and ranked against one
+// another on the composite (key << 32 | ~token); the chosen tokens are set in the bitmap, and a chosen token's place in
+// the ascending output is the number of set bits before it (popcounts: a running count per 16 bytes of bitmap + the
+// bits before it in its own 16 bytes): one histogram pass over the candidates, no sort.  Everything needed from global
+// memory is requested before anything is waited for.  Returns false, with nothing but the cleared bitmap and histogram
+// touched, when it does not apply: the head has to collect again (too few candidates), more than 16 candidates per
+// thread, or a bin b with more than SMALL members.  The caller then selects the general way.
+// Shared memory: bitmap of 1024 U 16-byte groups (U per thread), one group skipped after every 8 so that the threads of
+// a quarter warp, each reading its own U consecutive groups, hit different banks; running counts [1024 U] u16; tokens
+// in output order [k].
+constexpr int FINE_BINS = 2048, FINE_SHIFT = 13;
+__device__ __forceinline__ uint32_t fine_bin(float score, float lo) {
+  const uint32_t key = ordered_key(score), base = ordered_key(lo);
+  return min((key > base ? key - base : 0u) >> FINE_SHIFT, (uint32_t)(FINE_BINS - 1));
+}
+constexpr int FAST_MAXU = 12;                                 // 16-byte bitmap groups per thread: sequences of up to 1.5M tokens
+__host__ __device__ inline long long fast_select_groups(long long n) { return ((n + 127) / 128 + FIN_THREADS - 1) / FIN_THREADS; }   // U
+__host__ __device__ inline long long fast_select_bytes(long long n, int k) {
+  const long long G = fast_select_groups(n) * FIN_THREADS;
+  return (G + (G >> 3)) * 16 + G * 2 + (long long)k * 4;
+}
+constexpr int FAST_EPT = 8;                                   // candidates per thread and round of loads
+// ROUNDS = 1: lists of up to 8192 candidates; 2: up to 16384 (a second round of loads once the length is known)
+template <int SMALL, int ROUNDS>
+__device__ __forceinline__ bool select_by_fine_histogram_rounds(
+    const float* __restrict__ cs, const int32_t* __restrict__ ci, uint32_t m, const float (&sc0)[FAST_EPT], const int32_t (&ix0)[FAST_EPT],
+    uint32_t want, float lo, long long n, int k,
+    Forced F, unsigned char* s_dyn, uint32_t* s_fine, uint32_t* s_warp, int32_t* __restrict__ out, uint32_t* __restrict__ dev_status) {
+  constexpr int EPT = FAST_EPT;
+  constexpr int FPT = FINE_BINS / FIN_THREADS;                 // fine bins per thread
+  constexpr uint32_t TOKEN_BITS = 21, NONE = 0xffffffffu;      // a candidate in a register: fine bin << 21 | token
+  static_assert((long long)FAST_MAXU * FIN_THREADS * 128 <= (1ll << TOKEN_BITS) - 1, "tokens must fit beside the bin, NONE must be no token");
+  static_assert(SMALL * 8 <= FINE_BINS * 4, "the members of the split bin are listed where the fine histogram was");
+  __shared__ uint32_t s_bin, s_need_in, s_members, s_nsmall;
+  uint64_t* s_small = reinterpret_cast<uint64_t*>(s_fine);     // (free once every thread has read its bins)
+  const int tid = threadIdx.x;
+  const uint32_t U = (uint32_t)fast_select_groups(n), G = U * FIN_THREADS;
+  uint32_t* s_bits = reinterpret_cast<uint32_t*>(s_dyn);
+  const uint4* s_bits4 = reinterpret_cast<const uint4*>(s_dyn);
+  uint16_t* s_pref = reinterpret_cast<uint16_t*>(s_dyn + (size_t)(G + (G >> 3)) * 16);
+  int32_t* s_out = reinterpret_cast<int32_t*>(s_dyn + (size_t)(G + (G >> 3)) * 16 + (size_t)G * 2);
+  auto group_at = [](uint32_t g) { return g + (g >> 3); };     // where group g of the bitmap sits
+  auto set_bit = [&](uint32_t t) {
+    const uint32_t w = t >> 5;
+    atomicOr(&s_bits[(group_at(w >> 2) << 2) | (w & 3u)], 1u << (t & 31u));
+  };
+  uint32_t cand[ROUNDS * EPT];
+  if (tid == 0) { s_nsmall = 0u; s_bin = 0u; s_need_in = 0u; s_members = 0u; }
+#pragma unroll
+  for (int u = 0; u < EPT; ++u)
+    cand[u] = (uint32_t)u * FIN_THREADS + tid < m ? (fine_bin(sc0[u], lo) << TOKEN_BITS) | (uint32_t)ix0[u] : NONE;
+  if (ROUNDS == 2) {
+    float sc[EPT];
+    int32_t ix[EPT];
+#pragma unroll
+    for (int u = 0; u < EPT; ++u) {
+      const uint32_t c = (uint32_t)(EPT + u) * FIN_THREADS + tid;
+      sc[u] = c < m ? __ldcg(cs + c) : 0.0f;
+      ix[u] = c < m ? __ldcg(ci + c) : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < EPT; ++u)
+      cand[EPT + u] = (uint32_t)(EPT + u) * FIN_THREADS + tid < m ? (fine_bin(sc[u], lo) << TOKEN_BITS) | (uint32_t)ix[u] : NONE;
+  }
+  const uint32_t need0 = min(want, m);
+#pragma unroll
+  for (int u = 0; u < ROUNDS * EPT; ++u)                      // (s_fine was cleared before the wait)
+    if (cand[u] != NONE) atomicAdd(&s_fine[cand[u] >> TOKEN_BITS], 1u);
+  __syncthreads();
+  uint32_t fh[FPT], local = 0;
+#pragma unroll
+  for (int x = 0; x < FPT; ++x) {                             // descending: the block prefix is a suffix count
+    fh[x] = s_fine[FINE_BINS - 1 - (FPT * tid + x)];
+    local += fh[x];
+  }
+  uint32_t total;
+  const uint32_t above = block_exclusive_scan(local, s_warp, &total);
+  if (need0 > 0 && need0 < m && above < need0 && above + local >= need0) {
+    uint32_t run = above;
+#pragma unroll
+    for (int x = 0; x < FPT; ++x) {
+      if (run < need0 && run + fh[x] >= need0) {
+        s_bin = (uint32_t)(FINE_BINS - 1 - (FPT * tid + x));
+        s_need_in = need0 - run;
+        s_members = fh[x];
+      }
+      run += fh[x];
+    }
+  }
+  __syncthreads();
+  const uint32_t members = s_members, need_in = s_need_in;
+  const bool ranked = need0 > 0 && need0 < m && need_in != members;       // bin b is split: its members are ranked
+  if (ranked && members > (uint32_t)SMALL) return false;
+  // ---- candidates whose bin reaches take_from are chosen outright; the members of a split bin are listed (their
+  //      scores are read again: a few dozen loads per head)
+  const uint32_t take_from = need0 == 0 ? (uint32_t)FINE_BINS : (need0 >= m ? 0u : (ranked ? s_bin + 1u : s_bin));
+  const uint32_t split_bin = ranked ? s_bin : NONE;
+  uint32_t chosen = 0;                                        // bit u: my u-th candidate is chosen
+#pragma unroll
+  for (int u = 0; u < ROUNDS * EPT; ++u) {
+    if (cand[u] != NONE) {
+      const uint32_t fb = cand[u] >> TOKEN_BITS, t = cand[u] & ((1u << TOKEN_BITS) - 1u);
+      if (fb >= take_from) {
+        set_bit(t);
+        chosen |= 1u << u;
+      } else if (fb == split_bin) {
+        const uint32_t pos = atomicAdd(&s_nsmall, 1u);
+        if (pos < (uint32_t)SMALL) s_small[pos] = (((uint64_t)ordered_key(__ldcg(cs + (uint32_t)u * FIN_THREADS + tid))) << 32) | (uint32_t)~t;
+      }
+    }
+  }
+  __syncthreads();
+  uint32_t member_token = 0;
+  bool member_chosen = false;
+  if (ranked && (uint32_t)tid < members) {
+    const uint64_t mine = s_small[tid];
+    uint32_t larger = 0;
+    for (uint32_t j = 0; j < members; ++j) larger += s_small[j] > mine;
+    if (larger < need_in) {
+      member_token = ~(uint32_t)mine;
+      member_chosen = true;
+      set_bit(member_token);
+    }
+  }
+  __syncthreads();
+  // ---- set bits before every 16-byte group of the bitmap: a thread counts its own U groups, the block prefix does the rest
+  uint32_t before[FAST_MAXU], mine = 0;
+#pragma unroll
+  for (int j = 0; j < FAST_MAXU; ++j) {
+    before[j] = mine;
+    if ((uint32_t)j < U) {
+      const uint4 x = s_bits4[group_at(U * tid + j)];
+      mine += __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w);
+    }
+  }
+  uint32_t cnt;
+  const uint32_t base = block_exclusive_scan(mine, s_warp, &cnt);
+  cnt = min(cnt, (uint32_t)k);                                // = need0
+#pragma unroll
+  for (int j = 0; j < FAST_MAXU; ++j)
+    if ((uint32_t)j < U) s_pref[U * tid + j] = (uint16_t)min(base + before[j], 0xffffu);
+  __syncthreads();
+  // ---- every chosen token to its place in the output
+  auto place = [&](uint32_t t) {
+    const uint32_t w = t >> 5, g = w >> 2, q = w & 3u;
+    const uint4 x = s_bits4[group_at(g)];
+    uint32_t p = s_pref[g];
+    p += (q > 0u ? __popc(x.x) : 0) + (q > 1u ? __popc(x.y) : 0) + (q > 2u ? __popc(x.z) : 0);
+    const uint32_t own = q == 0u ? x.x : (q == 1u ? x.y : (q == 2u ? x.z : x.w));
+    p += __popc(own & ((1u << (t & 31u)) - 1u));
+    if (p < (uint32_t)k) s_out[p] = (int32_t)t;
+  };
+#pragma unroll
+  for (int u = 0; u < ROUNDS * EPT; ++u)
+    if ((chosen >> u) & 1u) place(cand[u] & ((1u << TOKEN_BITS) - 1u));
+  if (member_chosen) place(member_token);
+  __syncthreads();
+  const uint32_t n_sink = (uint32_t)F.sink_end, n_loc = (uint32_t)(n - F.local_begin);
+  for (uint32_t e = tid; e < cnt; e += FIN_THREADS) out[n_sink + e] = s_out[e];
+  for (uint32_t e = tid; e < n_sink; e += FIN_THREADS) out[e] = (int32_t)e;
+  for (uint32_t e = tid; e < n_loc; e += FIN_THREADS) out[n_sink + cnt + e] = (int32_t)(F.local_begin + e);
+  const uint32_t filled = n_sink + cnt + n_loc;
+  if (filled != (uint32_t)k) {                                // short selection (non-finite scores)
+    if (tid == 0) atomicOr(dev_status, FATHOM_DEV_TOPK_SHORT);
+    for (uint32_t e = filled + tid; e < (uint32_t)k; e += FIN_THREADS) out[e] = (int32_t)(n - 1);   // pad with the last token
+  }
+  return true;
+}
+
+template <int SMALL>
+__device__ __forceinline__ bool select_by_fine_histogram(
+    const float* __restrict__ cs, const int32_t* __restrict__ ci, long long capacity, const uint32_t* __restrict__ count_ptr,
+    bool must_reach_want, uint32_t want, const uint32_t* __restrict__ lo_ptr, long long n, int k,
+    Forced F, unsigned char* s_dyn, uint32_t* s_fine, uint32_t* s_warp, int32_t* __restrict__ out, uint32_t* __restrict__ dev_status) {
+  // ---- all loads in flight together (the candidate loads are speculative: the list's length is not known yet)
+  const int tid = threadIdx.x;
+  const uint32_t listed = __ldcg(count_ptr);
+  const float lo = __uint_as_float(__ldcg(lo_ptr));
+  float sc[FAST_EPT];
+  int32_t ix[FAST_EPT];
+#pragma unroll
+  for (int u = 0; u < FAST_EPT; ++u) {
+    const long long c = (long long)u * FIN_THREADS + tid;
+    sc[u] = c < capacity ? __ldcg(cs + c) : 0.0f;
+    ix[u] = c < capacity ? __ldcg(ci + c) : 0;
+  }
+  const uint32_t m = (uint32_t)min((long long)listed, capacity);
+  if (must_reach_want && listed < want) return false;          // (all conditions are the same for every thread)
+  if (m <= (uint32_t)(FAST_EPT * FIN_THREADS))
+    return select_by_fine_histogram_rounds<SMALL, 1>(cs, ci, m, sc, ix, want, lo, n, k, F, s_dyn, s_fine, s_warp, out, dev_status);
+  if (m <= (uint32_t)(2 * FAST_EPT * FIN_THREADS))
+    return select_by_fine_histogram_rounds<SMALL, 2>(cs, ci, m, sc, ix, want, lo, n, k, F, s_dyn, s_fine, s_warp, out, dev_status);
+  return false;
+}
+
 // DIRECT = false: candidates are the tokens of the threshold bin (their 12 leading key bits agree), scores are read
 //                  from the dense score rows, the number needed comes from the histogram state; the chosen tokens are
 //                  OR-ed into the bitmap the filter started, and topk_emit_kernel writes the indices.
@@ -468,22 +698,45 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
                    const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
                    Gate gate, const float* __restrict__ collect_scores, long long collect_stride, float* __restrict__ collect_score_out,
-                   int32_t* __restrict__ collect_idx_out, int cache_entries) {
+                   int32_t* __restrict__ collect_idx_out, int cache_entries, int lo_word, int dyn_bytes) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
-  FATHOM_PDL_WAIT();                                          // the candidates come from the previous kernel
-  FATHOM_PDL_RELEASE();                                       // the attention that follows may become resident now
-  if (!fathom_gate_open(gate)) return;
-  __shared__ uint32_t s_hist[DIGITS];
+  static_assert(FIN_THREADS == 1024, "one pair of s_diff words per lane; digits and ranges per thread");
+  static_assert(DIGITS == FINE_BINS, "the short way counts its fine histogram in s_hist");
+  constexpr int SMALL_BUCKET = 256;                           // a chosen bucket this small is finished by ranking its members
+  __shared__ __align__(8) uint32_t s_hist[DIGITS];            // (also: the members of a small bucket, as 64-bit composites)
   __shared__ uint32_t s_warp[33];
+  __shared__ uint32_t s_diff[2 * (FIN_THREADS / 32)];
   __shared__ uint64_t s_prefix;                               // decided leading bits of the threshold composite
-  __shared__ uint32_t s_need, s_bucket, s_ntok;
+  __shared__ uint32_t s_need, s_bucket, s_ntok, s_nsmall;
   extern __shared__ __align__(16) unsigned char s_dyn[];      // composite cache; DIRECT: + range counters, chosen tokens, tokens by range
   uint64_t* s_comp = reinterpret_cast<uint64_t*>(s_dyn);                        // [cache_entries]
   uint32_t* s_range = reinterpret_cast<uint32_t*>(s_comp + cache_entries);      // [SORT_BUCKETS]
   int32_t* s_tok = reinterpret_cast<int32_t*>(s_range + SORT_BUCKETS);          // [k]
   int32_t* s_sorted = s_tok + k;                                                // [k]
   const int head = blockIdx.x, tid = threadIdx.x;
+  // the short way (select_by_fine_histogram) when the candidates were counted and the bitmap of n tokens fits
+  const bool counted = DIRECT && lo_word >= 0 && fast_select_groups(n) <= FAST_MAXU && fast_select_bytes(n, k) <= (long long)dyn_bytes;
+  if (DIRECT) {                                               // shared memory only: done while the previous kernel still runs
+    if (counted) {
+      const uint32_t G = (uint32_t)fast_select_groups(n) * FIN_THREADS;
+      for (uint32_t w = tid; w < G + (G >> 3); w += FIN_THREADS) reinterpret_cast<uint4*>(s_dyn)[w] = make_uint4(0u, 0u, 0u, 0u);
+      for (int d = tid; d < DIGITS; d += FIN_THREADS) s_hist[d] = 0u;
+    } else
+      for (int d = tid; d < SORT_BUCKETS; d += FIN_THREADS) s_range[d] = 0u;
+  }
+  FATHOM_PDL_WAIT();                                          // the candidates come from the previous kernel
+  FATHOM_PDL_RELEASE();                                       // the attention that follows may become resident now
+  if (!fathom_gate_open(gate)) return;
+  if (counted) {
+    if (select_by_fine_histogram<SMALL_BUCKET>(scores + (size_t)head * (size_t)cand_capacity, cand + (size_t)head * (size_t)cand_capacity,
+                                               cand_capacity, cand_count + head, gate.mode == 5 && collect_scores != nullptr, want_direct,
+                                               state + head * 8 + lo_word, n, k, F, s_dyn, s_hist, s_warp,
+                                               idx_out + (size_t)head * k, dev_status))
+      return;
+    __syncthreads();                                          // the general way: its range counters lie where the bitmap was
+    for (int d = tid; d < SORT_BUCKETS; d += FIN_THREADS) s_range[d] = 0u;
+  }
   // dense: scores row of the head, candidate tokens [n];  direct: candidate scores and tokens [cand_capacity]
   // (when the CTA collects its own candidates they are read back through the pointers they were written through)
   const bool own_list = DIRECT && collect_scores != nullptr &&
@@ -561,9 +814,31 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       atomicAdd(&tc[i / FILT_TILE], 1u);
     }
   };
-  if (tid == 0) s_ntok = 0u;
-  if (cached)
-    for (uint32_t c = tid; c < m; c += FIN_THREADS) s_comp[c] = composite(c);
+  if (tid == 0) { s_ntok = 0u; s_nsmall = 0u; }
+  const bool from_cache = DIRECT && cached;                   // every candidate sits in shared memory from the start
+  uint64_t first = 0;                                         // a member of the set, the same for every thread
+  if (cached && m > 0) {
+    // batches of 8 per thread so that a batch's loads are in flight together; on the way: the bits in which any
+    // candidate differs from the first one
+    first = composite(0);
+    uint64_t diff = 0;
+    for (uint32_t c0 = 0; c0 < m; c0 += FIN_THREADS * 8) {
+      uint64_t comp[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t c = c0 + u * FIN_THREADS + tid;
+        comp[u] = c < m ? composite(c) : first;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t c = c0 + u * FIN_THREADS + tid;
+        if (c < m) s_comp[c] = comp[u];
+        diff |= comp[u] ^ first;
+      }
+    }
+    const uint32_t dlo = __reduce_or_sync(0xffffffffu, (uint32_t)diff), dhi = __reduce_or_sync(0xffffffffu, (uint32_t)(diff >> 32));
+    if ((tid & 31) == 0) { s_diff[2 * (tid >> 5)] = dlo; s_diff[2 * (tid >> 5) + 1] = dhi; }
+  }
   __syncthreads();
 
   // ---- radix select of the need0 largest composites among the m candidates: 11-bit digits from the top
@@ -576,20 +851,12 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       // All candidates lie in a narrow band of scores, so their leading bits agree: a digit taken there would put
       // every candidate in one histogram bin (thousands of atomics on one address).  Start below the highest bit in
       // which any two composites differ.
-      const uint64_t first = s_comp[0];
-      uint64_t diff = 0;
-      for (uint32_t c = tid; c < m; c += FIN_THREADS) diff |= s_comp[c] ^ first;
-      uint32_t dlo = __reduce_or_sync(0xffffffffu, (uint32_t)diff), dhi = __reduce_or_sync(0xffffffffu, (uint32_t)(diff >> 32));
-      if ((tid & 31) == 0) { s_hist[2 * (tid >> 5)] = dlo; s_hist[2 * (tid >> 5) + 1] = dhi; }
-      __syncthreads();
-      dlo = 0; dhi = 0;
-#pragma unroll 8
-      for (int w = 0; w < FIN_THREADS / 32; ++w) { dlo |= s_hist[2 * w]; dhi |= s_hist[2 * w + 1]; }
-      diff = ((uint64_t)dhi << 32) | dlo;
+      const uint32_t dlo = __reduce_or_sync(0xffffffffu, s_diff[2 * (tid & 31)]);       // (32 warps: one pair of words per lane)
+      const uint32_t dhi = __reduce_or_sync(0xffffffffu, s_diff[2 * (tid & 31) + 1]);
+      const uint64_t diff = ((uint64_t)dhi << 32) | dlo;
       hi = 64 - __clzll((long long)diff);                     // diff != 0: composites are distinct and m > 1
       if (hi > TOP) hi = TOP;
       common = hi >= 64 ? 0ull : (first >> hi) << hi;
-      __syncthreads();                                        // s_hist is reused by the passes
     }
     if (tid == 0) { s_prefix = common; s_need = need0; s_ncache = 0u; }
     while (hi > 0) {
@@ -636,6 +903,26 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       __syncthreads();
       hi = lo;
       if (s_need == s_bucket) break;                          // the chosen bucket is taken entirely: done
+      if (cached && s_bucket <= (uint32_t)SMALL_BUCKET) {
+        // a handful of candidates share the chosen digit: list them, rank each against the others, and the one of rank
+        // s_need is the threshold itself (composites are distinct)
+        uint64_t* s_small = reinterpret_cast<uint64_t*>(s_hist);
+        const uint64_t pfx = s_prefix;
+        const uint32_t needed = s_need, members = s_bucket;
+        for (uint32_t c = tid; c < mc; c += FIN_THREADS) {
+          const uint64_t comp = s_comp[c];
+          if ((comp >> hi) == (pfx >> hi)) s_small[atomicAdd(&s_nsmall, 1u)] = comp;    // hi < 64 here: a digit has been taken
+        }
+        __syncthreads();
+        if ((uint32_t)tid < members) {
+          const uint64_t mine = s_small[tid];
+          uint32_t larger = 0;
+          for (uint32_t j = 0; j < members; ++j) larger += s_small[j] > mine;
+          if (larger + 1u == needed) s_prefix = mine;
+        }
+        __syncthreads();
+        break;
+      }
       if (!cached && s_bucket <= (uint32_t)cache_entries) {
         // the undecided bucket fits in shared memory: pull it in, take what ranks above it, go on from there
         const uint64_t pfx = s_prefix;
@@ -669,7 +956,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     }
     thr = s_prefix;                                           // undecided low bits are zero
   }
-  if (need0 > 0) {
+  if (need0 > 0 && !from_cache) {                             // (from the cache the chosen go straight to the counting sort)
     if (DIRECT && cached) {
       // chosen tokens -> list: the warp counts its chosen candidates over all its rounds first and reserves their
       // places with ONE atomic (an atomic per round would serialise the rounds on its return value)
@@ -678,6 +965,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
       unsigned takes = 0;
 #pragma unroll
       for (int r = 0; r < ROUNDS; ++r) {
+        if ((uint32_t)(r * FIN_THREADS) >= mc) break;         // (uniform)
         const uint32_t c = r * FIN_THREADS + tid;
         const bool take = c < mc && (need0 >= m || s_comp[c] >= thr);
         const unsigned tm = __ballot_sync(0xffffffffu, take);
@@ -710,36 +998,74 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
 
   if (DIRECT) {
     // ---- ascending output: sink tokens, the chosen tokens in token order, local tokens
-    for (int d = tid; d < SORT_BUCKETS; d += FIN_THREADS) s_range[d] = 0u;
+    // (the range counters were cleared at the start; chosen: the need0 largest composites = those that reach thr)
+    const bool chosen_all = need0 >= m;
+    const uint32_t listed = from_cache ? 0u : min(s_ntok, (uint32_t)k);
+    if (from_cache) {
+      if (need0 > 0)
+        for (uint32_t c = tid; c < m; c += FIN_THREADS) {
+          const uint64_t comp = s_comp[c];
+          if (chosen_all || comp >= thr) atomicAdd(&s_range[(~(uint32_t)comp) >> bucket_shift], 1u);
+        }
+    } else {
+      __syncthreads();                                        // the list of chosen tokens is complete
+      for (uint32_t e = tid; e < listed; e += FIN_THREADS) atomicAdd(&s_range[(uint32_t)s_tok[e] >> bucket_shift], 1u);
+    }
     __syncthreads();
-    const uint32_t cnt = min(s_ntok, (uint32_t)k);            // = need0
-    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) atomicAdd(&s_range[(uint32_t)s_tok[e] >> bucket_shift], 1u);
-    __syncthreads();
+    uint32_t cnt;                                             // chosen tokens = need0
     {                                                         // exclusive prefix over the ranges, in place
       constexpr int RPT = SORT_BUCKETS / FIN_THREADS;
       uint32_t c[RPT], local = 0;
 #pragma unroll
       for (int x = 0; x < RPT; ++x) { c[x] = s_range[RPT * tid + x]; local += c[x]; }
-      uint32_t total;
-      uint32_t run = block_exclusive_scan(local, s_warp, &total);
+      uint32_t run = block_exclusive_scan(local, s_warp, &cnt);
 #pragma unroll
       for (int x = 0; x < RPT; ++x) { s_range[RPT * tid + x] = run; run += c[x]; }
+      cnt = min(cnt, (uint32_t)k);
     }
     __syncthreads();
-    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) {       // afterwards s_range[r] is the END of range r
-      const int32_t t = s_tok[e];
-      s_sorted[atomicAdd(&s_range[(uint32_t)t >> bucket_shift], 1u)] = t;
+    if (from_cache) {                                         // afterwards s_range[r] is the END of range r
+      if (need0 > 0)
+        for (uint32_t c = tid; c < m; c += FIN_THREADS) {
+          const uint64_t comp = s_comp[c];
+          if (chosen_all || comp >= thr) {
+            const uint32_t t = ~(uint32_t)comp;
+            const uint32_t pos = atomicAdd(&s_range[t >> bucket_shift], 1u);
+            if (pos < (uint32_t)k) s_sorted[pos] = (int32_t)t;
+          }
+        }
+    } else {
+      for (uint32_t e = tid; e < listed; e += FIN_THREADS) {
+        const int32_t t = s_tok[e];
+        s_sorted[atomicAdd(&s_range[(uint32_t)t >> bucket_shift], 1u)] = t;
+      }
     }
     __syncthreads();
     int32_t* out = idx_out + (size_t)head * k;
     const uint32_t n_sink = (uint32_t)F.sink_end, n_loc = (uint32_t)(n - F.local_begin);
-    for (uint32_t e = tid; e < cnt; e += FIN_THREADS) {
-      const int32_t t = s_sorted[e];
-      const uint32_t r = (uint32_t)t >> bucket_shift;
-      const uint32_t beg = r ? s_range[r - 1] : 0u, end = s_range[r];
-      uint32_t rank = 0;
-      for (uint32_t j = beg; j < end; ++j) rank += s_sorted[j] < t;
-      out[n_sink + beg + rank] = t;
+    for (uint32_t e0 = 0; e0 < cnt; e0 += FIN_THREADS * 4) {  // four tokens per thread at a time: their loads overlap
+      int32_t t[4];
+      uint32_t beg[4], end[4], rank[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t e = e0 + u * FIN_THREADS + tid;
+        t[u] = e < cnt ? s_sorted[e] : 0;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t r = (uint32_t)t[u] >> bucket_shift;
+        beg[u] = r ? s_range[r - 1] : 0u;
+        end[u] = s_range[r];
+        rank[u] = 0;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t e = e0 + u * FIN_THREADS + tid;
+        if (e < cnt) {
+          for (uint32_t j = beg[u]; j < end[u]; ++j) rank[u] += s_sorted[j] < t[u];
+          out[n_sink + beg[u] + rank[u]] = t[u];
+        }
+      }
     }
     for (uint32_t e = tid; e < n_sink; e += FIN_THREADS) out[e] = (int32_t)e;
     for (uint32_t e = tid; e < n_loc; e += FIN_THREADS) out[n_sink + cnt + e] = (int32_t)(F.local_begin + e);
@@ -873,11 +1199,15 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
     attr_set[ctx->device] = true;
   }
   Gate g = {S.cand_count, want, Hq, gate_mode};
+  const int lo_word = gate_mode == 2 ? -1 : 6;                // state word with the score the candidates had to reach (-1: a bin, no short way)
+  size_t smem = direct_select_smem(k);                        // a little more when that makes room for the bitmap of n tokens
+  if (fast_select_groups(n) <= FAST_MAXU && (size_t)fast_select_bytes(n, k) > smem && fast_select_bytes(n, k) <= 216 * 1024)
+    smem = (size_t)fast_select_bytes(n, k);
   FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(
-      topk_select_kernel<true>, dim3(Hq), dim3(FIN_THREADS), direct_select_smem(k), st, (const float*)S.cand_score, n, 0LL, F,
+      topk_select_kernel<true>, dim3(Hq), dim3(FIN_THREADS), smem, st, (const float*)S.cand_score, n, 0LL, F,
       (const uint32_t*)S.state, (const int32_t*)S.cand, (uint32_t*)nullptr, 0LL, k, idx, ctx->dev_status, (uint32_t*)nullptr, 0,
       (const uint32_t*)(gate_mode == 2 ? S.cand_count2 : S.cand_count), n, want, bucket_shift_for(n), g,
-      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k)));
+      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k), lo_word, (int)smem));
   return FATHOM_OK;
 }
 
@@ -910,7 +1240,8 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     }
     topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
                                                                             S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
-                                                                            ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr, FIN_CACHE);
+                                                                            ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr, FIN_CACHE,
+                                                                            -1, 0);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens

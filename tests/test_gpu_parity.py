@@ -646,6 +646,34 @@ def test_rotation_and_covariance_kernels_both_paths(n, dtype, path, monkeypatch)
     ctx.close()
 
 
+@pytest.mark.parametrize("n,Hq,k,n_sink,n_local", [(300_000, 3, 6000, 0, 0),      # lists of 8192..16384: two rounds of loads
+                                                   (300_000, 3, 2500, 4, 32),   # short lists, forced tokens
+                                                   (1_700_000, 2, 2048, 0, 0),  # too long for the shared-memory bitmap
+                                                   (140_000, 2, 1024, 0, 64)])  # a sample of few chunks
+def test_topk_direct_select_short_and_general_way(n, Hq, k, n_sink, n_local):
+    """The selection among the collected candidates has a short way (fine histogram + bitmap in shared memory: lists of
+    up to 8192 and of up to 16384 candidates take different instantiations) and a general way (radix select + counting
+    sort: longer lists, sequences whose bitmap does not fit, a split bin with many equal scores).  Normal scores with a
+    slice of exact ties right at the threshold; every case must give the oracle's selection."""
+    from paper_2609_17652_b200 import binding as fb
+    lay = fb.make_layout(1, Hq, n)
+    assert fb.fathom_topk_passes(lay, k) == 1
+    r = np.random.default_rng(n + k)
+    s = np.zeros((Hq, lay.score_stride), dtype=np.float32)
+    s[:, :n] = r.standard_normal((Hq, n)).astype(np.float32)
+    kth = np.sort(s[Hq - 1, :n])[-k]                             # last head: 40 exact copies of its k-th largest score
+    s[Hq - 1, r.choice(n, 40, replace=False)] = kth
+    sc = torch.from_numpy(s).cuda()
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    idx = torch.full((Hq, k), -1, dtype=torch.int32, device="cuda")
+    for _ in range(2):                                           # scratch and counters reused
+        ctx.fathom_topk(lay, sc, k, n_sink, n_local, idx)
+    want = O.topk(s[:, :n].astype(np.float64), k, n_sink, n_local)
+    assert np.array_equal(idx.cpu().numpy(), want)
+    assert ctx.fathom_device_status() == 0
+    ctx.close()
+
+
 def test_topk_at_the_largest_k_on_every_path():
     """k = FATHOM_MAX_K (16384): the direct select then holds 2 x 16384 tokens, the composite cache and the range
     counters in shared memory at once.  Single-pass and two-pass selection and the fused scan + selection."""
