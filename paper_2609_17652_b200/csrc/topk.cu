@@ -483,55 +483,67 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
 }
 
 
-// The short way of the direct select, for a head whose candidates had to reach a known score `lo` and whose selection
-// bitmap fits in shared memory.  The candidates (at most 16 per thread, loaded once, kept in registers as bin and token) are counted in a
-// fine histogram of the key's distance from lo's key (2048 bins of 2^13 keys: 16 bins of the 12-bit histogram lo came
-// from; the last bin takes everything beyond).  Its suffix counts give the bin b that holds the wanted-th largest
-// candidate; candidates in bins above b are chosen at once, the few dozen members of b are listed and ranked against one
-// another on the composite (key << 32 | ~token); the chosen tokens are set in the bitmap, and a chosen token's place in
-// the ascending output is the number of set bits before it (popcounts: a running count per 16 bytes of bitmap + the
-// bits before it in its own 16 bytes): one histogram pass over the candidates, no sort.  Everything needed from global
-// memory is requested before anything is waited for.  Returns false, with nothing but the cleared bitmap and histogram
-// touched, when it does not apply: the head has to collect again (too few candidates), more than 16 candidates per
-// thread, or a bin b with more than SMALL members.  The caller then selects the general way.
+// The short way of the direct select, for a head whose candidates had to reach a known score `lo`.  FAST_PARTS CTAs
+// share a head without talking to one another: each loads all the candidates and finds the threshold itself, then
+// emits the chosen tokens of its own quarter of the sequence.
+// The candidates (at most 16 per thread, loaded once, kept in registers as bin and token) are counted in a fine
+// histogram of the key's distance from lo's key (2048 bins of 2^13 keys: 16 bins of the 12-bit histogram lo came from;
+// the last bin takes everything beyond).  Its suffix counts give the bin b that holds the wanted-th largest candidate;
+// candidates in bins above b are chosen at once, the few dozen members of b are listed and ranked against one another
+// on the composite (key << 32 | ~token).  A chosen token of the CTA's own quarter is set in a bitmap in shared memory,
+// one before the quarter is counted; the quarter's tokens are then read off the bitmap in ascending order, each thread
+// its own groups, at the place given by the count before the quarter plus the popcounts of the threads before it: one
+// histogram pass over the candidates, no sort.  Everything needed from global memory is requested before anything is
+// waited for.  Returns false, with nothing but the cleared bitmap and histogram touched, when it does not apply (the
+// same for all CTAs of a head): the head has to collect again (too few candidates), more than 16 candidates per
+// thread, or a bin b with more than SMALL members.  The head's first CTA then selects the general way.
 // Shared memory: bitmap of 1024 U 16-byte groups (U per thread), one group skipped after every 8 so that the threads of
-// a quarter warp, each reading its own U consecutive groups, hit different banks; running counts [1024 U] u16; tokens
-// in output order [k].
+// a quarter warp, each reading its own U consecutive groups, hit different banks.
 constexpr int FINE_BINS = 2048, FINE_SHIFT = 13;
 __device__ __forceinline__ uint32_t fine_bin(float score, float lo) {
   const uint32_t key = ordered_key(score), base = ordered_key(lo);
   return min((key > base ? key - base : 0u) >> FINE_SHIFT, (uint32_t)(FINE_BINS - 1));
 }
-constexpr int FAST_MAXU = 12;                                 // 16-byte bitmap groups per thread: sequences of up to 1.5M tokens
-__host__ __device__ inline long long fast_select_groups(long long n) { return ((n + 127) / 128 + FIN_THREADS - 1) / FIN_THREADS; }   // U
-__host__ __device__ inline long long fast_select_bytes(long long n, int k) {
+constexpr int FAST_PARTS = 4;                                 // CTAs per head
+constexpr int FAST_MAXU = 4;                                  // 16-byte bitmap groups per thread
+constexpr long long FAST_MAX_TOKENS = (1ll << 21) - 1;        // tokens are kept in 21 bits
+// 16-byte groups (128 tokens) of a part, and per thread of it
+__host__ __device__ inline long long fast_part_groups(long long n) { return ((n + 127) / 128 + FAST_PARTS - 1) / FAST_PARTS; }
+__host__ __device__ inline long long fast_select_groups(long long n) { return (fast_part_groups(n) + FIN_THREADS - 1) / FIN_THREADS; }   // U
+__host__ __device__ inline long long fast_select_bytes(long long n) {
   const long long G = fast_select_groups(n) * FIN_THREADS;
-  return (G + (G >> 3)) * 16 + G * 2 + (long long)k * 4;
+  return (G + (G >> 3)) * 16;
 }
+static_assert(FAST_MAX_TOKENS <= (long long)FAST_PARTS * FAST_MAXU * FIN_THREADS * 128, "the parts' bitmaps must cover every token");
 constexpr int FAST_EPT = 8;                                   // candidates per thread and round of loads
 // ROUNDS = 1: lists of up to 8192 candidates; 2: up to 16384 (a second round of loads once the length is known)
 template <int SMALL, int ROUNDS>
 __device__ __forceinline__ bool select_by_fine_histogram_rounds(
     const float* __restrict__ cs, const int32_t* __restrict__ ci, uint32_t m, const float (&sc0)[FAST_EPT], const int32_t (&ix0)[FAST_EPT],
-    uint32_t want, float lo, long long n, int k,
+    uint32_t want, float lo, long long n, int k, int part,
     Forced F, unsigned char* s_dyn, uint32_t* s_fine, uint32_t* s_warp, int32_t* __restrict__ out, uint32_t* __restrict__ dev_status) {
   constexpr int EPT = FAST_EPT;
   constexpr int FPT = FINE_BINS / FIN_THREADS;                 // fine bins per thread
   constexpr uint32_t TOKEN_BITS = 21, NONE = 0xffffffffu;      // a candidate in a register: fine bin << 21 | token
-  static_assert((long long)FAST_MAXU * FIN_THREADS * 128 <= (1ll << TOKEN_BITS) - 1, "tokens must fit beside the bin, NONE must be no token");
+  static_assert(FAST_MAX_TOKENS <= (1ll << TOKEN_BITS) - 1, "tokens must fit beside the bin, NONE must be no token");
   static_assert(SMALL * 8 <= FINE_BINS * 4, "the members of the split bin are listed where the fine histogram was");
   __shared__ uint32_t s_bin, s_need_in, s_members, s_nsmall;
   uint64_t* s_small = reinterpret_cast<uint64_t*>(s_fine);     // (free once every thread has read its bins)
   const int tid = threadIdx.x;
-  const uint32_t U = (uint32_t)fast_select_groups(n), G = U * FIN_THREADS;
+  const uint32_t U = (uint32_t)fast_select_groups(n);
+  const uint32_t first_token = (uint32_t)part * (uint32_t)fast_part_groups(n) * 128u;   // my part: [first_token, + part_tokens)
+  const uint32_t part_tokens = (uint32_t)fast_part_groups(n) * 128u;
   uint32_t* s_bits = reinterpret_cast<uint32_t*>(s_dyn);
   const uint4* s_bits4 = reinterpret_cast<const uint4*>(s_dyn);
-  uint16_t* s_pref = reinterpret_cast<uint16_t*>(s_dyn + (size_t)(G + (G >> 3)) * 16);
-  int32_t* s_out = reinterpret_cast<int32_t*>(s_dyn + (size_t)(G + (G >> 3)) * 16 + (size_t)G * 2);
   auto group_at = [](uint32_t g) { return g + (g >> 3); };     // where group g of the bitmap sits
-  auto set_bit = [&](uint32_t t) {
-    const uint32_t w = t >> 5;
-    atomicOr(&s_bits[(group_at(w >> 2) << 2) | (w & 3u)], 1u << (t & 31u));
+  uint32_t below = 0;                                         // chosen tokens before my part (my share of the count)
+  auto choose = [&](uint32_t t) {                              // a chosen token: into the bitmap, counted, or not mine to emit
+    const uint32_t r = t - first_token;
+    if (t < first_token) ++below;
+    else if (r < part_tokens) {
+      const uint32_t w = r >> 5;
+      atomicOr(&s_bits[(group_at(w >> 2) << 2) | (w & 3u)], 1u << (r & 31u));
+    }
   };
   uint32_t cand[ROUNDS * EPT];
   if (tid == 0) { s_nsmall = 0u; s_bin = 0u; s_need_in = 0u; s_members = 0u; }
@@ -584,68 +596,59 @@ __device__ __forceinline__ bool select_by_fine_histogram_rounds(
   //      scores are read again: a few dozen loads per head)
   const uint32_t take_from = need0 == 0 ? (uint32_t)FINE_BINS : (need0 >= m ? 0u : (ranked ? s_bin + 1u : s_bin));
   const uint32_t split_bin = ranked ? s_bin : NONE;
-  uint32_t chosen = 0;                                        // bit u: my u-th candidate is chosen
 #pragma unroll
   for (int u = 0; u < ROUNDS * EPT; ++u) {
     if (cand[u] != NONE) {
       const uint32_t fb = cand[u] >> TOKEN_BITS, t = cand[u] & ((1u << TOKEN_BITS) - 1u);
-      if (fb >= take_from) {
-        set_bit(t);
-        chosen |= 1u << u;
-      } else if (fb == split_bin) {
+      if (fb >= take_from) choose(t);
+      else if (fb == split_bin) {
         const uint32_t pos = atomicAdd(&s_nsmall, 1u);
         if (pos < (uint32_t)SMALL) s_small[pos] = (((uint64_t)ordered_key(__ldcg(cs + (uint32_t)u * FIN_THREADS + tid))) << 32) | (uint32_t)~t;
       }
     }
   }
   __syncthreads();
-  uint32_t member_token = 0;
-  bool member_chosen = false;
-  if (ranked && (uint32_t)tid < members) {
-    const uint64_t mine = s_small[tid];
-    uint32_t larger = 0;
-    for (uint32_t j = 0; j < members; ++j) larger += s_small[j] > mine;
-    if (larger < need_in) {
-      member_token = ~(uint32_t)mine;
-      member_chosen = true;
-      set_bit(member_token);
+  if (ranked) {                                               // a warp per member, its lanes over the others
+    const int lane = tid & 31, warp = tid >> 5;
+    for (uint32_t i = warp; i < members; i += FIN_THREADS / 32) {
+      const uint64_t mine = s_small[i];
+      uint32_t larger = 0;
+      for (uint32_t j = lane; j < members; j += 32) larger += s_small[j] > mine;
+      larger = __reduce_add_sync(0xffffffffu, larger);
+      if (lane == 0 && larger < need_in) choose(~(uint32_t)mine);
     }
   }
   __syncthreads();
-  // ---- set bits before every 16-byte group of the bitmap: a thread counts its own U groups, the block prefix does the rest
-  uint32_t before[FAST_MAXU], mine = 0;
-#pragma unroll
-  for (int j = 0; j < FAST_MAXU; ++j) {
-    before[j] = mine;
-    if ((uint32_t)j < U) {
-      const uint4 x = s_bits4[group_at(U * tid + j)];
-      mine += __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w);
-    }
-  }
-  uint32_t cnt;
-  const uint32_t base = block_exclusive_scan(mine, s_warp, &cnt);
-  cnt = min(cnt, (uint32_t)k);                                // = need0
+  // ---- my part's chosen tokens in ascending order: a thread reads its own U groups; its place is the chosen tokens
+  //      before the part (counted by all threads) plus those of the threads before it
+  uint32_t own = 0;
 #pragma unroll
   for (int j = 0; j < FAST_MAXU; ++j)
-    if ((uint32_t)j < U) s_pref[U * tid + j] = (uint16_t)min(base + before[j], 0xffffu);
-  __syncthreads();
-  // ---- every chosen token to its place in the output
-  auto place = [&](uint32_t t) {
-    const uint32_t w = t >> 5, g = w >> 2, q = w & 3u;
-    const uint4 x = s_bits4[group_at(g)];
-    uint32_t p = s_pref[g];
-    p += (q > 0u ? __popc(x.x) : 0) + (q > 1u ? __popc(x.y) : 0) + (q > 2u ? __popc(x.z) : 0);
-    const uint32_t own = q == 0u ? x.x : (q == 1u ? x.y : (q == 2u ? x.z : x.w));
-    p += __popc(own & ((1u << (t & 31u)) - 1u));
-    if (p < (uint32_t)k) s_out[p] = (int32_t)t;
-  };
+    if ((uint32_t)j < U) {
+      const uint4 x = s_bits4[group_at(U * tid + j)];
+      own += __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w);
+    }
+  uint32_t totals;                                            // low half: prefix of own; high half: sum of below (both <= 16384)
+  const uint32_t prefix = block_exclusive_scan(own | (below << 16), s_warp, &totals);
+  const uint32_t n_sink = (uint32_t)F.sink_end, n_loc = (uint32_t)(n - F.local_begin), cnt = need0;
+  uint32_t pos = (totals >> 16) + (prefix & 0xffffu);
 #pragma unroll
-  for (int u = 0; u < ROUNDS * EPT; ++u)
-    if ((chosen >> u) & 1u) place(cand[u] & ((1u << TOKEN_BITS) - 1u));
-  if (member_chosen) place(member_token);
-  __syncthreads();
-  const uint32_t n_sink = (uint32_t)F.sink_end, n_loc = (uint32_t)(n - F.local_begin);
-  for (uint32_t e = tid; e < cnt; e += FIN_THREADS) out[n_sink + e] = s_out[e];
+  for (int j = 0; j < FAST_MAXU; ++j)
+    if ((uint32_t)j < U) {
+      const uint4 x = s_bits4[group_at(U * tid + j)];
+      const uint32_t word[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t w = word[q];
+        while (w) {
+          const uint32_t b = (uint32_t)__ffs((int)w) - 1u;
+          w &= w - 1u;
+          if (pos < cnt) out[n_sink + pos] = (int32_t)(first_token + ((U * tid + j) << 7) + (q << 5) + b);
+          ++pos;
+        }
+      }
+    }
+  if (part != 0) return true;
   for (uint32_t e = tid; e < n_sink; e += FIN_THREADS) out[e] = (int32_t)e;
   for (uint32_t e = tid; e < n_loc; e += FIN_THREADS) out[n_sink + cnt + e] = (int32_t)(F.local_begin + e);
   const uint32_t filled = n_sink + cnt + n_loc;
@@ -659,7 +662,7 @@ __device__ __forceinline__ bool select_by_fine_histogram_rounds(
 template <int SMALL>
 __device__ __forceinline__ bool select_by_fine_histogram(
     const float* __restrict__ cs, const int32_t* __restrict__ ci, long long capacity, const uint32_t* __restrict__ count_ptr,
-    bool must_reach_want, uint32_t want, const uint32_t* __restrict__ lo_ptr, long long n, int k,
+    bool must_reach_want, uint32_t want, const uint32_t* __restrict__ lo_ptr, long long n, int k, int part,
     Forced F, unsigned char* s_dyn, uint32_t* s_fine, uint32_t* s_warp, int32_t* __restrict__ out, uint32_t* __restrict__ dev_status) {
   // ---- all loads in flight together (the candidate loads are speculative: the list's length is not known yet)
   const int tid = threadIdx.x;
@@ -676,9 +679,9 @@ __device__ __forceinline__ bool select_by_fine_histogram(
   const uint32_t m = (uint32_t)min((long long)listed, capacity);
   if (must_reach_want && listed < want) return false;          // (all conditions are the same for every thread)
   if (m <= (uint32_t)(FAST_EPT * FIN_THREADS))
-    return select_by_fine_histogram_rounds<SMALL, 1>(cs, ci, m, sc, ix, want, lo, n, k, F, s_dyn, s_fine, s_warp, out, dev_status);
+    return select_by_fine_histogram_rounds<SMALL, 1>(cs, ci, m, sc, ix, want, lo, n, k, part, F, s_dyn, s_fine, s_warp, out, dev_status);
   if (m <= (uint32_t)(2 * FAST_EPT * FIN_THREADS))
-    return select_by_fine_histogram_rounds<SMALL, 2>(cs, ci, m, sc, ix, want, lo, n, k, F, s_dyn, s_fine, s_warp, out, dev_status);
+    return select_by_fine_histogram_rounds<SMALL, 2>(cs, ci, m, sc, ix, want, lo, n, k, part, F, s_dyn, s_fine, s_warp, out, dev_status);
   return false;
 }
 
@@ -698,7 +701,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
                    const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
                    Gate gate, const float* __restrict__ collect_scores, long long collect_stride, float* __restrict__ collect_score_out,
-                   int32_t* __restrict__ collect_idx_out, int cache_entries, int lo_word, int dyn_bytes) {
+                   int32_t* __restrict__ collect_idx_out, int cache_entries, int lo_word, int parts) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   static_assert(FIN_THREADS == 1024, "one pair of s_diff words per lane; digits and ranges per thread");
@@ -714,9 +717,9 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   uint32_t* s_range = reinterpret_cast<uint32_t*>(s_comp + cache_entries);      // [SORT_BUCKETS]
   int32_t* s_tok = reinterpret_cast<int32_t*>(s_range + SORT_BUCKETS);          // [k]
   int32_t* s_sorted = s_tok + k;                                                // [k]
-  const int head = blockIdx.x, tid = threadIdx.x;
-  // the short way (select_by_fine_histogram) when the candidates were counted and the bitmap of n tokens fits
-  const bool counted = DIRECT && lo_word >= 0 && fast_select_groups(n) <= FAST_MAXU && fast_select_bytes(n, k) <= (long long)dyn_bytes;
+  // `parts` CTAs per head: 1, or FAST_PARTS when the short way (select_by_fine_histogram) may apply
+  const int head = blockIdx.x / parts, part = blockIdx.x % parts, tid = threadIdx.x;
+  const bool counted = DIRECT && parts == FAST_PARTS;
   if (DIRECT) {                                               // shared memory only: done while the previous kernel still runs
     if (counted) {
       const uint32_t G = (uint32_t)fast_select_groups(n) * FIN_THREADS;
@@ -731,9 +734,10 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   if (counted) {
     if (select_by_fine_histogram<SMALL_BUCKET>(scores + (size_t)head * (size_t)cand_capacity, cand + (size_t)head * (size_t)cand_capacity,
                                                cand_capacity, cand_count + head, gate.mode == 5 && collect_scores != nullptr, want_direct,
-                                               state + head * 8 + lo_word, n, k, F, s_dyn, s_hist, s_warp,
+                                               state + head * 8 + lo_word, n, k, part, F, s_dyn, s_hist, s_warp,
                                                idx_out + (size_t)head * k, dev_status))
       return;
+    if (part != 0) return;                                    // the general way is one CTA's work
     __syncthreads();                                          // the general way: its range counters lie where the bitmap was
     for (int d = tid; d < SORT_BUCKETS; d += FIN_THREADS) s_range[d] = 0u;
   }
@@ -1200,14 +1204,15 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
   }
   Gate g = {S.cand_count, want, Hq, gate_mode};
   const int lo_word = gate_mode == 2 ? -1 : 6;                // state word with the score the candidates had to reach (-1: a bin, no short way)
-  size_t smem = direct_select_smem(k);                        // a little more when that makes room for the bitmap of n tokens
-  if (fast_select_groups(n) <= FAST_MAXU && (size_t)fast_select_bytes(n, k) > smem && fast_select_bytes(n, k) <= 216 * 1024)
-    smem = (size_t)fast_select_bytes(n, k);
+  const size_t smem = direct_select_smem(k);
+  // the short way: a known score threshold, tokens that fit in 21 bits, a part's bitmap within the shared memory
+  const bool counted = lo_word >= 0 && n <= FAST_MAX_TOKENS && fast_select_groups(n) <= FAST_MAXU && (size_t)fast_select_bytes(n) <= smem;
+  const int parts = counted ? FAST_PARTS : 1;
   FATHOM_CUDA_TRY(ctx, fathom_launch_dependent(
-      topk_select_kernel<true>, dim3(Hq), dim3(FIN_THREADS), smem, st, (const float*)S.cand_score, n, 0LL, F,
+      topk_select_kernel<true>, dim3(Hq * parts), dim3(FIN_THREADS), smem, st, (const float*)S.cand_score, n, 0LL, F,
       (const uint32_t*)S.state, (const int32_t*)S.cand, (uint32_t*)nullptr, 0LL, k, idx, ctx->dev_status, (uint32_t*)nullptr, 0,
       (const uint32_t*)(gate_mode == 2 ? S.cand_count2 : S.cand_count), n, want, bucket_shift_for(n), g,
-      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k), lo_word, (int)smem));
+      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k), lo_word, parts));
   return FATHOM_OK;
 }
 
@@ -1241,7 +1246,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
                                                                             S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
                                                                             ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr, FIN_CACHE,
-                                                                            -1, 0);
+                                                                            -1, 1);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
