@@ -58,7 +58,12 @@ struct Geo {
   static_assert(ROWS * ROW_BYTES <= WORD_STAGE_BYTES && ROWS * SCALE_ELEMS * 2 <= SCALE_STAGE_BYTES, "stage buffers too small");
 };
 
-constexpr int CAND_CAP = 32;                                 // MODE 2: candidates a warp keeps per head before it appends them to the global lists
+// MODE 2.  A lane whose eight scores hold a candidate parks all eight in its warp's ring (three stores, no atomic, no
+// loop); when the ring may not take another round of 32, the warp sifts it with all lanes, one parked group per lane,
+// into the CTA's four candidate lists (one shared-memory atomic per head); the lists go to the heads' global lists once,
+// when the CTA has scanned its last tile (one global atomic per head and CTA).
+constexpr int PARK_RING = 64;                                // parked groups per warp
+constexpr int CAND_LIST = 256;                               // candidates per head the CTA keeps; beyond that: straight to the global list
 
 template <int MODE>
 struct alignas(16) Smem {
@@ -70,8 +75,12 @@ struct alignas(16) Smem {
   float wmax[WARPS][4];                                       // per warp: max_j |q_hj| of its channels
   float hscale[4], hinv[4];                                   // E_h and 1 / E_h
   float thr[4];                                               // MODE 2: score a token must reach, per head
-  uint32_t ccnt[WARPS][4];                                    // MODE 2: candidates in the warp's lists
-  uint2 cand[MODE == 2 ? WARPS * 4 * CAND_CAP : 1];           // MODE 2: (score bits, token) per warp and head
+  uint32_t ccount[4], cbase[4];                               // MODE 2: candidates in the CTA's lists; where they go in the global lists
+  uint32_t elig[2];                                           // MODE 2: eligible tokens lo <= t < hi of the session
+  alignas(16) float4 park_lo[MODE == 2 ? WARPS * PARK_RING : 1];     // MODE 2: scores 0..3 of a parked group
+  alignas(16) float4 park_hi[MODE == 2 ? WARPS * PARK_RING : 1];     //         scores 4..7
+  uint32_t park_tok[MODE == 2 ? WARPS * PARK_RING : 1];       //         its first token (30 bits) and the head within the CTA (2 bits)
+  uint2 clist[MODE == 2 ? 4 * CAND_LIST : 1];                 // MODE 2: (score bits, token) per head
   alignas(16) uint2 bfr[STAGE_KSTEPS][32];                    // right operand of the rows of a pass: per 16 rows, the two B registers of every lane
   alignas(16) unsigned char words[2][WORD_STAGE_BYTES];       // staged plane words, double buffered
   alignas(16) unsigned char scale[2][SCALE_STAGE_BYTES];      // staged fp16 scales, double buffered
@@ -137,7 +146,8 @@ __device__ __forceinline__ void mma_rows(float (&acc)[4][4], const unsigned char
 template <int NH, int MODE>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
 scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fathom_scan_fuse fz) {
-  __shared__ Smem<MODE> M;
+  extern __shared__ __align__(16) unsigned char scan_smem[];   // sizeof(Smem<MODE>): more than the static limit in MODE 2
+  Smem<MODE>& M = *reinterpret_cast<Smem<MODE>*>(scan_smem);
 
   FATHOM_PDL_WAIT();                                          // depths (and thresholds) come from the previous kernels
   if (MODE == 2 && !fathom_gate_open(fz.gate)) return;         // second attempt of the fused selection: may have nothing to do
@@ -150,7 +160,13 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
   const int kv = h0 / G;
   const int myh = t4 < NH ? t4 : 0;                            // the head whose scores this lane receives (lanes t4 >= NH: none)
-  if (MODE == 2 && tid < WARPS * 4) (&M.ccnt[0][0])[tid] = 0u;
+  if (MODE == 2 && tid < 4) M.ccount[tid] = 0u;
+  if (MODE == 2 && tid == 0) {                                 // (MODE 2 is launched with one session)
+    const long long n0 = B.n[0];
+    const long long hi = fz.local_begin < n0 ? fz.local_begin : n0, lo = fz.sink_end < hi ? fz.sink_end : hi;
+    M.elig[0] = (uint32_t)lo;
+    M.elig[1] = (uint32_t)hi;
+  }
   if (MODE == 2 && tid < NH)                                   // read after the barriers of the first item's row list
     M.thr[tid] = fz.state_is_score ? __uint_as_float(fz.state[(h0 + tid) * 8]) : fathom_bin_lower_edge(fz.state[(h0 + tid) * 8]);
 
@@ -286,11 +302,71 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   };
 
   float acc[4][4];                                             // [16-token slice of the block][c0..c3]
+  uint32_t parked = 0u, stages = 0u;                           // MODE 2: groups in my warp's ring (the same in every lane); stages done
 
   enter_item(g);
   const float my_thr = MODE == 2 ? M.thr[myh] : 0.0f;
   int u = 0, pass = 0, buf = 0;
   prefetch(g, 0, 0, 0);
+
+  // ---- MODE 2, whole warp: the parked groups, one per lane and round, into the CTA's candidate lists.  A lane marks the
+  //      candidates among its group's eight scores (score reaches the head's threshold, token eligible).  Nearly always
+  //      there is one: the lanes that have any are ranked per head with a ballot, lanes 0..3 reserve the heads' places
+  //      with one shared-memory atomic each, and every such lane writes its first candidate; further candidates of a
+  //      group take a place of their own.  All warps of a CTA sift at the same stages (every fourth): a warp that did
+  //      it alone would keep the others waiting at the stage barrier.
+  auto sift = [&]() {
+    if (MODE != 2) return;
+    __syncwarp();                                              // the parked groups are visible to the whole warp
+    const uint32_t elo = M.elig[0], ehi = M.elig[1];
+    auto append = [&](uint32_t h, uint32_t pos, float val, uint32_t token) {
+      if (pos < (uint32_t)CAND_LIST) {
+        M.clist[h * CAND_LIST + pos] = make_uint2(__float_as_uint(val), token);
+      } else {                                                 // list full (only with a threshold far too low): straight to the global list
+        const uint32_t at = atomicAdd(&fz.cand_count[h0 + h], 1u);
+        if ((long long)at < fz.capacity) {
+          fz.cand_score[(size_t)(h0 + h) * fz.capacity + at] = val;
+          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + at] = (int32_t)token;
+        }
+      }
+    };
+    for (uint32_t e0 = 0; e0 < parked; e0 += 32) {
+      const uint32_t e = warp * PARK_RING + e0 + lane;
+      const bool mine = e0 + lane < parked;
+      const uint32_t tk = mine ? M.park_tok[e] : 0u;
+      const uint32_t h = tk >> 30, tok = tk & 0x3fffffffu;
+      const float th = M.thr[h];
+      uint32_t mask = 0u;
+      if (mine) {
+        const float4 a = M.park_lo[e], b = M.park_hi[e];
+        const float w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int x = 0; x < 8; ++x) mask |= (w[x] >= th && tok + x - elo < ehi - elo ? 1u : 0u) << x;
+      }
+      auto score_at = [&](uint32_t x) { return reinterpret_cast<const float*>(x < 4u ? &M.park_lo[e] : &M.park_hi[e])[x & 3u]; };
+      uint32_t rank = 0u, tot = 0u, base = 0u;
+#pragma unroll
+      for (int hh = 0; hh < 4; ++hh) {
+        const unsigned with = __ballot_sync(0xffffffffu, mask != 0u && h == (uint32_t)hh);
+        if (h == (uint32_t)hh) rank = __popc(with & ((1u << lane) - 1u));
+        if (lane == hh) tot = __popc(with);
+      }
+      if (lane < 4 && tot) base = atomicAdd(&M.ccount[lane], tot);
+      base = __shfl_sync(0xffffffffu, base, (int)h);
+      if (mask) {
+        const uint32_t x = (uint32_t)__ffs((int)mask) - 1u;
+        mask &= mask - 1u;
+        append(h, base + rank, score_at(x), tok + x);
+      }
+      while (mask) {                                           // a second candidate in one group of eight: rare
+        const uint32_t x = (uint32_t)__ffs((int)mask) - 1u;
+        mask &= mask - 1u;
+        append(h, atomicAdd(&M.ccount[h], 1u), score_at(x), tok + x);
+      }
+    }
+    parked = 0u;
+    __syncwarp();                                              // the ring may be written again
+  };
 
   while (true) {
     // ---- the stage after this one: the next pass of the sub-tile, the next sub-tile of the tile, or my next tile
@@ -309,8 +385,9 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
 
     // ---- eight consecutive scores of head t4 (lanes with t4 < NH, tokens of an existing block): tokens tok .. tok + 7 of
     //      the session, written at position dst of the head's row (MODE 0, 1) or tested against the head's threshold (MODE 2)
-    auto emit = [&](const float (&v)[8], uint32_t tok, uint32_t dst, uint32_t n) {
+    auto emit = [&](const float (&v)[8], uint32_t tok, uint32_t dst, uint32_t n, bool live) {
       if (MODE != 2) {
+        if (!live) return;
         float* row = B.scores[item] + (size_t)(h0 + t4) * (size_t)B.score_stride[item] + dst;
         if (tok + 8 <= n) {
           store_scores8(row, v);
@@ -320,62 +397,22 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
             if (tok + x < n) row[x] = v[x];
         }
       } else {
-        // candidates: (score, token) pairs appended to the head's list; their order in the list is irrelevant.  They are
-        // rare (a fraction of a percent of the tokens), so the common path is a maximum and one comparison
+        // a lane with a candidate among its eight scores parks them (called by all lanes of the warp; `live`: the lane
+        // has scores at all).  Eligibility of the tokens is checked when the ring is sifted.
         const float vmax = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
-        if (vmax >= my_thr) {
-          uint32_t m = 0u;
-#pragma unroll
-          for (int x = 0; x < 8; ++x) m |= (v[x] >= my_thr ? 1u : 0u) << x;
-          const uint32_t hi = (uint32_t)(fz.local_begin < (long long)n ? fz.local_begin : (long long)n);   // eligible: lo <= token < hi
-          const uint32_t lo = (uint32_t)(fz.sink_end < (long long)hi ? fz.sink_end : (long long)hi);
-#pragma unroll 1
-          while (m) {
-            const int x = __ffs(m) - 1;
-            m &= m - 1;
-            const uint32_t ti = tok + x;
-            if (ti - lo < hi - lo) {
-              const float a01 = (x & 1) ? v[1] : v[0], a23 = (x & 1) ? v[3] : v[2], a45 = (x & 1) ? v[5] : v[4], a67 = (x & 1) ? v[7] : v[6];
-              const float a03 = (x & 2) ? a23 : a01, a47 = (x & 2) ? a67 : a45;
-              const float val = (x & 4) ? a47 : a03;
-              const uint32_t p = atomicAdd(&M.ccnt[warp][t4], 1u);
-              if (p < (uint32_t)CAND_CAP) {
-                M.cand[(warp * 4 + t4) * CAND_CAP + p] = make_uint2(__float_as_uint(val), ti);
-              } else {                                         // list full (only with a threshold far too low): straight to the global list
-                const uint32_t at = atomicAdd(&fz.cand_count[h0 + t4], 1u);
-                if ((long long)at < fz.capacity) {
-                  fz.cand_score[(size_t)(h0 + t4) * fz.capacity + at] = val;
-                  fz.cand_idx[(size_t)(h0 + t4) * fz.capacity + at] = (int32_t)ti;
-                }
-              }
-            }
+        const bool has = live && vmax >= my_thr;
+        const unsigned bal = __ballot_sync(0xffffffffu, has);
+        if (bal) {                                             // (the same for every lane)
+          if (has) {
+            const uint32_t e = warp * PARK_RING + parked + __popc(bal & ((1u << lane) - 1u));
+            M.park_lo[e] = make_float4(v[0], v[1], v[2], v[3]);
+            M.park_hi[e] = make_float4(v[4], v[5], v[6], v[7]);
+            M.park_tok[e] = tok | ((uint32_t)t4 << 30);
           }
+          parked += __popc(bal);
+          if (parked > (uint32_t)(PARK_RING - 32)) sift();
         }
       }
-    };
-
-    // ---- MODE 2, whole warp, after the last emit of a stage: once a list is half full (or at the end of the warp's work:
-    //      `final`) the warp's lists go to the heads' global lists, one atomic per head (same-address atomics are what the
-    //      global lists can take least of, and waiting for their result is what a warp can afford least often)
-    auto flush_candidates = [&](bool final) {
-      if (MODE != 2) return;
-      __syncwarp();
-      uint32_t c = 0u, base = 0u;
-      if (lane < NH) c = min(M.ccnt[warp][lane], (uint32_t)CAND_CAP);
-      if (!final && !__any_sync(0xffffffffu, c >= (uint32_t)(CAND_CAP / 2))) return;
-      if (c) base = atomicAdd(&fz.cand_count[h0 + lane], c);
-#pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        const uint32_t ch = __shfl_sync(0xffffffffu, c, h), bh = __shfl_sync(0xffffffffu, base, h);
-        if (lane < ch && (long long)(bh + lane) < fz.capacity) {
-          const uint2 it = M.cand[(warp * 4 + h) * CAND_CAP + lane];
-          fz.cand_score[(size_t)(h0 + h) * fz.capacity + bh + lane] = __uint_as_float(it.x);
-          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + bh + lane] = (int32_t)it.y;
-        }
-      }
-      __syncwarp();
-      if (lane < 4) M.ccnt[warp][lane] = 0u;
-      __syncwarp();
     };
 
     // ---- a whole stage of TB blocks and NKS x 16 rows, single pass: the warp's TB / 4 blocks are 16 TB tokens, and a lane
@@ -432,9 +469,8 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
           v[2 * j] = fmaf(acc[j][1], hs_tail, acc[j][0] * hs);
           v[2 * j + 1] = fmaf(acc[j][3], hs_tail, acc[j][2] * hs);
         }
-        if (t4 < NH) emit(v, tok0 + 8 * k, dst0 + 8 * k, n);
+        emit(v, tok0 + 8 * k, dst0 + 8 * k, n, t4 < NH);
       }
-      flush_candidates(!more);
     };
 
     auto compute = [&](auto tbc) {
@@ -476,15 +512,15 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
         }
         const bool have_block = blk0 + b < nb_item;
         const uint32_t tok = (uint32_t)(blk0 + b) * FATHOM_BLOCK + gq * 8;                     // my first token
-        if (t4 >= NH || !have_block) continue;
-        emit(v, tok, MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok, n);
+        emit(v, tok, MODE == 1 ? (uint32_t)g * (TILE_BLOCKS * FATHOM_BLOCK) + (uint32_t)(u * TB + b) * FATHOM_BLOCK + gq * 8 : tok, n,
+             t4 < NH && have_block);
       }
-      if (pass == npass - 1) flush_candidates(!more);
     };
     if (tb == 16) compute(std::integral_constant<int, 16>());
     else if (tb == 8) compute(std::integral_constant<int, 8>());
     else compute(std::integral_constant<int, 4>());
 
+    if (MODE == 2 && (++stages & 3u) == 0u) sift();            // (every warp of the CTA at the same stages)
     if (!more) break;
     g = g_next;
     u = u_next;
@@ -499,6 +535,28 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       fill_bfr(pass);                                          // plans of more than 160 rows: the right operand of the next pass
     }
   }
+  if (MODE == 2) {
+    // ---- the CTA has scanned its last tile: what is still parked is sifted, then the four lists go to the heads' global
+    //      lists, one atomic per head
+    sift();
+    __syncthreads();
+    if (tid < NH) {
+      const uint32_t c = min(M.ccount[tid], (uint32_t)CAND_LIST);
+      M.ccount[tid] = c;
+      M.cbase[tid] = c ? atomicAdd(&fz.cand_count[h0 + tid], c) : 0u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < NH && h < 4; ++h) {
+      const uint32_t c = M.ccount[h], at = M.cbase[h];
+      for (uint32_t e = tid; e < c; e += THREADS)
+        if ((long long)(at + e) < fz.capacity) {
+          const uint2 it = M.clist[h * CAND_LIST + e];
+          fz.cand_score[(size_t)(h0 + h) * fz.capacity + at + e] = __uint_as_float(it.x);
+          fz.cand_idx[(size_t)(h0 + h) * fz.capacity + at + e] = (int32_t)it.y;
+        }
+    }
+  }
 }
 
 template <int NH, int MODE>
@@ -508,12 +566,23 @@ int launch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const f
   if (tiles <= 0) return FATHOM_OK;
   const int plans = Hq / NH;
   dim3 grid((unsigned)fathom_scan_grid_ctas(tiles, plans, fathom_planes_in_host_memory(B.planes[0]), CTAS_PER_SM), (unsigned)plans);
+  constexpr size_t smem = sizeof(Smem<MODE>);                 // dynamic: MODE 2 needs more than the static limit
+  if (smem > 48 * 1024) {
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FATHOM_ERR_CUDA;
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+      if (cudaFuncSetAttribute(scan_kernel<NH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return FATHOM_ERR_CUDA;
+      configured[dev] = true;
+    }
+  }
   if (dependent) {                                            // may become resident while the previous kernel of the stream runs
-    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(THREADS), 0, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
+    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(THREADS), smem, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
       return FATHOM_ERR_CUDA;
     return FATHOM_OK;
   }
-  scan_kernel<NH, MODE><<<grid, THREADS, 0, st>>>(B, Hq / Hkv, heads_per_plan, fz);
+  scan_kernel<NH, MODE><<<grid, THREADS, smem, st>>>(B, Hq / Hkv, heads_per_plan, fz);
   return FATHOM_OK;
 }
 
