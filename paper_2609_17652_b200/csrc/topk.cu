@@ -1004,6 +1004,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
     // ---- ascending output: sink tokens, the chosen tokens in token order, local tokens
     // (the range counters were cleared at the start; chosen: the need0 largest composites = those that reach thr)
     const bool chosen_all = need0 >= m;
+    if (!from_cache) __syncthreads();                         // the list of chosen tokens and its length are complete
     const uint32_t listed = from_cache ? 0u : min(s_ntok, (uint32_t)k);
     if (from_cache) {
       if (need0 > 0)
@@ -1012,7 +1013,6 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
           if (chosen_all || comp >= thr) atomicAdd(&s_range[(~(uint32_t)comp) >> bucket_shift], 1u);
         }
     } else {
-      __syncthreads();                                        // the list of chosen tokens is complete
       for (uint32_t e = tid; e < listed; e += FIN_THREADS) atomicAdd(&s_range[(uint32_t)s_tok[e] >> bucket_shift], 1u);
     }
     __syncthreads();

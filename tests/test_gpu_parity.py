@@ -674,6 +674,67 @@ def test_topk_direct_select_short_and_general_way(n, Hq, k, n_sink, n_local):
     ctx.close()
 
 
+def test_topk_narrow_band_of_tied_scores():
+    """Scores 5 +- 0.004: a handful of fp32 values per token, all in two bins of the 12-bit histogram, so half of the
+    row is a candidate and about eighty tokens share every score.  The list is far too long for shared memory: radix
+    passes over global memory, the undecided digit pulled into the cache, its ties decided by the token index."""
+    from paper_2609_17652_b200 import binding as fb
+    n, Hq, k = 700_000, 3, 4096
+    lay = fb.make_layout(1, Hq, n)
+    assert fb.fathom_topk_passes(lay, k) == 1
+    r = np.random.default_rng(5)
+    s = np.zeros((Hq, lay.score_stride), dtype=np.float32)
+    s[:, :n] = (r.standard_normal((Hq, n)) * 1e-3 + 5.0).astype(np.float32)
+    sc = torch.from_numpy(s).cuda()
+    ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+    for n_sink, n_local in ((0, 0), (2, 15)):
+        idx = torch.full((Hq, k), -1, dtype=torch.int32, device="cuda")
+        ctx.fathom_topk(lay, sc, k, n_sink, n_local, idx)
+        assert np.array_equal(idx.cpu().numpy(), O.topk(s[:, :n].astype(np.float64), k, n_sink, n_local))
+        assert ctx.fathom_device_status() == 0
+    ctx.close()
+
+
+def test_topk_random_lengths_counts_and_score_distributions():
+    """Fifty seeded draws of (n, heads, k, forced tokens, score distribution): normal, rounded (ties), spread growing
+    along the row, two-sided exponential, a narrow band far from zero.  Between them they take the two-pass path, the
+    short and the general way of the single-pass selection, lists of every length and sequences too long for the
+    shared-memory bitmap; draw 49 (1.3 M tokens, k = 16384, narrow band) once lost winners to a list length that was
+    read before the list was complete."""
+    from paper_2609_17652_b200 import binding as fb
+    r = np.random.default_rng(7)
+    for it in range(50):
+        n = int(r.choice([66000, 70001, 131072, 200003, 262144 + 5, 400000, 1048576, 1300000, 2100000, 2500000]))
+        Hq = int(r.choice([1, 2, 3, 5]))
+        k = min(int(r.choice([256, 300, 1000, 2048, 4096, 6000, 8192, 16384])), n // 8)
+        lay = fb.make_layout(1, Hq, n)
+        dist = int(r.integers(0, 5))
+        s = np.zeros((Hq, lay.score_stride), dtype=np.float32)
+        if dist == 0:
+            x = r.standard_normal((Hq, n))
+        elif dist == 1:
+            x = np.round(r.standard_normal((Hq, n)), 2)
+        elif dist == 2:
+            x = r.standard_normal((Hq, n)) * np.linspace(0.2, 3, n)[None]
+        elif dist == 3:
+            x = r.exponential(1.0, (Hq, n)) * r.choice([-1, 1], (Hq, n))
+        else:
+            x = r.standard_normal((Hq, n)) * 1e-3 + 5.0
+        s[:, :n] = x.astype(np.float32)
+        n_sink, n_local = (0, 0) if r.random() < 0.5 else (int(r.integers(0, 9)), int(r.integers(0, 70)))
+        if n_sink + n_local > k:
+            n_sink, n_local = 0, 0
+        sc = torch.from_numpy(s).cuda()
+        ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+        idx = torch.full((Hq, k), -1, dtype=torch.int32, device="cuda")
+        ctx.fathom_topk(lay, sc, k, n_sink, n_local, idx)
+        want = O.topk(s[:, :n].astype(np.float64), k, n_sink, n_local)
+        assert np.array_equal(idx.cpu().numpy(), want), (it, n, Hq, k, dist, n_sink, n_local)
+        assert ctx.fathom_device_status() == 0, it
+        ctx.close()
+        del sc, idx
+
+
 def test_topk_at_the_largest_k_on_every_path():
     """k = FATHOM_MAX_K (16384): the direct select then holds 2 x 16384 tokens, the composite cache and the range
     counters in shared memory at once.  Single-pass and two-pass selection and the fused scan + selection."""
