@@ -356,6 +356,35 @@ def test_fused_scan_topk_equals_scan_then_topk(n, k, hpp):
     assert np.array_equal(idx, O.topk(s.astype(np.float64), k))
 
 
+def test_fused_scan_topk_random_shapes():
+    """Thirty seeded draws of (n, KV heads, group size, heads per plan, budget, k, forced tokens): fathom_topk of the
+    scan's scores and fathom_scan_topk must both give the oracle's selection of those scores."""
+    from paper_2609_17652_b200 import binding as fb
+    r = np.random.default_rng(3)
+    for it in range(30):
+        n = int(r.choice([300, 5000, 20000, 40001, 70001, 131072, 200003, 400000, 1048576]))
+        Hkv, G = [(1, 4), (2, 4), (1, 8), (2, 2), (1, 1), (4, 4)][int(r.integers(0, 6))]
+        Hq = Hkv * G
+        hpp = int(r.choice([h for h in (1, 2, 4, 8) if G % h == 0]))
+        B = int(r.choice([16, 48, 80, 136, 200]))
+        k = max(1, min(int(r.choice([64, 300, 1000, 2048, 4096, 8192])), n // 2))
+        n_sink, n_local = (0, 0) if r.random() < 0.5 else (int(r.integers(0, 5)), int(r.integers(0, 40)))
+        if n_sink + n_local > k:
+            n_sink, n_local = 0, 0
+        L = make_layer(n, Hkv, Hq, seed=100 + it, device="cuda")
+        g = run_gpu(L, B, k, hpp, n_sink=n_sink, n_local=n_local, stages=("scan", "topk"))
+        ref = O.topk(g["scores"].astype(np.float64), k, n_sink, n_local)
+        case = (it, n, Hkv, Hq, hpp, B, k, n_sink, n_local)
+        assert np.array_equal(g["idx"], ref), case
+        lay = fb.make_layout(Hkv, Hq, n)
+        ctx = fb.Context(0, fb.fathom_scratch_bytes(lay, k))
+        idx = torch.full((Hq, k), -1, dtype=torch.int32, device="cuda")
+        ctx.fathom_scan_topk(lay, g["planes_t"], g["scales_t"], L.q, torch.from_numpy(g["depth"]).cuda(), hpp, k, n_sink, n_local, idx)
+        assert np.array_equal(idx.cpu().numpy(), ref), case
+        assert ctx.fathom_device_status() == 0, case
+        ctx.close()
+
+
 def test_fused_scan_topk_with_forced_tokens_and_degenerate_scores():
     L = make_layer(50000, Hkv=2, Hq=8, seed=77, device="cuda")
     _fused_vs_unfused(L, 48, 200, 4, n_sink=4, n_local=32)
