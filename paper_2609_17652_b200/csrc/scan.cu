@@ -203,7 +203,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   };
 
   // ---- a new session: the active row list of this plan, ordered by channel then plane (thread = channel), the
-  //      heads' power-of-two scales and the right operand of every 16 rows
+  //      heads' power-of-two scales (the right operand of every 16 rows follows once the first stage has been requested)
   auto enter_item = [&](int tile) {
     int it = item < 0 ? 0 : item;
     while (tile >= B.tile_end[it]) ++it;                       // uniform over the CTA; items only move forward
@@ -254,7 +254,6 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     npass = nrows > rows_stage ? (nrows + rows_stage - 1) / rows_stage : 1;
     hs = M.hscale[myh];
     hs_tail = hs * 4.8828125e-4f;                              // 2^-11
-    fill_bfr(0);
   };
 
   // first block of launch tile `tile` within its session
@@ -307,7 +306,8 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   enter_item(g);
   const float my_thr = MODE == 2 ? M.thr[myh] : 0.0f;
   int u = 0, pass = 0, buf = 0;
-  prefetch(g, 0, 0, 0);
+  prefetch(g, 0, 0, 0);                                        // the first stage's rows are on their way ...
+  fill_bfr(0);                                                 // ... while the right operand is made
 
   // ---- MODE 2, whole warp: the parked groups, one per lane and round, into the CTA's candidate lists.  A lane marks the
   //      candidates among its group's eight scores (score reaches the head's threshold, token eligible).  Nearly always
@@ -530,6 +530,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
       __syncthreads();                                         // every warp is done with the previous session's row list
       enter_item(g);
       prefetch(g, 0, 0, buf);
+      fill_bfr(0);
     } else if (npass > 1) {
       __syncthreads();                                         // every warp is done with the previous pass's right operand
       fill_bfr(pass);                                          // plans of more than 160 rows: the right operand of the next pass
@@ -660,6 +661,7 @@ int fathom_launch_scan_sample(const fathom_layout* L, const uint64_t* planes, co
 int fathom_launch_scan_filter(const fathom_layout* L, const uint64_t* planes, const uint16_t* scales, const float* q,
                               const uint8_t* depth, int heads_per_plan, const fathom_scan_fuse& fz, cudaStream_t st) {
   // (a programmatic dependent: the second, gated attempt then costs no launch latency when it has nothing to do)
+  if (L->n > (1ll << 30)) return FATHOM_ERR_UNSUPPORTED;      // a parked group keeps its first token in 30 bits
   return dispatch_scan<2>(single_item(L, planes, scales, q, depth, nullptr, 0, 1), L->n_kv_heads, L->n_q_heads, heads_per_plan, fz,
                           true, st);
 }
