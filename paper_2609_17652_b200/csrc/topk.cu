@@ -180,7 +180,12 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
   if (lane == 31) s_warp[warp] = incl;
   __syncthreads();
   uint32_t above = incl - local;
-  for (int w = 0; w < warp; ++w) above += s_warp[w];          // a short serial carry over the warps before this one
+  {                                                           // + the totals of the warps before mine (lane l sums warp l's if l < warp)
+    uint32_t carry = (lane < warp && lane < THREADS / 32) ? s_warp[lane] : 0u;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) carry += __shfl_xor_sync(0xffffffffu, carry, o);
+    above += carry;
+  }
   auto search = [&](uint32_t rank, bool bound_slot) {
     if (rank == 0) {                                          // nothing to select: no bin is above or equal
       if (tid == 0) {
@@ -212,9 +217,9 @@ __device__ void find_threshold_bin(const uint32_t* __restrict__ h, uint32_t* __r
 }
 
 // Histogram of a head's sample (every 16th whole chunk of 1024 scores) by a cluster of SAMPLE_CLUSTER CTAs: each
-// histograms its share of the chunks in its own shared memory, the first CTA of the cluster adds the others' histograms
-// to its own through distributed shared memory and finds the estimated and the bound bin: no global histogram, no
-// flush, no ticket.  For rows of up to a few million scores.
+// histograms its share of the chunks in its own shared memory, the others add their non-empty bins to the first CTA's
+// through distributed shared memory (atomics: a few hundred bins of 4096 hold anything), and the first CTA finds the
+// estimated and the bound bin: no global histogram, no flush, no ticket.  For rows of up to a few million scores.
 constexpr int SAMPLE_THREADS = 1024;
 constexpr int SAMPLE_CLUSTER = 4;
 __global__ void __cluster_dims__(SAMPLE_CLUSTER, 1, 1) __launch_bounds__(SAMPLE_THREADS)
@@ -235,6 +240,7 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
   }
   for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) sh[b] = 0u;
   __syncthreads();
+  auto cleared = cluster.barrier_arrive();                    // my histogram is clear (the first CTA's will be added to)
   const float* row = scores + (size_t)head * (size_t)score_stride;
   // `sampled` whole chunks of 1024 scores, chunk_stride scores apart (16384: every 16th chunk of a score row; 1024: a
   // compact array of sampled scores); CTA `part` of the cluster takes every SAMPLE_CLUSTER-th group of 1024 float4
@@ -246,16 +252,16 @@ topk_sample_kernel(const float* __restrict__ scores, long long sampled, long lon
     atomicAdd(&sh[ordered_key(x.z) >> 20], 1u);
     atomicAdd(&sh[ordered_key(x.w) >> 20], 1u);
   }
-  cluster.sync();                                             // every CTA's histogram is complete
-  if (part == 0) {
+  __syncthreads();                                            // my histogram is complete
+  cluster.barrier_wait(std::move(cleared));                   // (everyone arrived long ago: no wait in practice)
+  if (part != 0) {                                            // my non-empty bins are added to the first CTA's: a few hundred of 4096
+    uint32_t* first = cluster.map_shared_rank(sh, 0);
     for (int b = threadIdx.x; b < FATHOM_TOPK_BINS; b += SAMPLE_THREADS) {
-      uint32_t c = sh[b];
-#pragma unroll
-      for (int r = 1; r < SAMPLE_CLUSTER; ++r) c += cluster.map_shared_rank(sh, r)[b];
-      sh[b] = c;
+      const uint32_t c = sh[b];
+      if (c) atomicAdd(first + b, c);
     }
   }
-  cluster.sync();                                             // the others' shared memory has been read: they may exit
+  cluster.sync();                                             // the additions are complete and visible
   if (part != 0) return;
   find_threshold_bin<SAMPLE_THREADS, false>(sh, state + head * 8, want, nullptr, s_warp, want_bound);
 }
@@ -430,7 +436,7 @@ topk_collect_kernel(const float* __restrict__ scores, long long n, long long sco
   if (total == 0u) return;                                    // (the same for every thread)
   if (threadIdx.x == 0) s_base = atomicAdd(&cand_count[head], total);
   __syncthreads();
-  if (mine == 0u) return;
+  if (mine == 0u || (long long)s_base + total > n) return;    // (a list holds at most n: every token is appended once per call)
   uint32_t pos = s_base + before + incl - cnt;
   float* cs = cand_score + (size_t)head * (size_t)n;
   int32_t* ci = cand_idx + (size_t)head * (size_t)n;
