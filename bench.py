@@ -39,14 +39,14 @@ WORKLOAD = dict(name="million-token session, one Qwen3-8B-shaped layer (config 3
                 n=1 << 20, Hkv=8, Hq=32, d=128, B=48, k=4096, heads_per_plan=4)
 # dram__bytes_read.sum + dram__bytes_write.sum per unit (one token of one KV head) from the ncu captures
 # summarised under profiles/: build at n = 131072 (596.1 MB / 1,048,576 units; traffic is proportional to
-# units), scan at n = 1,048,576 and B = 48 (139.7 MB / 8,388,608 units; part of the score writes is still in
-# L2 when the kernel ends), the three top-k kernels at n = 1,048,576, k = 4096 (8.4 + 134.25 + 1.7 MB read, 0.5 MB
-# written / 8,388,608 units; valid for the single-pass path only), attention at k = 4096 (66.1 MB read + 1.05 MB
+# units), scan at n = 1,048,576 and B = 48 (58.5 MB read + 81.9 MB written = 140.4 MB / 8,388,608 units; part of the
+# score writes is still in L2 when the kernel ends), the three top-k kernels at n = 1,048,576, k = 4096 (8.4 + 134.25 +
+# 2.2 MB read, 3.7 MB written / 8,388,608 units; valid for the single-pass path only), attention at k = 4096 (66.1 MB read + 1.05 MB
 # written; proportional to k, not to n: 67.1 MB / (32 heads x 4096 rows) = 512.3 B per selected row).
 # Multiplied by the units of a launch in the JSON line.
-NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.65, "topk_*": 17.3}
+NCU_TRAFFIC_BYTES_PER_TOKEN_KVHEAD = {"build_planes_kernel": 568.5, "scan_kernel": 16.74, "topk_*": 17.7}
 NCU_TRAFFIC_BYTES_PER_SELECTED_ROW = 512.3
-NCU_SCAN_WARP_INSTRUCTIONS_PER_BLOCK_OF_48_ROWS = 232.0         # smsp__inst_executed.sum / (n * Hkv / 64) at B = 48 (profiles/scan_kernel_n1M_B48.md)
+NCU_SCAN_WARP_INSTRUCTIONS_PER_BLOCK_OF_48_ROWS = 222.7         # smsp__inst_executed.sum / (n * Hkv / 64) at B = 48 (profiles/scan_kernel_n1M_B48.md)
 
 
 def parse_args():
