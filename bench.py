@@ -424,10 +424,20 @@ def run_ours(args):
     scan_s = stage_us["scan"] * 1e-6
     result["roofline"] = roof("scan", stage_us["scan"], "scan_kernel", n * Hkv)
     result["roofline"]["frac_index_bytes_only"] = round(plane_bytes_read / scan_s / 1e9 / peak, 4)
+    # what two events around ONE launch cost by themselves: a one-element fill kernel between two events
+    tiny = torch.zeros(1, device=dev)
+    ov = []
+    for _ in range(50):
+        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_.record(stream); tiny.fill_(1.0); b_.record(stream)
+        torch.cuda.synchronize()
+        ov.append(a_.elapsed_time(b_) * 1e3)
+    result["roofline"]["event_bracket_overhead_us"] = round(statistics.median(ov), 2)
     result["roofline"]["launch_us_back_to_back"] = round(scan_b2b_us, 2)
     result["roofline"]["frac_back_to_back"] = round(alg_bytes["scan"] / (scan_b2b_us * 1e-6) / 1e9 / peak, 4)
     result["roofline"]["note_back_to_back"] = ("launch_us is the stage time inside the decode step (an event on either side of the call: it "
-                                               "includes the launch latency the events expose); launch_us_back_to_back is the mean of 40 launches "
+                                               "includes the launch latency the events expose - event_bracket_overhead_us is what a one-element "
+                                               "fill kernel measures between two events); launch_us_back_to_back is the mean of 40 launches "
                                                "in a row over the four layers' stores in turn (no gaps; every launch reads rows evicted since their last use)")
     result["roofline"]["note"] = ("algorithmic bytes = plane words and scales read + fp32 scores written; frac_index_bytes_only counts the "
                                   "plane words and scales alone (the paper's GB/s convention); with the scores materialised that figure "
