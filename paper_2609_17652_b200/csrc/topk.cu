@@ -707,7 +707,7 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
                    uint32_t* __restrict__ dev_status, uint32_t* __restrict__ tile_count, int ntiles,
                    const uint32_t* __restrict__ cand_count, long long cand_capacity, uint32_t want_direct, int bucket_shift,
                    Gate gate, const float* __restrict__ collect_scores, long long collect_stride, float* __restrict__ collect_score_out,
-                   int32_t* __restrict__ collect_idx_out, int cache_entries, int lo_word, int parts) {
+                   int32_t* __restrict__ collect_idx_out, int cache_entries, int lo_word, int parts, const uint32_t* __restrict__ cand_count_second) {
   constexpr int DIGIT_BITS = 11, DIGITS = 1 << DIGIT_BITS;    // radix of the candidate select
   constexpr int DPT = DIGITS / FIN_THREADS;                    // digits per thread in the suffix scan
   static_assert(FIN_THREADS == 1024, "one pair of s_diff words per lane; digits and ranges per thread");
@@ -736,9 +736,21 @@ topk_select_kernel(const float* __restrict__ scores, long long n, long long scor
   }
   FATHOM_PDL_WAIT();                                          // the candidates come from the previous kernel
   FATHOM_PDL_RELEASE();                                       // the attention that follows may become resident now
-  if (!fathom_gate_open(gate)) return;
+  // gate mode 3: one launch serves both attempts of the fused path - the first attempt's lists if every head holds what
+  // it needs, else the lists the second filtering scan has written over them (counted in cand_count_second; their
+  // threshold was a bin, so the general way)
+  bool second = false;
+  if (gate.mode == 3) {
+    bool ok = true;
+    for (int h = tid; h < gate.heads; h += FIN_THREADS) ok = ok && (__ldcg(gate.counts + h) >= gate.want);
+    second = __syncthreads_and(ok) == 0;
+  } else if (!fathom_gate_open(gate)) {
+    return;
+  }
+  if (second) cand_count = cand_count_second;
   if (counted) {
-    if (select_by_fine_histogram<SMALL_BUCKET>(scores + (size_t)head * (size_t)cand_capacity, cand + (size_t)head * (size_t)cand_capacity,
+    if (!second &&
+        select_by_fine_histogram<SMALL_BUCKET>(scores + (size_t)head * (size_t)cand_capacity, cand + (size_t)head * (size_t)cand_capacity,
                                                cand_capacity, cand_count + head, gate.mode == 5 && collect_scores != nullptr, want_direct,
                                                state + head * 8 + lo_word, n, k, part, F, s_dyn, s_hist, s_warp,
                                                idx_out + (size_t)head * k, dev_status))
@@ -1198,6 +1210,8 @@ static size_t direct_select_smem(int k) { return (size_t)direct_cache_entries(k)
 
 // The two attempts of a sampled path on the candidates collected above the estimated bin (counts in S.cand_count)
 // and above the bound bin (S.cand_count2): the first runs if every head collected `want`, the second otherwise.
+// gate_mode 3: both attempts of the fused path in one launch (after both filtering scans): the first lists if every head
+// collected `want`, else the second.
 // gate_mode 0: a single attempt whose threshold is a bound (candidates counted in S.cand_count); 1 / 2: first and second
 // attempt of the fused path (all heads together, second list counted in S.cand_count2); 5: the single-pass top-k, head
 // by head in one launch - a head that collected too few collects again itself, above the bound bin, from `scores`.
@@ -1218,7 +1232,7 @@ static int launch_direct_select(fathom_ctx* ctx, long long n, int Hq, int k, For
       topk_select_kernel<true>, dim3(Hq * parts), dim3(FIN_THREADS), smem, st, (const float*)S.cand_score, n, 0LL, F,
       (const uint32_t*)S.state, (const int32_t*)S.cand, (uint32_t*)nullptr, 0LL, k, idx, ctx->dev_status, (uint32_t*)nullptr, 0,
       (const uint32_t*)(gate_mode == 2 ? S.cand_count2 : S.cand_count), n, want, bucket_shift_for(n), g,
-      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k), lo_word, parts));
+      (const float*)(gate_mode == 5 ? scores : nullptr), score_stride, S.cand_score, S.cand, direct_cache_entries(k), lo_word, parts, (const uint32_t*)(gate_mode == 3 ? S.cand_count2 : nullptr)));
   return FATHOM_OK;
 }
 
@@ -1252,7 +1266,7 @@ static int run_dense_topk(fathom_ctx* ctx, const float* scores, long long n, lon
     topk_select_kernel<false><<<Hq, FIN_THREADS, select_cache_smem(), st>>>(scores, n, score_stride, F, S.state, S.cand, S.bitmap,
                                                                             S.bitmap_words, k, idx, ctx->dev_status, S.tile_count,
                                                                             ntiles, nullptr, 0, 0u, 0, always, nullptr, 0, nullptr, nullptr, FIN_CACHE,
-                                                                            -1, 1);
+                                                                            -1, 1, nullptr);
     topk_emit_kernel<<<fgrid, FILT_TILE / 128, 0, st>>>(S.bitmap, S.bitmap_words, S.tile_count, n, k, idx);
   } else {
     // the sample histogram counts forced tokens too, so both ranks allow for all of them: at least k sampled tokens
@@ -1406,8 +1420,6 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
   fz.gate = fathom_gate{nullptr, 0u, 0, 0};
   rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
   if (rc != FATHOM_OK) return rc;
-  rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, two_attempts ? 1 : 0, st);
-  if (rc != FATHOM_OK) return rc;
   if (two_attempts) {                                         // stands by: runs only if some head's estimate was too high
     fz.state = S.state + 3;
     fz.state_is_score = 0;
@@ -1415,9 +1427,10 @@ extern "C" int fathom_scan_topk(fathom_ctx* ctx, const fathom_layout* L, const u
     fz.gate = fathom_gate{S.cand_count, want, Hq, 2};
     rc = fathom_launch_scan_filter(L, planes, scales, q, depth, heads_per_plan, fz, st);
     if (rc != FATHOM_OK) return rc;
-    rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, 2, st);
-    if (rc != FATHOM_OK) return rc;
   }
+  // one selection serves both outcomes (a kernel in the chain costs 2.5 us even when it has nothing to do)
+  rc = launch_direct_select(ctx, n, Hq, k, F, want, S, idx, two_attempts ? 3 : 0, st);
+  if (rc != FATHOM_OK) return rc;
   FATHOM_CUDA_TRY(ctx, cudaGetLastError());
   return FATHOM_OK;
 }

@@ -393,6 +393,13 @@ def test_fused_scan_topk_with_forced_tokens_and_degenerate_scores():
     # scores that grow along the sequence: the sampled tiles see the trend, the bound stays a bound
     L.K[:, :, :] = L.K * torch.linspace(0.2, 3.0, L.n, device="cuda")[None, :, None]
     _fused_vs_unfused(L, 48, 400, 4)
+    # keys five times larger in the sampled tiles (every 16th tile of 1024 tokens) than elsewhere: the estimate from the
+    # sample is far too high, the first filtering scan collects too few, and the second one (bound threshold) must serve
+    L2 = make_layer(70000, Hkv=2, Hq=8, seed=78, device="cuda")
+    tile = torch.arange(L2.n, device="cuda") // 1024
+    L2.K[:, :, :] = L2.K * torch.where(tile % 16 == 0, 5.0, 1.0)[None, :, None]
+    _fused_vs_unfused(L2, 48, 600, 4)
+    _fused_vs_unfused(L2, 48, 600, 1)
 
 
 @pytest.mark.parametrize("n", [5000, 8192 + 77])
