@@ -684,7 +684,9 @@ def test_rotation_and_covariance_kernels_both_paths(n, dtype, path, monkeypatch)
 
 @pytest.mark.parametrize("n,Hq,k,n_sink,n_local", [(300_000, 3, 6000, 0, 0),      # lists of 8192..16384: two rounds of loads
                                                    (300_000, 3, 2500, 4, 32),   # short lists, forced tokens
-                                                   (1_700_000, 2, 2048, 0, 0),  # too long for the shared-memory bitmap
+                                                   (1_700_000, 2, 2048, 0, 0),  # four bitmap groups per thread
+                                                   (2_097_151, 1, 4096, 0, 0),  # the longest sequence of the short way (tokens in 21 bits)
+                                                   (2_097_152 + 64, 1, 4096, 3, 40),   # one more block: the general way
                                                    (140_000, 2, 1024, 0, 64)])  # a sample of few chunks
 def test_topk_direct_select_short_and_general_way(n, Hq, k, n_sink, n_local):
     """The selection among the collected candidates has a short way (fine histogram + bitmap in shared memory: lists of
