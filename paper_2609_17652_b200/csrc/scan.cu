@@ -143,7 +143,8 @@ __device__ __forceinline__ void mma_rows(float (&acc)[4][4], const unsigned char
 // MODE 2: every tile is scanned, nothing is written but the tokens whose score reaches the head's threshold:
 //         (score, token) pairs appended to the head's candidate list.
 // grid = (CTAs per plan, groups of NH query heads); MODE 1 and 2 are launched with one item.
-template <int NH, int MODE>
+// IN_HBM: every store of the launch lies in device memory (its rows are staged past the L1).
+template <int NH, int MODE, bool IN_HBM>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
 scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fathom_scan_fuse fz) {
   extern __shared__ __align__(16) unsigned char scan_smem[];   // sizeof(Smem<MODE>): more than the static limit in MODE 2
@@ -155,6 +156,7 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
   int g = blockIdx.x;                                          // my current tile of the launch
   if (g >= total) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr bool in_hbm = IN_HBM;
   const int gq = lane >> 2, t4 = lane & 3;                     // mma fragment coordinates: lane = (row group, column pair)
   const int h0 = blockIdx.y * NH;                              // first of the NH query heads of this CTA
   const int plan = h0 / heads_per_plan;                        // NH divides heads_per_plan: one plan per CTA
@@ -278,16 +280,17 @@ scan_kernel(const __grid_constant__ ScanBatch B, int G, int heads_per_plan, fath
     const int c = tid & ((1 << sh) - 1);                       // my 16-byte column of every row I copy
     const bool valid = 2 * c < nblk;
     for (int r = tid >> sh; r < sc; r += THREADS >> sh)
-      fathom_copy_async<16>(wdst + r * row_bytes + c * 16, valid ? planes_kv + M.woff[s0 + r] + c : planes_kv, valid);
+      fathom_copy_async<16>(wdst + r * row_bytes + c * 16, valid ? planes_kv + M.woff[s0 + r] + c : planes_kv, valid, in_hbm);
     unsigned char* sdst = M.scale[buf];
     if (tb == 16) {
       const int cs = tid & 1;
       const bool vs = 8 * cs < nblk;
       for (int r = tid >> 1; r < sc; r += THREADS >> 1)
-        fathom_copy_async<16>(sdst + r * (Geo<16>::SCALE_ELEMS * 2) + cs * 16, vs ? scales_kv + (uint64_t)M.soff[s0 + r] * 16 + cs * 16 : scales_kv, vs);
+        fathom_copy_async<16>(sdst + r * (Geo<16>::SCALE_ELEMS * 2) + cs * 16, vs ? scales_kv + (uint64_t)M.soff[s0 + r] * 16 + cs * 16 : scales_kv, vs,
+                              in_hbm);
     } else if (tb == 8) {
       for (int r = tid; r < sc; r += THREADS)
-        fathom_copy_async<16>(sdst + r * (Geo<8>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.soff[s0 + r] * 16, true);
+        fathom_copy_async<16>(sdst + r * (Geo<8>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.soff[s0 + r] * 16, true, in_hbm);
     } else {
       for (int r = tid; r < sc; r += THREADS)
         fathom_copy_async<8>(sdst + r * (Geo<4>::SCALE_ELEMS * 2), scales_kv + (uint64_t)M.soff[s0 + r] * 16, true);
@@ -566,24 +569,26 @@ int launch_scan(const ScanBatch& B, int Hkv, int Hq, int heads_per_plan, const f
   const long long tiles = B.tile_end[B.items - 1];
   if (tiles <= 0) return FATHOM_OK;
   const int plans = Hq / NH;
-  dim3 grid((unsigned)fathom_scan_grid_ctas(tiles, plans, fathom_planes_in_host_memory(B.planes[0]), CTAS_PER_SM), (unsigned)plans);
+  bool host = false;                                          // any store of the launch in pinned host memory
+  for (int i = 0; i < B.items; ++i) host = host || fathom_planes_in_host_memory(B.planes[i]);
+  dim3 grid((unsigned)fathom_scan_grid_ctas(tiles, plans, host, CTAS_PER_SM), (unsigned)plans);
   constexpr size_t smem = sizeof(Smem<MODE>);                 // dynamic: MODE 2 needs more than the static limit
+  auto kernel = host ? scan_kernel<NH, MODE, false> : scan_kernel<NH, MODE, true>;
   if (smem > 48 * 1024) {
-    static bool configured[64] = {};
+    static bool configured[64][2] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return FATHOM_ERR_CUDA;
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-      if (cudaFuncSetAttribute(scan_kernel<NH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return FATHOM_ERR_CUDA;
-      configured[dev] = true;
+    if (dev >= 0 && dev < 64 && !configured[dev][host ? 0 : 1]) {
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return FATHOM_ERR_CUDA;
+      configured[dev][host ? 0 : 1] = true;
     }
   }
   if (dependent) {                                            // may become resident while the previous kernel of the stream runs
-    if (fathom_launch_dependent(scan_kernel<NH, MODE>, grid, dim3(THREADS), smem, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
+    if (fathom_launch_dependent(kernel, grid, dim3(THREADS), smem, st, B, Hq / Hkv, heads_per_plan, fz) != cudaSuccess)
       return FATHOM_ERR_CUDA;
     return FATHOM_OK;
   }
-  scan_kernel<NH, MODE><<<grid, THREADS, smem, st>>>(B, Hq / Hkv, heads_per_plan, fz);
+  kernel<<<grid, THREADS, smem, st>>>(B, Hq / Hkv, heads_per_plan, fz);
   return FATHOM_OK;
 }
 
