@@ -382,6 +382,17 @@ def run_ours(args):
     scan_b2b_us = a_.elapsed_time(b_) * 1e3 / 40
     result["scan"]["us_back_to_back_over_the_layers"] = round(scan_b2b_us, 2)
     result["scan"]["gbs_with_score_writes_back_to_back"] = round(alg_bytes["scan"] / (scan_b2b_us * 1e-6) / 1e9, 1)
+    # ---- the top-k chain (sample, collection, selection) without launch gaps: 40 calls in a row on the scores of the last scan
+    for rep in range(2):
+        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_.record(stream)
+        for it in range(40):
+            ctx.fathom_topk(lay, scores, k, 0, 0, idx, stream)
+        b_.record(stream)
+        torch.cuda.synchronize()
+    topk_b2b_us = a_.elapsed_time(b_) * 1e3 / 40
+    result["topk"] = {"us_in_the_step_between_events": round(stage_us["topk"], 2), "us_back_to_back": round(topk_b2b_us, 2),
+                      "score_bytes": alg_bytes["topk"], "gbs_back_to_back": round(alg_bytes["topk"] / (topk_b2b_us * 1e-6) / 1e9, 1)}
     # ---- the configuration's second budget (B = 80) through the same kernels: bytes read, scan time
     other = {}
     for B2 in (80,):
